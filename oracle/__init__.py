@@ -1,0 +1,220 @@
+"""CPU oracle for the W4A8-dINT linear layer: numpy front end of w4a8_oracle.c.
+
+TEST INFRASTRUCTURE ONLY.  Tests, the smoke check and the bench's CPU-baseline
+leg compare the CUDA library against these functions; the product never calls
+them.  The arithmetic lives in w4a8_oracle.c (plain C, one rounded binary32
+operation per written operation); this module only marshals numpy arrays.
+
+Paper passages: dINT quantize / dequantize are Eq. 5 / Eq. 6 (Section 4.2);
+the operand scaling is Eq. 1 (Section 3.2); the quantizer granularities
+(token-wise activations, output-channel-wise weights, Min-Max asymmetric) are
+Appendix A.1 "Quantization Settings".
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "w4a8_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+# No value-changing optimisation: no fast-math, no FMA contraction.
+CFLAGS = ["-O2", "-fPIC", "-shared", "-std=c11", "-ffp-contract=off",
+          "-fno-fast-math", "-fopenmp"]
+
+
+def build(force: bool = False) -> str:
+    """Compile w4a8_oracle.c to liboracle.so (gcc) when missing or stale."""
+    stale = (not os.path.exists(_LIB)
+             or os.path.getmtime(_LIB) < os.path.getmtime(_SRC))
+    if force or stale:
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.run(["gcc", *CFLAGS, "-o", tmp, _SRC, "-lm"], check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_half_to_float.restype = ctypes.c_float
+        _lib.oracle_half_to_float.argtypes = [ctypes.c_uint16]
+        _lib.oracle_float_to_bf16.restype = ctypes.c_uint16
+        _lib.oracle_float_to_bf16.argtypes = [ctypes.c_float]
+        _lib.oracle_dint_p.restype = ctypes.c_int
+        _lib.oracle_dint_p.argtypes = [ctypes.c_int]
+        _lib.oracle_dint_quantize.restype = ctypes.c_int
+        _lib.oracle_dint_quantize.argtypes = [ctypes.c_float, ctypes.c_float,
+                                              ctypes.c_int, ctypes.c_int]
+        _lib.oracle_dint_dequantize.restype = ctypes.c_float
+        _lib.oracle_dint_dequantize.argtypes = [ctypes.c_int, ctypes.c_float,
+                                                ctypes.c_int, ctypes.c_int]
+        _lib.oracle_get_threads.restype = ctypes.c_int
+    return _lib
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    if a.dtype != dtype:
+        raise TypeError(f"expected {dtype}, got {a.dtype}")
+    return a
+
+
+def set_threads(n: int) -> None:
+    lib().oracle_set_threads(ctypes.c_int(n))
+
+
+def get_threads() -> int:
+    return int(lib().oracle_get_threads())
+
+
+# ---------------------------------------------------------------------------
+# scalar format routines (Eq. 5, Eq. 6)
+# ---------------------------------------------------------------------------
+
+def dint_p(b: int = 4) -> int:
+    """Number of uniform steps p = 2^b - 3 (Section 4.2)."""
+    return int(lib().oracle_dint_p(b))
+
+
+def dint_quantize(x: float, s: float, z: int, b: int = 4) -> int:
+    """Eq. 5: real value -> dINT code (0..p integer levels, p+1 = c1, p+2 = c2)."""
+    return int(lib().oracle_dint_quantize(np.float32(x), np.float32(s), z, b))
+
+
+def dint_dequantize(code: int, s: float, z: int, b: int = 4) -> float:
+    """Eq. 6: dINT code -> real value (binary32)."""
+    return float(lib().oracle_dint_dequantize(code, np.float32(s), z, b))
+
+
+def dint_table2(z: int, b: int = 4) -> np.ndarray:
+    """Eq. 6 in units of s/2: 2(code - z) for integer levels, +1 / -1 for c1 / c2."""
+    t = np.zeros(1 << b, dtype=np.int8)
+    lib().oracle_dint_table2(ctypes.c_int(z), ctypes.c_int(b), _p(t))
+    return t
+
+
+def half_to_float(bits: int) -> float:
+    return float(lib().oracle_half_to_float(bits))
+
+
+def float_to_bf16(f: float) -> int:
+    return int(lib().oracle_float_to_bf16(np.float32(f)))
+
+
+# ---------------------------------------------------------------------------
+# the three calls of the path, on host arrays
+# ---------------------------------------------------------------------------
+
+def pack_weights(W: np.ndarray, s_in: np.ndarray | None = None, group: int = 0,
+                 clip: float = 1.0):
+    """Q(W diag(s)) of Eq. 1 in dINT4.  W is [N, K] float16.
+
+    Returns (codes [N, K/2] uint8, scales [G, N] float32, zeros [G, N] uint8).
+    """
+    W = _c(W, np.float16)
+    N, K = W.shape
+    if K % 2 or (group and K % group):
+        raise ValueError("K must be even and a multiple of the group size")
+    G = K // group if group else 1
+    if s_in is not None:
+        s_in = _c(s_in, np.float32)
+        assert s_in.shape == (K,)
+    codes = np.empty((N, K // 2), dtype=np.uint8)
+    scales = np.empty((G, N), dtype=np.float32)
+    zeros = np.empty((G, N), dtype=np.uint8)
+    lib().oracle_pack_weights(_p(W.view(np.uint16)), _p(s_in) if s_in is not None else None,
+                              ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group),
+                              ctypes.c_float(clip), _p(codes), _p(scales), _p(zeros))
+    return codes, scales, zeros
+
+
+def quantize_act(X: np.ndarray, inv_s_in: np.ndarray | None = None):
+    """Q(diag(s)^-1 X) of Eq. 1, token-wise INT8.  X is [M, K] float16.
+
+    Returns (Xq [M, K] int8, tok_scale [M] float32).
+    """
+    X = _c(X, np.float16)
+    M, K = X.shape
+    if inv_s_in is not None:
+        inv_s_in = _c(inv_s_in, np.float32)
+        assert inv_s_in.shape == (K,)
+    Xq = np.empty((M, K), dtype=np.int8)
+    tok = np.empty((M,), dtype=np.float32)
+    lib().oracle_quantize_act(_p(X.view(np.uint16)),
+                              _p(inv_s_in) if inv_s_in is not None else None,
+                              ctypes.c_int(M), ctypes.c_int(K), _p(Xq), _p(tok))
+    return Xq, tok
+
+
+def _shape(Xq, codes, zeros, group):
+    M, K = Xq.shape
+    N = codes.shape[0]
+    assert codes.shape == (N, K // 2)
+    G = K // group if group else 1
+    assert zeros.shape == (G, N)
+    return M, N, K, G
+
+
+def linear_acc(Xq, codes, zeros, group: int = 0, wide: bool = False) -> np.ndarray:
+    """Integer accumulators [G, M, N]; int64 when `wide`, else int32."""
+    Xq = _c(Xq, np.int8)
+    codes = _c(codes, np.uint8)
+    zeros = _c(zeros, np.uint8)
+    M, N, K, G = _shape(Xq, codes, zeros, group)
+    acc = np.empty((G, M, N), dtype=np.int64 if wide else np.int32)
+    fn = lib().oracle_linear_acc_i64 if wide else lib().oracle_linear_acc_i32
+    fn(_p(Xq), _p(codes), _p(zeros), ctypes.c_int(M), ctypes.c_int(N),
+       ctypes.c_int(K), ctypes.c_int(group), _p(acc))
+    return acc
+
+
+def linear(Xq, tok_scale, codes, scales, zeros, bias=None, group: int = 0) -> np.ndarray:
+    """BF16 output bits [M, N] (uint16) of the quantized linear layer."""
+    Xq = _c(Xq, np.int8)
+    codes = _c(codes, np.uint8)
+    zeros = _c(zeros, np.uint8)
+    scales = _c(scales, np.float32)
+    tok_scale = _c(tok_scale, np.float32)
+    M, N, K, G = _shape(Xq, codes, zeros, group)
+    if bias is not None:
+        bias = _c(bias, np.float32)
+    Y = np.empty((M, N), dtype=np.uint16)
+    lib().oracle_linear(_p(Xq), _p(tok_scale), _p(codes), _p(scales), _p(zeros),
+                        _p(bias) if bias is not None else None, ctypes.c_int(M),
+                        ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group), _p(Y))
+    return Y
+
+
+def linear_f64(Xq, tok_scale, codes, scales, zeros, bias=None, group: int = 0) -> np.ndarray:
+    """The same output in binary64, not rounded to BF16."""
+    Xq = _c(Xq, np.int8)
+    codes = _c(codes, np.uint8)
+    zeros = _c(zeros, np.uint8)
+    scales = _c(scales, np.float32)
+    tok_scale = _c(tok_scale, np.float32)
+    M, N, K, G = _shape(Xq, codes, zeros, group)
+    if bias is not None:
+        bias = _c(bias, np.float32)
+    Y = np.empty((M, N), dtype=np.float64)
+    lib().oracle_linear_f64(_p(Xq), _p(tok_scale), _p(codes), _p(scales), _p(zeros),
+                            _p(bias) if bias is not None else None, ctypes.c_int(M),
+                            ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group), _p(Y))
+    return Y
+
+
+def bf16_bits_to_float(bits: np.ndarray) -> np.ndarray:
+    """Widen BF16 bit patterns (uint16) to float32 values (exact)."""
+    return (bits.astype(np.uint32) << 16).view(np.float32)
