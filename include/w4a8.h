@@ -1,0 +1,157 @@
+/*
+ * w4a8.h - C ABI of the B200 (sm_100a) W4A8-dINT quantized linear layer.
+ *
+ * The layer computes  Y = Q(diag(s)^-1 X) * Q(W diag(s))^T  (+ bias)  of
+ * arXiv 2311.05161, Eq. 1, with
+ *   - weights W[N][K] (N output features, K input features) quantized per output
+ *     channel, or per group of 128 input features, to the 4-bit dINT format of
+ *     Section 4.2 (Eq. 5 quantize, Eq. 6 dequantize): integer levels 0..13 plus two
+ *     special codes worth +s/2 and -s/2;
+ *   - activations X[M][K] (M tokens) quantized per token to INT8 (Appendix A.1,
+ *     "token-wise quantization for activations"), symmetric absmax variant;
+ *   - an exact INT8 x INT8 -> INT32 contraction on the tensor cores, in which a dINT
+ *     code stands for the integer 2 * (value / s), so the half-step levels stay whole;
+ *   - an FP32 rescale by (token step) x (weight step / 2), optional FP32 bias, BF16 out.
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer owned by the caller unless marked "host".
+ *   - Row-major everywhere.  K % 128 == 0, N % 8 == 0, M >= 1, K < 2^19.
+ *   - group_size is 0 (one step size and zero-point per output channel) or 128.
+ *   - Base pointers must be 16-byte aligned, `packed` and `workspace` 256-byte aligned.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All work
+ *     is enqueued on it; no call synchronizes the device except w4a8_poll_status.
+ *   - The library allocates no device memory and keeps no device state between calls.
+ *   - Every call validates its arguments first and launches nothing when validation
+ *     fails.  Inputs holding NaN or Inf are a precondition violation.
+ *   - There is no CPU or other-architecture fallback: a device that is not compute
+ *     capability 10.x makes the compute calls return W4A8_ERR_UNSUPPORTED_ARCH.
+ */
+#ifndef W4A8_H_
+#define W4A8_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    W4A8_OK = 0,
+    W4A8_ERR_NULL = 1,              /* a required pointer is NULL */
+    W4A8_ERR_SHAPE = 2,             /* M, N, K, group_size or an option outside the rules */
+    W4A8_ERR_ALIGN = 3,             /* a pointer breaks the alignment rule */
+    W4A8_ERR_BUFFER_TOO_SMALL = 4,  /* packed_bytes / workspace_bytes below the query */
+    W4A8_ERR_UNSUPPORTED_ARCH = 5,  /* current device is not sm_100 */
+    W4A8_ERR_CUDA = 6,              /* a CUDA runtime or driver call failed */
+    W4A8_ERR_TIMEOUT = 7,           /* a bounded wait inside a kernel ran out */
+    W4A8_ERR_BAD_BLOB = 8           /* `packed` does not hold a blob of this N, K, group */
+} w4a8_status;
+
+/* Which kernel w4a8_linear_ex runs.  AUTO picks by shape. */
+typedef enum {
+    W4A8_PATH_AUTO = 0,
+    W4A8_PATH_SIMPLE = 1,   /* one thread per output, CUDA cores: slow cross-check */
+    W4A8_PATH_TCGEN05 = 2   /* TMA + in-register dINT decode + tcgen05 kind::i8 MMA */
+} w4a8_path;
+
+typedef struct {
+    int path;        /* w4a8_path */
+    int split_k;     /* 0 = automatic; else number of K slices (tcgen05 path) */
+    int tok_tile;    /* 0 = automatic; else tokens per tile: 16, 32, 64, 128 or 256 */
+    int reserved[5]; /* must be zero */
+} w4a8_opts;
+
+/* Bytes of the packed-weight blob for an [N][K] matrix; 0 if the shape is invalid.
+ * Blob = 256-byte header, step sizes FP32 [G][Npad], zero-points u8 [G][Npad], then the
+ * codes in 8 KiB tiles of 128 output rows x 128 input features (G = 1 or K/128,
+ * Npad = N rounded up to 128).  Inside a tile, byte q*2048 + r*16 + j holds the codes of
+ * row r for k = 32 q + 2 j (low nibble) and 32 q + 2 j + 1 (high nibble).  The blob can be
+ * copied, saved and reloaded byte for byte. */
+size_t w4a8_packed_bytes(int N, int K, int group_size);
+
+/* Weight side of Eq. 1 with the dINT4 quantizer of Eq. 5 (offline, once per layer).
+ *   W_f16   [N][K] IEEE binary16.
+ *   s_in    [K] FP32 per-input-channel scale s of Eq. 1, or NULL (all ones).
+ *   clip    ratio in (0, 1] applied to both ends of the Min-Max range (Appendix A.4
+ *           mentions an extra weight clipping after the scale search); 1.0f = Min-Max.
+ *   packed  out, packed_bytes >= w4a8_packed_bytes(N, K, group_size).
+ * Per row (or per 128-wide group): w' = W * s, lo = min(0, min w') * clip,
+ * hi = max(0, max w') * clip, step = (hi - lo) / 13 (1 if zero),
+ * zero-point = clamp(rint(-lo / step), 0, 13), codes by Eq. 5 with c1 = 14, c2 = 15. */
+w4a8_status w4a8_pack_weights(const void *W_f16, const float *s_in, int N, int K,
+                              int group_size, float clip, void *packed,
+                              size_t packed_bytes, void *stream);
+
+/* Activation side of Eq. 1, token-wise INT8 (Appendix A.1), every forward pass.
+ *   X_f16     [M][K] IEEE binary16.
+ *   inv_s_in  [K] FP32 reciprocal of the Eq. 1 scale, or NULL.
+ *   Xq        out [M][K] INT8;  tok_scale out [M] FP32.
+ * Per token: x' = X * inv_s, amax = max |x'|, tok_scale = amax / 127,
+ * q = clamp(rint(x' * (127 / amax)), -127, 127); an all-zero token gives scale 0. */
+w4a8_status w4a8_quantize_act(const void *X_f16, const float *inv_s_in, int M, int K,
+                              int8_t *Xq, float *tok_scale, void *stream);
+
+/* Scratch bytes w4a8_linear needs for this shape (always >= 256: the first 256 bytes
+ * hold the status block read by w4a8_poll_status).  The caller zero-fills the workspace
+ * once after allocating it (w4a8_workspace_init); calls leave it ready for reuse.  Calls
+ * that may overlap on the device need separate workspaces.  The _ex form answers for
+ * explicit options (NULL = automatic); 0 means the shape or the options are invalid. */
+size_t w4a8_linear_workspace_bytes(int M, int N, int K, int group_size);
+size_t w4a8_linear_workspace_bytes_ex(int M, int N, int K, int group_size,
+                                      const w4a8_opts *opts);
+
+/* Zero-fill a workspace (enqueued on `stream`). */
+w4a8_status w4a8_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
+
+/* The quantized matmul of Eq. 1 with the dINT dequantization of Eq. 6 folded in.
+ *   Xq, tok_scale  as written by w4a8_quantize_act ([M][K] INT8, [M] FP32).
+ *   packed         as written by w4a8_pack_weights for the same N, K, group_size.
+ *   bias           [N] FP32 or NULL.
+ *   Y_bf16         out [M][N] bfloat16.
+ * acc[m][n](g) = sum_k Xq[m][k] * t2(code[n][k]),  t2 = 2 (code - z) | +1 | -1   (INT32)
+ * per channel : y = (float(acc) * tok_scale[m]) * (0.5 * step[n])
+ * group 128   : y = (sum_g float(acc_g) * (0.5 * step[g][n])) * tok_scale[m]     (FP32)
+ * then y += bias[n], rounded to BF16 nearest-even.
+ * Returns W4A8_OK once the work is enqueued; kernel-side failures (a wait that ran out,
+ * a blob that does not match) are reported by w4a8_poll_status. */
+w4a8_status w4a8_linear(const int8_t *Xq, const float *tok_scale, const void *packed,
+                        const float *bias, int M, int N, int K, int group_size,
+                        void *Y_bf16, void *workspace, size_t workspace_bytes,
+                        void *stream);
+
+/* Same as w4a8_linear with the kernel, K split and token tile chosen by the caller
+ * (opts == NULL behaves like w4a8_linear).  Unsupported combinations return
+ * W4A8_ERR_SHAPE. */
+w4a8_status w4a8_linear_ex(const int8_t *Xq, const float *tok_scale, const void *packed,
+                           const float *bias, int M, int N, int K, int group_size,
+                           void *Y_bf16, void *workspace, size_t workspace_bytes,
+                           void *stream, const w4a8_opts *opts);
+
+/* Test export: the INT32 accumulators of the contraction, acc [G][M][N], before any
+ * rescale (Eq. 6 in units of step/2).  Uses the same kernels as w4a8_linear_ex. */
+w4a8_status w4a8_linear_acc_i32(const int8_t *Xq, const void *packed, int M, int N, int K,
+                                int group_size, int32_t *acc, void *workspace,
+                                size_t workspace_bytes, void *stream,
+                                const w4a8_opts *opts);
+
+/* Test export: undo the tiling.  codes [N][K/2] with byte k/2 = code[k] | code[k+1] << 4,
+ * scales [G][N] FP32, zeros [G][N] u8. */
+w4a8_status w4a8_unpack_codes(const void *packed, int N, int K, int group_size,
+                              uint8_t *codes, float *scales, uint8_t *zeros, void *stream);
+
+/* Synchronizes `stream`, then reads and clears the status block of `workspace`:
+ * W4A8_OK, W4A8_ERR_TIMEOUT or W4A8_ERR_BAD_BLOB (first failure since the last poll). */
+w4a8_status w4a8_poll_status(void *workspace, void *stream);
+
+/* Host: Eq. 6 in units of step/2 for zero-point z: out[code] = 2 (code - z) for
+ * code <= 13, +1 for 14, -1 for 15.  `out` is a host array of 16. */
+void w4a8_dint4_table(int z, int8_t *out);
+
+/* Host: version string with static storage. */
+const char *w4a8_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* W4A8_H_ */

@@ -1,0 +1,150 @@
+// Token-wise INT8 activation quantizer: Q(diag(s)^-1 X) of Eq. 1 (Appendix A.1,
+// "token-wise quantization for activations"), symmetric absmax variant.
+// One CTA per token; the token stays in registers between the absmax pass and the
+// rounding pass, so HBM sees 2 bytes read and 1 byte written per element.
+#include "common.cuh"
+
+namespace w4a8 {
+
+namespace {
+
+constexpr int kActThreads = 256;
+
+__device__ __forceinline__ void scaled8(const uint4 &v, const float *__restrict__ inv_s, int k0,
+                                        float (&x)[8])
+{
+    const __half2 *h2 = reinterpret_cast<const __half2 *>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(h2[i]);
+        x[2 * i] = f.x;
+        x[2 * i + 1] = f.y;
+    }
+    if (inv_s) {
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(inv_s + k0));
+        const float4 b = __ldg(reinterpret_cast<const float4 *>(inv_s + k0 + 4));
+        x[0] = __fmul_rn(x[0], a.x); x[1] = __fmul_rn(x[1], a.y);
+        x[2] = __fmul_rn(x[2], a.z); x[3] = __fmul_rn(x[3], a.w);
+        x[4] = __fmul_rn(x[4], b.x); x[5] = __fmul_rn(x[5], b.y);
+        x[6] = __fmul_rn(x[6], b.z); x[7] = __fmul_rn(x[7], b.w);
+    }
+}
+
+__device__ __forceinline__ uint32_t round_clamp(float x, float r)
+{
+    int q = __float2int_rn(__fmul_rn(x, r));
+    q = q < -127 ? -127 : (q > 127 ? 127 : q);
+    return (uint32_t)q & 0xffu;
+}
+
+__device__ __forceinline__ uint2 quantize8(const float (&x)[8], float r)
+{
+    uint2 o;
+    o.x = round_clamp(x[0], r) | (round_clamp(x[1], r) << 8) | (round_clamp(x[2], r) << 16) |
+          (round_clamp(x[3], r) << 24);
+    o.y = round_clamp(x[4], r) | (round_clamp(x[5], r) << 8) | (round_clamp(x[6], r) << 16) |
+          (round_clamp(x[7], r) << 24);
+    return o;
+}
+
+__device__ __forceinline__ float block_max(float v, float *smem)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    if ((threadIdx.x & 31) == 0) smem[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float m = smem[0];
+#pragma unroll
+    for (int w = 1; w < kActThreads / 32; ++w) m = fmaxf(m, smem[w]);
+    return m;
+}
+
+// NV = 16-byte vectors per thread held in registers (K <= 2048 * NV); NV == 0 re-reads
+// the token from global memory (L2) in the second pass, for any K.
+template <int NV>
+__global__ void __launch_bounds__(kActThreads)
+act_quant_kernel(const __half *__restrict__ X, const float *__restrict__ inv_s, int M, int K,
+                 int8_t *__restrict__ Xq, float *__restrict__ tok_scale)
+{
+    __shared__ float red[kActThreads / 32];
+    const int m = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int nvec = K >> 3;
+    const uint4 *row = reinterpret_cast<const uint4 *>(X + (size_t)m * K);
+    uint2 *out = reinterpret_cast<uint2 *>(Xq + (size_t)m * K);
+    constexpr int NR = NV > 0 ? NV : 1;
+    uint4 v[NR];
+    float amax = 0.0f;
+    if (NV > 0) {
+#pragma unroll
+        for (int i = 0; i < NR; ++i) {
+            const int idx = tid + i * kActThreads;
+            v[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (idx < nvec) v[i] = __ldcs(row + idx);
+        }
+#pragma unroll
+        for (int i = 0; i < NR; ++i) {
+            const int idx = tid + i * kActThreads;
+            if (idx < nvec) {
+                float x[8];
+                scaled8(v[i], inv_s, idx * 8, x);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(x[e]));
+            }
+        }
+    } else {
+        for (int idx = tid; idx < nvec; idx += kActThreads) {
+            float x[8];
+            scaled8(__ldg(row + idx), inv_s, idx * 8, x);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(x[e]));
+        }
+    }
+    amax = block_max(amax, red);
+    if (amax == 0.0f) {
+        if (tid == 0) tok_scale[m] = 0.0f;
+        for (int idx = tid; idx < nvec; idx += kActThreads) out[idx] = make_uint2(0u, 0u);
+        return;
+    }
+    const float r = __fdiv_rn(127.0f, amax);
+    if (tid == 0) tok_scale[m] = __fdiv_rn(amax, 127.0f);
+    if (NV > 0) {
+#pragma unroll
+        for (int i = 0; i < NR; ++i) {
+            const int idx = tid + i * kActThreads;
+            if (idx < nvec) {
+                float x[8];
+                scaled8(v[i], inv_s, idx * 8, x);
+                out[idx] = quantize8(x, r);
+            }
+        }
+    } else {
+        for (int idx = tid; idx < nvec; idx += kActThreads) {
+            float x[8];
+            scaled8(__ldg(row + idx), inv_s, idx * 8, x);
+            out[idx] = quantize8(x, r);
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_quantize_act(const __half *X, const float *inv_s, int M, int K, int8_t *Xq,
+                                float *tok_scale, cudaStream_t st)
+{
+    const int nvec = K / 8;
+    const int per_thread = (nvec + kActThreads - 1) / kActThreads;
+    if (per_thread <= 1)
+        act_quant_kernel<1><<<M, kActThreads, 0, st>>>(X, inv_s, M, K, Xq, tok_scale);
+    else if (per_thread <= 2)
+        act_quant_kernel<2><<<M, kActThreads, 0, st>>>(X, inv_s, M, K, Xq, tok_scale);
+    else if (per_thread <= 4)
+        act_quant_kernel<4><<<M, kActThreads, 0, st>>>(X, inv_s, M, K, Xq, tok_scale);
+    else if (per_thread <= 8)
+        act_quant_kernel<8><<<M, kActThreads, 0, st>>>(X, inv_s, M, K, Xq, tok_scale);
+    else
+        act_quant_kernel<0><<<M, kActThreads, 0, st>>>(X, inv_s, M, K, Xq, tok_scale);
+    return cudaGetLastError();
+}
+
+}  // namespace w4a8

@@ -1,0 +1,154 @@
+// Shared declarations of the W4A8-dINT CUDA library: blob layout, status block,
+// exact-arithmetic helpers.  sm_100a only.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string.h>
+
+#include "w4a8.h"
+
+namespace w4a8 {
+
+// ---------------------------------------------------------------------------
+// packed-weight blob
+// ---------------------------------------------------------------------------
+constexpr int kTileN = 128;        // output rows per code tile
+constexpr int kTileK = 128;        // input features per code tile (= one quantization group)
+constexpr int kTileBytes = 8192;   // 128 x 128 nibbles
+constexpr int kQuarterBytes = 2048;
+constexpr int kHeaderBytes = 256;
+constexpr uint32_t kBlobMagic = 0x38413457u;   // "W4A8"
+constexpr uint32_t kBlobVersion = 1u;
+constexpr uint32_t kBlobLayoutQuarterRow16 = 1u;
+
+struct BlobHeader {
+    uint32_t magic, version, layout, group;
+    int32_t N, K, G, n_tiles, k_blocks, n_pad;
+    uint32_t pad0[2];
+    uint64_t off_scales, off_zeros, off_codes, total_bytes;
+    float clip;
+    uint32_t pad1[43];
+};
+static_assert(sizeof(BlobHeader) == kHeaderBytes, "blob header is 256 bytes");
+
+struct BlobLayout {
+    int N, K, group, G, n_tiles, k_blocks, n_pad;
+    size_t off_scales, off_zeros, off_codes, total_bytes;
+};
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+__host__ __device__ inline BlobLayout make_layout(int N, int K, int group)
+{
+    BlobLayout L;
+    L.N = N;
+    L.K = K;
+    L.group = group;
+    L.G = group ? K / group : 1;
+    L.n_tiles = (N + kTileN - 1) / kTileN;
+    L.k_blocks = K / kTileK;
+    L.n_pad = L.n_tiles * kTileN;
+    L.off_scales = kHeaderBytes;
+    L.off_zeros = align_up(L.off_scales + (size_t)L.G * L.n_pad * sizeof(float), 256);
+    L.off_codes = align_up(L.off_zeros + (size_t)L.G * L.n_pad, 256);
+    L.total_bytes = L.off_codes + (size_t)L.n_tiles * L.k_blocks * kTileBytes;
+    return L;
+}
+
+// Byte offset, inside the code section, of the byte holding code[n][k] (k even: low nibble).
+__host__ __device__ inline size_t code_byte_offset(const BlobLayout &L, int n, int k)
+{
+    const int nt = n / kTileN, r = n % kTileN;
+    const int kb = k / kTileK, kk = k % kTileK;
+    const int q = kk / 32, j = (kk % 32) / 2;
+    return ((size_t)nt * L.k_blocks + kb) * kTileBytes + (size_t)q * kQuarterBytes + r * 16 + j;
+}
+
+inline bool shape_ok(int N, int K, int group)
+{
+    if (N < 8 || N % 8 != 0) return false;
+    if (K < 128 || K % 128 != 0 || K >= (1 << 19)) return false;
+    if (group != 0 && group != 128) return false;
+    return true;
+}
+
+__device__ inline bool header_matches(const uint8_t *blob, const BlobLayout &L)
+{
+    const BlobHeader *h = reinterpret_cast<const BlobHeader *>(blob);
+    return h->magic == kBlobMagic && h->version == kBlobVersion &&
+           h->layout == kBlobLayoutQuarterRow16 && h->N == L.N && h->K == L.K &&
+           h->group == (uint32_t)L.group;
+}
+
+// ---------------------------------------------------------------------------
+// status block (first 256 bytes of a workspace)
+// ---------------------------------------------------------------------------
+struct StatusBlock {
+    int status;       // 0, W4A8_ERR_TIMEOUT or W4A8_ERR_BAD_BLOB: first failure wins
+    int where;        // site code of the wait that gave up
+    int block;        // CTA that reported
+    int pad[61];
+};
+static_assert(sizeof(StatusBlock) == 256, "status block is 256 bytes");
+
+__device__ inline void report_failure(StatusBlock *sb, int status, int where)
+{
+    if (atomicCAS(&sb->status, 0, status) == 0) {
+        sb->where = where;
+        sb->block = (int)blockIdx.x;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// dINT4 decode in units of step/2 (Eq. 6 doubled)
+// ---------------------------------------------------------------------------
+__host__ __device__ inline int dint4_t2(int code, int z)
+{
+    return code <= 13 ? 2 * (code - z) : (code == 14 ? 1 : -1);
+}
+
+// ---------------------------------------------------------------------------
+// output rescale, one rounded FP32 operation per step
+// ---------------------------------------------------------------------------
+__device__ inline float rescale_channel(int acc, float tok_scale, float half_step)
+{
+    return __fmul_rn(__fmul_rn((float)acc, tok_scale), half_step);
+}
+
+__device__ inline float add_bias(float t, const float *bias, int n)
+{
+    return bias ? __fadd_rn(t, bias[n]) : t;
+}
+
+// ---------------------------------------------------------------------------
+// plan of the tensor-core kernel (shared by the workspace query and the launcher)
+// ---------------------------------------------------------------------------
+struct LinearPlan {
+    int tok_tile;     // tokens per tile (UMMA N): 16, 32, 64, 128, 256
+    int tok_tiles;    // ceil(M / tok_tile)
+    int split_k;      // K slices (1 = none)
+    int kb_per_split; // k-blocks per slice (last slice may be shorter)
+    size_t off_counters, off_partials, workspace_bytes;
+};
+
+// launchers (defined in the .cu files, called by api.cu)
+cudaError_t launch_pack(const __half *W, const float *s_in, const BlobLayout &L, float clip,
+                        uint8_t *blob, cudaStream_t st);
+cudaError_t launch_unpack(const uint8_t *blob, const BlobLayout &L, uint8_t *codes,
+                          float *scales, uint8_t *zeros, cudaStream_t st);
+cudaError_t launch_quantize_act(const __half *X, const float *inv_s, int M, int K, int8_t *Xq,
+                                float *tok_scale, cudaStream_t st);
+cudaError_t launch_linear_simple(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
+                                 const BlobLayout &L, const float *bias, int M,
+                                 __nv_bfloat16 *Y, int32_t *acc, StatusBlock *sb,
+                                 cudaStream_t st);
+bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *plan);
+w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
+                                  const BlobLayout &L, const float *bias, int M,
+                                  __nv_bfloat16 *Y, int32_t *acc, uint8_t *workspace,
+                                  const LinearPlan &plan, cudaStream_t st);
+
+}  // namespace w4a8

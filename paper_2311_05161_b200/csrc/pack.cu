@@ -1,0 +1,222 @@
+// Weight packing: Q(W diag(s)) of Eq. 1 with the dINT4 quantizer of Eq. 5, written in
+// the tiled blob layout, and its inverse (test export).
+#include "common.cuh"
+
+namespace w4a8 {
+
+namespace {
+
+constexpr int kPackThreads = 256;
+
+// Eq. 5 for b = 4: codes 0..13 integer levels, 14 = c1 (+s/2), 15 = c2 (-s/2).
+__device__ __forceinline__ uint32_t dint4_quantize(float x, float s, int z, float quarter,
+                                                   float threeq)
+{
+    if (x > quarter && x <= threeq) return 14u;
+    if (x < -quarter && x >= -threeq) return 15u;
+    float r = rintf(__fdiv_rn(x, s));
+    r = fminf(fmaxf(r, -1048576.0f), 1048576.0f);
+    int q = (int)r + z;
+    q = q < 0 ? 0 : (q > 13 ? 13 : q);
+    return (uint32_t)q;
+}
+
+__device__ __forceinline__ void step_and_zero(float lo, float hi, float clip, float &s, int &z)
+{
+    lo = __fmul_rn(lo, clip);
+    hi = __fmul_rn(hi, clip);
+    s = __fdiv_rn(__fsub_rn(hi, lo), 13.0f);
+    if (s == 0.0f) s = 1.0f;
+    float r = rintf(__fdiv_rn(-lo, s));
+    r = fminf(fmaxf(r, -1048576.0f), 1048576.0f);
+    z = (int)r;
+    z = z < 0 ? 0 : (z > 13 ? 13 : z);
+}
+
+__device__ __forceinline__ float scaled(const __half h, const float *s_in, int k)
+{
+    const float w = __half2float(h);
+    return s_in ? __fmul_rn(w, s_in[k]) : w;
+}
+
+__device__ __forceinline__ void write_header(uint8_t *blob, const BlobLayout &L, float clip)
+{
+    BlobHeader h;
+    memset(&h, 0, sizeof(h));
+    h.magic = kBlobMagic;
+    h.version = kBlobVersion;
+    h.layout = kBlobLayoutQuarterRow16;
+    h.group = (uint32_t)L.group;
+    h.N = L.N; h.K = L.K; h.G = L.G;
+    h.n_tiles = L.n_tiles; h.k_blocks = L.k_blocks; h.n_pad = L.n_pad;
+    h.off_scales = L.off_scales; h.off_zeros = L.off_zeros;
+    h.off_codes = L.off_codes; h.total_bytes = L.total_bytes;
+    h.clip = clip;
+    *reinterpret_cast<BlobHeader *>(blob) = h;
+}
+
+// One CTA per output row; the whole row is one quantization group.
+__global__ void __launch_bounds__(kPackThreads)
+pack_rows_kernel(const __half *__restrict__ W, const float *__restrict__ s_in, BlobLayout L,
+                 float clip, uint8_t *__restrict__ blob)
+{
+    const int n = blockIdx.x;
+    const int tid = threadIdx.x;
+    float *scales = reinterpret_cast<float *>(blob + L.off_scales);
+    uint8_t *zeros = blob + L.off_zeros;
+    uint8_t *codes = blob + L.off_codes;
+    if (n == 0 && tid == 0) write_header(blob, L, clip);
+
+    __shared__ float s_lo[kPackThreads / 32], s_hi[kPackThreads / 32];
+    __shared__ float s_step;
+    __shared__ int s_zero;
+
+    const bool real = n < L.N;
+    const __half *row = W + (size_t)n * L.K;
+    float lo = 0.0f, hi = 0.0f;
+    if (real) {
+        for (int k0 = tid * 8; k0 < L.K; k0 += kPackThreads * 8) {
+            const uint4 v = *reinterpret_cast<const uint4 *>(row + k0);
+            const __half *h = reinterpret_cast<const __half *>(&v);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float w = scaled(h[i], s_in, k0 + i);
+                if (w < lo) lo = w;
+                if (w > hi) hi = w;
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float l2 = __shfl_xor_sync(0xffffffffu, lo, o);
+        const float h2 = __shfl_xor_sync(0xffffffffu, hi, o);
+        if (l2 < lo) lo = l2;
+        if (h2 > hi) hi = h2;
+    }
+    if ((tid & 31) == 0) { s_lo[tid >> 5] = lo; s_hi[tid >> 5] = hi; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < kPackThreads / 32; ++w) {
+            if (s_lo[w] < lo) lo = s_lo[w];
+            if (s_hi[w] > hi) hi = s_hi[w];
+        }
+        float s; int z;
+        step_and_zero(lo, hi, clip, s, z);
+        s_step = s; s_zero = z;
+        scales[n] = s;
+        zeros[n] = (uint8_t)z;
+    }
+    __syncthreads();
+    const float s = s_step;
+    const int z = s_zero;
+    const float quarter = __fmul_rn(0.25f, s), threeq = __fmul_rn(0.75f, s);
+    for (int k0 = tid * 8; k0 < L.K; k0 += kPackThreads * 8) {
+        uint32_t word = 0;
+        if (real) {
+            const uint4 v = *reinterpret_cast<const uint4 *>(row + k0);
+            const __half *h = reinterpret_cast<const __half *>(&v);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                word |= dint4_quantize(scaled(h[i], s_in, k0 + i), s, z, quarter, threeq) << (4 * i);
+        }
+        *reinterpret_cast<uint32_t *>(codes + code_byte_offset(L, n, k0)) = word;
+    }
+}
+
+// One CTA per output row; each warp takes one 128-wide group at a time.
+__global__ void __launch_bounds__(kPackThreads)
+pack_groups_kernel(const __half *__restrict__ W, const float *__restrict__ s_in, BlobLayout L,
+                   float clip, uint8_t *__restrict__ blob)
+{
+    const int n = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float *scales = reinterpret_cast<float *>(blob + L.off_scales);
+    uint8_t *zeros = blob + L.off_zeros;
+    uint8_t *codes = blob + L.off_codes;
+    if (n == 0 && threadIdx.x == 0) write_header(blob, L, clip);
+    const bool real = n < L.N;
+    const __half *row = W + (size_t)n * L.K;
+    for (int g = warp; g < L.G; g += kPackThreads / 32) {
+        const int k0 = g * 128 + lane * 4;
+        float w[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        if (real) {
+            const uint2 v = *reinterpret_cast<const uint2 *>(row + k0);
+            const __half *h = reinterpret_cast<const __half *>(&v);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) w[i] = scaled(h[i], s_in, k0 + i);
+        }
+        float lo = 0.0f, hi = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (w[i] < lo) lo = w[i];
+            if (w[i] > hi) hi = w[i];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float l2 = __shfl_xor_sync(0xffffffffu, lo, o);
+            const float h2 = __shfl_xor_sync(0xffffffffu, hi, o);
+            if (l2 < lo) lo = l2;
+            if (h2 > hi) hi = h2;
+        }
+        float s; int z;
+        step_and_zero(lo, hi, clip, s, z);
+        if (lane == 0) {
+            scales[(size_t)g * L.n_pad + n] = s;
+            zeros[(size_t)g * L.n_pad + n] = (uint8_t)z;
+        }
+        const float quarter = __fmul_rn(0.25f, s), threeq = __fmul_rn(0.75f, s);
+        uint32_t half_word = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            half_word |= dint4_quantize(w[i], s, z, quarter, threeq) << (4 * i);
+        *reinterpret_cast<uint16_t *>(codes + code_byte_offset(L, n, k0)) = (uint16_t)half_word;
+    }
+}
+
+__global__ void unpack_kernel(const uint8_t *__restrict__ blob, BlobLayout L,
+                              uint8_t *__restrict__ out_codes, float *__restrict__ out_scales,
+                              uint8_t *__restrict__ out_zeros)
+{
+    const size_t half_k = (size_t)L.K / 2;
+    const size_t total = (size_t)L.N * half_k;
+    const float *scales = reinterpret_cast<const float *>(blob + L.off_scales);
+    const uint8_t *zeros = blob + L.off_zeros;
+    const uint8_t *codes = blob + L.off_codes;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (size_t)gridDim.x * blockDim.x) {
+        const int n = (int)(i / half_k);
+        const int k = (int)(i % half_k) * 2;
+        out_codes[i] = codes[code_byte_offset(L, n, k)];
+    }
+    const size_t meta = (size_t)L.G * L.N;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < meta;
+         i += (size_t)gridDim.x * blockDim.x) {
+        const int g = (int)(i / L.N), n = (int)(i % L.N);
+        out_scales[i] = scales[(size_t)g * L.n_pad + n];
+        out_zeros[i] = zeros[(size_t)g * L.n_pad + n];
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_pack(const __half *W, const float *s_in, const BlobLayout &L, float clip,
+                        uint8_t *blob, cudaStream_t st)
+{
+    if (L.group == 0)
+        pack_rows_kernel<<<L.n_pad, kPackThreads, 0, st>>>(W, s_in, L, clip, blob);
+    else
+        pack_groups_kernel<<<L.n_pad, kPackThreads, 0, st>>>(W, s_in, L, clip, blob);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_unpack(const uint8_t *blob, const BlobLayout &L, uint8_t *codes,
+                          float *scales, uint8_t *zeros, cudaStream_t st)
+{
+    const size_t total = (size_t)L.N * L.K / 2;
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    unpack_kernel<<<blocks, 256, 0, st>>>(blob, L, codes, scales, zeros);
+    return cudaGetLastError();
+}
+
+}  // namespace w4a8
