@@ -1,0 +1,222 @@
+"""ctypes binding of libw4a8.so: argument marshalling only.
+
+Every function here has the name of the C entry point it calls (include/w4a8.h) minus the
+`w4a8_` prefix.  torch supplies device memory and the current stream; all arithmetic of
+the path runs in the library's CUDA kernels.  There is no fallback: a missing library or a
+non-zero status raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libw4a8.so")
+
+STATUS_NAMES = {
+    0: "W4A8_OK", 1: "W4A8_ERR_NULL", 2: "W4A8_ERR_SHAPE", 3: "W4A8_ERR_ALIGN",
+    4: "W4A8_ERR_BUFFER_TOO_SMALL", 5: "W4A8_ERR_UNSUPPORTED_ARCH", 6: "W4A8_ERR_CUDA",
+    7: "W4A8_ERR_TIMEOUT", 8: "W4A8_ERR_BAD_BLOB",
+}
+PATH_AUTO, PATH_SIMPLE, PATH_TCGEN05 = 0, 1, 2
+
+EXPORTS = (
+    "w4a8_packed_bytes", "w4a8_pack_weights", "w4a8_quantize_act",
+    "w4a8_linear_workspace_bytes", "w4a8_linear_workspace_bytes_ex", "w4a8_workspace_init",
+    "w4a8_linear", "w4a8_linear_ex", "w4a8_linear_acc_i32", "w4a8_unpack_codes",
+    "w4a8_poll_status", "w4a8_dint4_table", "w4a8_version",
+)
+
+
+class W4A8Error(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {STATUS_NAMES.get(status, status)}")
+
+
+class Opts(ctypes.Structure):
+    _fields_ = [("path", ctypes.c_int), ("split_k", ctypes.c_int), ("tok_tile", ctypes.c_int),
+                ("reserved", ctypes.c_int * 5)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python __graft_entry__.py` "
+            "(nvcc, sm_100a). There is no fallback path.")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci, sz, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_float
+    op = ctypes.POINTER(Opts)
+    lib.w4a8_packed_bytes.restype = sz
+    lib.w4a8_packed_bytes.argtypes = [ci, ci, ci]
+    lib.w4a8_pack_weights.restype = ci
+    lib.w4a8_pack_weights.argtypes = [vp, vp, ci, ci, ci, cf, vp, sz, vp]
+    lib.w4a8_quantize_act.restype = ci
+    lib.w4a8_quantize_act.argtypes = [vp, vp, ci, ci, vp, vp, vp]
+    lib.w4a8_linear_workspace_bytes.restype = sz
+    lib.w4a8_linear_workspace_bytes.argtypes = [ci, ci, ci, ci]
+    lib.w4a8_linear_workspace_bytes_ex.restype = sz
+    lib.w4a8_linear_workspace_bytes_ex.argtypes = [ci, ci, ci, ci, op]
+    lib.w4a8_workspace_init.restype = ci
+    lib.w4a8_workspace_init.argtypes = [vp, sz, vp]
+    lib.w4a8_linear.restype = ci
+    lib.w4a8_linear.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, vp]
+    lib.w4a8_linear_ex.restype = ci
+    lib.w4a8_linear_ex.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, vp, op]
+    lib.w4a8_linear_acc_i32.restype = ci
+    lib.w4a8_linear_acc_i32.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, sz, vp, op]
+    lib.w4a8_unpack_codes.restype = ci
+    lib.w4a8_unpack_codes.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp]
+    lib.w4a8_poll_status.restype = ci
+    lib.w4a8_poll_status.argtypes = [vp, vp]
+    lib.w4a8_dint4_table.restype = None
+    lib.w4a8_dint4_table.argtypes = [ci, vp]
+    lib.w4a8_version.restype = ctypes.c_char_p
+    lib.w4a8_version.argtypes = []
+    return lib
+
+
+lib = _load()
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(status: int, what: str):
+    if status != 0:
+        raise W4A8Error(status, what)
+
+
+def _dev(t, dtype, what):
+    if t is None:
+        return None
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{what}: expected a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+def make_opts(path: int = PATH_AUTO, split_k: int = 0, tok_tile: int = 0) -> Opts:
+    o = Opts()
+    o.path, o.split_k, o.tok_tile = path, split_k, tok_tile
+    return o
+
+
+def version() -> str:
+    return lib.w4a8_version().decode()
+
+
+def dint4_table(z: int):
+    buf = (ctypes.c_int8 * 16)()
+    lib.w4a8_dint4_table(z, buf)
+    return list(buf)
+
+
+def packed_bytes(N: int, K: int, group: int = 0) -> int:
+    return int(lib.w4a8_packed_bytes(N, K, group))
+
+
+def pack_weights(W, s_in=None, group: int = 0, clip: float = 1.0, out=None):
+    """W [N, K] float16 (CUDA) -> packed blob (uint8 CUDA tensor)."""
+    W = _dev(W, torch.float16, "W")
+    s_in = _dev(s_in, torch.float32, "s_in")
+    N, K = W.shape
+    nbytes = packed_bytes(N, K, group)
+    if nbytes == 0:
+        raise W4A8Error(2, "w4a8_packed_bytes")
+    if out is None:
+        out = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
+    _check(lib.w4a8_pack_weights(_ptr(W), _ptr(s_in), N, K, group, clip, _ptr(out),
+                                 out.numel(), _stream()), "w4a8_pack_weights")
+    return out
+
+
+def quantize_act(X, inv_s_in=None, out=None):
+    """X [M, K] float16 (CUDA) -> (Xq [M, K] int8, tok_scale [M] float32)."""
+    X = _dev(X, torch.float16, "X")
+    inv_s_in = _dev(inv_s_in, torch.float32, "inv_s_in")
+    M, K = X.shape
+    if out is None:
+        out = (torch.empty((M, K), dtype=torch.int8, device=X.device),
+               torch.empty((M,), dtype=torch.float32, device=X.device))
+    Xq, tok = out
+    _check(lib.w4a8_quantize_act(_ptr(X), _ptr(inv_s_in), M, K, _ptr(Xq), _ptr(tok), _stream()),
+           "w4a8_quantize_act")
+    return Xq, tok
+
+
+def linear_workspace_bytes(M: int, N: int, K: int, group: int = 0, opts: Opts | None = None) -> int:
+    if opts is None:
+        return int(lib.w4a8_linear_workspace_bytes(M, N, K, group))
+    return int(lib.w4a8_linear_workspace_bytes_ex(M, N, K, group, ctypes.byref(opts)))
+
+
+def workspace_init(ws):
+    _check(lib.w4a8_workspace_init(_ptr(ws), ws.numel(), _stream()), "w4a8_workspace_init")
+
+
+def new_workspace(M: int, N: int, K: int, group: int = 0, opts: Opts | None = None, device="cuda"):
+    nbytes = linear_workspace_bytes(M, N, K, group, opts)
+    if nbytes == 0:
+        raise W4A8Error(2, "w4a8_linear_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    workspace_init(ws)
+    return ws
+
+
+def linear(Xq, tok_scale, packed, bias, N: int, group: int, workspace, opts: Opts | None = None,
+           out=None):
+    """Quantized linear layer: returns Y [M, N] bfloat16."""
+    Xq = _dev(Xq, torch.int8, "Xq")
+    tok_scale = _dev(tok_scale, torch.float32, "tok_scale")
+    bias = _dev(bias, torch.float32, "bias")
+    M, K = Xq.shape
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=Xq.device)
+    if opts is None:
+        st = lib.w4a8_linear(_ptr(Xq), _ptr(tok_scale), _ptr(packed), _ptr(bias), M, N, K, group,
+                             _ptr(out), _ptr(workspace), workspace.numel(), _stream())
+    else:
+        st = lib.w4a8_linear_ex(_ptr(Xq), _ptr(tok_scale), _ptr(packed), _ptr(bias), M, N, K,
+                                group, _ptr(out), _ptr(workspace), workspace.numel(), _stream(),
+                                ctypes.byref(opts))
+    _check(st, "w4a8_linear")
+    return out
+
+
+def linear_acc_i32(Xq, packed, N: int, group: int, workspace, opts: Opts | None = None):
+    """INT32 accumulators [G, M, N] of the contraction (test export)."""
+    Xq = _dev(Xq, torch.int8, "Xq")
+    M, K = Xq.shape
+    G = K // group if group else 1
+    acc = torch.empty((G, M, N), dtype=torch.int32, device=Xq.device)
+    _check(lib.w4a8_linear_acc_i32(_ptr(Xq), _ptr(packed), M, N, K, group, _ptr(acc),
+                                   _ptr(workspace), workspace.numel(), _stream(),
+                                   ctypes.byref(opts) if opts is not None else None),
+           "w4a8_linear_acc_i32")
+    return acc
+
+
+def unpack_codes(packed, N: int, K: int, group: int = 0):
+    """Blob -> (codes [N, K/2] uint8, scales [G, N] float32, zeros [G, N] uint8)."""
+    G = K // group if group else 1
+    codes = torch.empty((N, K // 2), dtype=torch.uint8, device=packed.device)
+    scales = torch.empty((G, N), dtype=torch.float32, device=packed.device)
+    zeros = torch.empty((G, N), dtype=torch.uint8, device=packed.device)
+    _check(lib.w4a8_unpack_codes(_ptr(packed), N, K, group, _ptr(codes), _ptr(scales),
+                                 _ptr(zeros), _stream()), "w4a8_unpack_codes")
+    return codes, scales, zeros
+
+
+def poll_status(workspace) -> int:
+    return int(lib.w4a8_poll_status(_ptr(workspace), _stream()))
+
+
+def check_status(workspace):
+    _check(poll_status(workspace), "w4a8_poll_status")

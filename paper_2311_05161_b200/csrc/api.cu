@@ -1,0 +1,191 @@
+// extern "C" entry points: argument validation and dispatch.  See include/w4a8.h.
+#include "common.cuh"
+
+using namespace w4a8;
+
+namespace {
+
+inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// W4A8_OK when the current device is compute capability 10.x.
+w4a8_status check_arch()
+{
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return W4A8_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+        return W4A8_ERR_CUDA;
+    return major == 10 ? W4A8_OK : W4A8_ERR_UNSUPPORTED_ARCH;
+}
+
+bool opts_ok(const w4a8_opts *o)
+{
+    if (!o) return true;
+    if (o->path < W4A8_PATH_AUTO || o->path > W4A8_PATH_TCGEN05) return false;
+    if (o->split_k < 0 || o->tok_tile < 0) return false;
+    for (int i = 0; i < 5; ++i)
+        if (o->reserved[i] != 0) return false;
+    return true;
+}
+
+w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *packed,
+                          const float *bias, int M, int N, int K, int group, void *Y,
+                          int32_t *acc, void *workspace, size_t workspace_bytes, void *stream,
+                          const w4a8_opts *opts)
+{
+    if (!Xq || !packed || !workspace) return W4A8_ERR_NULL;
+    if (!Y && !acc) return W4A8_ERR_NULL;
+    if (Y && !tok_scale) return W4A8_ERR_NULL;
+    if (!shape_ok(N, K, group) || M < 1 || !opts_ok(opts)) return W4A8_ERR_SHAPE;
+    if (!aligned(Xq, 16) || !aligned(tok_scale, 4) || !aligned(bias, 4) || !aligned(Y, 16) ||
+        !aligned(acc, 16) || !aligned(packed, 256) || !aligned(workspace, 256))
+        return W4A8_ERR_ALIGN;
+    const size_t need = w4a8_linear_workspace_bytes_ex(M, N, K, group, opts);
+    if (need == 0) return W4A8_ERR_SHAPE;
+    if (workspace_bytes < need) return W4A8_ERR_BUFFER_TOO_SMALL;
+    const w4a8_status arch = check_arch();
+    if (arch != W4A8_OK) return arch;
+    const BlobLayout L = make_layout(N, K, group);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint8_t *blob = static_cast<const uint8_t *>(packed);
+    if (opts && opts->path == W4A8_PATH_SIMPLE) {
+        const cudaError_t e =
+            launch_linear_simple(Xq, tok_scale, blob, L, bias, M, static_cast<__nv_bfloat16 *>(Y),
+                                 acc, static_cast<StatusBlock *>(workspace), st);
+        if (e == cudaErrorInvalidValue) return W4A8_ERR_SHAPE;
+        return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+    }
+    LinearPlan plan;
+    if (!make_plan(M, L, opts, &plan)) return W4A8_ERR_SHAPE;
+    return launch_linear_tcgen05(Xq, tok_scale, blob, L, bias, M, static_cast<__nv_bfloat16 *>(Y),
+                                 acc, static_cast<uint8_t *>(workspace), plan, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t w4a8_packed_bytes(int N, int K, int group_size)
+{
+    if (!shape_ok(N, K, group_size)) return 0;
+    return make_layout(N, K, group_size).total_bytes;
+}
+
+w4a8_status w4a8_pack_weights(const void *W_f16, const float *s_in, int N, int K, int group_size,
+                              float clip, void *packed, size_t packed_bytes, void *stream)
+{
+    if (!W_f16 || !packed) return W4A8_ERR_NULL;
+    if (!shape_ok(N, K, group_size) || !(clip > 0.0f && clip <= 1.0f)) return W4A8_ERR_SHAPE;
+    if (!aligned(W_f16, 16) || !aligned(s_in, 16) || !aligned(packed, 256)) return W4A8_ERR_ALIGN;
+    const BlobLayout L = make_layout(N, K, group_size);
+    if (packed_bytes < L.total_bytes) return W4A8_ERR_BUFFER_TOO_SMALL;
+    const w4a8_status arch = check_arch();
+    if (arch != W4A8_OK) return arch;
+    const cudaError_t e = launch_pack(static_cast<const __half *>(W_f16), s_in, L, clip,
+                                      static_cast<uint8_t *>(packed),
+                                      static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+w4a8_status w4a8_quantize_act(const void *X_f16, const float *inv_s_in, int M, int K,
+                              int8_t *Xq, float *tok_scale, void *stream)
+{
+    if (!X_f16 || !Xq || !tok_scale) return W4A8_ERR_NULL;
+    if (M < 1 || K < 128 || K % 128 != 0 || K >= (1 << 19)) return W4A8_ERR_SHAPE;
+    if (!aligned(X_f16, 16) || !aligned(inv_s_in, 16) || !aligned(Xq, 16) ||
+        !aligned(tok_scale, 4))
+        return W4A8_ERR_ALIGN;
+    const w4a8_status arch = check_arch();
+    if (arch != W4A8_OK) return arch;
+    const cudaError_t e =
+        launch_quantize_act(static_cast<const __half *>(X_f16), inv_s_in, M, K, Xq, tok_scale,
+                            static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+size_t w4a8_linear_workspace_bytes_ex(int M, int N, int K, int group_size, const w4a8_opts *opts)
+{
+    if (!shape_ok(N, K, group_size) || M < 1 || !opts_ok(opts)) return 0;
+    if (opts && opts->path == W4A8_PATH_SIMPLE) return sizeof(StatusBlock);
+    LinearPlan plan;
+    if (!make_plan(M, make_layout(N, K, group_size), opts, &plan)) return 0;
+    return plan.workspace_bytes;
+}
+
+size_t w4a8_linear_workspace_bytes(int M, int N, int K, int group_size)
+{
+    return w4a8_linear_workspace_bytes_ex(M, N, K, group_size, nullptr);
+}
+
+w4a8_status w4a8_workspace_init(void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!workspace) return W4A8_ERR_NULL;
+    if (!aligned(workspace, 256)) return W4A8_ERR_ALIGN;
+    if (workspace_bytes < sizeof(StatusBlock)) return W4A8_ERR_BUFFER_TOO_SMALL;
+    const cudaError_t e =
+        cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+w4a8_status w4a8_linear(const int8_t *Xq, const float *tok_scale, const void *packed,
+                        const float *bias, int M, int N, int K, int group_size, void *Y_bf16,
+                        void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!Y_bf16) return W4A8_ERR_NULL;
+    return linear_common(Xq, tok_scale, packed, bias, M, N, K, group_size, Y_bf16, nullptr,
+                         workspace, workspace_bytes, stream, nullptr);
+}
+
+w4a8_status w4a8_linear_ex(const int8_t *Xq, const float *tok_scale, const void *packed,
+                           const float *bias, int M, int N, int K, int group_size, void *Y_bf16,
+                           void *workspace, size_t workspace_bytes, void *stream,
+                           const w4a8_opts *opts)
+{
+    if (!Y_bf16) return W4A8_ERR_NULL;
+    return linear_common(Xq, tok_scale, packed, bias, M, N, K, group_size, Y_bf16, nullptr,
+                         workspace, workspace_bytes, stream, opts);
+}
+
+w4a8_status w4a8_linear_acc_i32(const int8_t *Xq, const void *packed, int M, int N, int K,
+                                int group_size, int32_t *acc, void *workspace,
+                                size_t workspace_bytes, void *stream, const w4a8_opts *opts)
+{
+    if (!acc) return W4A8_ERR_NULL;
+    return linear_common(Xq, nullptr, packed, nullptr, M, N, K, group_size, nullptr, acc,
+                         workspace, workspace_bytes, stream, opts);
+}
+
+w4a8_status w4a8_unpack_codes(const void *packed, int N, int K, int group_size, uint8_t *codes,
+                              float *scales, uint8_t *zeros, void *stream)
+{
+    if (!packed || !codes || !scales || !zeros) return W4A8_ERR_NULL;
+    if (!shape_ok(N, K, group_size)) return W4A8_ERR_SHAPE;
+    if (!aligned(packed, 256) || !aligned(scales, 4)) return W4A8_ERR_ALIGN;
+    const w4a8_status arch = check_arch();
+    if (arch != W4A8_OK) return arch;
+    const cudaError_t e =
+        launch_unpack(static_cast<const uint8_t *>(packed), make_layout(N, K, group_size), codes,
+                      scales, zeros, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+w4a8_status w4a8_poll_status(void *workspace, void *stream)
+{
+    if (!workspace) return W4A8_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return W4A8_ERR_CUDA;
+    int host[3] = {0, 0, 0};
+    if (cudaMemcpy(host, workspace, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return W4A8_ERR_CUDA;
+    if (host[0] == 0) return W4A8_OK;
+    if (cudaMemset(workspace, 0, sizeof(StatusBlock)) != cudaSuccess) return W4A8_ERR_CUDA;
+    return host[0] == W4A8_ERR_BAD_BLOB ? W4A8_ERR_BAD_BLOB : W4A8_ERR_TIMEOUT;
+}
+
+void w4a8_dint4_table(int z, int8_t *out)
+{
+    for (int c = 0; c < 16; ++c) out[c] = (int8_t)dint4_t2(c, z);
+}
+
+const char *w4a8_version(void) { return "w4a8-dint 0.1 (sm_100a)"; }
+
+}  // extern "C"

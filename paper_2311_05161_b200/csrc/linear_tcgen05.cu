@@ -1,0 +1,792 @@
+// Tensor-core kernel of the W4A8-dINT linear layer (Eq. 1 contraction with the Eq. 6
+// dequantization folded into an integer lookup), sm_100a.
+//
+// Orientation: the 128 output features of a tile are the M side of the MMA (operand A,
+// decoded weights), the tokens are the N side (operand B, INT8 activations), so the
+// accumulator in tensor memory has one feature per lane and one token per column.  Per
+// 128-wide k-block:
+//   producer thread   TMA tile load of TOK x 128 INT8 activations (128-byte swizzle) and one
+//                     bulk copy of the 8 KiB packed-code tile into a shared-memory ring
+//   decode warps      one thread per feature row: 4-bit codes -> INT8 through a 16-entry
+//                     byte table held in four registers (byte permute), written in the
+//                     128-byte-swizzled K-major layout the MMA reads
+//   MMA thread        4 x tcgen05.mma kind::i8 (128 x TOK x 32) into tensor memory, INT32
+//   epilogue warps    tcgen05.ld, FP32 rescale (token step x weight step / 2), bias, BF16
+// Per-channel weights accumulate over the whole K slice in tensor memory; group-128
+// weights hand every k-block's INT32 partial to the epilogue warps, which scale it by the
+// group's step and add it to FP32 registers, while the next k-block accumulates into the
+// other tensor-memory buffer.  Split-K slices leave partial tiles in the workspace and the
+// last slice to finish a tile (an atomic counter, no spinning) reduces them in slice order.
+//
+// Every wait is bounded: a wait that runs out records a status, raises a flag that all
+// roles poll, and the CTA drains its copies, frees tensor memory and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace w4a8 {
+
+namespace {
+
+constexpr int kDecodeWarps = 4;
+constexpr int kFirstDecodeWarp = 2;
+constexpr int kFirstEpiWarp = kFirstDecodeWarp + kDecodeWarps;
+constexpr int kABytes = kTileN * kTileK;            // decoded INT8 tile, 16 KiB
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr unsigned long long kDrainLimitNs = 200000000ull;
+
+template <int TOK, bool GROUPED>
+struct Cfg {
+    static constexpr int kEpiGroups = (GROUPED && TOK >= 64) ? 2 : 1;   // warpgroups
+    static constexpr int kEpiWarps = 4 * kEpiGroups;
+    static constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
+    static constexpr int kColsPerThread = TOK / kEpiGroups;
+    static constexpr int kChunk = kColsPerThread >= 32 ? 32 : 16;
+    static constexpr int kTokBytes = TOK * kTileK;
+    static constexpr int kStageBytes = kABytes + kTokBytes + kTileBytes;
+    static constexpr int kStages = TOK == 256 ? 3 : TOK == 128 ? 5 : TOK == 64 ? 6 : 7;
+    static constexpr int kTmemCols = 2 * TOK < 32 ? 32 : 2 * TOK;
+    static constexpr int kBarrierBytes = 1024;
+    static constexpr int kSmemBytes = kStages * kStageBytes + kBarrierBytes + 1024;
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
+    static_assert(!GROUPED || TOK <= 128, "group mode keeps its FP32 sums in registers");
+};
+
+struct Params {
+    const uint8_t *blob;
+    const uint8_t *codes;
+    const float *scales;
+    const uint8_t *zeros;
+    const float *tok_scale;
+    const float *bias;
+    __nv_bfloat16 *Y;
+    int32_t *acc_out;
+    StatusBlock *sb;
+    int *counters;
+    void *partials;
+    BlobLayout L;
+    int M, tok_tiles, m_pad, split_k, kb_per_split, total_units;
+};
+
+// --------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes,
+                                          uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
+            "r"(dst),
+        "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before()
+{
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after()
+{
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::
+                     "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),
+          "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]),
+          "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld()
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+__device__ __forceinline__ void named_bar_sync(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+// Barrier over `threads` threads that also ANDs a predicate: every caller gets the same answer.
+__device__ __forceinline__ bool named_bar_and(int id, int threads, bool pred)
+{
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %3, 0;\n\t"
+        "bar.red.and.pred q, %1, %2, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(out)
+        : "r"(id), "r"(threads), "r"((uint32_t)pred)
+        : "memory");
+    return out != 0;
+}
+
+// Shared-memory matrix descriptor of a K-major operand tile with 128-byte rows and
+// 128-byte swizzle: 8-row groups are 1024 bytes apart; `addr` may be advanced by 32 bytes
+// per 32-deep MMA step inside the swizzle span.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+{
+    const uint32_t lo = ((addr & 0x3FFFFu) >> 4) | (1u << 16);
+    const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    return ((uint64_t)hi << 32) | lo;
+}
+
+// Instruction descriptor: signed 8-bit A and B, both K-major, INT32 accumulate, M = 128.
+__host__ __device__ constexpr uint32_t instr_desc_i8(int n)
+{
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// --------------------------------------------------------------------------- bounded wait
+struct Ctl {
+    volatile int abort;
+    int is_last;
+    uint32_t tmem_base;
+};
+
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Ctl *ctl,
+                                             StatusBlock *sb, int where,
+                                             unsigned long long limit = kWaitLimitNs)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t i = 1;; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 255u) == 0u) {
+            if (ctl->abort) return false;
+            if (global_ns() - t0 > limit) {
+                ctl->abort = 1;
+                report_failure(sb, W4A8_ERR_TIMEOUT, where);
+                return false;
+            }
+        }
+    }
+}
+
+// --------------------------------------------------------------------------- decode
+// Byte tables of Eq. 6 in units of step/2 for zero-point z: t[c / 4] byte c % 4 holds
+// 2 (c - z) for c <= 13, +1 for c = 14, -1 for c = 15.
+__device__ __forceinline__ void build_tables(int z, uint32_t (&t)[4])
+{
+    const uint32_t zz = (uint32_t)(2 * z) * 0x01010101u;
+    // per byte: (0x80 + 2c) - 2z never borrows; the XOR removes the 0x80 again
+    t[0] = ((0x86848280u) - zz) ^ 0x80808080u;
+    t[1] = ((0x8E8C8A88u) - zz) ^ 0x80808080u;
+    t[2] = ((0x96949290u) - zz) ^ 0x80808080u;
+    t[3] = ((((0x00009A98u) - (zz & 0xFFFFu)) ^ 0x00008080u) & 0xFFFFu) | 0xFF010000u;
+}
+
+// Eight codes (nibble i = code of k0 + i) -> eight INT8 values, bytes in k order.
+__device__ __forceinline__ void decode8(uint32_t w, const uint32_t (&t)[4], uint32_t &o0,
+                                        uint32_t &o1)
+{
+    const uint32_t idx = w & 0x77777777u;
+    const uint32_t e = w << 4;
+    const uint32_t idx_hi = idx >> 16;
+    const uint32_t a0 = prmt(t[0], t[1], idx), b0 = prmt(t[2], t[3], idx);
+    const uint32_t a1 = prmt(t[0], t[1], idx_hi), b1 = prmt(t[2], t[3], idx_hi);
+    const uint32_t m0 = prmt(e, w, 0xD9C8u), m1 = prmt(e, w, 0xFBEAu);   // bit 3 -> byte mask
+    o0 = (a0 & ~m0) | (b0 & m0);
+    o1 = (a1 & ~m1) | (b1 & m1);
+}
+
+// --------------------------------------------------------------------------- the kernel
+template <int TOK, bool GROUPED>
+__global__ void __launch_bounds__(Cfg<TOK, GROUPED>::kThreads, 1)
+linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map, const Params P)
+{
+    using C = Cfg<TOK, GROUPED>;
+    constexpr int S = C::kStages;
+    extern __shared__ uint8_t smem_raw[];
+
+    if (!header_matches(P.blob, P.L)) {
+        if (threadIdx.x == 0) report_failure(P.sb, W4A8_ERR_BAD_BLOB, 2);
+        return;
+    }
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bar_base = base + S * C::kStageBytes;
+    const uint32_t bar_full = bar_base;                  // S: TMA bytes landed
+    const uint32_t bar_dec = bar_base + 8 * S;           // S: decoded operand written
+    const uint32_t bar_empty = bar_base + 16 * S;        // S: MMAs of the stage retired
+    const uint32_t bar_acc_full = bar_base + 24 * S;     // 2
+    const uint32_t bar_acc_empty = bar_acc_full + 16;    // 2
+    const uint32_t bar_drain = bar_acc_empty + 16;       // 1
+    Ctl *ctl = reinterpret_cast<Ctl *>(gen_base + S * C::kStageBytes + 24 * S + 48);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_dec + 8 * s, kDecodeWarps);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_acc_full + 8 * b, 1);
+            mbar_init(bar_acc_empty + 8 * b, C::kEpiWarps);
+        }
+        mbar_init(bar_drain, 1);
+        ctl->abort = 0;
+        ctl->is_last = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         smem_u32(&ctl->tmem_base)),
+                     "r"((uint32_t)C::kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    const int n_tiles = P.L.n_tiles, k_blocks = P.L.k_blocks;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
+                const int s = u % P.split_k, rest = u / P.split_k;
+                const int nt = rest % n_tiles, tt = rest / n_tiles;
+                const int kb0 = s * P.kb_per_split;
+                const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                    const int st = it % S;
+                    const uint32_t fill = it / S;
+                    if (!wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 10)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t stage = base + st * C::kStageBytes;
+                    mbar_arrive_expect_tx(bar_full + 8 * st, C::kTokBytes + kTileBytes);
+                    tma_load_2d(stage + kABytes, &tok_map, kb * kTileK, tt * TOK,
+                                bar_full + 8 * st);
+                    bulk_load(stage + kABytes + C::kTokBytes,
+                              P.codes + ((size_t)nt * k_blocks + kb) * kTileBytes, kTileBytes,
+                              bar_full + 8 * st);
+                }
+            }
+            if (!ok) {
+                // copies already issued must land before the CTA gives its memory back
+                const uint32_t first = it > (uint32_t)S ? it - S : 0u;
+                for (uint32_t j = first; j < it; ++j)
+                    wait_bounded(bar_full + 8 * (j % S), (j / S) & 1u, ctl, P.sb, 11,
+                                 kDrainLimitNs);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_i8(TOK);
+            uint32_t it = 0, phase = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
+                const int s = u % P.split_k;
+                const int kb0 = s * P.kb_per_split;
+                const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                    const int st = it % S;
+                    const uint32_t fill = it / S;
+                    const bool first = GROUPED || kb == kb0;
+                    const bool last = GROUPED || kb == kb1 - 1;
+                    const uint32_t buf = phase & 1u;
+                    if (first &&
+                        !wait_bounded(bar_acc_empty + 8 * buf, ((phase >> 1) & 1u) ^ 1u, ctl, P.sb,
+                                      20)) {
+                        ok = false;
+                        break;
+                    }
+                    if (!wait_bounded(bar_dec + 8 * st, fill & 1u, ctl, P.sb, 21)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t stage = base + st * C::kStageBytes;
+                    const uint32_t d = tmem_base + buf * TOK;
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        tc_mma_i8(d, smem_desc_sw128(stage + ks * 32),
+                                  smem_desc_sw128(stage + kABytes + ks * 32), idesc,
+                                  (!first || ks > 0) ? 1u : 0u);
+                    }
+                    tc_commit(bar_empty + 8 * st);
+                    if (last) {
+                        tc_commit(bar_acc_full + 8 * buf);
+                        ++phase;
+                    }
+                }
+            }
+            // nothing issued may still be running when tensor memory is freed
+            tc_commit(bar_drain);
+            wait_bounded(bar_drain, 0u, ctl, P.sb, 22, ok ? kWaitLimitNs : kDrainLimitNs);
+        }
+        __syncwarp();
+    } else if (warp < kFirstEpiWarp) {
+        // ------------------------------------------------------------------ decode warps
+        const int r = threadIdx.x - 32 * kFirstDecodeWarp;       // feature row in the tile
+        uint32_t it = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
+            const int s = u % P.split_k, rest = u / P.split_k;
+            const int nt = rest % n_tiles;
+            const int kb0 = s * P.kb_per_split;
+            const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
+            const int n = nt * kTileN + r;
+            uint32_t t[4];
+            int z_next = GROUPED ? P.zeros[(size_t)kb0 * P.L.n_pad + n] : P.zeros[n];
+            if (!GROUPED) build_tables(z_next, t);
+            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                if (GROUPED) {
+                    build_tables(z_next, t);
+                    if (kb + 1 < kb1) z_next = P.zeros[(size_t)(kb + 1) * P.L.n_pad + n];
+                }
+                const int st = it % S;
+                const uint32_t fill = it / S;
+                ok = wait_bounded(bar_full + 8 * st, fill & 1u, ctl, P.sb, 30);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                uint8_t *stage = gen_base + st * C::kStageBytes;
+                const uint8_t *pk = stage + kABytes + C::kTokBytes + r * 16;
+                uint8_t *arow = stage + r * 128;
+                const int sw = r & 7;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint4 w = *reinterpret_cast<const uint4 *>(pk + q * kQuarterBytes);
+                    uint4 c0, c1;
+                    decode8(w.x, t, c0.x, c0.y);
+                    decode8(w.y, t, c0.z, c0.w);
+                    decode8(w.z, t, c1.x, c1.y);
+                    decode8(w.w, t, c1.z, c1.w);
+                    *reinterpret_cast<uint4 *>(arow + (((2 * q) ^ sw) << 4)) = c0;
+                    *reinterpret_cast<uint4 *>(arow + (((2 * q + 1) ^ sw) << 4)) = c1;
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_dec + 8 * st);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int ew = warp - kFirstEpiWarp;
+        const int quarter = warp & 3;                     // tensor-memory lane quarter
+        const int col_group = ew >> 2;                    // which share of the columns
+        const int col0 = col_group * C::kColsPerThread;
+        constexpr int kEpiThreads = 32 * C::kEpiWarps;
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
+            const int s = u % P.split_k, rest = u / P.split_k;
+            const int nt = rest % n_tiles, tt = rest / n_tiles;
+            const int kb0 = s * P.kb_per_split;
+            const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
+            const int n = nt * kTileN + quarter * 32 + lane;
+            const bool n_ok = n < P.L.N;
+            const int tok0 = tt * TOK + col0;
+            int valid = P.M - tok0;                       // columns of this thread that are tokens
+            valid = valid < 0 ? 0 : (valid > C::kColsPerThread ? C::kColsPerThread : valid);
+            const float bias_n = (P.bias && n_ok) ? P.bias[n] : 0.0f;
+
+            if (!GROUPED) {
+                const float half_step = __fmul_rn(0.5f, P.scales[n]);
+                const uint32_t buf = phase & 1u;
+                ok = wait_bounded(bar_acc_full + 8 * buf, (phase >> 1) & 1u, ctl, P.sb, 40);
+                ok = __all_sync(0xffffffffu, ok);
+                if (P.split_k > 1) ok = named_bar_and(1, kEpiThreads, ok);
+                if (!ok) break;
+                tc_fence_after();
+                ++phase;
+                int32_t *part = reinterpret_cast<int32_t *>(P.partials);
+#pragma unroll 1
+                for (int c = 0; c < C::kColsPerThread; c += C::kChunk) {
+                    uint32_t v[32];
+                    const uint32_t taddr = tmem_base + lane_base + buf * TOK + col0 + c;
+                    if (C::kChunk == 32) tc_ld32(taddr, v); else tc_ld16(taddr, v);
+                    tc_wait_ld();
+                    if (c + C::kChunk >= C::kColsPerThread) {
+                        // the accumulator is in registers: hand the buffer back
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+                    }
+                    if (P.split_k == 1) {
+#pragma unroll
+                        for (int j = 0; j < C::kChunk; ++j) {
+                            if (c + j < valid && n_ok) {
+                                const int m = tok0 + c + j;
+                                const int acc = (int)v[j];
+                                if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = acc;
+                                if (P.Y) {
+                                    float tv = rescale_channel(acc, __ldg(P.tok_scale + m), half_step);
+                                    if (P.bias) tv = __fadd_rn(tv, bias_n);
+                                    P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(tv);
+                                }
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < C::kChunk; ++j) {
+                            if (c + j < valid) {
+                                const int m = tok0 + c + j;
+                                part[((size_t)s * P.m_pad + m) * P.L.n_pad + n] = (int)v[j];
+                            }
+                        }
+                    }
+                }
+                if (P.split_k > 1) {
+                    __threadfence();
+                    named_bar_sync(1, kEpiThreads);
+                    if (threadIdx.x == 32 * kFirstEpiWarp) {
+                        const int old = atomicAdd(P.counters + (size_t)tt * n_tiles + nt, 1);
+                        const int last = old == P.split_k - 1;
+                        if (last) P.counters[(size_t)tt * n_tiles + nt] = 0;
+                        ctl->is_last = last;
+                    }
+                    named_bar_sync(1, kEpiThreads);
+                    const bool is_last = ctl->is_last != 0;
+                    named_bar_sync(1, kEpiThreads);
+                    if (is_last && n_ok) {
+                        __threadfence();
+                        for (int j = 0; j < valid; ++j) {
+                            const int m = tok0 + j;
+                            int acc = 0;
+                            for (int ss = 0; ss < P.split_k; ++ss)
+                                acc += __ldcg(part + ((size_t)ss * P.m_pad + m) * P.L.n_pad + n);
+                            if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = acc;
+                            if (P.Y) {
+                                float tv = rescale_channel(acc, __ldg(P.tok_scale + m), half_step);
+                                if (P.bias) tv = __fadd_rn(tv, bias_n);
+                                P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(tv);
+                            }
+                        }
+                    }
+                }
+            } else {
+                float usum[C::kColsPerThread];
+#pragma unroll
+                for (int j = 0; j < C::kColsPerThread; ++j) usum[j] = 0.0f;
+                float h_next = __fmul_rn(0.5f, P.scales[(size_t)kb0 * P.L.n_pad + n]);
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    const float h = h_next;
+                    if (kb + 1 < kb1)
+                        h_next = __fmul_rn(0.5f, P.scales[(size_t)(kb + 1) * P.L.n_pad + n]);
+                    const uint32_t buf = phase & 1u;
+                    ok = wait_bounded(bar_acc_full + 8 * buf, (phase >> 1) & 1u, ctl, P.sb, 41);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                    ++phase;
+#pragma unroll
+                    for (int c = 0; c < C::kColsPerThread; c += C::kChunk) {
+                        uint32_t v[32];
+                        const uint32_t taddr = tmem_base + lane_base + buf * TOK + col0 + c;
+                        if (C::kChunk == 32) tc_ld32(taddr, v); else tc_ld16(taddr, v);
+                        tc_wait_ld();
+                        if (c + C::kChunk >= C::kColsPerThread) {
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+                        }
+#pragma unroll
+                        for (int j = 0; j < C::kChunk; ++j)
+                            usum[c + j] = fmaf((float)(int)v[j], h, usum[c + j]);
+                        if (P.acc_out && n_ok) {
+#pragma unroll
+                            for (int j = 0; j < C::kChunk; ++j)
+                                if (c + j < valid)
+                                    P.acc_out[((size_t)kb * P.M + tok0 + c + j) * P.L.N + n] =
+                                        (int)v[j];
+                        }
+                    }
+                }
+                if (P.split_k > 1) ok = named_bar_and(1, kEpiThreads, ok);
+                if (!ok) break;
+                if (P.split_k == 1) {
+                    if (P.Y && n_ok) {
+#pragma unroll
+                        for (int j = 0; j < C::kColsPerThread; ++j) {
+                            if (j < valid) {
+                                const int m = tok0 + j;
+                                float tv = __fmul_rn(usum[j], __ldg(P.tok_scale + m));
+                                if (P.bias) tv = __fadd_rn(tv, bias_n);
+                                P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(tv);
+                            }
+                        }
+                    }
+                } else {
+                    float *part = reinterpret_cast<float *>(P.partials);
+#pragma unroll
+                    for (int j = 0; j < C::kColsPerThread; ++j)
+                        if (j < valid)
+                            part[((size_t)s * P.m_pad + tok0 + j) * P.L.n_pad + n] = usum[j];
+                    __threadfence();
+                    named_bar_sync(1, kEpiThreads);
+                    if (threadIdx.x == 32 * kFirstEpiWarp) {
+                        const int old = atomicAdd(P.counters + (size_t)tt * n_tiles + nt, 1);
+                        const int last = old == P.split_k - 1;
+                        if (last) P.counters[(size_t)tt * n_tiles + nt] = 0;
+                        ctl->is_last = last;
+                    }
+                    named_bar_sync(1, kEpiThreads);
+                    const bool is_last = ctl->is_last != 0;
+                    named_bar_sync(1, kEpiThreads);
+                    if (is_last && n_ok && P.Y) {
+                        __threadfence();
+                        for (int j = 0; j < valid; ++j) {
+                            const int m = tok0 + j;
+                            float usm = 0.0f;
+                            for (int ss = 0; ss < P.split_k; ++ss)
+                                usm = __fadd_rn(
+                                    usm, __ldcg(part + ((size_t)ss * P.m_pad + m) * P.L.n_pad + n));
+                            float tv = __fmul_rn(usm, __ldg(P.tok_scale + m));
+                            if (P.bias) tv = __fadd_rn(tv, bias_n);
+                            P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(tv);
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                     "r"((uint32_t)C::kTmemCols)
+                     : "memory");
+    }
+}
+
+// --------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) ==
+                cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n = v;
+        else
+            return 148;
+    }
+    return n;
+}
+
+template <int TOK, bool GROUPED>
+w4a8_status launch_one(const CUtensorMap &map, const Params &P, cudaStream_t st)
+{
+    using C = Cfg<TOK, GROUPED>;
+    auto kern = linear_tcgen05_kernel<TOK, GROUPED>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) !=
+        cudaSuccess)
+        return W4A8_ERR_CUDA;
+    int grid = P.total_units < sm_count() ? P.total_units : sm_count();
+    kern<<<grid, C::kThreads, C::kSmemBytes, st>>>(map, P);
+    return cudaGetLastError() == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+}  // namespace
+
+bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *plan)
+{
+    const bool grouped = L.group != 0;
+    const int cap = grouped ? 128 : 256;
+    int tok = opts ? opts->tok_tile : 0;
+    if (tok == 0) {
+        tok = 16;
+        while (tok < M && tok < cap) tok *= 2;
+    }
+    if (tok != 16 && tok != 32 && tok != 64 && tok != 128 && tok != 256) return false;
+    if (tok > cap) return false;
+    const int tok_tiles = (M + tok - 1) / tok;
+    const long long tiles = (long long)tok_tiles * L.n_tiles;
+    int split = opts ? opts->split_k : 0;
+    if (split == 0) {
+        split = 1;
+        const int sms = sm_count();
+        if (M <= 256 && tiles < sms) {
+            split = (int)((2LL * sms) / tiles);
+            const int max_split = L.k_blocks / 4 > 0 ? L.k_blocks / 4 : 1;   // >= 4 k-blocks each
+            if (split > max_split) split = max_split;
+            if (split < 1) split = 1;
+        }
+    }
+    if (split < 1 || split > L.k_blocks) return false;
+    const int kb_per = (L.k_blocks + split - 1) / split;
+    split = (L.k_blocks + kb_per - 1) / kb_per;              // no empty slice
+    if (tiles * split > 0x7fffffffLL) return false;
+    plan->tok_tile = tok;
+    plan->tok_tiles = tok_tiles;
+    plan->split_k = split;
+    plan->kb_per_split = kb_per;
+    plan->off_counters = sizeof(StatusBlock);
+    plan->off_partials = align_up(plan->off_counters + (size_t)tiles * sizeof(int), 256);
+    const size_t m_pad = (size_t)tok_tiles * tok;
+    plan->workspace_bytes =
+        plan->off_partials + (split > 1 ? (size_t)split * m_pad * L.n_pad * 4 : 0);
+    return true;
+}
+
+w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
+                                  const BlobLayout &L, const float *bias, int M,
+                                  __nv_bfloat16 *Y, int32_t *acc, uint8_t *workspace,
+                                  const LinearPlan &plan, cudaStream_t st)
+{
+    EncodeTiledFn enc = encode_tiled();
+    if (!enc) return W4A8_ERR_CUDA;
+    CUtensorMap map;
+    const cuuint64_t dims[2] = {(cuuint64_t)L.K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)L.K};
+    const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)plan.tok_tile};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(Xq), dims, strides, box,
+            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return W4A8_ERR_CUDA;
+
+    Params P;
+    P.blob = blob;
+    P.codes = blob + L.off_codes;
+    P.scales = reinterpret_cast<const float *>(blob + L.off_scales);
+    P.zeros = blob + L.off_zeros;
+    P.tok_scale = tok_scale;
+    P.bias = bias;
+    P.Y = Y;
+    P.acc_out = acc;
+    P.sb = reinterpret_cast<StatusBlock *>(workspace);
+    P.counters = reinterpret_cast<int *>(workspace + plan.off_counters);
+    P.partials = workspace + plan.off_partials;
+    P.L = L;
+    P.M = M;
+    P.tok_tiles = plan.tok_tiles;
+    P.m_pad = plan.tok_tiles * plan.tok_tile;
+    P.split_k = plan.split_k;
+    P.kb_per_split = plan.kb_per_split;
+    P.total_units = plan.tok_tiles * L.n_tiles * plan.split_k;
+
+    const bool g = L.group != 0;
+    switch (plan.tok_tile) {
+    case 16: return g ? launch_one<16, true>(map, P, st) : launch_one<16, false>(map, P, st);
+    case 32: return g ? launch_one<32, true>(map, P, st) : launch_one<32, false>(map, P, st);
+    case 64: return g ? launch_one<64, true>(map, P, st) : launch_one<64, false>(map, P, st);
+    case 128: return g ? launch_one<128, true>(map, P, st) : launch_one<128, false>(map, P, st);
+    case 256: return g ? W4A8_ERR_SHAPE : launch_one<256, false>(map, P, st);
+    }
+    return W4A8_ERR_SHAPE;
+}
+
+}  // namespace w4a8

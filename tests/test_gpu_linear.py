@@ -1,0 +1,120 @@
+"""GPU parity of the quantized linear layer against the CPU oracle, through the C ABI:
+INT32 accumulators bit-exact; BF16 outputs bit-exact for per-channel weights and within
+1 BF16 ulp (+ the FP32 reordering allowance) for group-128 weights and split-K."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2311_05161_b200 as w4a8
+from util import Problem, bf16_bits, check_y
+
+pytestmark = pytest.mark.gpu
+
+
+def run_linear(prob, opts=None, packed=None, want_acc=True):
+    d = prob.dev
+    if packed is None:
+        packed = w4a8.pack_weights(d["W"], d["s"], prob.group)
+    Xq, tok = w4a8.quantize_act(d["X"], d["inv_s"])
+    ws = w4a8.new_workspace(prob.M, prob.N, prob.K, prob.group, opts)
+    Y = w4a8.linear(Xq, tok, packed, d["bias"], prob.N, prob.group, ws, opts)
+    acc = w4a8.linear_acc_i32(Xq, packed, prob.N, prob.group, ws, opts) if want_acc else None
+    w4a8.check_status(ws)
+    return bf16_bits(Y), (acc.cpu().numpy() if want_acc else None)
+
+
+@pytest.mark.parametrize("group", [0, 128])
+def test_simple_path_config1(group):
+    prob = Problem(768, 768, 16, group, seed=0)
+    Y, acc = run_linear(prob, w4a8.make_opts(w4a8.PATH_SIMPLE))
+    assert np.array_equal(acc, prob.oracle_acc())
+    check_y(prob, Y, exact=True)      # same FP32 order as the oracle in both modes
+
+
+@pytest.mark.parametrize("group", [0, 128])
+def test_tcgen05_config1(group):
+    prob = Problem(768, 768, 16, group, seed=0)
+    Y, acc = run_linear(prob, w4a8.make_opts(w4a8.PATH_TCGEN05))
+    assert np.array_equal(acc, prob.oracle_acc())
+    check_y(prob, Y, exact=(group == 0))
+
+
+@pytest.mark.parametrize("group", [0, 128])
+@pytest.mark.parametrize("tok_tile", [16, 32, 64, 128, 256])
+def test_tcgen05_token_tiles_and_ragged_edges(tok_tile, group):
+    if group and tok_tile == 256:
+        pytest.skip("group mode tiles at most 128 tokens")
+    # M spans several token tiles with a ragged tail; N = 200 is not a multiple of 128
+    M = tok_tile * 2 + 5
+    prob = Problem(1024, 200, M, group, seed=tok_tile + group, dist="laplace", outliers=0.01,
+                   mult=20.0)
+    Y, acc = run_linear(prob, w4a8.make_opts(w4a8.PATH_TCGEN05, tok_tile=tok_tile))
+    assert np.array_equal(acc, prob.oracle_acc())
+    check_y(prob, Y, exact=(group == 0))
+
+
+@pytest.mark.parametrize("group", [0, 128])
+@pytest.mark.parametrize("M,split", [(1, 2), (5, 3), (16, 8), (40, 5)])
+def test_tcgen05_split_k(M, split, group):
+    prob = Problem(1024, 384, M, group, seed=M + split + group)
+    opts = w4a8.make_opts(w4a8.PATH_TCGEN05, split_k=split)
+    packed = w4a8.pack_weights(prob.dev["W"], prob.dev["s"], group)
+    for _ in range(2):                       # second call reuses the self-cleaned workspace
+        Y, acc = run_linear(prob, opts, packed)
+        assert np.array_equal(acc, prob.oracle_acc())
+        check_y(prob, Y, exact=(group == 0))
+
+
+@pytest.mark.parametrize("group", [0, 128])
+def test_auto_path_matches_simple_path_and_oracle(group):
+    prob = Problem(2048, 1536, 300, group, seed=77, dist="laplace", outliers=0.01, mult=20.0)
+    Y, acc = run_linear(prob)
+    Ys, accs = run_linear(prob, w4a8.make_opts(w4a8.PATH_SIMPLE))
+    assert np.array_equal(acc, accs)
+    assert np.array_equal(acc, prob.oracle_acc())
+    check_y(prob, Y, exact=(group == 0))
+    check_y(prob, Ys, exact=True)
+
+
+def test_no_bias_no_scale_and_persistent_many_tiles():
+    # more tiles than SMs, so every CTA walks several tiles and both accumulator buffers
+    prob = Problem(512, 128 * 40, 130, 0, seed=9, scaled=False, with_bias=False)
+    Y, acc = run_linear(prob, w4a8.make_opts(w4a8.PATH_TCGEN05, tok_tile=16))
+    assert np.array_equal(acc, prob.oracle_acc())
+    check_y(prob, Y, exact=True)
+
+
+def test_worst_case_magnitudes_do_not_overflow():
+    K, N, M = 36864, 128, 4
+    W = np.zeros((N, K), dtype=np.float16)
+    W[:, :] = 1.0
+    W[:, 0] = 0.0                      # lo = 0, hi = 1 -> z = 0, every other code 13 (t2 = 26)
+    W[1::2] *= -1                      # negative rows: z = 13, codes 0 (t2 = -26)
+    X = np.full((M, K), 3.0, dtype=np.float16)
+    X[1] = -3.0
+    prob = Problem.__new__(Problem)
+    prob.K, prob.N, prob.M, prob.group, prob.rows = K, N, M, 0, None
+    prob.host = {"W": W, "X": X, "s": None, "inv_s": None, "bias": None}
+    prob.dev = {k: (torch.from_numpy(v).cuda() if v is not None else None) for k, v in prob.host.items()}
+    prob.codes, prob.scales, prob.zeros = oracle.pack_weights(W, None, 0)
+    prob.Xq, prob.tok = oracle.quantize_act(X, None)
+    prob.bias_sel = None
+    Y, acc = run_linear(prob)
+    want = prob.oracle_acc()
+    assert np.abs(want).max() == 127 * 26 * (K - 1)
+    assert np.array_equal(acc, want)
+    check_y(prob, Y, exact=True)
+
+
+def test_wrong_blob_is_reported_not_computed():
+    prob = Problem(768, 768, 16, 0, seed=0)
+    packed = w4a8.pack_weights(prob.dev["W"], prob.dev["s"], 128)      # packed for group mode
+    Xq, tok = w4a8.quantize_act(prob.dev["X"], prob.dev["inv_s"])
+    for path in (w4a8.PATH_SIMPLE, w4a8.PATH_TCGEN05):
+        ws = w4a8.new_workspace(16, 768, 768, 0)
+        buf = torch.zeros(max(packed.numel(), w4a8.packed_bytes(768, 768, 0)), dtype=torch.uint8, device="cuda")
+        buf[:packed.numel()] = packed
+        w4a8.linear(Xq, tok, buf, None, 768, 0, ws, w4a8.make_opts(path))
+        assert w4a8.poll_status(ws) == 8          # W4A8_ERR_BAD_BLOB
+        assert w4a8.poll_status(ws) == 0          # cleared by the poll
