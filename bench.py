@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Throughput of the W4A8-dINT quantized linear path on B200.
+
+One step = one pass of the hot path over the four linears of an OPT-6.7B-shaped decoder
+block at M = 2048 tokens: for each linear, the token-wise INT8 activation quantizer followed
+by the tensor-core linear (weights are packed once, before timing, as the method does
+offline).  Inputs are seeded synthetic tensors (see paper_2311_05161_b200/synth.py).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is TOPS (2*M*N*K per linear) with inputs resident in HBM;
+`e2e` is the same metric with host buffers and the copies inside the timed region;
+`roofline` describes the tensor-core kernel; `decode` gives the M = 1 weight-streaming
+GB/s of the same block; `cpu_baseline` is the CPU checker timed on a bounded sample.
+With --impl reference the CPU checker itself is the timed program.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+CONFIG = 2            # OPT-6.7B-shaped block
+M_PREFILL = 2048
+M_DECODE = 1
+CPU_SAMPLE_TOKENS = 48
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_burst": p["bf16_tflops"],
+                "bf16_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "20"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.perf_counter(), line.strip()))
+
+    def wait_first(self, timeout=5.0):
+        t0 = time.perf_counter()
+        while self.proc is not None and not self.lines and time.perf_counter() - t0 < timeout:
+            time.sleep(0.01)
+
+    def mark(self):
+        """Samples taken before this moment are dropped."""
+        self.t_mark = time.perf_counter()
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, line in self.lines:
+            if ts < getattr(self, "t_mark", 0.0):
+                continue
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def cpu_sample_time(layers_host, tokens):
+    """CPU checker on the first `tokens` tokens of every linear: seconds and op count."""
+    import oracle
+    ops = 0
+    t0 = time.perf_counter()
+    for lay in layers_host:
+        X = lay["X"][:tokens]
+        codes, scales, zeros = lay["oracle_pack"]
+        Xq, tok = oracle.quantize_act(X, lay["inv_s"])
+        oracle.linear(Xq, tok, codes, scales, zeros, lay["bias"], lay["group"])
+        ops += 2 * X.shape[0] * lay["W"].shape[0] * lay["W"].shape[1]
+    return time.perf_counter() - t0, ops
+
+
+def host_layers(M, with_oracle_pack=False):
+    from paper_2311_05161_b200 import synth
+    wl = synth.WORKLOADS[CONFIG]
+    out = []
+    for i, (K, N, label) in enumerate(wl.shapes):
+        lay = synth.workload_layer(CONFIG, i, M)
+        lay.update(K=K, N=N, label=label, group=wl.group)
+        if with_oracle_pack:
+            import oracle
+            lay["oracle_pack"] = oracle.pack_weights(lay["W"], lay["s"], wl.group)
+        out.append(lay)
+    return out
+
+
+def run_reference(args):
+    """The CPU checker as the timed program (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    layers = host_layers(CPU_SAMPLE_TOKENS, with_oracle_pack=True)
+    for _ in range(min(args.warmup, 1)):
+        cpu_sample_time(layers, CPU_SAMPLE_TOKENS)
+    total_t, total_ops = 0.0, 0
+    for _ in range(args.steps):
+        t, ops = cpu_sample_time(layers, CPU_SAMPLE_TOKENS)
+        total_t += t
+        total_ops += ops
+    tops = total_ops / total_t / 1e12
+    sample = f"first {CPU_SAMPLE_TOKENS} of {M_PREFILL} tokens of each of the 4 linears per step"
+    line = {
+        "impl": "reference", "metric": "w4a8_dint_linear_tops", "value": tops, "unit": "TOPS",
+        "n_gpus": 0, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * total_t / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": "opt-6.7b block linears, M=2048 prefill (CPU sample)",
+                   "sample": sample},
+        "cpu_baseline": {"value": tops, "unit": "TOPS", "cores": oracle.get_threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": tops, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2311_05161_b200 as w4a8
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+    peaks = read_peaks()
+    warmup = max(args.warmup, 3)
+
+    # ------------------------------------------------------------------ set-up (untimed)
+    layers = host_layers(M_PREFILL, with_oracle_pack=(rank == 0 and not args.no_cpu_baseline))
+    group = layers[0]["group"]
+    L = []
+    for lay in layers:
+        K, N = lay["K"], lay["N"]
+        d = {k: torch.from_numpy(lay[k]).to(dev) for k in ("W", "X", "s", "inv_s", "bias")}
+        d["packed"] = w4a8.pack_weights(d["W"], d["s"], group)
+        del d["W"]
+        d["Xq"] = torch.empty((M_PREFILL, K), dtype=torch.int8, device=dev)
+        d["tok"] = torch.empty((M_PREFILL,), dtype=torch.float32, device=dev)
+        d["Y"] = torch.empty((M_PREFILL, N), dtype=torch.bfloat16, device=dev)
+        d["ws"] = w4a8.new_workspace(M_PREFILL, N, K, group)
+        d["K"], d["N"] = K, N
+        d["X_host"] = torch.from_numpy(lay["X"]).pin_memory()
+        d["Y_host"] = torch.empty((M_PREFILL, N), dtype=torch.bfloat16).pin_memory()
+        # decode (M = 1): three rotating blob copies so that every launch streams from HBM
+        d["packed_rot"] = [d["packed"]] + [d["packed"].clone() for _ in range(2)]
+        d["X1"] = d["X"][:M_DECODE].contiguous()
+        d["Xq1"] = torch.empty((M_DECODE, K), dtype=torch.int8, device=dev)
+        d["tok1"] = torch.empty((M_DECODE,), dtype=torch.float32, device=dev)
+        d["Y1"] = torch.empty((M_DECODE, N), dtype=torch.bfloat16, device=dev)
+        d["ws1"] = w4a8.new_workspace(M_DECODE, N, K, group)
+        L.append(d)
+    ops_per_step = sum(2 * M_PREFILL * d["K"] * d["N"] for d in L)
+
+    def step(record=None):
+        for i, d in enumerate(L):
+            w4a8.quantize_act(d["X"], d["inv_s"], out=(d["Xq"], d["tok"]))
+            if record is not None:
+                record[i][0].record()
+            w4a8.linear(d["Xq"], d["tok"], d["packed"], d["bias"], d["N"], group, d["ws"],
+                        out=d["Y"])
+            if record is not None:
+                record[i][1].record()
+
+    def step_e2e():
+        for d in L:
+            d["X"].copy_(d["X_host"], non_blocking=True)
+            w4a8.quantize_act(d["X"], d["inv_s"], out=(d["Xq"], d["tok"]))
+            w4a8.linear(d["Xq"], d["tok"], d["packed"], d["bias"], d["N"], group, d["ws"],
+                        out=d["Y"])
+            d["Y_host"].copy_(d["Y"], non_blocking=True)
+
+    def step_decode(it):
+        for d in L:
+            w4a8.quantize_act(d["X1"], d["inv_s"], out=(d["Xq1"], d["tok1"]))
+            w4a8.linear(d["Xq1"], d["tok1"], d["packed_rot"][it % 3], d["bias"], d["N"], group,
+                        d["ws1"], out=d["Y1"])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for it in range(steps):
+            fn(it)
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    # ------------------------------------------------------------------ prefill, resident
+    for _ in range(warmup):
+        step()
+    for d in L:
+        w4a8.check_status(d["ws"])
+    records = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                for _ in L] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    sampler.wait_first()
+    for _ in range(warmup):
+        step()
+    sampler.mark()
+    ms = timed(lambda it: step(records[it]), args.steps)
+    clocks = sampler.stop()
+    lin_ms = [statistics.mean(records[it][i][0].elapsed_time(records[it][i][1])
+                              for it in range(args.steps)) for i in range(len(L))]
+    ms_per_step = ms / args.steps
+    tops = world * ops_per_step / (ms_per_step * 1e-3) / 1e12
+    lin_tops = ops_per_step / (sum(lin_ms) * 1e-3) / 1e12
+    peak_tops = 2.0 * peaks["bf16_sustained"]        # INT8 dense = 2 x BF16 dense (nominal ratio)
+
+    # ------------------------------------------------------------------ prefill, host buffers
+    for _ in range(3):
+        step_e2e()
+    e2e_steps = max(3, min(args.steps, 10))
+    ms_e2e = timed(lambda it: step_e2e(), e2e_steps) / e2e_steps
+    h2d = sum(d["X_host"].numel() * 2 for d in L)
+    d2h = sum(d["Y_host"].numel() * 2 for d in L)
+
+    # ------------------------------------------------------------------ decode (M = 1)
+    for it in range(6):
+        step_decode(it)
+    dec_steps = 60
+    ms_dec = timed(step_decode, dec_steps) / dec_steps
+    dec_bytes = sum(d["K"] * d["N"] // 2 + 5 * d["N"] + M_DECODE * (d["K"] + 4) + 2 * M_DECODE * d["N"]
+                    + 4 * d["N"] for d in L)
+    dec_gbs = dec_bytes / (ms_dec * 1e-3) / 1e9
+    for d in L:
+        w4a8.check_status(d["ws"])
+        w4a8.check_status(d["ws1"])
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        import oracle
+        t, ops = cpu_sample_time(layers, CPU_SAMPLE_TOKENS)
+        cpu = {"value": ops / t / 1e12, "unit": "TOPS", "cores": oracle.get_threads(),
+               "kind": "oracle", "seconds": t,
+               "sample": f"first {CPU_SAMPLE_TOKENS} of {M_PREFILL} tokens of each of the 4 linears"}
+
+    line = {
+        "metric": "w4a8_dint_linear_tops", "value": tops, "unit": "TOPS", "n_gpus": world,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
+        "data": "synthetic",
+        "config": {"workload": "opt-6.7b block linears (qkv 4096->12288, out 4096->4096, "
+                               "fc1 4096->16384, fc2 16384->4096), M=2048 prefill, per-channel dINT4",
+                   "step": "4 x (quantize_act + linear); weights packed once before timing",
+                   "l2": "inputs larger than L2 (about 400 MB touched per step)",
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "clocks": clocks,
+        "e2e": {"value": world * ops_per_step / (ms_e2e * 1e-3) / 1e12, "unit": "TOPS",
+                "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": 2 * len(L) * args.steps,
+        "roofline": {"bound": "tensor", "kernel": "linear_tcgen05_kernel<256,false>",
+                     "achieved": lin_tops, "peak": peak_tops, "unit": "TOPS",
+                     "frac": lin_tops / peak_tops,
+                     "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS TFLOP/s",
+                     "frac_of_nominal_4500": lin_tops / 4500.0,
+                     "per_linear_ms": dict(zip([lay["label"] for lay in layers], lin_ms)),
+                     "traffic": None},
+        "decode": {"metric": "w4a8_dint_linear_hbm_gbs", "value": dec_gbs, "unit": "GB/s", "M": M_DECODE,
+                   "ms_per_step": ms_dec, "bytes_per_step": dec_bytes,
+                   "frac_of_measured_copy": dec_gbs / peaks["hbm_gbs"],
+                   "frac_of_nominal_8000": dec_gbs / 8000.0,
+                   "note": "quantize_act + linear per shape, 3 rotating blob copies (> L2)"},
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
