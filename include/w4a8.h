@@ -128,6 +128,28 @@ w4a8_status w4a8_linear_ex(const int8_t *Xq, const float *tok_scale, const void 
                            void *Y_bf16, void *workspace, size_t workspace_bytes,
                            void *stream, const w4a8_opts *opts);
 
+/* w4a8_linear for callers that must not allocate device memory and therefore have no
+ * workspace to pass: code running after a host framework has claimed the whole device for
+ * its own pool (a cudaMalloc there fails or stalls the device), plug-ins whose host forbids
+ * allocation once serving has started, and real-time loops that may not risk the implicit
+ * synchronisation of an allocation.  The paper has no counterpart of this call; it is
+ * w4a8_linear with the same kernel, the same automatic plan and the same results, and it
+ * calls no allocating routine.
+ *   The scratch is an 8 MiB array inside the library image (each GPU that loads the
+ *   library holds it until the process ends).  Shapes whose plan needs more than that
+ *   (large split-K cases; w4a8_linear_workspace_bytes tells) return
+ *   W4A8_ERR_BUFFER_TOO_SMALL and launch nothing.
+ *   The first call on each device looks up the array's device address; make that first
+ *   call outside any stream capture.
+ *   All calls on one device share the array: the call clears the part that must start at
+ *   zero, on `stream`, before its kernel.  Two calls that can overlap on the GPU (different
+ *   streams without an ordering between them) race on it and give undefined results.
+ *   Failures inside the kernel are not reported through this call: there is no workspace
+ *   to poll. */
+w4a8_status w4a8_linear_static(const int8_t *Xq, const float *tok_scale, const void *packed,
+                               const float *bias, int M, int N, int K, int group_size,
+                               void *Y_bf16, void *stream);
+
 /* Test export: the INT32 accumulators of the contraction, acc [G][M][N], before any
  * rescale (Eq. 6 in units of step/2).  Uses the same kernels as w4a8_linear_ex. */
 w4a8_status w4a8_linear_acc_i32(const int8_t *Xq, const void *packed, int M, int N, int K,

@@ -25,7 +25,7 @@ PATH_AUTO, PATH_SIMPLE, PATH_TCGEN05 = 0, 1, 2
 EXPORTS = (
     "w4a8_packed_bytes", "w4a8_pack_weights", "w4a8_quantize_act",
     "w4a8_linear_workspace_bytes", "w4a8_linear_workspace_bytes_ex", "w4a8_workspace_init",
-    "w4a8_linear", "w4a8_linear_ex", "w4a8_linear_acc_i32", "w4a8_unpack_codes",
+    "w4a8_linear", "w4a8_linear_ex", "w4a8_linear_static", "w4a8_linear_acc_i32", "w4a8_unpack_codes",
     "w4a8_poll_status", "w4a8_dint4_table", "w4a8_version",
 )
 
@@ -65,6 +65,8 @@ def _load() -> ctypes.CDLL:
     lib.w4a8_linear.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, vp]
     lib.w4a8_linear_ex.restype = ci
     lib.w4a8_linear_ex.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, vp, op]
+    lib.w4a8_linear_static.restype = ci
+    lib.w4a8_linear_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp]
     lib.w4a8_linear_acc_i32.restype = ci
     lib.w4a8_linear_acc_i32.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, sz, vp, op]
     lib.w4a8_unpack_codes.restype = ci
@@ -187,6 +189,20 @@ def linear(Xq, tok_scale, packed, bias, N: int, group: int, workspace, opts: Opt
                                 group, _ptr(out), _ptr(workspace), workspace.numel(), _stream(),
                                 ctypes.byref(opts))
     _check(st, "w4a8_linear")
+    return out
+
+
+def linear_static(Xq, tok_scale, packed, bias, N: int, group: int, out):
+    """w4a8_linear without a workspace: the library's built-in scratch array is used, and
+    nothing is allocated here either, so the caller passes the output tensor `out`
+    ([M, N] bfloat16).  For callers that may not allocate device memory."""
+    Xq = _dev(Xq, torch.int8, "Xq")
+    tok_scale = _dev(tok_scale, torch.float32, "tok_scale")
+    bias = _dev(bias, torch.float32, "bias")
+    out = _dev(out, torch.bfloat16, "out")
+    M, K = Xq.shape
+    _check(lib.w4a8_linear_static(_ptr(Xq), _ptr(tok_scale), _ptr(packed), _ptr(bias), M, N, K,
+                                  group, _ptr(out), _stream()), "w4a8_linear_static")
     return out
 
 
