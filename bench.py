@@ -169,6 +169,76 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_case(args):
+    """One linear shape: quantize_act + linear, each timed with its own CUDA events.
+    Rotates over enough copies of the weights and activations to exceed L2."""
+    import torch
+
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2311_05161_b200 as w4a8
+    from paper_2311_05161_b200 import synth
+
+    vals = [int(v) for v in args.case.split(",")]
+    K, N, M, group = vals[:4]
+    tok_tile = vals[4] if len(vals) > 4 else 0
+    split_k = vals[5] if len(vals) > 5 else 0
+    dw = vals[6] if len(vals) > 6 else 0
+    opts = w4a8.make_opts(w4a8.PATH_TCGEN05, split_k, tok_tile, dw) if (tok_tile or split_k or dw) else None
+    torch.cuda.set_device(0)
+    peaks = read_peaks()
+    lay = synth.make_layer(K, N, M, seed=7, dist="normal", outliers=0.001, mult=60.0)
+    d = {k: torch.from_numpy(lay[k]).cuda() for k in ("W", "X", "s", "inv_s", "bias")}
+    packed = w4a8.pack_weights(d["W"], d["s"], group)
+    del d["W"]
+    per_copy = packed.numel() + M * K * 3 + M * N * 2
+    copies = max(1, min(8, -(-(256 << 20) // per_copy)))
+    packs = [packed] + [packed.clone() for _ in range(copies - 1)]
+    Xs = [d["X"]] + [d["X"].clone() for _ in range(copies - 1)]
+    Xq = [torch.empty((M, K), dtype=torch.int8, device="cuda") for _ in range(copies)]
+    tok = [torch.empty((M,), dtype=torch.float32, device="cuda") for _ in range(copies)]
+    Y = [torch.empty((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(copies)]
+    ws = w4a8.new_workspace(M, N, K, group, opts)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+
+    def one(it, e=None):
+        c = it % copies
+        if e:
+            e[0].record()
+        w4a8.quantize_act(Xs[c], d["inv_s"], out=(Xq[c], tok[c]))
+        if e:
+            e[1].record()
+        w4a8.linear(Xq[c], tok[c], packs[c], d["bias"], N, group, ws, opts, out=Y[c])
+        if e:
+            e[2].record()
+
+    for it in range(max(args.warmup, 3)):
+        one(it)
+    torch.cuda.synchronize()
+    w4a8.check_status(ws)
+    for it in range(args.steps):
+        one(it, ev[it])
+    torch.cuda.synchronize()
+    w4a8.check_status(ws)
+    q_ms = statistics.median(e[0].elapsed_time(e[1]) for e in ev)
+    l_ms = statistics.median(e[1].elapsed_time(e[2]) for e in ev)
+    G = K // group if group else 1
+    ops = 2.0 * M * N * K
+    lin_bytes = N * K / 2 + 5 * N * G + M * K + 4 * M + 2 * M * N + 4 * N
+    q_bytes = 3.0 * M * K + 4 * M
+    line = {
+        "case": {"K": K, "N": N, "M": M, "group": group, "tok_tile": tok_tile, "split_k": split_k,
+                 "decode_warps": dw, "copies": copies},
+        "linear_ms": l_ms, "linear_tops": ops / l_ms / 1e9, "linear_gbs": lin_bytes / l_ms / 1e6,
+        "linear_frac_tensor": ops / l_ms / 1e9 / (2 * peaks["bf16_burst"]),
+        "linear_frac_hbm": lin_bytes / l_ms / 1e6 / peaks["hbm_gbs"],
+        "quant_ms": q_ms, "quant_gbs": q_bytes / q_ms / 1e6,
+        "quant_frac_hbm": q_bytes / q_ms / 1e6 / peaks["hbm_gbs"],
+        "peaks": peaks, "steps": args.steps,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -176,9 +246,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--case", default=None,
+                    help="K,N,M,group[,tok_tile[,split_k[,decode_warps]]]: time one linear shape instead of "
+                         "the block (profiling and sweeps); prints its own JSON line")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.case:
+        run_case(args)
         return
 
     import numpy as np

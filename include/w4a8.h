@@ -59,7 +59,8 @@ typedef struct {
     int path;        /* w4a8_path */
     int split_k;     /* 0 = automatic; else number of K slices (tcgen05 path) */
     int tok_tile;    /* 0 = automatic; else tokens per tile: 16, 32, 64, 128 or 256 */
-    int reserved[5]; /* must be zero */
+    int decode_warps;/* 0 = automatic; else warps that expand codes to INT8: 4, 8 or 16 */
+    int reserved[4]; /* must be zero */
 } w4a8_opts;
 
 /* Bytes of the packed-weight blob for an [N][K] matrix; 0 if the shape is invalid.

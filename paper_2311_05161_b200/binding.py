@@ -38,7 +38,7 @@ class W4A8Error(RuntimeError):
 
 class Opts(ctypes.Structure):
     _fields_ = [("path", ctypes.c_int), ("split_k", ctypes.c_int), ("tok_tile", ctypes.c_int),
-                ("reserved", ctypes.c_int * 5)]
+                ("decode_warps", ctypes.c_int), ("reserved", ctypes.c_int * 4)]
 
 
 def _load() -> ctypes.CDLL:
@@ -104,9 +104,10 @@ def _dev(t, dtype, what):
     return t
 
 
-def make_opts(path: int = PATH_AUTO, split_k: int = 0, tok_tile: int = 0) -> Opts:
+def make_opts(path: int = PATH_AUTO, split_k: int = 0, tok_tile: int = 0,
+              decode_warps: int = 0) -> Opts:
     o = Opts()
-    o.path, o.split_k, o.tok_tile = path, split_k, tok_tile
+    o.path, o.split_k, o.tok_tile, o.decode_warps = path, split_k, tok_tile, decode_warps
     return o
 
 

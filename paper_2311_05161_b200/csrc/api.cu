@@ -21,8 +21,8 @@ bool opts_ok(const w4a8_opts *o)
 {
     if (!o) return true;
     if (o->path < W4A8_PATH_AUTO || o->path > W4A8_PATH_TCGEN05) return false;
-    if (o->split_k < 0 || o->tok_tile < 0) return false;
-    for (int i = 0; i < 5; ++i)
+    if (o->split_k < 0 || o->tok_tile < 0 || o->decode_warps < 0) return false;
+    for (int i = 0; i < 4; ++i)
         if (o->reserved[i] != 0) return false;
     return true;
 }

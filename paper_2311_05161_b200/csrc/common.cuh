@@ -130,6 +130,7 @@ struct LinearPlan {
     int tok_tile;     // tokens per tile (UMMA N): 16, 32, 64, 128, 256
     int tok_tiles;    // ceil(M / tok_tile)
     int split_k;      // K slices (1 = none)
+    int decode_warps; // warps converting codes to INT8: 4, 8 or 16
     int kb_per_split; // k-blocks per slice (last slice may be shorter)
     size_t off_counters, off_partials, workspace_bytes;
 };

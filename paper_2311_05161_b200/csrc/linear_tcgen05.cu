@@ -28,15 +28,16 @@ namespace w4a8 {
 
 namespace {
 
-constexpr int kDecodeWarps = 4;
 constexpr int kFirstDecodeWarp = 2;
-constexpr int kFirstEpiWarp = kFirstDecodeWarp + kDecodeWarps;
 constexpr int kABytes = kTileN * kTileK;            // decoded INT8 tile, 16 KiB
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 constexpr unsigned long long kDrainLimitNs = 200000000ull;
 
-template <int TOK, bool GROUPED>
+template <int TOK, bool GROUPED, int DW>
 struct Cfg {
+    static constexpr int kDecodeWarps = DW;                 // 4, 8 or 16: 4 / 2 / 1 quarters of a row each
+    static constexpr int kQuartersPerThread = 16 / DW;
+    static constexpr int kFirstEpiWarp = kFirstDecodeWarp + DW;
     static constexpr int kEpiGroups = (GROUPED && TOK >= 64) ? 2 : 1;   // warpgroups
     static constexpr int kEpiWarps = 4 * kEpiGroups;
     static constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
@@ -44,10 +45,17 @@ struct Cfg {
     static constexpr int kChunk = kColsPerThread >= 32 ? 32 : 16;
     static constexpr int kTokBytes = TOK * kTileK;
     static constexpr int kStageBytes = kABytes + kTokBytes + kTileBytes;
-    static constexpr int kStages = TOK == 256 ? 3 : TOK == 128 ? 5 : TOK == 64 ? 6 : 7;
+    // output staging: two buffers of kChunk tokens x 128 features BF16 per epilogue group
+    static constexpr int kStagingBytes = kEpiGroups * 2 * kChunk * kTileN * 2;
+    static constexpr int kTailBytes = kStagingBytes + 1024 /* token steps */ + 1024 /* barriers */;
+    static constexpr int kMaxStages = (232448 - 1024 - kTailBytes) / kStageBytes;
+    static constexpr int kStages = kMaxStages > 7 ? 7 : kMaxStages;
     static constexpr int kTmemCols = 2 * TOK < 32 ? 32 : 2 * TOK;
-    static constexpr int kBarrierBytes = 1024;
-    static constexpr int kSmemBytes = kStages * kStageBytes + kBarrierBytes + 1024;
+    static constexpr int kOffStaging = kStages * kStageBytes;
+    static constexpr int kOffTok = kOffStaging + kStagingBytes;
+    static constexpr int kOffBarriers = kOffTok + 1024;
+    static constexpr int kSmemBytes = kOffBarriers + 1024 + 1024 /* alignment slack */;
+    static_assert(kStages >= 3, "pipeline depth");
     static_assert(kSmemBytes <= 232448, "shared memory budget");
     static_assert(!GROUPED || TOK <= 128, "group mode keeps its FP32 sums in registers");
 };
@@ -121,6 +129,22 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
             "r"(dst),
         "l"(src), "r"(bytes), "r"(bar)
         : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::
+                     "l"(map),
+                 "r"(src), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit()
+{
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async()
 {
@@ -232,12 +256,15 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Ctl 
                                              unsigned long long limit = kWaitLimitNs)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
+    // the timer is slow to read: it is only consulted after many failed polls
+    unsigned long long t0 = 0;
     for (uint32_t i = 1;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 0u) {
+        if ((i & 1023u) == 0u) {
             if (ctl->abort) return false;
-            if (global_ns() - t0 > limit) {
+            if (t0 == 0) {
+                t0 = global_ns();
+            } else if (global_ns() - t0 > limit) {
                 ctl->abort = 1;
                 report_failure(sb, W4A8_ERR_TIMEOUT, where);
                 return false;
@@ -274,11 +301,13 @@ __device__ __forceinline__ void decode8(uint32_t w, const uint32_t (&t)[4], uint
 }
 
 // --------------------------------------------------------------------------- the kernel
-template <int TOK, bool GROUPED>
-__global__ void __launch_bounds__(Cfg<TOK, GROUPED>::kThreads, 1)
-linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map, const Params P)
+template <int TOK, bool GROUPED, int DW>
+__global__ void __launch_bounds__(Cfg<TOK, GROUPED, DW>::kThreads, 1)
+linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
+                      const __grid_constant__ CUtensorMap y_map, const Params P)
 {
-    using C = Cfg<TOK, GROUPED>;
+    using C = Cfg<TOK, GROUPED, DW>;
+    constexpr int kFirstEpiWarp = C::kFirstEpiWarp;
     constexpr int S = C::kStages;
     extern __shared__ uint8_t smem_raw[];
 
@@ -289,21 +318,21 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map, const Params 
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t bar_base = base + S * C::kStageBytes;
+    const uint32_t bar_base = base + C::kOffBarriers;
     const uint32_t bar_full = bar_base;                  // S: TMA bytes landed
     const uint32_t bar_dec = bar_base + 8 * S;           // S: decoded operand written
     const uint32_t bar_empty = bar_base + 16 * S;        // S: MMAs of the stage retired
     const uint32_t bar_acc_full = bar_base + 24 * S;     // 2
     const uint32_t bar_acc_empty = bar_acc_full + 16;    // 2
     const uint32_t bar_drain = bar_acc_empty + 16;       // 1
-    Ctl *ctl = reinterpret_cast<Ctl *>(gen_base + S * C::kStageBytes + 24 * S + 48);
+    Ctl *ctl = reinterpret_cast<Ctl *>(gen_base + C::kOffBarriers + 24 * S + 48);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_dec + 8 * s, kDecodeWarps);
+            mbar_init(bar_dec + 8 * s, DW);
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -414,7 +443,9 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map, const Params 
         __syncwarp();
     } else if (warp < kFirstEpiWarp) {
         // ------------------------------------------------------------------ decode warps
-        const int r = threadIdx.x - 32 * kFirstDecodeWarp;       // feature row in the tile
+        const int dt = threadIdx.x - 32 * kFirstDecodeWarp;
+        const int r = dt & 127;                                  // feature row in the tile
+        const int q_first = dt >> 7;                             // first 32-wide quarter it decodes
         uint32_t it = 0;
         bool ok = true;
         for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
@@ -441,7 +472,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map, const Params 
                 uint8_t *arow = stage + r * 128;
                 const int sw = r & 7;
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
+                for (int qi = 0; qi < C::kQuartersPerThread; ++qi) {
+                    const int q = q_first + qi * (DW / 4);
                     const uint4 w = *reinterpret_cast<const uint4 *>(pk + q * kQuarterBytes);
                     uint4 c0, c1;
                     decode8(w.x, t, c0.x, c0.y);
@@ -462,28 +494,65 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map, const Params 
         const int quarter = warp & 3;                     // tensor-memory lane quarter
         const int col_group = ew >> 2;                    // which share of the columns
         const int col0 = col_group * C::kColsPerThread;
+        const int f = quarter * 32 + lane;                // feature row inside the tile
         constexpr int kEpiThreads = 32 * C::kEpiWarps;
+        const int et = threadIdx.x - 32 * kFirstEpiWarp;
+        const bool elected = et == col_group * 128;       // issues this group's bulk stores
+        const int group_bar = 2 + col_group;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        uint32_t phase = 0;
+        float *s_tok = reinterpret_cast<float *>(gen_base + C::kOffTok);
+        __nv_bfloat16 *stg =
+            reinterpret_cast<__nv_bfloat16 *>(gen_base + C::kOffStaging) +
+            col_group * 2 * C::kChunk * kTileN;
+        // Outputs leave through shared memory: the accumulator has one feature per thread,
+        // the output row is one token, so a chunk of kChunk tokens x 128 features is
+        // transposed into a staging buffer and written by one bulk tensor store.
+        const bool bulk_out = P.Y != nullptr && P.split_k == 1;
+        uint32_t phase = 0, stores = 0;
         bool ok = true;
+
+        auto emit = [&](const float (&tv)[32], int nt, int tok_row) {
+            const uint32_t sbuf = stores & 1u;
+            if (elected) bulk_wait_read<1>();             // the store before last has been read
+            named_bar_sync(group_bar, 128);
+            __nv_bfloat16 *dst = stg + sbuf * (C::kChunk * kTileN) + f;
+#pragma unroll
+            for (int j = 0; j < C::kChunk; ++j) dst[j * kTileN] = __float2bfloat16_rn(tv[j]);
+            fence_proxy_async();
+            named_bar_sync(group_bar, 128);
+            if (elected) {
+                tma_store_2d(&y_map, smem_u32(stg + sbuf * (C::kChunk * kTileN)), nt * kTileN,
+                             tok_row);
+                bulk_commit();
+            }
+            ++stores;
+        };
+
         for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
             const int s = u % P.split_k, rest = u / P.split_k;
             const int nt = rest % n_tiles, tt = rest / n_tiles;
             const int kb0 = s * P.kb_per_split;
             const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
-            const int n = nt * kTileN + quarter * 32 + lane;
+            const int n = nt * kTileN + f;
             const bool n_ok = n < P.L.N;
             const int tok0 = tt * TOK + col0;
             int valid = P.M - tok0;                       // columns of this thread that are tokens
             valid = valid < 0 ? 0 : (valid > C::kColsPerThread ? C::kColsPerThread : valid);
             const float bias_n = (P.bias && n_ok) ? P.bias[n] : 0.0f;
 
+            if (P.Y) {
+                // token step sizes of this tile, shared by all epilogue threads
+                named_bar_sync(1, kEpiThreads);
+                for (int i = et; i < TOK; i += kEpiThreads)
+                    s_tok[i] = (tt * TOK + i < P.M) ? __ldg(P.tok_scale + tt * TOK + i) : 0.0f;
+                named_bar_sync(1, kEpiThreads);
+            }
+
             if (!GROUPED) {
                 const float half_step = __fmul_rn(0.5f, P.scales[n]);
                 const uint32_t buf = phase & 1u;
                 ok = wait_bounded(bar_acc_full + 8 * buf, (phase >> 1) & 1u, ctl, P.sb, 40);
-                ok = __all_sync(0xffffffffu, ok);
-                if (P.split_k > 1) ok = named_bar_and(1, kEpiThreads, ok);
+                ok = named_bar_and(1, kEpiThreads, ok);
                 if (!ok) break;
                 tc_fence_after();
                 ++phase;
@@ -500,21 +569,23 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map, const Params 
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
                     }
-                    if (P.split_k == 1) {
+                    if (c >= valid) continue;             // uniform over the column group
+                    if (P.acc_out && P.split_k == 1 && n_ok) {
+#pragma unroll
+                        for (int j = 0; j < C::kChunk; ++j)
+                            if (c + j < valid)
+                                P.acc_out[(size_t)(tok0 + c + j) * P.L.N + n] = (int)v[j];
+                    }
+                    if (bulk_out) {
+                        float tv[32];
 #pragma unroll
                         for (int j = 0; j < C::kChunk; ++j) {
-                            if (c + j < valid && n_ok) {
-                                const int m = tok0 + c + j;
-                                const int acc = (int)v[j];
-                                if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = acc;
-                                if (P.Y) {
-                                    float tv = rescale_channel(acc, __ldg(P.tok_scale + m), half_step);
-                                    if (P.bias) tv = __fadd_rn(tv, bias_n);
-                                    P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(tv);
-                                }
-                            }
+                            float x = rescale_channel((int)v[j], s_tok[col0 + c + j], half_step);
+                            if (P.bias) x = __fadd_rn(x, bias_n);
+                            tv[j] = x;
                         }
-                    } else {
+                        emit(tv, nt, tok0 + c);
+                    } else if (P.split_k > 1) {
 #pragma unroll
                         for (int j = 0; j < C::kChunk; ++j) {
                             if (c + j < valid) {
@@ -527,7 +598,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map, const Params 
                 if (P.split_k > 1) {
                     __threadfence();
                     named_bar_sync(1, kEpiThreads);
-                    if (threadIdx.x == 32 * kFirstEpiWarp) {
+                    if (et == 0) {
                         const int old = atomicAdd(P.counters + (size_t)tt * n_tiles + nt, 1);
                         const int last = old == P.split_k - 1;
                         if (last) P.counters[(size_t)tt * n_tiles + nt] = 0;
@@ -545,9 +616,9 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map, const Params 
                                 acc += __ldcg(part + ((size_t)ss * P.m_pad + m) * P.L.n_pad + n);
                             if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = acc;
                             if (P.Y) {
-                                float tv = rescale_channel(acc, __ldg(P.tok_scale + m), half_step);
-                                if (P.bias) tv = __fadd_rn(tv, bias_n);
-                                P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(tv);
+                                float x = rescale_channel(acc, s_tok[col0 + j], half_step);
+                                if (P.bias) x = __fadd_rn(x, bias_n);
+                                P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(x);
                             }
                         }
                     }
@@ -590,21 +661,23 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map, const Params 
                         }
                     }
                 }
-                if (P.split_k > 1) ok = named_bar_and(1, kEpiThreads, ok);
+                ok = named_bar_and(1, kEpiThreads, ok);
                 if (!ok) break;
-                if (P.split_k == 1) {
-                    if (P.Y && n_ok) {
+                if (bulk_out) {
 #pragma unroll
-                        for (int j = 0; j < C::kColsPerThread; ++j) {
-                            if (j < valid) {
-                                const int m = tok0 + j;
-                                float tv = __fmul_rn(usum[j], __ldg(P.tok_scale + m));
-                                if (P.bias) tv = __fadd_rn(tv, bias_n);
-                                P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(tv);
+                    for (int c = 0; c < C::kColsPerThread; c += C::kChunk) {
+                        if (c < valid) {
+                            float tv[32];
+#pragma unroll
+                            for (int j = 0; j < C::kChunk; ++j) {
+                                float x = __fmul_rn(usum[c + j], s_tok[col0 + c + j]);
+                                if (P.bias) x = __fadd_rn(x, bias_n);
+                                tv[j] = x;
                             }
+                            emit(tv, nt, tok0 + c);
                         }
                     }
-                } else {
+                } else if (P.split_k > 1) {
                     float *part = reinterpret_cast<float *>(P.partials);
 #pragma unroll
                     for (int j = 0; j < C::kColsPerThread; ++j)
@@ -612,7 +685,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map, const Params 
                             part[((size_t)s * P.m_pad + tok0 + j) * P.L.n_pad + n] = usum[j];
                     __threadfence();
                     named_bar_sync(1, kEpiThreads);
-                    if (threadIdx.x == 32 * kFirstEpiWarp) {
+                    if (et == 0) {
                         const int old = atomicAdd(P.counters + (size_t)tt * n_tiles + nt, 1);
                         const int last = old == P.split_k - 1;
                         if (last) P.counters[(size_t)tt * n_tiles + nt] = 0;
@@ -629,14 +702,16 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map, const Params 
                             for (int ss = 0; ss < P.split_k; ++ss)
                                 usm = __fadd_rn(
                                     usm, __ldcg(part + ((size_t)ss * P.m_pad + m) * P.L.n_pad + n));
-                            float tv = __fmul_rn(usm, __ldg(P.tok_scale + m));
-                            if (P.bias) tv = __fadd_rn(tv, bias_n);
-                            P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(tv);
+                            float x = __fmul_rn(usm, s_tok[col0 + j]);
+                            if (P.bias) x = __fadd_rn(x, bias_n);
+                            P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(x);
                         }
                     }
                 }
             }
         }
+        // the staging buffers must have been read before the CTA gives its memory back
+        if (elected) bulk_wait_read<0>();
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -686,17 +761,31 @@ int sm_count()
     return n;
 }
 
-template <int TOK, bool GROUPED>
-w4a8_status launch_one(const CUtensorMap &map, const Params &P, cudaStream_t st)
+struct Maps {
+    CUtensorMap tok, y16, y32;      // activations; output with 16- and 32-token boxes
+};
+
+template <int TOK, bool GROUPED, int DW>
+w4a8_status launch_dw(const Maps &maps, const Params &P, cudaStream_t st)
 {
-    using C = Cfg<TOK, GROUPED>;
-    auto kern = linear_tcgen05_kernel<TOK, GROUPED>;
+    using C = Cfg<TOK, GROUPED, DW>;
+    auto kern = linear_tcgen05_kernel<TOK, GROUPED, DW>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) !=
         cudaSuccess)
         return W4A8_ERR_CUDA;
     int grid = P.total_units < sm_count() ? P.total_units : sm_count();
-    kern<<<grid, C::kThreads, C::kSmemBytes, st>>>(map, P);
+    kern<<<grid, C::kThreads, C::kSmemBytes, st>>>(maps.tok, C::kChunk == 32 ? maps.y32 : maps.y16,
+                                                   P);
     return cudaGetLastError() == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+template <int TOK, bool GROUPED>
+w4a8_status launch_one(const Maps &maps, const Params &P, int dw, cudaStream_t st)
+{
+    if (dw == 4) return launch_dw<TOK, GROUPED, 4>(maps, P, st);
+    if (dw == 8) return launch_dw<TOK, GROUPED, 8>(maps, P, st);
+    if (dw == 16 && !GROUPED) return launch_dw<TOK, false, 16>(maps, P, st);
+    return W4A8_ERR_SHAPE;
 }
 
 }  // namespace
@@ -729,6 +818,10 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     const int kb_per = (L.k_blocks + split - 1) / split;
     split = (L.k_blocks + kb_per - 1) / kb_per;              // no empty slice
     if (tiles * split > 0x7fffffffLL) return false;
+    int dw = opts ? opts->decode_warps : 0;
+    if (dw == 0) dw = 8;
+    if (dw != 4 && dw != 8 && !(dw == 16 && !grouped)) return false;
+    plan->decode_warps = dw;
     plan->tok_tile = tok;
     plan->tok_tiles = tok_tiles;
     plan->split_k = split;
@@ -748,15 +841,29 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
 {
     EncodeTiledFn enc = encode_tiled();
     if (!enc) return W4A8_ERR_CUDA;
-    CUtensorMap map;
+    Maps maps;
+    memset(&maps, 0, sizeof(maps));
     const cuuint64_t dims[2] = {(cuuint64_t)L.K, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)L.K};
     const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)plan.tok_tile};
     const cuuint32_t estr[2] = {1, 1};
-    if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(Xq), dims, strides, box,
-            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+    if (enc(&maps.tok, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(Xq), dims, strides,
+            box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return W4A8_ERR_CUDA;
+    if (Y && plan.split_k == 1) {
+        // output tiles of 128 features x 16 or 32 tokens; parts beyond N or M are clipped
+        const cuuint64_t ydims[2] = {(cuuint64_t)L.N, (cuuint64_t)M};
+        const cuuint64_t ystrides[1] = {(cuuint64_t)L.N * 2};
+        for (int rows = 16; rows <= 32; rows += 16) {
+            const cuuint32_t ybox[2] = {(cuuint32_t)kTileN, (cuuint32_t)rows};
+            if (enc(rows == 16 ? &maps.y16 : &maps.y32, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y,
+                    ydims, ystrides, ybox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return W4A8_ERR_CUDA;
+        }
+    }
 
     Params P;
     P.blob = blob;
@@ -780,11 +887,11 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
 
     const bool g = L.group != 0;
     switch (plan.tok_tile) {
-    case 16: return g ? launch_one<16, true>(map, P, st) : launch_one<16, false>(map, P, st);
-    case 32: return g ? launch_one<32, true>(map, P, st) : launch_one<32, false>(map, P, st);
-    case 64: return g ? launch_one<64, true>(map, P, st) : launch_one<64, false>(map, P, st);
-    case 128: return g ? launch_one<128, true>(map, P, st) : launch_one<128, false>(map, P, st);
-    case 256: return g ? W4A8_ERR_SHAPE : launch_one<256, false>(map, P, st);
+    case 16: return g ? launch_one<16, true>(maps, P, plan.decode_warps, st) : launch_one<16, false>(maps, P, plan.decode_warps, st);
+    case 32: return g ? launch_one<32, true>(maps, P, plan.decode_warps, st) : launch_one<32, false>(maps, P, plan.decode_warps, st);
+    case 64: return g ? launch_one<64, true>(maps, P, plan.decode_warps, st) : launch_one<64, false>(maps, P, plan.decode_warps, st);
+    case 128: return g ? launch_one<128, true>(maps, P, plan.decode_warps, st) : launch_one<128, false>(maps, P, plan.decode_warps, st);
+    case 256: return g ? W4A8_ERR_SHAPE : launch_one<256, false>(maps, P, plan.decode_warps, st);
     }
     return W4A8_ERR_SHAPE;
 }
