@@ -220,8 +220,34 @@ def run_case(args):
         one(it, ev[it])
     torch.cuda.synchronize()
     w4a8.check_status(ws)
-    q_ms = statistics.median(e[0].elapsed_time(e[1]) for e in ev)
-    l_ms = statistics.median(e[1].elapsed_time(e[2]) for e in ev)
+    q_ms_ev = statistics.median(e[0].elapsed_time(e[1]) for e in ev)
+    l_ms_ev = statistics.median(e[1].elapsed_time(e[2]) for e in ev)
+    q_ms, l_ms = q_ms_ev, l_ms_ev
+    if not args.no_graph:
+        # Short kernels are launch-bound from Python: replay the same launches from a CUDA
+        # graph so that the device runs them back to back, and time the replay.
+        def graph_ms(fn):
+            g = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(g, stream=side):
+                    for it in range(args.steps):
+                        fn(it)
+            torch.cuda.synchronize()
+            g.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / args.steps
+
+        q_ms = graph_ms(lambda it: w4a8.quantize_act(Xs[it % copies], d["inv_s"],
+                                                     out=(Xq[it % copies], tok[it % copies])))
+        l_ms = graph_ms(lambda it: w4a8.linear(Xq[it % copies], tok[it % copies], packs[it % copies],
+                                               d["bias"], N, group, ws, opts, out=Y[it % copies]))
+        w4a8.check_status(ws)
     G = K // group if group else 1
     ops = 2.0 * M * N * K
     lin_bytes = N * K / 2 + 5 * N * G + M * K + 4 * M + 2 * M * N + 4 * N
@@ -234,6 +260,8 @@ def run_case(args):
         "linear_frac_hbm": lin_bytes / l_ms / 1e6 / peaks["hbm_gbs"],
         "quant_ms": q_ms, "quant_gbs": q_bytes / q_ms / 1e6,
         "quant_frac_hbm": q_bytes / q_ms / 1e6 / peaks["hbm_gbs"],
+        "linear_ms_events": l_ms_ev, "quant_ms_events": q_ms_ev,
+        "timing": "events per launch" if args.no_graph else "CUDA graph replay of `steps` launches",
         "peaks": peaks, "steps": args.steps,
     }
     print(json.dumps(line), flush=True)
@@ -246,6 +274,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true",
+                    help="--case only: time with per-launch events, no CUDA graph replay")
     ap.add_argument("--case", default=None,
                     help="K,N,M,group[,tok_tile[,split_k[,decode_warps]]]: time one linear shape instead of "
                          "the block (profiling and sweeps); prints its own JSON line")

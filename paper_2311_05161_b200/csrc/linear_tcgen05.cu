@@ -35,7 +35,6 @@ constexpr unsigned long long kDrainLimitNs = 200000000ull;
 
 template <int TOK, bool GROUPED, int DW>
 struct Cfg {
-    static constexpr int kDecodeWarps = DW;                 // 4, 8 or 16: 4 / 2 / 1 quarters of a row each
     static constexpr int kQuartersPerThread = 16 / DW;
     static constexpr int kFirstEpiWarp = kFirstDecodeWarp + DW;
     static constexpr int kEpiGroups = (GROUPED && TOK >= 64) ? 2 : 1;   // warpgroups
