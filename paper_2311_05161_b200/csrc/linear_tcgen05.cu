@@ -43,7 +43,12 @@ struct Cfg {
     static constexpr int kColsPerThread = TOK / kEpiGroups;
     static constexpr int kChunk = kColsPerThread >= 32 ? 32 : 16;
     static constexpr int kTokBytes = TOK * kTileK;
-    static constexpr int kStageBytes = kABytes + kTokBytes + kTileBytes;
+    // Codes reach the decode threads either through the shared-memory ring (bulk copies:
+    // deep prefetch for weight-streaming shapes) or, for wide token tiles where shared-memory
+    // bandwidth is the scarce resource, straight from global memory into registers.
+    static constexpr bool kDirect = TOK >= 128;
+    static constexpr int kTeams = DW / 4;              // teams of 4 warps take k-blocks in turn
+    static constexpr int kStageBytes = kABytes + kTokBytes + (kDirect ? 0 : kTileBytes);
     // output staging: two buffers of kChunk tokens x 128 features BF16 per epilogue group
     static constexpr int kStagingBytes = kEpiGroups * 2 * kChunk * kTileN * 2;
     static constexpr int kTailBytes = kStagingBytes + 1024 /* token steps */ + 1024 /* barriers */;
@@ -272,6 +277,50 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Ctl 
     }
 }
 
+// Position of a CTA in its list of k-blocks: units (token tile, row tile, K slice) are dealt
+// round-robin to the CTAs, each unit is a run of k-blocks, `it` counts k-blocks from zero.
+struct KbCursor {
+    int u, step, total_units, split_k, kb_per_split, k_blocks;
+    int kb, kb1;
+    uint32_t it;
+    __device__ __forceinline__ void open_unit()
+    {
+        if (u < total_units) {
+            const int s = u % split_k;
+            kb = s * kb_per_split;
+            kb1 = min(k_blocks, kb + kb_per_split);
+        }
+    }
+    __device__ __forceinline__ void start(int first, int stride, int total, int split, int per,
+                                          int kbs)
+    {
+        u = first; step = stride; total_units = total; split_k = split; kb_per_split = per;
+        k_blocks = kbs; it = 0; kb = kb1 = 0;
+        open_unit();
+    }
+    __device__ __forceinline__ bool valid() const { return u < total_units; }
+    __device__ __forceinline__ void advance(int n)
+    {
+        for (int i = 0; i < n && valid(); ++i) {
+            ++it;
+            if (++kb >= kb1) {
+                u += step;
+                open_unit();
+            }
+        }
+    }
+};
+
+// 16-byte global load that does not allocate in L1 (each code byte is used once per CTA).
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
 // --------------------------------------------------------------------------- decode
 // Byte tables of Eq. 6 in units of step/2 for zero-point z: t[c / 4] byte c % 4 holds
 // 2 (c - z) for c <= 13, +1 for c = 14, -1 for c = 15.
@@ -331,7 +380,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_dec + 8 * s, DW);
+            mbar_init(bar_dec + 8 * s, 4);
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -376,12 +425,14 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         break;
                     }
                     const uint32_t stage = base + st * C::kStageBytes;
-                    mbar_arrive_expect_tx(bar_full + 8 * st, C::kTokBytes + kTileBytes);
+                    mbar_arrive_expect_tx(bar_full + 8 * st,
+                                          C::kTokBytes + (C::kDirect ? 0 : kTileBytes));
                     tma_load_2d(stage + kABytes, &tok_map, kb * kTileK, tt * TOK,
                                 bar_full + 8 * st);
-                    bulk_load(stage + kABytes + C::kTokBytes,
-                              P.codes + ((size_t)nt * k_blocks + kb) * kTileBytes, kTileBytes,
-                              bar_full + 8 * st);
+                    if (!C::kDirect)
+                        bulk_load(stage + kABytes + C::kTokBytes,
+                                  P.codes + ((size_t)nt * k_blocks + kb) * kTileBytes, kTileBytes,
+                                  bar_full + 8 * st);
                 }
             }
             if (!ok) {
@@ -415,7 +466,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         ok = false;
                         break;
                     }
-                    if (!wait_bounded(bar_dec + 8 * st, fill & 1u, ctl, P.sb, 21)) {
+                    if (!wait_bounded(bar_dec + 8 * st, fill & 1u, ctl, P.sb, 21) ||
+                        (C::kDirect && !wait_bounded(bar_full + 8 * st, fill & 1u, ctl, P.sb, 23))) {
                         ok = false;
                         break;
                     }
@@ -442,50 +494,73 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         __syncwarp();
     } else if (warp < kFirstEpiWarp) {
         // ------------------------------------------------------------------ decode warps
+        // Four warps (one thread per feature row) form a team; teams take k-blocks in turn,
+        // so the fixed latency of one k-block (barrier wait, loads, proxy fence, arrive)
+        // overlaps the table lookups of the other teams.
         const int dt = threadIdx.x - 32 * kFirstDecodeWarp;
         const int r = dt & 127;                                  // feature row in the tile
-        const int q_first = dt >> 7;                             // first 32-wide quarter it decodes
-        uint32_t it = 0;
-        bool ok = true;
-        for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
-            const int s = u % P.split_k, rest = u / P.split_k;
-            const int nt = rest % n_tiles;
-            const int kb0 = s * P.kb_per_split;
-            const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
+        const int team = dt >> 7;
+        constexpr int T = C::kTeams;
+        KbCursor cur;
+        cur.start(blockIdx.x, gridDim.x, P.total_units, P.split_k, P.kb_per_split, k_blocks);
+        cur.advance(team);
+        uint4 w[4];
+        int z = 0;
+        auto fetch = [&](const KbCursor &c, uint4 (&dst)[4], int &zz) {
+            const int nt = (c.u / P.split_k) % n_tiles;
             const int n = nt * kTileN + r;
-            uint32_t t[4];
-            int z_next = GROUPED ? P.zeros[(size_t)kb0 * P.L.n_pad + n] : P.zeros[n];
-            if (!GROUPED) build_tables(z_next, t);
-            for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                if (GROUPED) {
-                    build_tables(z_next, t);
-                    if (kb + 1 < kb1) z_next = P.zeros[(size_t)(kb + 1) * P.L.n_pad + n];
-                }
-                const int st = it % S;
-                const uint32_t fill = it / S;
-                ok = wait_bounded(bar_full + 8 * st, fill & 1u, ctl, P.sb, 30);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                uint8_t *stage = gen_base + st * C::kStageBytes;
-                const uint8_t *pk = stage + kABytes + C::kTokBytes + r * 16;
-                uint8_t *arow = stage + r * 128;
-                const int sw = r & 7;
+            zz = GROUPED ? P.zeros[(size_t)c.kb * P.L.n_pad + n] : P.zeros[n];
+            if (C::kDirect) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(
+                    P.codes + ((size_t)nt * k_blocks + c.kb) * kTileBytes + r * 16);
 #pragma unroll
-                for (int qi = 0; qi < C::kQuartersPerThread; ++qi) {
-                    const int q = q_first + qi * (DW / 4);
-                    const uint4 w = *reinterpret_cast<const uint4 *>(pk + q * kQuarterBytes);
-                    uint4 c0, c1;
-                    decode8(w.x, t, c0.x, c0.y);
-                    decode8(w.y, t, c0.z, c0.w);
-                    decode8(w.z, t, c1.x, c1.y);
-                    decode8(w.w, t, c1.z, c1.w);
-                    *reinterpret_cast<uint4 *>(arow + (((2 * q) ^ sw) << 4)) = c0;
-                    *reinterpret_cast<uint4 *>(arow + (((2 * q + 1) ^ sw) << 4)) = c1;
-                }
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_dec + 8 * st);
+                for (int q = 0; q < 4; ++q) dst[q] = ld_stream(src + q * (kQuarterBytes / 16));
             }
+        };
+        if (cur.valid()) fetch(cur, w, z);
+        bool ok = true;
+        while (cur.valid() && ok) {
+            KbCursor nxt = cur;
+            nxt.advance(T);
+            uint4 wn[4];
+            int zn = 0;
+            if (nxt.valid()) fetch(nxt, wn, zn);                 // prefetch the team's next k-block
+            const int st = cur.it % S;
+            const uint32_t fill = cur.it / S;
+            if (C::kDirect)   // the operand buffer is free once the MMAs of its last use retired
+                ok = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
+            else
+                ok = wait_bounded(bar_full + 8 * st, fill & 1u, ctl, P.sb, 30);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            uint8_t *stage = gen_base + st * C::kStageBytes;
+            uint8_t *arow = stage + r * 128;
+            const int sw = r & 7;
+            uint32_t t[4];
+            build_tables(z, t);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint4 wq;
+                if (C::kDirect)
+                    wq = w[q];
+                else
+                    wq = *reinterpret_cast<const uint4 *>(stage + kABytes + C::kTokBytes +
+                                                          q * kQuarterBytes + r * 16);
+                uint4 c0, c1;
+                decode8(wq.x, t, c0.x, c0.y);
+                decode8(wq.y, t, c0.z, c0.w);
+                decode8(wq.z, t, c1.x, c1.y);
+                decode8(wq.w, t, c1.z, c1.w);
+                *reinterpret_cast<uint4 *>(arow + (((2 * q) ^ sw) << 4)) = c0;
+                *reinterpret_cast<uint4 *>(arow + (((2 * q + 1) ^ sw) << 4)) = c1;
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_dec + 8 * st);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) w[q] = wn[q];
+            z = zn;
+            cur = nxt;
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
