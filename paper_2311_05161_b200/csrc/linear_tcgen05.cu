@@ -43,12 +43,12 @@ struct Cfg {
     static constexpr int kColsPerThread = TOK / kEpiGroups;
     static constexpr int kChunk = kColsPerThread >= 32 ? 32 : 16;
     static constexpr int kTokBytes = TOK * kTileK;
-    // Codes reach the decode threads either through the shared-memory ring (bulk copies:
-    // deep prefetch for weight-streaming shapes) or, for wide token tiles where shared-memory
-    // bandwidth is the scarce resource, straight from global memory into registers.
-    static constexpr bool kDirect = TOK >= 128;
+    // Codes go from global memory straight into the decode threads' registers (shared-memory
+    // bandwidth and capacity are the scarce resources); for weight-streaming shapes the
+    // producer thread runs ahead with L2 prefetches of the code tiles.
     static constexpr int kTeams = DW / 4;              // teams of 4 warps take k-blocks in turn
-    static constexpr int kStageBytes = kABytes + kTokBytes + (kDirect ? 0 : kTileBytes);
+    static constexpr int kStageBytes = kABytes + kTokBytes;
+    static constexpr int kPrefetchAhead = 16;          // k-blocks of codes requested into L2
     // output staging: two buffers of kChunk tokens x 128 features BF16 per epilogue group
     static constexpr int kStagingBytes = kEpiGroups * 2 * kChunk * kTileN * 2;
     static constexpr int kTailBytes = kStagingBytes + 1024 /* token steps */ + 1024 /* barriers */;
@@ -77,7 +77,7 @@ struct Params {
     int *counters;
     void *partials;
     BlobLayout L;
-    int M, tok_tiles, m_pad, split_k, kb_per_split, total_units;
+    int M, tok_tiles, m_pad, split_k, kb_per_split, total_units, prefetch_codes;
 };
 
 // --------------------------------------------------------------------------- PTX wrappers
@@ -311,6 +311,12 @@ struct KbCursor {
     }
 };
 
+// Ask for `bytes` (a multiple of 16) at `p` to be brought into L2; nothing waits for it.
+__device__ __forceinline__ void prefetch_l2(const void *p, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
 // 16-byte global load that does not allocate in L1 (each code byte is used once per CTA).
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p)
 {
@@ -412,9 +418,11 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
+            KbCursor pf;
+            pf.start(blockIdx.x, gridDim.x, P.total_units, P.split_k, P.kb_per_split, k_blocks);
             for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
                 const int s = u % P.split_k, rest = u / P.split_k;
-                const int nt = rest % n_tiles, tt = rest / n_tiles;
+                const int tt = rest / n_tiles;
                 const int kb0 = s * P.kb_per_split;
                 const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
@@ -425,14 +433,18 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         break;
                     }
                     const uint32_t stage = base + st * C::kStageBytes;
-                    mbar_arrive_expect_tx(bar_full + 8 * st,
-                                          C::kTokBytes + (C::kDirect ? 0 : kTileBytes));
+                    mbar_arrive_expect_tx(bar_full + 8 * st, C::kTokBytes);
                     tma_load_2d(stage + kABytes, &tok_map, kb * kTileK, tt * TOK,
                                 bar_full + 8 * st);
-                    if (!C::kDirect)
-                        bulk_load(stage + kABytes + C::kTokBytes,
-                                  P.codes + ((size_t)nt * k_blocks + kb) * kTileBytes, kTileBytes,
-                                  bar_full + 8 * st);
+                    if (P.prefetch_codes) {
+                        // keep the code stream kPrefetchAhead k-blocks ahead of the decode warps
+                        while (pf.valid() && pf.it < it + C::kPrefetchAhead) {
+                            const int pnt = (pf.u / P.split_k) % n_tiles;
+                            prefetch_l2(P.codes + ((size_t)pnt * k_blocks + pf.kb) * kTileBytes,
+                                        kTileBytes);
+                            pf.advance(1);
+                        }
+                    }
                 }
             }
             if (!ok) {
@@ -467,7 +479,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         break;
                     }
                     if (!wait_bounded(bar_dec + 8 * st, fill & 1u, ctl, P.sb, 21) ||
-                        (C::kDirect && !wait_bounded(bar_full + 8 * st, fill & 1u, ctl, P.sb, 23))) {
+                        !wait_bounded(bar_full + 8 * st, fill & 1u, ctl, P.sb, 23)) {
                         ok = false;
                         break;
                     }
@@ -510,12 +522,10 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             const int nt = (c.u / P.split_k) % n_tiles;
             const int n = nt * kTileN + r;
             zz = GROUPED ? P.zeros[(size_t)c.kb * P.L.n_pad + n] : P.zeros[n];
-            if (C::kDirect) {
-                const uint4 *src = reinterpret_cast<const uint4 *>(
-                    P.codes + ((size_t)nt * k_blocks + c.kb) * kTileBytes + r * 16);
+            const uint4 *src = reinterpret_cast<const uint4 *>(
+                P.codes + ((size_t)nt * k_blocks + c.kb) * kTileBytes + r * 16);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) dst[q] = ld_stream(src + q * (kQuarterBytes / 16));
-            }
+            for (int q = 0; q < 4; ++q) dst[q] = ld_stream(src + q * (kQuarterBytes / 16));
         };
         if (cur.valid()) fetch(cur, w, z);
         bool ok = true;
@@ -527,10 +537,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             if (nxt.valid()) fetch(nxt, wn, zn);                 // prefetch the team's next k-block
             const int st = cur.it % S;
             const uint32_t fill = cur.it / S;
-            if (C::kDirect)   // the operand buffer is free once the MMAs of its last use retired
-                ok = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
-            else
-                ok = wait_bounded(bar_full + 8 * st, fill & 1u, ctl, P.sb, 30);
+            // the operand buffer is free once the MMAs of its last use have retired
+            ok = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             uint8_t *stage = gen_base + st * C::kStageBytes;
@@ -540,12 +548,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             build_tables(z, t);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                uint4 wq;
-                if (C::kDirect)
-                    wq = w[q];
-                else
-                    wq = *reinterpret_cast<const uint4 *>(stage + kABytes + C::kTokBytes +
-                                                          q * kQuarterBytes + r * 16);
+                const uint4 wq = w[q];
                 uint4 c0, c1;
                 decode8(wq.x, t, c0.x, c0.y);
                 decode8(wq.y, t, c0.z, c0.w);
@@ -893,7 +896,7 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     split = (L.k_blocks + kb_per - 1) / kb_per;              // no empty slice
     if (tiles * split > 0x7fffffffLL) return false;
     int dw = opts ? opts->decode_warps : 0;
-    if (dw == 0) dw = 8;
+    if (dw == 0) dw = grouped ? 8 : 16;
     if (dw != 4 && dw != 8 && !(dw == 16 && !grouped)) return false;
     plan->decode_warps = dw;
     plan->tok_tile = tok;
@@ -958,6 +961,7 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     P.split_k = plan.split_k;
     P.kb_per_split = plan.kb_per_split;
     P.total_units = plan.tok_tiles * L.n_tiles * plan.split_k;
+    P.prefetch_codes = plan.tok_tiles == 1 ? 1 : 0;   // every code tile is read exactly once
 
     const bool g = L.group != 0;
     switch (plan.tok_tile) {
