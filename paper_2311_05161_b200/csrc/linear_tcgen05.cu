@@ -277,6 +277,30 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Ctl 
     }
 }
 
+// The same wait for the roles with many threads (decode, epilogue): between polls the thread
+// sleeps, so that its warp leaves the issue slots to the producer and MMA threads, whose
+// per-k-block loops are the serial part of the pipeline.
+__device__ __forceinline__ bool wait_bounded_idle(uint32_t bar, uint32_t parity, Ctl *ctl,
+                                                  StatusBlock *sb, int where)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    unsigned long long t0 = 0;
+    for (uint32_t i = 1;; ++i) {
+        __nanosleep(64);
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 1023u) == 0u) {
+            if (ctl->abort) return false;
+            if (t0 == 0) {
+                t0 = global_ns();
+            } else if (global_ns() - t0 > kWaitLimitNs) {
+                ctl->abort = 1;
+                report_failure(sb, W4A8_ERR_TIMEOUT, where);
+                return false;
+            }
+        }
+    }
+}
+
 // Position of a CTA in its list of k-blocks: units (token tile, row tile, K slice) are dealt
 // round-robin to the CTAs, each unit is a run of k-blocks, `it` counts k-blocks from zero.
 struct KbCursor {
@@ -538,7 +562,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             const int st = cur.it % S;
             const uint32_t fill = cur.it / S;
             // the operand buffer is free once the MMAs of its last use have retired
-            ok = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
+            ok = wait_bounded_idle(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             uint8_t *stage = gen_base + st * C::kStageBytes;
@@ -628,7 +652,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             if (!GROUPED) {
                 const float half_step = __fmul_rn(0.5f, P.scales[n]);
                 const uint32_t buf = phase & 1u;
-                ok = wait_bounded(bar_acc_full + 8 * buf, (phase >> 1) & 1u, ctl, P.sb, 40);
+                ok = wait_bounded_idle(bar_acc_full + 8 * buf, (phase >> 1) & 1u, ctl, P.sb, 40);
                 ok = named_bar_and(1, kEpiThreads, ok);
                 if (!ok) break;
                 tc_fence_after();
@@ -710,7 +734,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     if (kb + 1 < kb1)
                         h_next = __fmul_rn(0.5f, P.scales[(size_t)(kb + 1) * P.L.n_pad + n]);
                     const uint32_t buf = phase & 1u;
-                    ok = wait_bounded(bar_acc_full + 8 * buf, (phase >> 1) & 1u, ctl, P.sb, 41);
+                    ok = wait_bounded_idle(bar_acc_full + 8 * buf, (phase >> 1) & 1u, ctl, P.sb, 41);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after();
