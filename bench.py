@@ -169,6 +169,22 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """Slowest rank's time: replicas run independently, the job ends when the last one does."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(ops_per_step: float, world: int, ms_per_step: float) -> float:
+    """Whole-job TOPS of `world` independent replicas that each do `ops_per_step` per step."""
+    return world * ops_per_step / (ms_per_step * 1e-3) / 1e12
+
+
 def run_case(args):
     """One linear shape: quantize_act + linear, each timed with its own CUDA events.
     Rotates over enough copies of the weights and activations to exceed L2."""
@@ -368,12 +384,7 @@ def main():
             fn(it)
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), world, dev)
 
     # ------------------------------------------------------------------ prefill, resident
     for _ in range(warmup):
@@ -393,7 +404,7 @@ def main():
     lin_ms = [statistics.mean(records[it][i][0].elapsed_time(records[it][i][1])
                               for it in range(args.steps)) for i in range(len(L))]
     ms_per_step = ms / args.steps
-    tops = world * ops_per_step / (ms_per_step * 1e-3) / 1e12
+    tops = replica_throughput(ops_per_step, world, ms_per_step)
     lin_tops = ops_per_step / (sum(lin_ms) * 1e-3) / 1e12
     peak_tops = 2.0 * peaks["bf16_sustained"]        # INT8 dense = 2 x BF16 dense (nominal ratio)
 
@@ -453,7 +464,7 @@ def main():
                    "l2": "inputs larger than L2 (about 400 MB touched per step)",
                    "parallelism": "replicas" if world > 1 else "single"},
         "clocks": clocks,
-        "e2e": {"value": world * ops_per_step / (ms_e2e * 1e-3) / 1e12, "unit": "TOPS",
+        "e2e": {"value": replica_throughput(ops_per_step, world, ms_e2e), "unit": "TOPS",
                 "ms_per_step": ms_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": 2 * len(L) * args.steps,
         "roofline": {"bound": "tensor", "kernel": "linear_tcgen05_kernel<256,false>",
