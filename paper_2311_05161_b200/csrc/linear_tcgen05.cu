@@ -54,7 +54,13 @@ struct Cfg {
     static constexpr int kTailBytes = kStagingBytes + 1024 /* token steps */ + 1024 /* barriers */;
     static constexpr int kMaxStages = (232448 - 1024 - kTailBytes) / kStageBytes;
     static constexpr int kStages = kMaxStages > 7 ? 7 : kMaxStages;
-    static constexpr int kTmemCols = 2 * TOK < 32 ? 32 : 2 * TOK;
+    // accumulator buffers in tensor memory: two for per-channel weights (epilogue of one unit
+    // overlaps the main loop of the next); group mode hands over every k-block, and a hand-over
+    // costs several hundred cycles of latency, so it rotates over as many buffers as fit
+    static constexpr int kAccBufs = !GROUPED ? 2 : (512 / TOK > 8 ? 8 : 512 / TOK);
+    static constexpr int kTmemNeed = kAccBufs * TOK;
+    static constexpr int kTmemCols = kTmemNeed <= 32 ? 32 : kTmemNeed <= 64 ? 64 : kTmemNeed <= 128 ? 128
+                                     : kTmemNeed <= 256 ? 256 : 512;
     static constexpr int kOffStaging = kStages * kStageBytes;
     static constexpr int kOffTok = kOffStaging + kStagingBytes;
     static constexpr int kOffBarriers = kOffTok + 1024;
@@ -400,10 +406,11 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     const uint32_t bar_full = bar_base;                  // S: TMA bytes landed
     const uint32_t bar_dec = bar_base + 8 * S;           // S: decoded operand written
     const uint32_t bar_empty = bar_base + 16 * S;        // S: MMAs of the stage retired
-    const uint32_t bar_acc_full = bar_base + 24 * S;     // 2
-    const uint32_t bar_acc_empty = bar_acc_full + 16;    // 2
-    const uint32_t bar_drain = bar_acc_empty + 16;       // 1
-    Ctl *ctl = reinterpret_cast<Ctl *>(gen_base + C::kOffBarriers + 24 * S + 48);
+    constexpr int NB = C::kAccBufs;
+    const uint32_t bar_acc_full = bar_base + 24 * S;          // NB
+    const uint32_t bar_acc_empty = bar_acc_full + 8 * NB;     // NB
+    const uint32_t bar_drain = bar_acc_empty + 8 * NB;        // 1
+    Ctl *ctl = reinterpret_cast<Ctl *>(gen_base + C::kOffBarriers + 24 * S + 16 * NB + 16);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -413,7 +420,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             mbar_init(bar_dec + 8 * s, 4);
             mbar_init(bar_empty + 8 * s, 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < NB; ++b) {
             mbar_init(bar_acc_full + 8 * b, 1);
             mbar_init(bar_acc_empty + 8 * b, C::kEpiWarps);
         }
@@ -495,9 +502,9 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     const uint32_t fill = it / S;
                     const bool first = GROUPED || kb == kb0;
                     const bool last = GROUPED || kb == kb1 - 1;
-                    const uint32_t buf = phase & 1u;
+                    const uint32_t buf = phase % NB;
                     if (first &&
-                        !wait_bounded(bar_acc_empty + 8 * buf, ((phase >> 1) & 1u) ^ 1u, ctl, P.sb,
+                        !wait_bounded(bar_acc_empty + 8 * buf, ((phase / NB) & 1u) ^ 1u, ctl, P.sb,
                                       20)) {
                         ok = false;
                         break;
@@ -651,8 +658,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
 
             if (!GROUPED) {
                 const float half_step = __fmul_rn(0.5f, P.scales[n]);
-                const uint32_t buf = phase & 1u;
-                ok = wait_bounded_idle(bar_acc_full + 8 * buf, (phase >> 1) & 1u, ctl, P.sb, 40);
+                const uint32_t buf = phase % NB;
+                ok = wait_bounded_idle(bar_acc_full + 8 * buf, (phase / NB) & 1u, ctl, P.sb, 40);
                 ok = named_bar_and(1, kEpiThreads, ok);
                 if (!ok) break;
                 tc_fence_after();
@@ -733,8 +740,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     const float h = h_next;
                     if (kb + 1 < kb1)
                         h_next = __fmul_rn(0.5f, P.scales[(size_t)(kb + 1) * P.L.n_pad + n]);
-                    const uint32_t buf = phase & 1u;
-                    ok = wait_bounded_idle(bar_acc_full + 8 * buf, (phase >> 1) & 1u, ctl, P.sb, 41);
+                    const uint32_t buf = phase % NB;
+                    ok = wait_bounded_idle(bar_acc_full + 8 * buf, (phase / NB) & 1u, ctl, P.sb, 41);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after();
@@ -900,7 +907,7 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
         tok = 16;
         while (tok < M && tok < cap) tok *= 2;
     }
-    if (tok != 16 && tok != 32 && tok != 64 && tok != 128 && tok != 256) return false;
+    if (tok != 16 && tok != 32 && tok != 64 && tok != 128 && tok != 192 && tok != 256) return false;
     if (tok > cap) return false;
     const int tok_tiles = (M + tok - 1) / tok;
     const long long tiles = (long long)tok_tiles * L.n_tiles;
@@ -993,6 +1000,7 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     case 32: return g ? launch_one<32, true>(maps, P, plan.decode_warps, st) : launch_one<32, false>(maps, P, plan.decode_warps, st);
     case 64: return g ? launch_one<64, true>(maps, P, plan.decode_warps, st) : launch_one<64, false>(maps, P, plan.decode_warps, st);
     case 128: return g ? launch_one<128, true>(maps, P, plan.decode_warps, st) : launch_one<128, false>(maps, P, plan.decode_warps, st);
+    case 192: return g ? W4A8_ERR_SHAPE : launch_one<192, false>(maps, P, plan.decode_warps, st);
     case 256: return g ? W4A8_ERR_SHAPE : launch_one<256, false>(maps, P, plan.decode_warps, st);
     }
     return W4A8_ERR_SHAPE;
