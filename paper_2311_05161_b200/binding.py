@@ -20,7 +20,7 @@ STATUS_NAMES = {
     4: "W4A8_ERR_BUFFER_TOO_SMALL", 5: "W4A8_ERR_UNSUPPORTED_ARCH", 6: "W4A8_ERR_CUDA",
     7: "W4A8_ERR_TIMEOUT", 8: "W4A8_ERR_BAD_BLOB",
 }
-PATH_AUTO, PATH_SIMPLE, PATH_TCGEN05 = 0, 1, 2
+PATH_AUTO, PATH_SIMPLE, PATH_TCGEN05, PATH_GEMV = 0, 1, 2, 3
 
 EXPORTS = (
     "w4a8_packed_bytes", "w4a8_pack_weights", "w4a8_quantize_act",

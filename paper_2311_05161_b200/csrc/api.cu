@@ -20,11 +20,20 @@ w4a8_status check_arch()
 bool opts_ok(const w4a8_opts *o)
 {
     if (!o) return true;
-    if (o->path < W4A8_PATH_AUTO || o->path > W4A8_PATH_TCGEN05) return false;
+    if (o->path < W4A8_PATH_AUTO || o->path > W4A8_PATH_GEMV) return false;
     if (o->split_k < 0 || o->tok_tile < 0 || o->decode_warps < 0) return false;
     for (int i = 0; i < 4; ++i)
         if (o->reserved[i] != 0) return false;
     return true;
+}
+
+// The weight-streaming kernel serves one to four tokens: by default there, or on request.
+bool use_gemv(int M, const w4a8_opts *o)
+{
+    const int path = o ? o->path : W4A8_PATH_AUTO;
+    if (path == W4A8_PATH_GEMV) return true;
+    return path == W4A8_PATH_AUTO && M <= gemv_max_tokens() &&
+           !(o && (o->split_k || o->tok_tile || o->decode_warps));
 }
 
 w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *packed,
@@ -55,6 +64,11 @@ w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *
         return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
     }
     LinearPlan plan;
+    if (use_gemv(M, opts)) {
+        gemv_plan(M, L, &plan);
+        return launch_linear_gemv(Xq, tok_scale, blob, L, bias, M, static_cast<__nv_bfloat16 *>(Y),
+                                  acc, static_cast<uint8_t *>(workspace), plan, st);
+    }
     if (!make_plan(M, L, opts, &plan)) return W4A8_ERR_SHAPE;
     return launch_linear_tcgen05(Xq, tok_scale, blob, L, bias, M, static_cast<__nv_bfloat16 *>(Y),
                                  acc, static_cast<uint8_t *>(workspace), plan, st);
@@ -107,6 +121,11 @@ size_t w4a8_linear_workspace_bytes_ex(int M, int N, int K, int group_size, const
     if (!shape_ok(N, K, group_size) || M < 1 || !opts_ok(opts)) return 0;
     if (opts && opts->path == W4A8_PATH_SIMPLE) return sizeof(StatusBlock);
     LinearPlan plan;
+    if (use_gemv(M, opts)) {
+        if (M > gemv_max_tokens()) return 0;
+        gemv_plan(M, make_layout(N, K, group_size), &plan);
+        return plan.workspace_bytes;
+    }
     if (!make_plan(M, make_layout(N, K, group_size), opts, &plan)) return 0;
     return plan.workspace_bytes;
 }

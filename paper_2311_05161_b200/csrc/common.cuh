@@ -152,4 +152,11 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
                                   __nv_bfloat16 *Y, int32_t *acc, uint8_t *workspace,
                                   const LinearPlan &plan, cudaStream_t st);
 
+int gemv_max_tokens();
+void gemv_plan(int M, const BlobLayout &L, LinearPlan *plan);
+w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
+                               const BlobLayout &L, const float *bias, int M, __nv_bfloat16 *Y,
+                               int32_t *acc, uint8_t *workspace, const LinearPlan &plan,
+                               cudaStream_t st);
+
 }  // namespace w4a8

@@ -1,0 +1,260 @@
+// Weight-streaming kernel of the W4A8-dINT linear layer for one to four tokens (decode).
+//
+// With so few tokens the layer is a scan of the packed weights: 0.5 byte per weight from HBM,
+// about two integer instructions per weight on the CUDA cores, nothing for the tensor cores to
+// win.  One CTA of 128 threads takes one 128-row tile and up to four 128-wide k-blocks of it;
+// thread r owns output row r, issues all of its 16-byte code loads at once (up to 256 bytes in
+// flight per thread), expands eight codes at a time through the same 16-entry byte table as the
+// tensor-core kernel (Eq. 6 in units of step/2) and accumulates with dp4a against the INT8 tokens
+// held in shared memory.  K slices leave partial sums in the workspace; the last slice of a row
+// tile to finish (an atomic counter, nobody waits) adds them in slice order and applies the
+// FP32 rescale, so results do not depend on scheduling.
+#include "common.cuh"
+
+namespace w4a8 {
+
+namespace {
+
+constexpr int kGemvKb = 4;          // k-blocks per CTA
+constexpr int kGemvMaxTokens = 4;
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+__device__ __forceinline__ void build_tables(int z, uint32_t (&t)[4])
+{
+    const uint32_t zz = (uint32_t)(2 * z) * 0x01010101u;
+    t[0] = ((0x86848280u) - zz) ^ 0x80808080u;
+    t[1] = ((0x8E8C8A88u) - zz) ^ 0x80808080u;
+    t[2] = ((0x96949290u) - zz) ^ 0x80808080u;
+    t[3] = ((((0x00009A98u) - (zz & 0xFFFFu)) ^ 0x00008080u) & 0xFFFFu) | 0xFF010000u;
+}
+
+__device__ __forceinline__ void decode8(uint32_t w, const uint32_t (&t)[4], uint32_t &o0,
+                                        uint32_t &o1)
+{
+    const uint32_t idx = w & 0x77777777u;
+    const uint32_t e = w << 4;
+    const uint32_t idx_hi = idx >> 16;
+    const uint32_t a0 = prmt(t[0], t[1], idx), b0 = prmt(t[2], t[3], idx);
+    const uint32_t a1 = prmt(t[0], t[1], idx_hi), b1 = prmt(t[2], t[3], idx_hi);
+    const uint32_t m0 = prmt(e, w, 0xD9C8u), m1 = prmt(e, w, 0xFBEAu);
+    o0 = (a0 & ~m0) | (b0 & m0);
+    o1 = (a1 & ~m1) | (b1 & m1);
+}
+
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+struct GemvParams {
+    const uint8_t *blob;
+    const uint8_t *codes;
+    const float *scales;
+    const uint8_t *zeros;
+    const int8_t *Xq;
+    const float *tok_scale;
+    const float *bias;
+    __nv_bfloat16 *Y;
+    int32_t *acc_out;
+    StatusBlock *sb;
+    int *counters;
+    void *partials;
+    BlobLayout L;
+    int M, slices;
+};
+
+template <int MT, bool GROUPED>
+__global__ void __launch_bounds__(128)
+linear_gemv_kernel(const GemvParams P)
+{
+    __shared__ __align__(16) int8_t s_x[MT][kGemvKb * kTileK];
+    __shared__ int s_last;
+    if (!header_matches(P.blob, P.L)) {
+        if (threadIdx.x == 0) report_failure(P.sb, W4A8_ERR_BAD_BLOB, 3);
+        return;
+    }
+    const int nt = blockIdx.x, slice = blockIdx.y, r = threadIdx.x;
+    const int n = nt * kTileN + r;
+    const int kb0 = slice * kGemvKb;
+    const int nkb = min(kGemvKb, P.L.k_blocks - kb0);
+
+    // all code loads of this thread first: they are the long-latency part
+    uint4 w[kGemvKb][4];
+    const uint4 *src = reinterpret_cast<const uint4 *>(
+        P.codes + ((size_t)nt * P.L.k_blocks + kb0) * kTileBytes + r * 16);
+#pragma unroll
+    for (int b = 0; b < kGemvKb; ++b)
+        if (b < nkb) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                w[b][q] = ld_stream(src + (size_t)b * (kTileBytes / 16) + q * (kQuarterBytes / 16));
+        }
+    // tokens of this K slice: MT rows of nkb * 128 INT8
+    for (int i = r; i < MT * kGemvKb * (kTileK / 16); i += 128) {
+        const int m = i / (kGemvKb * (kTileK / 16)), c = i % (kGemvKb * (kTileK / 16));
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (m < P.M && c < nkb * (kTileK / 16))
+            v = __ldg(reinterpret_cast<const uint4 *>(P.Xq + (size_t)m * P.L.K + kb0 * kTileK) + c);
+        reinterpret_cast<uint4 *>(&s_x[m][0])[c] = v;
+    }
+    __syncthreads();
+
+    int acc[MT];
+    float usum[MT];
+#pragma unroll
+    for (int m = 0; m < MT; ++m) { acc[m] = 0; usum[m] = 0.0f; }
+    uint32_t t[4];
+    if (!GROUPED) build_tables(P.zeros[n], t);
+#pragma unroll
+    for (int b = 0; b < kGemvKb; ++b) {
+        if (b < nkb) {
+            const int kb = kb0 + b;
+            if (GROUPED) {
+                build_tables(P.zeros[(size_t)kb * P.L.n_pad + n], t);
+#pragma unroll
+                for (int m = 0; m < MT; ++m) acc[m] = 0;
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t words[4] = {w[b][q].x, w[b][q].y, w[b][q].z, w[b][q].w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    uint32_t d0, d1;
+                    decode8(words[i], t, d0, d1);
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) {
+                        const uint2 x = *reinterpret_cast<const uint2 *>(
+                            &s_x[m][b * kTileK + q * 32 + i * 8]);
+                        acc[m] = __dp4a((int)d0, (int)x.x, acc[m]);
+                        acc[m] = __dp4a((int)d1, (int)x.y, acc[m]);
+                    }
+                }
+            }
+            if (GROUPED) {
+                const float h = __fmul_rn(0.5f, P.scales[(size_t)kb * P.L.n_pad + n]);
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    usum[m] = fmaf((float)acc[m], h, usum[m]);
+                    if (P.acc_out && m < P.M && n < P.L.N)
+                        P.acc_out[((size_t)kb * P.M + m) * P.L.N + n] = acc[m];
+                }
+            }
+        }
+    }
+
+    // partial sums of this slice, then find out whether every slice of the tile is in
+    if (GROUPED) {
+        float *part = reinterpret_cast<float *>(P.partials);
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+            if (m < P.M) part[((size_t)slice * P.M + m) * P.L.n_pad + n] = usum[m];
+    } else {
+        int32_t *part = reinterpret_cast<int32_t *>(P.partials);
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+            if (m < P.M) part[((size_t)slice * P.M + m) * P.L.n_pad + n] = acc[m];
+    }
+    __threadfence();
+    __syncthreads();
+    if (r == 0) {
+        const int old = atomicAdd(P.counters + nt, 1);
+        const int last = old == P.slices - 1;
+        if (last) P.counters[nt] = 0;            // ready for the next call
+        s_last = last;
+    }
+    __syncthreads();
+    if (!s_last || n >= P.L.N) return;
+    __threadfence();
+    const float bias_n = P.bias ? P.bias[n] : 0.0f;
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+        if (m >= P.M) break;
+        float tv;
+        if (GROUPED) {
+            const float *part = reinterpret_cast<const float *>(P.partials);
+            float u = 0.0f;
+            for (int s = 0; s < P.slices; ++s)
+                u = __fadd_rn(u, __ldcg(part + ((size_t)s * P.M + m) * P.L.n_pad + n));
+            tv = __fmul_rn(u, P.tok_scale ? P.tok_scale[m] : 0.0f);
+        } else {
+            const int32_t *part = reinterpret_cast<const int32_t *>(P.partials);
+            int a = 0;
+            for (int s = 0; s < P.slices; ++s)
+                a += __ldcg(part + ((size_t)s * P.M + m) * P.L.n_pad + n);
+            if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = a;
+            tv = rescale_channel(a, P.tok_scale ? P.tok_scale[m] : 0.0f,
+                                 __fmul_rn(0.5f, P.scales[n]));
+        }
+        if (P.bias) tv = __fadd_rn(tv, bias_n);
+        if (P.Y) P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(tv);
+    }
+}
+
+}  // namespace
+
+int gemv_max_tokens() { return kGemvMaxTokens; }
+
+// Workspace of the GEMV path: status block, one counter per row tile, partial sums
+// [slices][M][n_pad] (4 bytes each).
+void gemv_plan(int M, const BlobLayout &L, LinearPlan *plan)
+{
+    const int slices = (L.k_blocks + kGemvKb - 1) / kGemvKb;
+    plan->tok_tile = 0;
+    plan->tok_tiles = 1;
+    plan->split_k = slices;
+    plan->kb_per_split = kGemvKb;
+    plan->decode_warps = 0;
+    plan->off_counters = sizeof(StatusBlock);
+    plan->off_partials = align_up(plan->off_counters + (size_t)L.n_tiles * sizeof(int), 256);
+    plan->workspace_bytes = plan->off_partials + (size_t)slices * M * L.n_pad * 4;
+}
+
+w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
+                               const BlobLayout &L, const float *bias, int M, __nv_bfloat16 *Y,
+                               int32_t *acc, uint8_t *workspace, const LinearPlan &plan,
+                               cudaStream_t st)
+{
+    if (M < 1 || M > kGemvMaxTokens) return W4A8_ERR_SHAPE;
+    GemvParams P;
+    P.blob = blob;
+    P.codes = blob + L.off_codes;
+    P.scales = reinterpret_cast<const float *>(blob + L.off_scales);
+    P.zeros = blob + L.off_zeros;
+    P.Xq = Xq;
+    P.tok_scale = tok_scale;
+    P.bias = bias;
+    P.Y = Y;
+    P.acc_out = acc;
+    P.sb = reinterpret_cast<StatusBlock *>(workspace);
+    P.counters = reinterpret_cast<int *>(workspace + plan.off_counters);
+    P.partials = workspace + plan.off_partials;
+    P.L = L;
+    P.M = M;
+    P.slices = plan.split_k;
+    if (P.slices > 65535) return W4A8_ERR_SHAPE;
+    const dim3 grid(L.n_tiles, P.slices);
+    const bool g = L.group != 0;
+    if (M == 1) {
+        if (g) linear_gemv_kernel<1, true><<<grid, 128, 0, st>>>(P);
+        else linear_gemv_kernel<1, false><<<grid, 128, 0, st>>>(P);
+    } else if (M == 2) {
+        if (g) linear_gemv_kernel<2, true><<<grid, 128, 0, st>>>(P);
+        else linear_gemv_kernel<2, false><<<grid, 128, 0, st>>>(P);
+    } else {
+        if (g) linear_gemv_kernel<4, true><<<grid, 128, 0, st>>>(P);
+        else linear_gemv_kernel<4, false><<<grid, 128, 0, st>>>(P);
+    }
+    return cudaGetLastError() == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+}  // namespace w4a8

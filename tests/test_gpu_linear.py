@@ -118,3 +118,23 @@ def test_wrong_blob_is_reported_not_computed():
         w4a8.linear(Xq, tok, buf, None, 768, 0, ws, w4a8.make_opts(path))
         assert w4a8.poll_status(ws) == 8          # W4A8_ERR_BAD_BLOB
         assert w4a8.poll_status(ws) == 0          # cleared by the poll
+
+
+@pytest.mark.parametrize("group", [0, 128])
+@pytest.mark.parametrize("M", [1, 2, 3, 4])
+def test_gemv_path_small_token_counts(M, group):
+    # K = 1280 is ten k-blocks: K slices of 4 + 4 + 2; N = 200 is not a multiple of the row tile
+    prob = Problem(1280, 200, M, group, seed=50 + M + group, dist="laplace", outliers=0.01, mult=20.0)
+    opts = w4a8.make_opts(w4a8.PATH_GEMV)
+    packed = w4a8.pack_weights(prob.dev["W"], prob.dev["s"], group)
+    for _ in range(2):                       # the second call reuses the self-cleaned workspace
+        Y, acc = run_linear(prob, opts, packed)
+        assert np.array_equal(acc, prob.oracle_acc())
+        check_y(prob, Y, exact=(group == 0))
+    # the automatic choice for these token counts is the same kernel: identical bits
+    Ya, _ = run_linear(prob, None, packed)
+    assert np.array_equal(Ya, Y)
+
+
+def test_gemv_path_rejects_more_than_four_tokens():
+    assert w4a8.linear_workspace_bytes(5, 256, 256, 0, w4a8.make_opts(w4a8.PATH_GEMV)) == 0
