@@ -2,9 +2,9 @@
 //
 // With so few tokens the layer is a scan of the packed weights: 0.5 byte per weight from HBM,
 // about two integer instructions per weight on the CUDA cores, nothing for the tensor cores to
-// win.  One CTA of 128 threads takes one 128-row tile and up to four 128-wide k-blocks of it;
-// thread r owns output row r, issues all of its 16-byte code loads at once (up to 256 bytes in
-// flight per thread), expands eight codes at a time through the same 16-entry byte table as the
+// win.  One CTA of 128 threads takes one 128-row tile and up to two 128-wide k-blocks of it;
+// thread r owns output row r, issues all of its 16-byte code loads at once (128 bytes in
+// flight per thread, eight CTAs per SM), expands eight codes at a time through the same 16-entry byte table as the
 // tensor-core kernel (Eq. 6 in units of step/2) and accumulates with dp4a against the INT8 tokens
 // held in shared memory.  K slices leave partial sums in the workspace; the last slice of a row
 // tile to finish (an atomic counter, nobody waits) adds them in slice order and applies the
@@ -15,7 +15,7 @@ namespace w4a8 {
 
 namespace {
 
-constexpr int kGemvKb = 4;          // k-blocks per CTA
+constexpr int kGemvKb = 2;          // k-blocks per CTA
 constexpr int kGemvMaxTokens = 4;
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
@@ -74,7 +74,7 @@ struct GemvParams {
 };
 
 template <int MT, bool GROUPED>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, 8)
 linear_gemv_kernel(const GemvParams P)
 {
     __shared__ __align__(16) int8_t s_x[MT][kGemvKb * kTileK];

@@ -123,7 +123,7 @@ def test_wrong_blob_is_reported_not_computed():
 @pytest.mark.parametrize("group", [0, 128])
 @pytest.mark.parametrize("M", [1, 2, 3, 4])
 def test_gemv_path_small_token_counts(M, group):
-    # K = 1280 is ten k-blocks: K slices of 4 + 4 + 2; N = 200 is not a multiple of the row tile
+    # K = 1280 is ten k-blocks: K slices of 2 k-blocks; N = 200 is not a multiple of the row tile
     prob = Problem(1280, 200, M, group, seed=50 + M + group, dist="laplace", outliers=0.01, mult=20.0)
     opts = w4a8.make_opts(w4a8.PATH_GEMV)
     packed = w4a8.pack_weights(prob.dev["W"], prob.dev["s"], group)
