@@ -2,9 +2,9 @@
 //
 // With so few tokens the layer is a scan of the packed weights: 0.5 byte per weight from HBM,
 // about two integer instructions per weight on the CUDA cores, nothing for the tensor cores to
-// win.  One CTA of 128 threads takes one 128-row tile and up to two 128-wide k-blocks of it;
-// thread r owns output row r, issues all of its 16-byte code loads at once (128 bytes in
-// flight per thread, eight CTAs per SM), expands eight codes at a time through the same 16-entry byte table as the
+// win.  One CTA of 128 threads takes one 128-row tile and a K slice of two to eight 128-wide
+// k-blocks of it; thread r owns output row r, loads its codes two k-blocks (128 bytes) at a
+// time, one step ahead of the arithmetic, expands eight codes at a time through the same 16-entry byte table as the
 // tensor-core kernel (Eq. 6 in units of step/2) and accumulates with dp4a against the INT8 tokens
 // held in shared memory.  K slices leave partial sums in the workspace; the last slice of a row
 // tile to finish (an atomic counter, nobody waits) adds them in slice order and applies the
@@ -15,7 +15,8 @@ namespace w4a8 {
 
 namespace {
 
-constexpr int kGemvKb = 2;          // k-blocks per CTA
+constexpr int kGemvKb = 2;          // k-blocks per pipeline step (128 bytes of codes per thread)
+constexpr int kGemvMaxSteps = 4;    // steps per CTA: a K slice is at most 8 k-blocks
 constexpr int kGemvMaxTokens = 4;
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
@@ -70,14 +71,14 @@ struct GemvParams {
     int *counters;
     void *partials;
     BlobLayout L;
-    int M, slices;
+    int M, slices, kb_per_slice;
 };
 
 template <int MT, bool GROUPED>
-__global__ void __launch_bounds__(128, 8)
+__global__ void __launch_bounds__(128, 4)
 linear_gemv_kernel(const GemvParams P)
 {
-    __shared__ __align__(16) int8_t s_x[MT][kGemvKb * kTileK];
+    __shared__ __align__(16) int8_t s_x[MT][kGemvMaxSteps * kGemvKb * kTileK];
     __shared__ int s_last;
     if (!header_matches(P.blob, P.L)) {
         if (threadIdx.x == 0) report_failure(P.sb, W4A8_ERR_BAD_BLOB, 3);
@@ -85,26 +86,33 @@ linear_gemv_kernel(const GemvParams P)
     }
     const int nt = blockIdx.x, slice = blockIdx.y, r = threadIdx.x;
     const int n = nt * kTileN + r;
-    const int kb0 = slice * kGemvKb;
-    const int nkb = min(kGemvKb, P.L.k_blocks - kb0);
+    const int kb_first = slice * P.kb_per_slice;
+    const int kb_count = min(P.kb_per_slice, P.L.k_blocks - kb_first);
+    const int steps = (kb_count + kGemvKb - 1) / kGemvKb;
 
-    // all code loads of this thread first: they are the long-latency part
-    uint4 w[kGemvKb][4];
+    // The codes are the long-latency part: the loads of a step are issued one step ahead of
+    // its arithmetic, so that a CTA always has 128 bytes per thread in flight.
     const uint4 *src = reinterpret_cast<const uint4 *>(
-        P.codes + ((size_t)nt * P.L.k_blocks + kb0) * kTileBytes + r * 16);
+        P.codes + ((size_t)nt * P.L.k_blocks + kb_first) * kTileBytes + r * 16);
+    auto load_step = [&](int step, uint4 (&dst)[kGemvKb][4]) {
 #pragma unroll
-    for (int b = 0; b < kGemvKb; ++b)
-        if (b < nkb) {
+        for (int b = 0; b < kGemvKb; ++b)
+            if (step * kGemvKb + b < kb_count) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-                w[b][q] = ld_stream(src + (size_t)b * (kTileBytes / 16) + q * (kQuarterBytes / 16));
-        }
-    // tokens of this K slice: MT rows of nkb * 128 INT8
-    for (int i = r; i < MT * kGemvKb * (kTileK / 16); i += 128) {
-        const int m = i / (kGemvKb * (kTileK / 16)), c = i % (kGemvKb * (kTileK / 16));
+                for (int q = 0; q < 4; ++q)
+                    dst[b][q] = ld_stream(src + (size_t)(step * kGemvKb + b) * (kTileBytes / 16) +
+                                          q * (kQuarterBytes / 16));
+            }
+    };
+    uint4 w[kGemvKb][4];
+    load_step(0, w);
+    // tokens of this K slice: MT rows of kb_count * 128 INT8
+    constexpr int kRowChunks = kGemvMaxSteps * kGemvKb * (kTileK / 16);
+    for (int i = r; i < MT * kRowChunks; i += 128) {
+        const int m = i / kRowChunks, c = i % kRowChunks;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (m < P.M && c < nkb * (kTileK / 16))
-            v = __ldg(reinterpret_cast<const uint4 *>(P.Xq + (size_t)m * P.L.K + kb0 * kTileK) + c);
+        if (m < P.M && c < kb_count * (kTileK / 16))
+            v = __ldg(reinterpret_cast<const uint4 *>(P.Xq + (size_t)m * P.L.K + kb_first * kTileK) + c);
         reinterpret_cast<uint4 *>(&s_x[m][0])[c] = v;
     }
     __syncthreads();
@@ -115,40 +123,52 @@ linear_gemv_kernel(const GemvParams P)
     for (int m = 0; m < MT; ++m) { acc[m] = 0; usum[m] = 0.0f; }
     uint32_t t[4];
     if (!GROUPED) build_tables(P.zeros[n], t);
+#pragma unroll 1
+    for (int step = 0; step < steps; ++step) {
+        uint4 wn[kGemvKb][4];
+        if (step + 1 < steps) load_step(step + 1, wn);
 #pragma unroll
-    for (int b = 0; b < kGemvKb; ++b) {
-        if (b < nkb) {
-            const int kb = kb0 + b;
-            if (GROUPED) {
-                build_tables(P.zeros[(size_t)kb * P.L.n_pad + n], t);
+        for (int b = 0; b < kGemvKb; ++b) {
+            const int kl = step * kGemvKb + b;             // k-block inside the slice
+            if (kl < kb_count) {
+                const int kb = kb_first + kl;
+                if (GROUPED) {
+                    build_tables(P.zeros[(size_t)kb * P.L.n_pad + n], t);
 #pragma unroll
-                for (int m = 0; m < MT; ++m) acc[m] = 0;
-            }
+                    for (int m = 0; m < MT; ++m) acc[m] = 0;
+                }
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint32_t words[4] = {w[b][q].x, w[b][q].y, w[b][q].z, w[b][q].w};
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t words[4] = {w[b][q].x, w[b][q].y, w[b][q].z, w[b][q].w};
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    uint32_t d0, d1;
-                    decode8(words[i], t, d0, d1);
+                    for (int i = 0; i < 4; ++i) {
+                        uint32_t d0, d1;
+                        decode8(words[i], t, d0, d1);
+#pragma unroll
+                        for (int m = 0; m < MT; ++m) {
+                            const uint2 x = *reinterpret_cast<const uint2 *>(
+                                &s_x[m][kl * kTileK + q * 32 + i * 8]);
+                            acc[m] = __dp4a((int)d0, (int)x.x, acc[m]);
+                            acc[m] = __dp4a((int)d1, (int)x.y, acc[m]);
+                        }
+                    }
+                }
+                if (GROUPED) {
+                    const float h = __fmul_rn(0.5f, P.scales[(size_t)kb * P.L.n_pad + n]);
 #pragma unroll
                     for (int m = 0; m < MT; ++m) {
-                        const uint2 x = *reinterpret_cast<const uint2 *>(
-                            &s_x[m][b * kTileK + q * 32 + i * 8]);
-                        acc[m] = __dp4a((int)d0, (int)x.x, acc[m]);
-                        acc[m] = __dp4a((int)d1, (int)x.y, acc[m]);
+                        usum[m] = fmaf((float)acc[m], h, usum[m]);
+                        if (P.acc_out && m < P.M && n < P.L.N)
+                            P.acc_out[((size_t)kb * P.M + m) * P.L.N + n] = acc[m];
                     }
                 }
             }
-            if (GROUPED) {
-                const float h = __fmul_rn(0.5f, P.scales[(size_t)kb * P.L.n_pad + n]);
+        }
+        if (step + 1 < steps) {
 #pragma unroll
-                for (int m = 0; m < MT; ++m) {
-                    usum[m] = fmaf((float)acc[m], h, usum[m]);
-                    if (P.acc_out && m < P.M && n < P.L.N)
-                        P.acc_out[((size_t)kb * P.M + m) * P.L.N + n] = acc[m];
-                }
-            }
+            for (int b = 0; b < kGemvKb; ++b)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) w[b][q] = wn[b][q];
         }
     }
 
@@ -208,11 +228,18 @@ int gemv_max_tokens() { return kGemvMaxTokens; }
 // [slices][M][n_pad] (4 bytes each).
 void gemv_plan(int M, const BlobLayout &L, LinearPlan *plan)
 {
-    const int slices = (L.k_blocks + kGemvKb - 1) / kGemvKb;
+    // enough K slices for about four CTAs per SM, each slice between 2 and 8 k-blocks
+    const int target_ctas = 148 * 4;
+    int slices = (target_ctas + L.n_tiles - 1) / L.n_tiles;
+    int per = (L.k_blocks + slices - 1) / slices;
+    if (per < kGemvKb) per = kGemvKb;
+    if (per > kGemvKb * kGemvMaxSteps) per = kGemvKb * kGemvMaxSteps;
+    if (per > L.k_blocks) per = L.k_blocks;
+    slices = (L.k_blocks + per - 1) / per;
     plan->tok_tile = 0;
     plan->tok_tiles = 1;
     plan->split_k = slices;
-    plan->kb_per_split = kGemvKb;
+    plan->kb_per_split = per;
     plan->decode_warps = 0;
     plan->off_counters = sizeof(StatusBlock);
     plan->off_partials = align_up(plan->off_counters + (size_t)L.n_tiles * sizeof(int), 256);
@@ -241,6 +268,7 @@ w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const u
     P.L = L;
     P.M = M;
     P.slices = plan.split_k;
+    P.kb_per_slice = plan.kb_per_split;
     if (P.slices > 65535) return W4A8_ERR_SHAPE;
     const dim3 grid(L.n_tiles, P.slices);
     const bool g = L.group != 0;
