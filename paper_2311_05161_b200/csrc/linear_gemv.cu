@@ -104,6 +104,14 @@ linear_gemv_kernel(const GemvParams P)
                                           q * (kQuarterBytes / 16));
             }
     };
+    // One thread asks for the rest of the slice to be brought into L2 right away: that puts the
+    // whole slice in flight from HBM, far more than the registers of the CTA could hold.
+    if (r == 0)
+        for (int kl = kGemvKb; kl < kb_count; ++kl)
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(
+                             P.codes + ((size_t)nt * P.L.k_blocks + kb_first + kl) * kTileBytes),
+                         "r"((uint32_t)kTileBytes)
+                         : "memory");
     uint4 w[kGemvKb][4];
     load_step(0, w);
     // tokens of this K slice: MT rows of kb_count * 128 INT8
