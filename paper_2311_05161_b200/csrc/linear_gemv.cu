@@ -16,7 +16,9 @@ namespace w4a8 {
 namespace {
 
 constexpr int kGemvKb = 2;          // k-blocks per pipeline step (128 bytes of codes per thread)
-constexpr int kGemvMaxSteps = 4;    // steps per CTA: a K slice is at most 8 k-blocks
+constexpr int kGemvMaxSteps = 8;    // steps per CTA: a K slice is at most 16 k-blocks
+constexpr int kGemvDepth = 4;       // steps of codes in flight per thread (asynchronous copies)
+constexpr int kGemvRingBytes = kGemvDepth * kGemvKb * 4 * 128 * 16;   // 64 KiB per CTA
 constexpr int kGemvMaxTokens = 4;
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
@@ -75,10 +77,14 @@ struct GemvParams {
 };
 
 template <int MT, bool GROUPED>
-__global__ void __launch_bounds__(128, 4)
+__global__ void __launch_bounds__(128, 3)
 linear_gemv_kernel(const GemvParams P)
 {
-    __shared__ __align__(16) int8_t s_x[MT][kGemvMaxSteps * kGemvKb * kTileK];
+    // dynamic shared memory: the code ring, then the tokens of the K slice
+    extern __shared__ __align__(16) uint8_t gemv_smem[];
+    uint4 *ring = reinterpret_cast<uint4 *>(gemv_smem);
+    int8_t (*s_x)[kGemvMaxSteps * kGemvKb * kTileK] =
+        reinterpret_cast<int8_t (*)[kGemvMaxSteps * kGemvKb * kTileK]>(gemv_smem + kGemvRingBytes);
     __shared__ int s_last;
     if (!header_matches(P.blob, P.L)) {
         if (threadIdx.x == 0) report_failure(P.sb, W4A8_ERR_BAD_BLOB, 3);
@@ -90,30 +96,30 @@ linear_gemv_kernel(const GemvParams P)
     const int kb_count = min(P.kb_per_slice, P.L.k_blocks - kb_first);
     const int steps = (kb_count + kGemvKb - 1) / kGemvKb;
 
-    // The codes are the long-latency part: the loads of a step are issued one step ahead of
-    // its arithmetic, so that a CTA always has 128 bytes per thread in flight.
-    const uint4 *src = reinterpret_cast<const uint4 *>(
-        P.codes + ((size_t)nt * P.L.k_blocks + kb_first) * kTileBytes + r * 16);
-    auto load_step = [&](int step, uint4 (&dst)[kGemvKb][4]) {
+    // The codes are the long-latency part.  Every thread copies its own 16-byte pieces
+    // asynchronously into a private ring in shared memory, kGemvDepth steps ahead of the
+    // arithmetic (512 bytes in flight per thread, no registers held, no cross-thread hand-off).
+    const uint8_t *src = P.codes + ((size_t)nt * P.L.k_blocks + kb_first) * kTileBytes + r * 16;
+    auto issue = [&](int step) {
+        if (step < steps) {
 #pragma unroll
-        for (int b = 0; b < kGemvKb; ++b)
-            if (step * kGemvKb + b < kb_count) {
+            for (int b = 0; b < kGemvKb; ++b)
+                if (step * kGemvKb + b < kb_count) {
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    dst[b][q] = ld_stream(src + (size_t)(step * kGemvKb + b) * (kTileBytes / 16) +
-                                          q * (kQuarterBytes / 16));
-            }
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(
+                            ring + (((step % kGemvDepth) * kGemvKb + b) * 4 + q) * 128 + r);
+                        const uint8_t *g = src + (size_t)(step * kGemvKb + b) * kTileBytes +
+                                           q * kQuarterBytes;
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(g)
+                                     : "memory");
+                    }
+                }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");     // one group per step, even if empty
     };
-    // One thread asks for the rest of the slice to be brought into L2 right away: that puts the
-    // whole slice in flight from HBM, far more than the registers of the CTA could hold.
-    if (r == 0)
-        for (int kl = kGemvKb; kl < kb_count; ++kl)
-            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(
-                             P.codes + ((size_t)nt * P.L.k_blocks + kb_first + kl) * kTileBytes),
-                         "r"((uint32_t)kTileBytes)
-                         : "memory");
-    uint4 w[kGemvKb][4];
-    load_step(0, w);
+#pragma unroll
+    for (int s = 0; s < kGemvDepth; ++s) issue(s);
     // tokens of this K slice: MT rows of kb_count * 128 INT8
     constexpr int kRowChunks = kGemvMaxSteps * kGemvKb * (kTileK / 16);
     for (int i = r; i < MT * kRowChunks; i += 128) {
@@ -133,8 +139,15 @@ linear_gemv_kernel(const GemvParams P)
     if (!GROUPED) build_tables(P.zeros[n], t);
 #pragma unroll 1
     for (int step = 0; step < steps; ++step) {
-        uint4 wn[kGemvKb][4];
-        if (step + 1 < steps) load_step(step + 1, wn);
+        // the group of this step is the oldest of kGemvDepth outstanding ones
+        asm volatile("cp.async.wait_group %0;" ::"n"(kGemvDepth - 1) : "memory");
+        uint4 w[kGemvKb][4];
+#pragma unroll
+        for (int b = 0; b < kGemvKb; ++b)
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                w[b][q] = ring[(((step % kGemvDepth) * kGemvKb + b) * 4 + q) * 128 + r];
+        issue(step + kGemvDepth);                            // refill the slot just read
 #pragma unroll
         for (int b = 0; b < kGemvKb; ++b) {
             const int kl = step * kGemvKb + b;             // k-block inside the slice
@@ -171,12 +184,6 @@ linear_gemv_kernel(const GemvParams P)
                     }
                 }
             }
-        }
-        if (step + 1 < steps) {
-#pragma unroll
-            for (int b = 0; b < kGemvKb; ++b)
-#pragma unroll
-                for (int q = 0; q < 4; ++q) w[b][q] = wn[b][q];
         }
     }
 
@@ -228,6 +235,15 @@ linear_gemv_kernel(const GemvParams P)
     }
 }
 
+template <int MT, bool GROUPED>
+void launch_gemv(dim3 grid, const GemvParams &P, cudaStream_t st)
+{
+    constexpr int smem = kGemvRingBytes + MT * kGemvMaxSteps * kGemvKb * kTileK;
+    cudaFuncSetAttribute(linear_gemv_kernel<MT, GROUPED>,
+                         cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    linear_gemv_kernel<MT, GROUPED><<<grid, 128, smem, st>>>(P);
+}
+
 }  // namespace
 
 int gemv_max_tokens() { return kGemvMaxTokens; }
@@ -236,9 +252,11 @@ int gemv_max_tokens() { return kGemvMaxTokens; }
 // [slices][M][n_pad] (4 bytes each).
 void gemv_plan(int M, const BlobLayout &L, LinearPlan *plan)
 {
-    // enough K slices for about four CTAs per SM, each slice between 2 and 8 k-blocks
-    const int target_ctas = 148 * 4;
-    int slices = (target_ctas + L.n_tiles - 1) / L.n_tiles;
+    // K slices so that the grid fills, but does not exceed, three CTAs per SM when it can;
+    // a slice is between 2 and 16 k-blocks
+    const int target_ctas = 148 * 3;
+    int slices = target_ctas / L.n_tiles;
+    if (slices < 1) slices = 1;
     int per = (L.k_blocks + slices - 1) / slices;
     if (per < kGemvKb) per = kGemvKb;
     if (per > kGemvKb * kGemvMaxSteps) per = kGemvKb * kGemvMaxSteps;
@@ -281,14 +299,14 @@ w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const u
     const dim3 grid(L.n_tiles, P.slices);
     const bool g = L.group != 0;
     if (M == 1) {
-        if (g) linear_gemv_kernel<1, true><<<grid, 128, 0, st>>>(P);
-        else linear_gemv_kernel<1, false><<<grid, 128, 0, st>>>(P);
+        if (g) launch_gemv<1, true>(grid, P, st);
+        else launch_gemv<1, false>(grid, P, st);
     } else if (M == 2) {
-        if (g) linear_gemv_kernel<2, true><<<grid, 128, 0, st>>>(P);
-        else linear_gemv_kernel<2, false><<<grid, 128, 0, st>>>(P);
+        if (g) launch_gemv<2, true>(grid, P, st);
+        else launch_gemv<2, false>(grid, P, st);
     } else {
-        if (g) linear_gemv_kernel<4, true><<<grid, 128, 0, st>>>(P);
-        else linear_gemv_kernel<4, false><<<grid, 128, 0, st>>>(P);
+        if (g) launch_gemv<4, true>(grid, P, st);
+        else launch_gemv<4, false>(grid, P, st);
     }
     return cudaGetLastError() == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
