@@ -17,8 +17,8 @@ namespace {
 
 constexpr int kGemvKb = 2;          // k-blocks per pipeline step (128 bytes of codes per thread)
 constexpr int kGemvMaxSteps = 8;    // steps per CTA: a K slice is at most 16 k-blocks
-constexpr int kGemvDepth = 4;       // steps of codes in flight per thread (asynchronous copies)
-constexpr int kGemvRingBytes = kGemvDepth * kGemvKb * 4 * 128 * 16;   // 64 KiB per CTA
+constexpr int kGemvDepth = 2;       // steps of codes in flight per thread (asynchronous copies)
+constexpr int kGemvRingBytes = kGemvDepth * kGemvKb * 4 * 128 * 16;   // 32 KiB per CTA
 constexpr int kGemvMaxTokens = 4;
 
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
@@ -77,7 +77,7 @@ struct GemvParams {
 };
 
 template <int MT, bool GROUPED>
-__global__ void __launch_bounds__(128, 3)
+__global__ void __launch_bounds__(128, 6)
 linear_gemv_kernel(const GemvParams P)
 {
     // dynamic shared memory: the code ring, then the tokens of the K slice
@@ -98,7 +98,7 @@ linear_gemv_kernel(const GemvParams P)
 
     // The codes are the long-latency part.  Every thread copies its own 16-byte pieces
     // asynchronously into a private ring in shared memory, kGemvDepth steps ahead of the
-    // arithmetic (512 bytes in flight per thread, no registers held, no cross-thread hand-off).
+    // arithmetic (256 bytes in flight per thread, no registers held, no cross-thread hand-off).
     const uint8_t *src = P.codes + ((size_t)nt * P.L.k_blocks + kb_first) * kTileBytes + r * 16;
     auto issue = [&](int step) {
         if (step < steps) {
@@ -252,9 +252,9 @@ int gemv_max_tokens() { return kGemvMaxTokens; }
 // [slices][M][n_pad] (4 bytes each).
 void gemv_plan(int M, const BlobLayout &L, LinearPlan *plan)
 {
-    // K slices so that the grid fills, but does not exceed, three CTAs per SM when it can;
+    // K slices so that the grid fills, but does not exceed, six CTAs per SM when it can;
     // a slice is between 2 and 16 k-blocks
-    const int target_ctas = 148 * 3;
+    const int target_ctas = 148 * 6;
     int slices = target_ctas / L.n_tiles;
     if (slices < 1) slices = 1;
     int per = (L.k_blocks + slices - 1) / slices;
