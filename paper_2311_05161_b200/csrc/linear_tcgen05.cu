@@ -37,7 +37,10 @@ template <int TOK, bool GROUPED, int DW>
 struct Cfg {
     static constexpr int kQuartersPerThread = 16 / DW;
     static constexpr int kFirstEpiWarp = kFirstDecodeWarp + DW;
-    static constexpr int kEpiGroups = (GROUPED && TOK >= 64) ? 2 : 1;   // warpgroups
+    // epilogue warpgroups: group mode spreads the per-k-block FP32 accumulation over
+    // 32 columns per thread (more warps in flight, fewer registers each)
+    static constexpr int kEpiGroups = !GROUPED ? 1 : (TOK >= 128 ? 4 : TOK >= 64 ? 2 : 1);
+    static constexpr int kStageBufs = GROUPED ? 1 : 2;      // output staging buffers per group
     static constexpr int kEpiWarps = 4 * kEpiGroups;
     static constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
     static constexpr int kColsPerThread = TOK / kEpiGroups;
@@ -50,7 +53,7 @@ struct Cfg {
     static constexpr int kStageBytes = kABytes + kTokBytes;
     static constexpr int kPrefetchAhead = 16;          // k-blocks of codes requested into L2
     // output staging: two buffers of kChunk tokens x 128 features BF16 per epilogue group
-    static constexpr int kStagingBytes = kEpiGroups * 2 * kChunk * kTileN * 2;
+    static constexpr int kStagingBytes = kEpiGroups * kStageBufs * kChunk * kTileN * 2;
     static constexpr int kTailBytes = kStagingBytes + 1024 /* token steps */ + 1024 /* barriers */;
     static constexpr int kMaxStages = (232448 - 1024 - kTailBytes) / kStageBytes;
     static constexpr int kStages = kMaxStages > 7 ? 7 : kMaxStages;
@@ -611,7 +614,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         float *s_tok = reinterpret_cast<float *>(gen_base + C::kOffTok);
         __nv_bfloat16 *stg =
             reinterpret_cast<__nv_bfloat16 *>(gen_base + C::kOffStaging) +
-            col_group * 2 * C::kChunk * kTileN;
+            col_group * C::kStageBufs * C::kChunk * kTileN;
         // Outputs leave through shared memory: the accumulator has one feature per thread,
         // the output row is one token, so a chunk of kChunk tokens x 128 features is
         // transposed into a staging buffer and written by one bulk tensor store.
@@ -620,8 +623,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         bool ok = true;
 
         auto emit = [&](const float (&tv)[32], int nt, int tok_row) {
-            const uint32_t sbuf = stores & 1u;
-            if (elected) bulk_wait_read<1>();             // the store before last has been read
+            const uint32_t sbuf = stores % C::kStageBufs;
+            if (elected) bulk_wait_read<C::kStageBufs - 1>();   // the buffer's last store has been read
             named_bar_sync(group_bar, 128);
             __nv_bfloat16 *dst = stg + sbuf * (C::kChunk * kTileN) + f;
 #pragma unroll
