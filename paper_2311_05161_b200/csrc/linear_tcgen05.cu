@@ -572,7 +572,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             const int st = cur.it % S;
             const uint32_t fill = cur.it / S;
             // the operand buffer is free once the MMAs of its last use have retired
-            ok = wait_bounded_idle(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
+            ok = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             uint8_t *stage = gen_base + st * C::kStageBytes;
@@ -744,7 +744,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     if (kb + 1 < kb1)
                         h_next = __fmul_rn(0.5f, P.scales[(size_t)(kb + 1) * P.L.n_pad + n]);
                     const uint32_t buf = phase % NB;
-                    ok = wait_bounded_idle(bar_acc_full + 8 * buf, (phase / NB) & 1u, ctl, P.sb, 41);
+                    ok = wait_bounded(bar_acc_full + 8 * buf, (phase / NB) & 1u, ctl, P.sb, 41);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after();
