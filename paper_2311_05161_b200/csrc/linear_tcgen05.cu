@@ -738,11 +738,12 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 float usum[C::kColsPerThread];
 #pragma unroll
                 for (int j = 0; j < C::kColsPerThread; ++j) usum[j] = 0.0f;
-                float h_next = __fmul_rn(0.5f, P.scales[(size_t)kb0 * P.L.n_pad + n]);
+                // the next group's step is loaded one k-block ahead and only touched when used,
+                // so the warp never stalls on that load
+                float step_next = P.scales[(size_t)kb0 * P.L.n_pad + n];
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    const float h = h_next;
-                    if (kb + 1 < kb1)
-                        h_next = __fmul_rn(0.5f, P.scales[(size_t)(kb + 1) * P.L.n_pad + n]);
+                    const float h = __fmul_rn(0.5f, step_next);
+                    if (kb + 1 < kb1) step_next = P.scales[(size_t)(kb + 1) * P.L.n_pad + n];
                     const uint32_t buf = phase % NB;
                     ok = wait_bounded(bar_acc_full + 8 * buf, (phase / NB) & 1u, ctl, P.sb, 41);
                     ok = __all_sync(0xffffffffu, ok);
