@@ -31,6 +31,9 @@ namespace {
 constexpr int kFirstDecodeWarp = 2;
 constexpr int kABytes = kTileN * kTileK;            // decoded INT8 tile, 16 KiB
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+// how long a waiting thread may stay suspended in hardware before it polls again (it is woken
+// at once when the barrier phase completes); keeps waiting warps out of the issue slots
+constexpr uint32_t kSuspendHintNs = 20000u;
 constexpr unsigned long long kDrainLimitNs = 200000000ull;
 
 template <int TOK, bool GROUPED, int DW>
@@ -118,10 +121,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     return ok != 0;
 }
@@ -273,7 +276,7 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Ctl 
     unsigned long long t0 = 0;
     for (uint32_t i = 1;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 1023u) == 0u) {
+        if ((i & 63u) == 0u) {
             if (ctl->abort) return false;
             if (t0 == 0) {
                 t0 = global_ns();
