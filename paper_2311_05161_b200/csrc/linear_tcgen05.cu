@@ -53,18 +53,26 @@ struct Cfg {
     // bandwidth and capacity are the scarce resources); for weight-streaming shapes the
     // producer thread runs ahead with L2 prefetches of the code tiles.
     static constexpr int kTeams = DW / 4;              // teams of 4 warps take k-blocks in turn
-    static constexpr int kStageBytes = kABytes + kTokBytes;
+    // The decoded weights (operand A) live in tensor memory when there is room beside the
+    // accumulators: they are then written with tcgen05.st and read by the MMA without touching
+    // shared memory, whose bandwidth (operand reads + TMA writes + decode stores) is the
+    // limiter of the wide tiles.  Otherwise they go through the shared-memory stage.
+    static constexpr bool kATmem = !GROUPED && TOK <= 192;
+    static constexpr int kASlots = 4;                  // operand-A buffers of 32 columns each
+    static constexpr int kStageBytes = (kATmem ? 0 : kABytes) + kTokBytes;
+    static constexpr int kTokOff = kATmem ? 0 : kABytes;   // tokens inside a stage
     static constexpr int kPrefetchAhead = 16;          // k-blocks of codes requested into L2
     // output staging: two buffers of kChunk tokens x 128 features BF16 per epilogue group
     static constexpr int kStagingBytes = kEpiGroups * kStageBufs * kChunk * kTileN * 2;
     static constexpr int kTailBytes = kStagingBytes + 1024 /* token steps */ + 1024 /* barriers */;
     static constexpr int kMaxStages = (232448 - 1024 - kTailBytes) / kStageBytes;
-    static constexpr int kStages = kMaxStages > 7 ? 7 : kMaxStages;
+    static constexpr int kStages = kMaxStages > 8 ? 8 : kMaxStages;
     // accumulator buffers in tensor memory: two for per-channel weights (epilogue of one unit
     // overlaps the main loop of the next); group mode hands over every k-block, and a hand-over
     // costs several hundred cycles of latency, so it rotates over as many buffers as fit
     static constexpr int kAccBufs = !GROUPED ? 2 : (512 / TOK > 8 ? 8 : 512 / TOK);
-    static constexpr int kTmemNeed = kAccBufs * TOK;
+    static constexpr int kAColBase = kAccBufs * TOK;   // first operand-A column
+    static constexpr int kTmemNeed = kAccBufs * TOK + (kATmem ? kASlots * 32 : 0);
     static constexpr int kTmemCols = kTmemNeed <= 32 ? 32 : kTmemNeed <= 64 ? 64 : kTmemNeed <= 128 ? 128
                                      : kTmemNeed <= 256 ? 256 : 512;
     static constexpr int kOffStaging = kStages * kStageBytes;
@@ -72,6 +80,8 @@ struct Cfg {
     static constexpr int kOffBarriers = kOffTok + 1024;
     static constexpr int kSmemBytes = kOffBarriers + 1024 + 1024 /* alignment slack */;
     static_assert(kStages >= 3, "pipeline depth");
+    static_assert(!kATmem || kStages > kASlots, "a stage outlives an operand-A buffer");
+    static_assert(kTmemNeed <= 512, "tensor memory budget");
     static_assert(kSmemBytes <= 232448, "shared memory budget");
     static_assert(!GROUPED || TOK <= 128, "group mode keeps its FP32 sums in registers");
 };
@@ -189,6 +199,34 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint
         "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
         "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
+}
+// A from tensor memory, B from shared memory
+__device__ __forceinline__ void tc_mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
+                                             uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]),
+        "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
+        "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_st()
+{
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
 {
@@ -423,7 +461,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_dec + 8 * s, 4);
+            mbar_init(bar_dec + 8 * s, 4);   // indexed by stage, or by operand-A slot
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int b = 0; b < NB; ++b) {
@@ -471,7 +509,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     }
                     const uint32_t stage = base + st * C::kStageBytes;
                     mbar_arrive_expect_tx(bar_full + 8 * st, C::kTokBytes);
-                    tma_load_2d(stage + kABytes, &tok_map, kb * kTileK, tt * TOK,
+                    tma_load_2d(stage + C::kTokOff, &tok_map, kb * kTileK, tt * TOK,
                                 bar_full + 8 * st);
                     if (P.prefetch_codes) {
                         // keep the code stream kPrefetchAhead k-blocks ahead of the decode warps
@@ -515,7 +553,10 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         ok = false;
                         break;
                     }
-                    if (!wait_bounded(bar_dec + 8 * st, fill & 1u, ctl, P.sb, 21) ||
+                    // decoded weights: per stage in shared memory, or per slot in tensor memory
+                    const int aslot = C::kATmem ? (int)(it % C::kASlots) : st;
+                    const uint32_t afill = C::kATmem ? it / C::kASlots : fill;
+                    if (!wait_bounded(bar_dec + 8 * aslot, afill & 1u, ctl, P.sb, 21) ||
                         !wait_bounded(bar_full + 8 * st, fill & 1u, ctl, P.sb, 23)) {
                         ok = false;
                         break;
@@ -525,9 +566,13 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     const uint32_t d = tmem_base + buf * TOK;
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
-                        tc_mma_i8(d, smem_desc_sw128(stage + ks * 32),
-                                  smem_desc_sw128(stage + kABytes + ks * 32), idesc,
-                                  (!first || ks > 0) ? 1u : 0u);
+                        const uint32_t acc_flag = (!first || ks > 0) ? 1u : 0u;
+                        if (C::kATmem)
+                            tc_mma_i8_ts(d, tmem_base + C::kAColBase + aslot * 32 + ks * 8,
+                                         smem_desc_sw128(stage + C::kTokOff + ks * 32), idesc, acc_flag);
+                        else
+                            tc_mma_i8(d, smem_desc_sw128(stage + ks * 32),
+                                      smem_desc_sw128(stage + C::kTokOff + ks * 32), idesc, acc_flag);
                     }
                     tc_commit(bar_empty + 8 * st);
                     if (last) {
@@ -547,7 +592,9 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         // so the fixed latency of one k-block (barrier wait, loads, proxy fence, arrive)
         // overlaps the table lookups of the other teams.
         const int dt = threadIdx.x - 32 * kFirstDecodeWarp;
-        const int r = dt & 127;                                  // feature row in the tile
+        // row r of the tile; with the operand in tensor memory a warp may only touch the lane
+        // quarter (warp index mod 4), so rows follow the warp index there
+        const int r = C::kATmem ? ((warp & 3) * 32 + lane) : (dt & 127);
         const int team = dt >> 7;
         constexpr int T = C::kTeams;
         KbCursor cur;
@@ -574,29 +621,56 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             if (nxt.valid()) fetch(nxt, wn, zn);                 // prefetch the team's next k-block
             const int st = cur.it % S;
             const uint32_t fill = cur.it / S;
-            // the operand buffer is free once the MMAs of its last use have retired
-            ok = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            uint8_t *stage = gen_base + st * C::kStageBytes;
-            uint8_t *arow = stage + r * 128;
-            const int sw = r & 7;
             uint32_t t[4];
             build_tables(z, t);
+            if (C::kATmem) {
+                // The operand-A slot is free once the MMAs of the k-block that used it last
+                // (kASlots k-blocks ago) have retired: that is the stage barrier of that k-block.
+                const int aslot = cur.it % C::kASlots;
+                if (cur.it >= (uint32_t)C::kASlots) {
+                    const uint32_t j = cur.it - C::kASlots;
+                    ok = wait_bounded(bar_empty + 8 * (j % S), (j / S) & 1u, ctl, P.sb, 32);
+                }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                uint32_t a[32];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint4 wq = w[q];
-                uint4 c0, c1;
-                decode8(wq.x, t, c0.x, c0.y);
-                decode8(wq.y, t, c0.z, c0.w);
-                decode8(wq.z, t, c1.x, c1.y);
-                decode8(wq.w, t, c1.z, c1.w);
-                *reinterpret_cast<uint4 *>(arow + (((2 * q) ^ sw) << 4)) = c0;
-                *reinterpret_cast<uint4 *>(arow + (((2 * q + 1) ^ sw) << 4)) = c1;
+                for (int q = 0; q < 4; ++q) {
+                    const uint4 wq = w[q];
+                    decode8(wq.x, t, a[8 * q + 0], a[8 * q + 1]);
+                    decode8(wq.y, t, a[8 * q + 2], a[8 * q + 3]);
+                    decode8(wq.z, t, a[8 * q + 4], a[8 * q + 5]);
+                    decode8(wq.w, t, a[8 * q + 6], a[8 * q + 7]);
+                }
+                // lane = row, 32 columns of four INT8 each = the 128 k of this k-block
+                tc_st32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + C::kAColBase + aslot * 32, a);
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_dec + 8 * aslot);
+            } else {
+                // the operand buffer is free once the MMAs of its last use have retired
+                ok = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                uint8_t *stage = gen_base + st * C::kStageBytes;
+                uint8_t *arow = stage + r * 128;
+                const int sw = r & 7;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint4 wq = w[q];
+                    uint4 c0, c1;
+                    decode8(wq.x, t, c0.x, c0.y);
+                    decode8(wq.y, t, c0.z, c0.w);
+                    decode8(wq.z, t, c1.x, c1.y);
+                    decode8(wq.w, t, c1.z, c1.w);
+                    *reinterpret_cast<uint4 *>(arow + (((2 * q) ^ sw) << 4)) = c0;
+                    *reinterpret_cast<uint4 *>(arow + (((2 * q + 1) ^ sw) << 4)) = c1;
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_dec + 8 * st);
             }
-            fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_dec + 8 * st);
 #pragma unroll
             for (int q = 0; q < 4; ++q) w[q] = wn[q];
             z = zn;
