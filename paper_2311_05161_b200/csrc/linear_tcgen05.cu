@@ -534,51 +534,58 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
+            // This loop is the serial spine of the kernel (one thread, once per k-block): all
+            // counters are kept incrementally and the descriptors are an add away.
             constexpr uint32_t idesc = instr_desc_i8(TOK);
-            uint32_t it = 0, phase = 0;
+            constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+            const uint32_t a_lo0 = ((base & 0x3FFFFu) >> 4) | (1u << 16);
+            const uint32_t b_lo0 = (((base + C::kTokOff) & 0x3FFFFu) >> 4) | (1u << 16);
+            uint32_t st = 0, st_par = 0;                 // stage and its fill parity
+            uint32_t as = 0, as_par = 0;                 // operand-A slot and its parity
+            uint32_t buf = 0, buf_par = 0;               // accumulator buffer and its parity
             bool ok = true;
             for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
                 const int s = u % P.split_k;
                 const int kb0 = s * P.kb_per_split;
-                const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
-                for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                    const int st = it % S;
-                    const uint32_t fill = it / S;
-                    const bool first = GROUPED || kb == kb0;
-                    const bool last = GROUPED || kb == kb1 - 1;
-                    const uint32_t buf = phase % NB;
+                const int nkb = min(k_blocks, kb0 + P.kb_per_split) - kb0;
+                for (int i = 0; i < nkb; ++i) {
+                    const bool first = GROUPED || i == 0;
+                    const bool last = GROUPED || i == nkb - 1;
                     if (first &&
-                        !wait_bounded(bar_acc_empty + 8 * buf, ((phase / NB) & 1u) ^ 1u, ctl, P.sb,
-                                      20)) {
+                        !wait_bounded(bar_acc_empty + 8 * buf, buf_par ^ 1u, ctl, P.sb, 20)) {
                         ok = false;
                         break;
                     }
                     // decoded weights: per stage in shared memory, or per slot in tensor memory
-                    const int aslot = C::kATmem ? (int)(it % C::kASlots) : st;
-                    const uint32_t afill = C::kATmem ? it / C::kASlots : fill;
-                    if (!wait_bounded(bar_dec + 8 * aslot, afill & 1u, ctl, P.sb, 21) ||
-                        !wait_bounded(bar_full + 8 * st, fill & 1u, ctl, P.sb, 23)) {
+                    const uint32_t dslot = C::kATmem ? as : st;
+                    const uint32_t dpar = C::kATmem ? as_par : st_par;
+                    if (!wait_bounded(bar_dec + 8 * dslot, dpar, ctl, P.sb, 21) ||
+                        !wait_bounded(bar_full + 8 * st, st_par, ctl, P.sb, 23)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t stage = base + st * C::kStageBytes;
                     const uint32_t d = tmem_base + buf * TOK;
+                    const uint32_t soff = st * (C::kStageBytes >> 4);
+                    const uint64_t a_desc = ((uint64_t)kDescHi << 32) | (a_lo0 + soff);
+                    const uint64_t b_desc = ((uint64_t)kDescHi << 32) | (b_lo0 + soff);
+                    const uint32_t a_tm = tmem_base + C::kAColBase + as * 32;
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
                         const uint32_t acc_flag = (!first || ks > 0) ? 1u : 0u;
                         if (C::kATmem)
-                            tc_mma_i8_ts(d, tmem_base + C::kAColBase + aslot * 32 + ks * 8,
-                                         smem_desc_sw128(stage + C::kTokOff + ks * 32), idesc, acc_flag);
+                            tc_mma_i8_ts(d, a_tm + ks * 8, b_desc + (uint64_t)(ks * 2), idesc, acc_flag);
                         else
-                            tc_mma_i8(d, smem_desc_sw128(stage + ks * 32),
-                                      smem_desc_sw128(stage + C::kTokOff + ks * 32), idesc, acc_flag);
+                            tc_mma_i8(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
+                                      acc_flag);
                     }
                     tc_commit(bar_empty + 8 * st);
                     if (last) {
                         tc_commit(bar_acc_full + 8 * buf);
-                        ++phase;
+                        if (++buf == (uint32_t)NB) { buf = 0; buf_par ^= 1u; }
                     }
+                    if (++st == (uint32_t)S) { st = 0; st_par ^= 1u; }
+                    if (++as == (uint32_t)C::kASlots) { as = 0; as_par ^= 1u; }
                 }
             }
             // nothing issued may still be running when tensor memory is freed
