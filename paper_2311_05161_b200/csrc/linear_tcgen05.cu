@@ -461,7 +461,9 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_dec + 8 * s, 4);   // indexed by stage, or by operand-A slot
+            // per operand-A slot in tensor-memory mode (4 decode warps); per stage otherwise, where the
+            // token copy completes on the same barrier (4 decode warps + the producer's arrival)
+            mbar_init(bar_dec + 8 * s, C::kATmem ? 4 : 5);
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int b = 0; b < NB; ++b) {
@@ -508,9 +510,9 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         break;
                     }
                     const uint32_t stage = base + st * C::kStageBytes;
-                    mbar_arrive_expect_tx(bar_full + 8 * st, C::kTokBytes);
-                    tma_load_2d(stage + C::kTokOff, &tok_map, kb * kTileK, tt * TOK,
-                                bar_full + 8 * st);
+                    const uint32_t tok_bar = C::kATmem ? bar_full + 8 * st : bar_dec + 8 * st;
+                    mbar_arrive_expect_tx(tok_bar, C::kTokBytes);
+                    tma_load_2d(stage + C::kTokOff, &tok_map, kb * kTileK, tt * TOK, tok_bar);
                     if (P.prefetch_codes) {
                         // keep the code stream kPrefetchAhead k-blocks ahead of the decode warps
                         while (pf.valid() && pf.it < it + C::kPrefetchAhead) {
@@ -526,8 +528,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 // copies already issued must land before the CTA gives its memory back
                 const uint32_t first = it > (uint32_t)S ? it - S : 0u;
                 for (uint32_t j = first; j < it; ++j)
-                    wait_bounded(bar_full + 8 * (j % S), (j / S) & 1u, ctl, P.sb, 11,
-                                 kDrainLimitNs);
+                    wait_bounded((C::kATmem ? bar_full : bar_dec) + 8 * (j % S), (j / S) & 1u, ctl,
+                                 P.sb, 11, kDrainLimitNs);
             }
         }
         __syncwarp();
@@ -560,7 +562,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     const uint32_t dslot = C::kATmem ? as : st;
                     const uint32_t dpar = C::kATmem ? as_par : st_par;
                     if (!wait_bounded(bar_dec + 8 * dslot, dpar, ctl, P.sb, 21) ||
-                        !wait_bounded(bar_full + 8 * st, st_par, ctl, P.sb, 23)) {
+                        (C::kATmem && !wait_bounded(bar_full + 8 * st, st_par, ctl, P.sb, 23))) {
                         ok = false;
                         break;
                     }
