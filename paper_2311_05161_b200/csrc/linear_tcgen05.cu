@@ -982,6 +982,7 @@ w4a8_status launch_one(const Maps &maps, const Params &P, int dw, cudaStream_t s
 {
     if (dw == 4) return launch_dw<TOK, GROUPED, 4>(maps, P, st);
     if (dw == 8) return launch_dw<TOK, GROUPED, 8>(maps, P, st);
+    if (dw == 12 && !GROUPED) return launch_dw<TOK, false, 12>(maps, P, st);
     if (dw == 16 && !GROUPED) return launch_dw<TOK, false, 16>(maps, P, st);
     return W4A8_ERR_SHAPE;
 }
@@ -1018,7 +1019,7 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     if (tiles * split > 0x7fffffffLL) return false;
     int dw = opts ? opts->decode_warps : 0;
     if (dw == 0) dw = grouped ? 8 : 16;
-    if (dw != 4 && dw != 8 && !(dw == 16 && !grouped)) return false;
+    if (dw != 4 && dw != 8 && !((dw == 12 || dw == 16) && !grouped)) return false;
     plan->decode_warps = dw;
     plan->tok_tile = tok;
     plan->tok_tiles = tok_tiles;
