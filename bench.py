@@ -157,11 +157,12 @@ def run_reference(args):
     sample = f"first {CPU_SAMPLE_TOKENS} of {M_PREFILL} tokens of each of the 4 linears per step"
     line = {
         "impl": "reference", "metric": "w4a8_dint_linear_tops", "value": tops, "unit": "TOPS",
-        "n_gpus": 0, "steps": args.steps, "warmup": args.warmup,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * total_t / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-        "config": {"workload": "opt-6.7b block linears, M=2048 prefill (CPU sample)",
-                   "sample": sample},
+        "config": {"workload": "opt-6.7b block linears (qkv 4096->12288, out 4096->4096, "
+                               "fc1 4096->16384, fc2 16384->4096), M=2048 prefill, per-channel dINT4",
+                   "step": "CPU oracle on a bounded sample of the same step", "sample": sample},
         "cpu_baseline": {"value": tops, "unit": "TOPS", "cores": oracle.get_threads(),
                          "kind": "oracle", "sample": sample},
         "e2e": {"value": tops, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
