@@ -68,7 +68,9 @@ struct Cfg {
     // shared memory, whose bandwidth (operand reads + TMA writes + decode stores) is the
     // limiter of the wide tiles.  Otherwise they go through the shared-memory stage.
     static constexpr bool kATmem = !GROUPED && TOK <= 192;
-    static constexpr int kASlots = 4;                  // operand-A buffers of 32 columns each
+    // operand-A buffers of 32 columns each: as many as fit beside the two accumulators
+    static constexpr int kASlotsFit = (512 - 2 * TOK) / 32;
+    static constexpr int kASlots = !kATmem ? 4 : (kASlotsFit > 8 ? 8 : kASlotsFit);
     static constexpr int kStageBytes = (kATmem ? 0 : kABytes) + kTokBytes;
     static constexpr int kTokOff = kATmem ? 0 : kABytes;   // tokens inside a stage
     static constexpr int kPrefetchAhead = 16;          // k-blocks of codes requested into L2
