@@ -45,17 +45,7 @@ struct Cfg {
     static constexpr int kEpiGroups = !GROUPED ? 1 : (TOK >= 128 ? 4 : TOK >= 64 ? 2 : 1);
     static constexpr int kStageBufs = GROUPED ? 1 : 2;      // output staging buffers per group
     static constexpr int kEpiWarps = 4 * kEpiGroups;
-    // Warp layout.  A warp runs on scheduler (warp index mod 4).  The producer and MMA threads
-    // are the serial spine of the pipeline and starve when they share a scheduler with busy
-    // decode warps, so in the "spine" layout scheduler 0 only hosts them (warps 0 and 4) and
-    // one light epilogue warp per column group; decode warps and the other epilogue warps
-    // take the indices that are not multiples of four.  The tensor-memory operand path needs
-    // decode warps on all four lane quarters and keeps the plain layout.
-    static constexpr bool kSpine = !GROUPED && TOK > 192;
-    static constexpr int kSpineRowsA = 2 + kEpiGroups;                       // scheduler-0 column
-    static constexpr int kSpineRowsB = (DW + 3 * kEpiGroups + 2) / 3;        // the other three
-    static constexpr int kSpineRows = kSpineRowsA > kSpineRowsB ? kSpineRowsA : kSpineRowsB;
-    static constexpr int kThreads = kSpine ? 128 * kSpineRows : 32 * (kFirstEpiWarp + kEpiWarps);
+    static constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
     static constexpr int kColsPerThread = TOK / kEpiGroups;
     static constexpr int kChunk = kColsPerThread >= 32 ? 32 : 16;
     static constexpr int kTokBytes = TOK * kTileK;
@@ -469,25 +459,6 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     Ctl *ctl = reinterpret_cast<Ctl *>(gen_base + C::kOffBarriers + 24 * S + 16 * NB + 16);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // role of this warp: 0 producer, 1 MMA, 2 decode (index di), 3 epilogue (index ei =
-    // 4 * column group + lane quarter), 4 none
-    int role, di = 0, ei = 0;
-    if (C::kSpine) {
-        const int res = warp & 3, row = warp >> 2;
-        if (res == 0) {
-            role = row == 0 ? 0 : row == 1 ? 1 : (row < 2 + C::kEpiGroups ? 3 : 4);
-            ei = (row - 2) * 4;
-        } else {
-            const int slot = row * 3 + res - 1;
-            if (slot < DW) { role = 2; di = slot; }
-            else if (slot < DW + 3 * C::kEpiGroups) { role = 3; ei = ((slot - DW) / 3) * 4 + res; }
-            else role = 4;
-        }
-    } else {
-        role = warp == 0 ? 0 : warp == 1 ? 1 : warp < kFirstEpiWarp ? 2 : 3;
-        di = warp - kFirstDecodeWarp;
-        ei = ((warp - kFirstEpiWarp) >> 2) * 4 + (warp & 3);
-    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -507,7 +478,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
-    if (role == 1) {
+    if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                          smem_u32(&ctl->tmem_base)),
                      "r"((uint32_t)C::kTmemCols)
@@ -521,7 +492,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
 
     const int n_tiles = P.L.n_tiles, k_blocks = P.L.k_blocks;
 
-    if (role == 0) {
+    if (warp == 0) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
             uint32_t it = 0;
@@ -564,7 +535,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             }
         }
         __syncwarp();
-    } else if (role == 1) {
+    } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             // This loop is the serial spine of the kernel (one thread, once per k-block): all
@@ -626,12 +597,12 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             wait_bounded(bar_drain, 0u, ctl, P.sb, 22, ok ? kWaitLimitNs : kDrainLimitNs);
         }
         __syncwarp();
-    } else if (role == 2) {
+    } else if (warp < kFirstEpiWarp) {
         // ------------------------------------------------------------------ decode warps
         // Four warps (one thread per feature row) form a team; teams take k-blocks in turn,
         // so the fixed latency of one k-block (barrier wait, loads, proxy fence, arrive)
         // overlaps the table lookups of the other teams.
-        const int dt = di * 32 + lane;
+        const int dt = threadIdx.x - 32 * kFirstDecodeWarp;
         // row r of the tile; with the operand in tensor memory a warp may only touch the lane
         // quarter (warp index mod 4), so rows follow the warp index there
         const int r = C::kATmem ? ((warp & 3) * 32 + lane) : (dt & 127);
@@ -716,15 +687,16 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             z = zn;
             cur = nxt;
         }
-    } else if (role == 3) {
+    } else {
         // ------------------------------------------------------------------ epilogue warps
+        const int ew = warp - kFirstEpiWarp;
         const int quarter = warp & 3;                     // tensor-memory lane quarter
-        const int col_group = ei >> 2;                    // which share of the columns
+        const int col_group = ew >> 2;                    // which share of the columns
         const int col0 = col_group * C::kColsPerThread;
         const int f = quarter * 32 + lane;                // feature row inside the tile
         constexpr int kEpiThreads = 32 * C::kEpiWarps;
-        const int et = ei * 32 + lane;                    // index among the epilogue threads
-        const bool elected = quarter == 0 && lane == 0;   // issues this group's bulk stores
+        const int et = threadIdx.x - 32 * kFirstEpiWarp;
+        const bool elected = et == col_group * 128;       // issues this group's bulk stores
         const int group_bar = 2 + col_group;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         float *s_tok = reinterpret_cast<float *>(gen_base + C::kOffTok);
@@ -945,7 +917,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     // ---------------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
-    if (role == 1) {
+    if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                      "r"((uint32_t)C::kTmemCols)
