@@ -68,7 +68,7 @@ struct Cfg {
     static constexpr int kStagingBytes = kEpiGroups * kStageBufs * kChunk * kTileN * 2;
     static constexpr int kTailBytes = kStagingBytes + 1024 /* token steps */ + 1024 /* barriers */;
     static constexpr int kMaxStages = (232448 - 1024 - kTailBytes) / kStageBytes;
-    static constexpr int kStages = kMaxStages > 8 ? 8 : kMaxStages;
+    static constexpr int kStages = kMaxStages > 9 ? 9 : kMaxStages;
     // accumulator buffers in tensor memory: two for per-channel weights (epilogue of one unit
     // overlaps the main loop of the next); group mode hands over every k-block, and a hand-over
     // costs several hundred cycles of latency, so it rotates over as many buffers as fit
