@@ -548,19 +548,10 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             uint32_t as = 0, as_par = 0;                 // operand-A slot and its parity
             uint32_t buf = 0, buf_par = 0;               // accumulator buffer and its parity
             bool ok = true;
-            // operands of the k-block at (stage st, slot as) are in place
-            auto operands_ready = [&](uint32_t s_, uint32_t sp_, uint32_t a_, uint32_t ap_) {
-                const uint32_t dslot = C::kATmem ? a_ : s_;
-                const uint32_t dpar = C::kATmem ? ap_ : sp_;
-                return wait_bounded(bar_dec + 8 * dslot, dpar, ctl, P.sb, 21) &&
-                       (!C::kATmem || wait_bounded(bar_full + 8 * s_, sp_, ctl, P.sb, 23));
-            };
-            bool have = false;                           // operands of the coming k-block checked
             for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
                 const int s = u % P.split_k;
                 const int kb0 = s * P.kb_per_split;
                 const int nkb = min(k_blocks, kb0 + P.kb_per_split) - kb0;
-                const bool more_units = u + (int)gridDim.x < P.total_units;
                 for (int i = 0; i < nkb; ++i) {
                     const bool first = GROUPED || i == 0;
                     const bool last = GROUPED || i == nkb - 1;
@@ -569,7 +560,11 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         ok = false;
                         break;
                     }
-                    if (!have && !operands_ready(st, st_par, as, as_par)) {
+                    // decoded weights: per stage in shared memory, or per slot in tensor memory
+                    const uint32_t dslot = C::kATmem ? as : st;
+                    const uint32_t dpar = C::kATmem ? as_par : st_par;
+                    if (!wait_bounded(bar_dec + 8 * dslot, dpar, ctl, P.sb, 21) ||
+                        (C::kATmem && !wait_bounded(bar_full + 8 * st, st_par, ctl, P.sb, 23))) {
                         ok = false;
                         break;
                     }
@@ -579,35 +574,22 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     const uint64_t a_desc = ((uint64_t)kDescHi << 32) | (a_lo0 + soff);
                     const uint64_t b_desc = ((uint64_t)kDescHi << 32) | (b_lo0 + soff);
                     const uint32_t a_tm = tmem_base + C::kAColBase + as * 32;
-                    auto issue = [&](int ks) {
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
                         const uint32_t acc_flag = (!first || ks > 0) ? 1u : 0u;
                         if (C::kATmem)
                             tc_mma_i8_ts(d, a_tm + ks * 8, b_desc + (uint64_t)(ks * 2), idesc, acc_flag);
                         else
                             tc_mma_i8(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
                                       acc_flag);
-                    };
-                    issue(0);
-                    issue(1);
-                    // While those two run, look at the next k-block's barriers: the wait (and the
-                    // loop bookkeeping) then overlaps queued tensor work instead of idling the pipe.
-                    uint32_t nst = st + 1, nsp = st_par, nas = as + 1, nap = as_par;
-                    if (nst == (uint32_t)S) { nst = 0; nsp ^= 1u; }
-                    if (nas == (uint32_t)C::kASlots) { nas = 0; nap ^= 1u; }
-                    have = false;
-                    if (i + 1 < nkb || more_units) {
-                        if (!operands_ready(nst, nsp, nas, nap)) ok = false;
-                        have = ok;
                     }
-                    issue(2);
-                    issue(3);
                     tc_commit(bar_empty + 8 * st);
                     if (last) {
                         tc_commit(bar_acc_full + 8 * buf);
                         if (++buf == (uint32_t)NB) { buf = 0; buf_par ^= 1u; }
                     }
-                    st = nst; st_par = nsp; as = nas; as_par = nap;
-                    if (!ok) break;
+                    if (++st == (uint32_t)S) { st = 0; st_par ^= 1u; }
+                    if (++as == (uint32_t)C::kASlots) { as = 0; as_par ^= 1u; }
                 }
             }
             // nothing issued may still be running when tensor memory is freed
