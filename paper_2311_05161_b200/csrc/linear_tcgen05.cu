@@ -259,6 +259,42 @@ __device__ __forceinline__ void tc_wait_ld()
 {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+
+// Two FP32 values in one 64-bit register for the packed FP32 instructions.
+__device__ __forceinline__ uint64_t pack_f32x2(uint32_t lo, uint32_t hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float &lo, float &hi)
+{
+    uint32_t a, b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+    lo = __uint_as_float(a);
+    hi = __uint_as_float(b);
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+// A group's INT32 partial sum is below 2^22 in magnitude (128 products of at most 127 * 26), so
+// its low 23 bits with bit 22 flipped, under the exponent of 2^23, are the FP32 number
+// 1.5 * 2^23 + sum: one logic instruction instead of a conversion, which runs at an eighth of
+// the FP32 rate.  Subtracting 1.5 * 2^23 afterwards is exact.
+constexpr uint32_t kMagicBits = 0x4B400000u;          // 1.5 * 2^23 = 12582912.0f
+__device__ __forceinline__ uint32_t biased_float_bits(uint32_t acc)
+{
+    return (acc & 0x007FFFFFu) ^ kMagicBits;
+}
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 {
     uint32_t d;
@@ -823,14 +859,21 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     }
                 }
             } else {
-                float usum[C::kColsPerThread];
+                // FP32 sums over the groups, two tokens per 64-bit register: each k-block adds
+                // float(partial) * step/2 with one packed add and one packed fused multiply-add
+                // per pair (same roundings as the scalar fmaf)
+                uint64_t usum2[C::kColsPerThread / 2];
 #pragma unroll
-                for (int j = 0; j < C::kColsPerThread; ++j) usum[j] = 0.0f;
+                for (int j = 0; j < C::kColsPerThread / 2; ++j) usum2[j] = 0ull;
+                const uint32_t neg_magic = __float_as_uint(-12582912.0f);
+                const uint64_t neg_magic2 = pack_f32x2(neg_magic, neg_magic);
                 // the next group's step is loaded one k-block ahead and only touched when used,
                 // so the warp never stalls on that load
                 float step_next = P.scales[(size_t)kb0 * P.L.n_pad + n];
+                constexpr int kAcc = 16;          // columns per tensor-memory load while accumulating
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    const float h = __fmul_rn(0.5f, step_next);
+                    const uint32_t h_bits = __float_as_uint(__fmul_rn(0.5f, step_next));
+                    const uint64_t h2 = pack_f32x2(h_bits, h_bits);
                     if (kb + 1 < kb1) step_next = P.scales[(size_t)(kb + 1) * P.L.n_pad + n];
                     const uint32_t buf = phase % NB;
                     ok = wait_bounded(bar_acc_full + 8 * buf, (phase / NB) & 1u, ctl, P.sb, 41);
@@ -839,22 +882,26 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     tc_fence_after();
                     ++phase;
 #pragma unroll
-                    for (int c = 0; c < C::kColsPerThread; c += C::kChunk) {
+                    for (int c = 0; c < C::kColsPerThread; c += kAcc) {
                         uint32_t v[32];
                         const uint32_t taddr = tmem_base + lane_base + buf * TOK + col0 + c;
-                        if (C::kChunk == 32) tc_ld32(taddr, v); else tc_ld16(taddr, v);
+                        if (kAcc == 32) tc_ld32(taddr, v); else tc_ld16(taddr, v);
                         tc_wait_ld();
-                        if (c + C::kChunk >= C::kColsPerThread) {
+                        if (c + kAcc >= C::kColsPerThread) {
                             tc_fence_before();
                             __syncwarp();
                             if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
                         }
 #pragma unroll
-                        for (int j = 0; j < C::kChunk; ++j)
-                            usum[c + j] = fmaf((float)(int)v[j], h, usum[c + j]);
+                        for (int j = 0; j < kAcc; j += 2) {
+                            const uint64_t biased =
+                                pack_f32x2(biased_float_bits(v[j]), biased_float_bits(v[j + 1]));
+                            usum2[(c + j) >> 1] =
+                                fma_f32x2(add_f32x2(biased, neg_magic2), h2, usum2[(c + j) >> 1]);
+                        }
                         if (P.acc_out && n_ok) {
 #pragma unroll
-                            for (int j = 0; j < C::kChunk; ++j)
+                            for (int j = 0; j < kAcc; ++j)
                                 if (c + j < valid)
                                     P.acc_out[((size_t)kb * P.M + tok0 + c + j) * P.L.N + n] =
                                         (int)v[j];
@@ -863,6 +910,10 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 }
                 ok = named_bar_and(1, kEpiThreads, ok);
                 if (!ok) break;
+                float usum[C::kColsPerThread];
+#pragma unroll
+                for (int j = 0; j < C::kColsPerThread / 2; ++j)
+                    unpack_f32x2(usum2[j], usum[2 * j], usum[2 * j + 1]);
                 if (bulk_out) {
 #pragma unroll
                     for (int c = 0; c < C::kColsPerThread; c += C::kChunk) {
