@@ -28,7 +28,7 @@ namespace w4a8 {
 
 namespace {
 
-constexpr int kFirstDecodeWarp = 4;           // warp 0 producer, warps 1-2 MMA issuers, warp 3 spare
+constexpr int kFirstDecodeWarp = 2;
 constexpr int kABytes = kTileN * kTileK;            // decoded INT8 tile, 16 KiB
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 // how long a waiting thread may stay suspended in hardware before it polls again (it is woken
@@ -491,9 +491,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     constexpr int NB = C::kAccBufs;
     const uint32_t bar_acc_full = bar_base + 24 * S;          // NB
     const uint32_t bar_acc_empty = bar_acc_full + 8 * NB;     // NB
-    const uint32_t bar_unit = bar_acc_empty + 8 * NB;         // NB: a unit's first MMAs are queued
-    const uint32_t bar_drain = bar_unit + 8 * NB;             // 1
-    Ctl *ctl = reinterpret_cast<Ctl *>(gen_base + C::kOffBarriers + 24 * S + 24 * NB + 16);
+    const uint32_t bar_drain = bar_acc_empty + 8 * NB;        // 1
+    Ctl *ctl = reinterpret_cast<Ctl *>(gen_base + C::kOffBarriers + 24 * S + 16 * NB + 16);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -506,12 +505,10 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int b = 0; b < NB; ++b) {
-            // per-channel units are shared by the two issuing threads: each commits its own MMAs
-            mbar_init(bar_acc_full + 8 * b, GROUPED ? 1 : 2);
+            mbar_init(bar_acc_full + 8 * b, 1);
             mbar_init(bar_acc_empty + 8 * b, C::kEpiWarps);
-            mbar_init(bar_unit + 8 * b, 1);
         }
-        mbar_init(bar_drain, 2);
+        mbar_init(bar_drain, 1);
         ctl->abort = 0;
         ctl->is_last = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -574,21 +571,11 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             }
         }
         __syncwarp();
-    } else if (warp == 1 || warp == 2) {
-        // ------------------------------------------------------------------ MMA issuers
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            // Two threads on two schedulers issue alternate k-blocks.  The tensor pipe takes only
-            // a couple of MMAs ahead of the one it executes, so a single issuing thread leaves it
-            // idle while it commits, polls the next k-block's barriers and rebuilds descriptors
-            // (several hundred cycles of dependent instructions per k-block); with two threads that
-            // bookkeeping overlaps the other thread's MMAs.  Integer accumulation commutes, so the
-            // only order that matters inside a per-channel unit is that its first MMA (the one that
-            // overwrites the accumulator) is queued first: thread 0 owns the even k-blocks of every
-            // unit and announces the unit on bar_unit once those MMAs are issued; thread 1 waits
-            // for that before its first k-block of the unit.  Each thread commits its own MMAs to
-            // the stage barriers and to the accumulator barrier (two arrivals per unit).  Group mode
-            // hands a fresh accumulator to every k-block, so there the threads are independent.
-            const uint32_t me = (uint32_t)(warp - 1);
+            // This loop is the serial spine of the kernel (one thread, once per k-block): all
+            // counters are kept incrementally and the descriptors are an add away.
             constexpr uint32_t idesc = instr_desc_i8(TOK);
             constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
             const uint32_t a_lo0 = ((base & 0x3FFFFu) >> 4) | (1u << 16);
@@ -596,76 +583,49 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             uint32_t st = 0, st_par = 0;                 // stage and its fill parity
             uint32_t as = 0, as_par = 0;                 // operand-A slot and its parity
             uint32_t buf = 0, buf_par = 0;               // accumulator buffer and its parity
-            uint32_t turn = 0;                           // whose k-block it is in group mode
             bool ok = true;
             for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
                 const int s = u % P.split_k;
                 const int kb0 = s * P.kb_per_split;
                 const int nkb = min(k_blocks, kb0 + P.kb_per_split) - kb0;
-                for (int i = 0; i < nkb && ok; ++i) {
-                    const bool mine = GROUPED ? (turn == me) : (((uint32_t)i & 1u) == me);
-                    if (mine) {
-                        const bool first = GROUPED || i == 0;
-                        if (first &&
-                            !wait_bounded(bar_acc_empty + 8 * buf, buf_par ^ 1u, ctl, P.sb, 20)) {
-                            ok = false;
-                            break;
-                        }
-                        if (!GROUPED && i == 1 &&
-                            !wait_bounded(bar_unit + 8 * buf, buf_par, ctl, P.sb, 24)) {
-                            ok = false;
-                            break;
-                        }
-                        // decoded weights: per stage in shared memory, or per slot in tensor memory
-                        const uint32_t dslot = C::kATmem ? as : st;
-                        const uint32_t dpar = C::kATmem ? as_par : st_par;
-                        if (!wait_bounded(bar_dec + 8 * dslot, dpar, ctl, P.sb, 21) ||
-                            (C::kATmem && !wait_bounded(bar_full + 8 * st, st_par, ctl, P.sb, 23))) {
-                            ok = false;
-                            break;
-                        }
-                        tc_fence_after();
-                        const uint32_t d = tmem_base + buf * TOK;
-                        const uint32_t soff = st * (C::kStageBytes >> 4);
-                        const uint64_t a_desc = ((uint64_t)kDescHi << 32) | (a_lo0 + soff);
-                        const uint64_t b_desc = ((uint64_t)kDescHi << 32) | (b_lo0 + soff);
-                        const uint32_t a_tm = tmem_base + C::kAColBase + as * 32;
-#pragma unroll
-                        for (int ks = 0; ks < 4; ++ks) {
-                            const uint32_t acc_flag = (!first || ks > 0) ? 1u : 0u;
-                            if (C::kATmem)
-                                tc_mma_i8_ts(d, a_tm + ks * 8, b_desc + (uint64_t)(ks * 2), idesc,
-                                             acc_flag);
-                            else
-                                tc_mma_i8(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2),
-                                          idesc, acc_flag);
-                        }
-                        tc_commit(bar_empty + 8 * st);
-                        if (!GROUPED && i == 0) {
-                            tc_fence_before();
-                            mbar_arrive(bar_unit + 8 * buf);
-                        }
-                        // this thread's last k-block of the unit: its MMAs count towards "full"
-                        if (GROUPED || i + 2 >= nkb) tc_commit(bar_acc_full + 8 * buf);
+                for (int i = 0; i < nkb; ++i) {
+                    const bool first = GROUPED || i == 0;
+                    const bool last = GROUPED || i == nkb - 1;
+                    if (first &&
+                        !wait_bounded(bar_acc_empty + 8 * buf, buf_par ^ 1u, ctl, P.sb, 20)) {
+                        ok = false;
+                        break;
                     }
-                    if (GROUPED) {
+                    // decoded weights: per stage in shared memory, or per slot in tensor memory
+                    const uint32_t dslot = C::kATmem ? as : st;
+                    const uint32_t dpar = C::kATmem ? as_par : st_par;
+                    if (!wait_bounded(bar_dec + 8 * dslot, dpar, ctl, P.sb, 21) ||
+                        (C::kATmem && !wait_bounded(bar_full + 8 * st, st_par, ctl, P.sb, 23))) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t d = tmem_base + buf * TOK;
+                    const uint32_t soff = st * (C::kStageBytes >> 4);
+                    const uint64_t a_desc = ((uint64_t)kDescHi << 32) | (a_lo0 + soff);
+                    const uint64_t b_desc = ((uint64_t)kDescHi << 32) | (b_lo0 + soff);
+                    const uint32_t a_tm = tmem_base + C::kAColBase + as * 32;
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint32_t acc_flag = (!first || ks > 0) ? 1u : 0u;
+                        if (C::kATmem)
+                            tc_mma_i8_ts(d, a_tm + ks * 8, b_desc + (uint64_t)(ks * 2), idesc, acc_flag);
+                        else
+                            tc_mma_i8(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
+                                      acc_flag);
+                    }
+                    tc_commit(bar_empty + 8 * st);
+                    if (last) {
+                        tc_commit(bar_acc_full + 8 * buf);
                         if (++buf == (uint32_t)NB) { buf = 0; buf_par ^= 1u; }
-                        turn ^= 1u;
                     }
                     if (++st == (uint32_t)S) { st = 0; st_par ^= 1u; }
                     if (++as == (uint32_t)C::kASlots) { as = 0; as_par ^= 1u; }
-                }
-                if (!GROUPED && ok) {
-                    if (me == 1u && nkb == 1) {
-                        // nothing of this unit was mine: arrive once the unit is under way, so that
-                        // the arrival cannot be counted for an earlier use of the buffer
-                        if (!wait_bounded(bar_unit + 8 * buf, buf_par, ctl, P.sb, 25)) {
-                            ok = false;
-                            break;
-                        }
-                        mbar_arrive(bar_acc_full + 8 * buf);
-                    }
-                    if (++buf == (uint32_t)NB) { buf = 0; buf_par ^= 1u; }
                 }
             }
             // nothing issued may still be running when tensor memory is freed
@@ -673,8 +633,6 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             wait_bounded(bar_drain, 0u, ctl, P.sb, 22, ok ? kWaitLimitNs : kDrainLimitNs);
         }
         __syncwarp();
-    } else if (warp < kFirstDecodeWarp) {
-        // spare warp: keeps the decode and epilogue warps aligned to the tensor-memory lane quarters
     } else if (warp < kFirstEpiWarp) {
         // ------------------------------------------------------------------ decode warps
         // Four warps (one thread per feature row) form a team; teams take k-blocks in turn,
