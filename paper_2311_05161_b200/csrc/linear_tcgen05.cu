@@ -647,6 +647,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         KbCursor cur;
         cur.start(blockIdx.x, gridDim.x, P.total_units, P.split_k, P.kb_per_split, k_blocks);
         cur.advance(team);
+        uint4 w[4];
+        int z = 0;
         auto fetch = [&](const KbCursor &c, uint4 (&dst)[4], int &zz) {
             const int nt = (c.u / P.split_k) % n_tiles;
             const int n = nt * kTileN + r;
@@ -656,21 +658,14 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
 #pragma unroll
             for (int q = 0; q < 4; ++q) dst[q] = ld_stream(src + q * (kQuarterBytes / 16));
         };
-        // Codes are requested two of the team's k-blocks ahead of their use: a load from L2 or
-        // HBM under the traffic of 148 such CTAs takes longer than one turn of the team.  Three
-        // register sets rotate by name (the loop is unrolled by three), so no copy ever waits
-        // for a load that has just been issued.
-        KbCursor far = cur;                                  // the k-block being requested
-        uint4 w0[4], w1[4], w2[4];
-        int z0 = 0, z1 = 0, z2 = 0;
-        if (far.valid()) fetch(far, w0, z0);
-        far.advance(T);
-        if (far.valid()) fetch(far, w1, z1);
-        far.advance(T);
+        if (cur.valid()) fetch(cur, w, z);
         bool ok = true;
-        auto process = [&](const uint4 (&w)[4], const int z, uint4 (&wl)[4], int &zl) -> bool {
-            if (far.valid()) fetch(far, wl, zl);
-            far.advance(T);
+        while (cur.valid() && ok) {
+            KbCursor nxt = cur;
+            nxt.advance(T);
+            uint4 wn[4];
+            int zn = 0;
+            if (nxt.valid()) fetch(nxt, wn, zn);                 // prefetch the team's next k-block
             const int st = cur.it % S;
             const uint32_t fill = cur.it / S;
             uint32_t t[4];
@@ -684,7 +679,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     ok = wait_bounded(bar_empty + 8 * (j % S), (j / S) & 1u, ctl, P.sb, 32);
                 }
                 ok = __all_sync(0xffffffffu, ok);
-                if (!ok) return false;
+                if (!ok) break;
                 uint32_t a[32];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
@@ -704,7 +699,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 // the operand buffer is free once the MMAs of its last use have retired
                 ok = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
                 ok = __all_sync(0xffffffffu, ok);
-                if (!ok) return false;
+                if (!ok) break;
                 uint8_t *stage = gen_base + st * C::kStageBytes;
                 uint8_t *arow = stage + r * 128;
                 const int sw = r & 7;
@@ -723,13 +718,10 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_dec + 8 * st);
             }
-            cur.advance(T);
-            return true;
-        };
-        while (true) {
-            if (!cur.valid() || !process(w0, z0, w2, z2)) break;
-            if (!cur.valid() || !process(w1, z1, w0, z0)) break;
-            if (!cur.valid() || !process(w2, z2, w1, z1)) break;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) w[q] = wn[q];
+            z = zn;
+            cur = nxt;
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
