@@ -392,22 +392,25 @@ __device__ __forceinline__ bool wait_bounded_idle(uint32_t bar, uint32_t parity,
 // Position of a CTA in its list of k-blocks: units (token tile, row tile, K slice) are dealt
 // round-robin to the CTAs, each unit is a run of k-blocks, `it` counts k-blocks from zero.
 struct KbCursor {
-    int u, step, total_units, split_k, kb_per_split, k_blocks;
+    int u, step, total_units, split_k, kb_per_split, k_blocks, n_tiles;
     int kb, kb1;
+    int nt;                    // row tile of the unit (integer divisions happen once per unit)
     uint32_t it;
     __device__ __forceinline__ void open_unit()
     {
         if (u < total_units) {
-            const int s = u % split_k;
+            const int rest = u / split_k;
+            const int s = u - rest * split_k;
+            nt = rest % n_tiles;
             kb = s * kb_per_split;
             kb1 = min(k_blocks, kb + kb_per_split);
         }
     }
     __device__ __forceinline__ void start(int first, int stride, int total, int split, int per,
-                                          int kbs)
+                                          int kbs, int tiles)
     {
         u = first; step = stride; total_units = total; split_k = split; kb_per_split = per;
-        k_blocks = kbs; it = 0; kb = kb1 = 0;
+        k_blocks = kbs; n_tiles = tiles; it = 0; kb = kb1 = 0; nt = 0;
         open_unit();
     }
     __device__ __forceinline__ bool valid() const { return u < total_units; }
@@ -534,7 +537,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             uint32_t it = 0;
             bool ok = true;
             KbCursor pf;
-            pf.start(blockIdx.x, gridDim.x, P.total_units, P.split_k, P.kb_per_split, k_blocks);
+            pf.start(blockIdx.x, gridDim.x, P.total_units, P.split_k, P.kb_per_split, k_blocks, n_tiles);
             for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
                 const int s = u % P.split_k, rest = u / P.split_k;
                 const int tt = rest / n_tiles;
@@ -554,7 +557,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     if (P.prefetch_codes) {
                         // keep the code stream kPrefetchAhead k-blocks ahead of the decode warps
                         while (pf.valid() && pf.it < it + C::kPrefetchAhead) {
-                            const int pnt = (pf.u / P.split_k) % n_tiles;
+                            const int pnt = pf.nt;
                             prefetch_l2(P.codes + ((size_t)pnt * k_blocks + pf.kb) * kTileBytes,
                                         kTileBytes);
                             pf.advance(1);
@@ -645,12 +648,12 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         const int team = dt >> 7;
         constexpr int T = C::kTeams;
         KbCursor cur;
-        cur.start(blockIdx.x, gridDim.x, P.total_units, P.split_k, P.kb_per_split, k_blocks);
+        cur.start(blockIdx.x, gridDim.x, P.total_units, P.split_k, P.kb_per_split, k_blocks, n_tiles);
         cur.advance(team);
         uint4 w[4];
         int z = 0;
         auto fetch = [&](const KbCursor &c, uint4 (&dst)[4], int &zz) {
-            const int nt = (c.u / P.split_k) % n_tiles;
+            const int nt = c.nt;
             const int n = nt * kTileN + r;
             zz = GROUPED ? P.zeros[(size_t)c.kb * P.L.n_pad + n] : P.zeros[n];
             const uint4 *src = reinterpret_cast<const uint4 *>(
