@@ -416,11 +416,6 @@ struct KbCursor {
     __device__ __forceinline__ bool valid() const { return u < total_units; }
     __device__ __forceinline__ void advance(int n)
     {
-        if (valid() && kb + n < kb1) {       // stays inside the unit: the common case
-            kb += n;
-            it += (uint32_t)n;
-            return;
-        }
         for (int i = 0; i < n && valid(); ++i) {
             ++it;
             if (++kb >= kb1) {
@@ -435,13 +430,6 @@ struct KbCursor {
 __device__ __forceinline__ void prefetch_l2(const void *p, uint32_t bytes)
 {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
-}
-
-__device__ __forceinline__ void sts128(uint32_t addr, const uint4 &v)
-{
-    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z),
-                 "r"(v.w)
-                 : "memory");
 }
 
 // 16-byte global load that does not allocate in L1 (each code byte is used once per CTA).
@@ -662,6 +650,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         KbCursor cur;
         cur.start(blockIdx.x, gridDim.x, P.total_units, P.split_k, P.kb_per_split, k_blocks, n_tiles);
         cur.advance(team);
+        uint4 w[4];
+        int z = 0;
         auto fetch = [&](const KbCursor &c, uint4 (&dst)[4], int &zz) {
             const int nt = c.nt;
             const int n = nt * kTileN + r;
@@ -671,18 +661,13 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
 #pragma unroll
             for (int q = 0; q < 4; ++q) dst[q] = ld_stream(src + q * (kQuarterBytes / 16));
         };
-        // row r of stage 0 in the 128-byte swizzle: 16-byte chunk c of the row lives at
-        // chunk c ^ (r & 7), i.e. at this address with bits 4-6 flipped by c
-        const uint32_t row_sw = (base + (uint32_t)r * 128u) | ((uint32_t)(r & 7) << 4);
-        // Two register sets alternate by name (the loop is unrolled by two): the codes of the
-        // team's next k-block are loaded while the current one is decoded, without copies.
-        uint4 wa[4], wb[4];
-        int za = 0, zb = 0;
-        if (cur.valid()) fetch(cur, wa, za);
+        if (cur.valid()) fetch(cur, w, z);
         bool ok = true;
-        auto process = [&](const uint4 (&w)[4], const int z, uint4 (&wn)[4], int &zn) -> bool {
+        while (cur.valid() && ok) {
             KbCursor nxt = cur;
             nxt.advance(T);
+            uint4 wn[4];
+            int zn = 0;
             if (nxt.valid()) fetch(nxt, wn, zn);                 // prefetch the team's next k-block
             const int st = cur.it % S;
             const uint32_t fill = cur.it / S;
@@ -697,7 +682,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     ok = wait_bounded(bar_empty + 8 * (j % S), (j / S) & 1u, ctl, P.sb, 32);
                 }
                 ok = __all_sync(0xffffffffu, ok);
-                if (!ok) return false;
+                if (!ok) break;
                 uint32_t a[32];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
@@ -717,8 +702,10 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 // the operand buffer is free once the MMAs of its last use have retired
                 ok = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
                 ok = __all_sync(0xffffffffu, ok);
-                if (!ok) return false;
-                const uint32_t row = row_sw + (uint32_t)(st * C::kStageBytes);
+                if (!ok) break;
+                uint8_t *stage = gen_base + st * C::kStageBytes;
+                uint8_t *arow = stage + r * 128;
+                const int sw = r & 7;
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const uint4 wq = w[q];
@@ -727,19 +714,17 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     decode8(wq.y, t, c0.z, c0.w);
                     decode8(wq.z, t, c1.x, c1.y);
                     decode8(wq.w, t, c1.z, c1.w);
-                    sts128(row ^ (uint32_t)((2 * q) << 4), c0);
-                    sts128(row ^ (uint32_t)((2 * q + 1) << 4), c1);
+                    *reinterpret_cast<uint4 *>(arow + (((2 * q) ^ sw) << 4)) = c0;
+                    *reinterpret_cast<uint4 *>(arow + (((2 * q + 1) ^ sw) << 4)) = c1;
                 }
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_dec + 8 * st);
             }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) w[q] = wn[q];
+            z = zn;
             cur = nxt;
-            return true;
-        };
-        while (true) {
-            if (!cur.valid() || !process(wa, za, wb, zb)) break;
-            if (!cur.valid() || !process(wb, zb, wa, za)) break;
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
