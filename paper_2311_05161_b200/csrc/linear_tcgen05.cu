@@ -213,70 +213,6 @@ __device__ __forceinline__ void tc_mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, u
         "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// One k-block of the main loop as a single instruction sequence: a non-blocking look at the
-// barriers of the NEXT k-block first, then the four MMAs of this one and the commit that
-// releases its stage, and only then the look's result.  The barrier test takes about a hundred
-// cycles to answer; placed ahead of the MMAs that time passes while they are issued, instead
-// of idling the tensor pipe between k-blocks.  `ready` returns bit 0 / bit 1 for the two tests.
-__device__ __forceinline__ uint32_t tc_kblock_ss(uint32_t d, uint64_t a_desc, uint64_t b_desc,
-                                                 uint32_t idesc, uint32_t accumulate,
-                                                 uint32_t bar_release, uint32_t next_bar0,
-                                                 uint32_t next_par0, uint32_t next_bar1,
-                                                 uint32_t next_par1)
-{
-    uint32_t ready;
-    asm volatile(
-        "{\n\t.reg .pred p, t, q0, q1;\n\t.reg .b32 r0, r1;\n\t.reg .b64 a, b;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 q0, [%7], %8;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 q1, [%9], %10;\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "setp.eq.b32 t, 0, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%1], %2, %3, %4, p;\n\t"
-        "add.u64 a, %2, 2;\n\tadd.u64 b, %3, 2;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%1], a, b, %4, t;\n\t"
-        "add.u64 a, %2, 4;\n\tadd.u64 b, %3, 4;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%1], a, b, %4, t;\n\t"
-        "add.u64 a, %2, 6;\n\tadd.u64 b, %3, 6;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%1], a, b, %4, t;\n\t"
-        "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%6];\n\t"
-        "selp.u32 r0, 1, 0, q0;\n\tselp.u32 r1, 2, 0, q1;\n\t"
-        "or.b32 %0, r0, r1;\n\t}"
-        : "=r"(ready)
-        : "r"(d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(bar_release),
-          "r"(next_bar0), "r"(next_par0), "r"(next_bar1), "r"(next_par1)
-        : "memory");
-    return ready;
-}
-// the same with operand A in tensor memory (32 columns per k-block, 8 per MMA)
-__device__ __forceinline__ uint32_t tc_kblock_ts(uint32_t d, uint32_t a_tmem, uint64_t b_desc,
-                                                 uint32_t idesc, uint32_t accumulate,
-                                                 uint32_t bar_release, uint32_t next_bar0,
-                                                 uint32_t next_par0, uint32_t next_bar1,
-                                                 uint32_t next_par1)
-{
-    uint32_t ready;
-    asm volatile(
-        "{\n\t.reg .pred p, t, q0, q1;\n\t.reg .b32 r0, r1, a;\n\t.reg .b64 b;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 q0, [%7], %8;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 q1, [%9], %10;\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "setp.eq.b32 t, 0, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%1], [%2], %3, %4, p;\n\t"
-        "add.u32 a, %2, 8;\n\tadd.u64 b, %3, 2;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%1], [a], b, %4, t;\n\t"
-        "add.u32 a, %2, 16;\n\tadd.u64 b, %3, 4;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%1], [a], b, %4, t;\n\t"
-        "add.u32 a, %2, 24;\n\tadd.u64 b, %3, 6;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%1], [a], b, %4, t;\n\t"
-        "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%6];\n\t"
-        "selp.u32 r0, 1, 0, q0;\n\tselp.u32 r1, 2, 0, q1;\n\t"
-        "or.b32 %0, r0, r1;\n\t}"
-        : "=r"(ready)
-        : "r"(d), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(bar_release),
-          "r"(next_bar0), "r"(next_par0), "r"(next_bar1), "r"(next_par1)
-        : "memory");
-    return ready;
-}
 __device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&r)[32])
 {
     asm volatile(
@@ -651,7 +587,6 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             uint32_t as = 0, as_par = 0;                 // operand-A slot and its parity
             uint32_t buf = 0, buf_par = 0;               // accumulator buffer and its parity
             bool ok = true;
-            bool ready = false;                          // operands of the coming k-block seen in place
             for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
                 const int s = u % P.split_k;
                 const int kb0 = s * P.kb_per_split;
@@ -667,41 +602,33 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     // decoded weights: per stage in shared memory, or per slot in tensor memory
                     const uint32_t dslot = C::kATmem ? as : st;
                     const uint32_t dpar = C::kATmem ? as_par : st_par;
-                    if (!ready &&
-                        (!wait_bounded(bar_dec + 8 * dslot, dpar, ctl, P.sb, 21) ||
-                         (C::kATmem && !wait_bounded(bar_full + 8 * st, st_par, ctl, P.sb, 23)))) {
+                    if (!wait_bounded(bar_dec + 8 * dslot, dpar, ctl, P.sb, 21) ||
+                        (C::kATmem && !wait_bounded(bar_full + 8 * st, st_par, ctl, P.sb, 23))) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    // where the next k-block's operands will be announced (the position after the
-                    // last k-block is tested too, harmlessly: its answer is never used)
-                    uint32_t nst = st + 1, nsp = st_par, nas = as + 1, nap = as_par;
-                    if (nst == (uint32_t)S) { nst = 0; nsp ^= 1u; }
-                    if (nas == (uint32_t)C::kASlots) { nas = 0; nap ^= 1u; }
-                    const uint32_t nbar0 = bar_dec + 8 * (C::kATmem ? nas : nst);
-                    const uint32_t npar0 = C::kATmem ? nap : nsp;
-                    const uint32_t nbar1 = C::kATmem ? bar_full + 8 * nst : nbar0;
-                    const uint32_t npar1 = C::kATmem ? nsp : npar0;
                     const uint32_t d = tmem_base + buf * TOK;
                     const uint32_t soff = st * (C::kStageBytes >> 4);
+                    const uint64_t a_desc = ((uint64_t)kDescHi << 32) | (a_lo0 + soff);
                     const uint64_t b_desc = ((uint64_t)kDescHi << 32) | (b_lo0 + soff);
-                    uint32_t seen;
-                    if (C::kATmem) {
-                        seen = tc_kblock_ts(d, tmem_base + C::kAColBase + as * 32, b_desc, idesc,
-                                            first ? 0u : 1u, bar_empty + 8 * st, nbar0, npar0, nbar1,
-                                            npar1);
-                    } else {
-                        const uint64_t a_desc = ((uint64_t)kDescHi << 32) | (a_lo0 + soff);
-                        seen = tc_kblock_ss(d, a_desc, b_desc, idesc, first ? 0u : 1u,
-                                            bar_empty + 8 * st, nbar0, npar0, nbar1, npar1);
+                    const uint32_t a_tm = tmem_base + C::kAColBase + as * 32;
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint32_t acc_flag = (!first || ks > 0) ? 1u : 0u;
+                        if (C::kATmem)
+                            tc_mma_i8_ts(d, a_tm + ks * 8, b_desc + (uint64_t)(ks * 2), idesc, acc_flag);
+                        else
+                            tc_mma_i8(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
+                                      acc_flag);
                     }
-                    ready = seen == 3u;
+                    tc_commit(bar_empty + 8 * st);
                     if (last) {
                         tc_commit(bar_acc_full + 8 * buf);
                         if (++buf == (uint32_t)NB) { buf = 0; buf_par ^= 1u; }
                     }
-                    st = nst; st_par = nsp; as = nas; as_par = nap;
+                    if (++st == (uint32_t)S) { st = 0; st_par ^= 1u; }
+                    if (++as == (uint32_t)C::kASlots) { as = 0; as_par ^= 1u; }
                 }
             }
             // nothing issued may still be running when tensor memory is freed
