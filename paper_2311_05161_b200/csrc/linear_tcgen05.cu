@@ -5,11 +5,13 @@
 // decoded weights), the tokens are the N side (operand B, INT8 activations), so the
 // accumulator in tensor memory has one feature per lane and one token per column.  Per
 // 128-wide k-block:
-//   producer thread   TMA tile load of TOK x 128 INT8 activations (128-byte swizzle) and one
-//                     bulk copy of the 8 KiB packed-code tile into a shared-memory ring
-//   decode warps      one thread per feature row: 4-bit codes -> INT8 through a 16-entry
-//                     byte table held in four registers (byte permute), written in the
-//                     128-byte-swizzled K-major layout the MMA reads
+//   producer thread   TMA tile load of TOK x 128 INT8 activations (128-byte swizzle) into the
+//                     stage; for weight-streaming shapes also L2 prefetches of the code tiles
+//   decode warps      teams of four warps take k-blocks in turn, one thread per feature row:
+//                     64 bytes of 4-bit codes straight from global memory into registers (one
+//                     of the team's k-blocks ahead), 4-bit codes -> INT8 through a 16-entry
+//                     byte table held in four registers (byte permute), written into the stage
+//                     in the 128-byte-swizzled K-major layout the MMA reads
 //   MMA thread        4 x tcgen05.mma kind::i8 (128 x TOK x 32) into tensor memory, INT32
 //   epilogue warps    tcgen05.ld, FP32 rescale (token step x weight step / 2), bias, BF16
 // Per-channel weights accumulate over the whole K slice in tensor memory; group-128
@@ -53,16 +55,11 @@ struct Cfg {
     // bandwidth and capacity are the scarce resources); for weight-streaming shapes the
     // producer thread runs ahead with L2 prefetches of the code tiles.
     static constexpr int kTeams = DW / 4;              // teams of 4 warps take k-blocks in turn
-    // The decoded weights (operand A) live in tensor memory when there is room beside the
-    // accumulators: they are then written with tcgen05.st and read by the MMA without touching
-    // shared memory, whose bandwidth (operand reads + TMA writes + decode stores) is the
-    // limiter of the wide tiles.  Otherwise they go through the shared-memory stage.
-    static constexpr bool kATmem = !GROUPED && TOK <= 192;
-    // operand-A buffers of 32 columns each: as many as fit beside the two accumulators
-    static constexpr int kASlotsFit = (512 - 2 * TOK) / 32;
-    static constexpr int kASlots = !kATmem ? 4 : (kASlotsFit > 8 ? 8 : kASlotsFit);
-    static constexpr int kStageBytes = (kATmem ? 0 : kABytes) + kTokBytes;
-    static constexpr int kTokOff = kATmem ? 0 : kABytes;   // tokens inside a stage
+    // One stage holds the decoded INT8 weights of a k-block (operand A, 16 KiB, written by the
+    // decode warps) and the tokens of the same k-block (operand B, written by TMA).  Keeping
+    // operand A in tensor memory instead was measured slower at every token tile.
+    static constexpr int kStageBytes = kABytes + kTokBytes;
+    static constexpr int kTokOff = kABytes;             // tokens inside a stage
     static constexpr int kPrefetchAhead = 16;          // k-blocks of codes requested into L2
     // output staging: two buffers of kChunk tokens x 128 features BF16 per epilogue group
     static constexpr int kStagingBytes = kEpiGroups * kStageBufs * kChunk * kTileN * 2;
@@ -73,8 +70,7 @@ struct Cfg {
     // overlaps the main loop of the next); group mode hands over every k-block, and a hand-over
     // costs several hundred cycles of latency, so it rotates over as many buffers as fit
     static constexpr int kAccBufs = !GROUPED ? 2 : (512 / TOK > 8 ? 8 : 512 / TOK);
-    static constexpr int kAColBase = kAccBufs * TOK;   // first operand-A column
-    static constexpr int kTmemNeed = kAccBufs * TOK + (kATmem ? kASlots * 32 : 0);
+    static constexpr int kTmemNeed = kAccBufs * TOK;
     static constexpr int kTmemCols = kTmemNeed <= 32 ? 32 : kTmemNeed <= 64 ? 64 : kTmemNeed <= 128 ? 128
                                      : kTmemNeed <= 256 ? 256 : 512;
     static constexpr int kOffStaging = kStages * kStageBytes;
@@ -82,7 +78,6 @@ struct Cfg {
     static constexpr int kOffBarriers = kOffTok + 1024;
     static constexpr int kSmemBytes = kOffBarriers + 1024 + 1024 /* alignment slack */;
     static_assert(kStages >= 3, "pipeline depth");
-    static_assert(!kATmem || kStages > kASlots, "a stage outlives an operand-A buffer");
     static_assert(kTmemNeed <= 512, "tensor memory budget");
     static_assert(kSmemBytes <= 232448, "shared memory budget");
     static_assert(!GROUPED || TOK <= 128, "group mode keeps its FP32 sums in registers");
@@ -201,34 +196,6 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint
         "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
         "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
-}
-// A from tensor memory, B from shared memory
-__device__ __forceinline__ void tc_mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
-                                             uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
-        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]),
-        "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
-        "r"(r[30]), "r"(r[31])
-        : "memory");
-}
-__device__ __forceinline__ void tc_wait_st()
-{
-    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
 {
@@ -488,23 +455,20 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t bar_base = base + C::kOffBarriers;
-    const uint32_t bar_full = bar_base;                  // S: TMA bytes landed
-    const uint32_t bar_dec = bar_base + 8 * S;           // S: decoded operand written
-    const uint32_t bar_empty = bar_base + 16 * S;        // S: MMAs of the stage retired
+    const uint32_t bar_dec = bar_base;                   // S: operands of the stage in place
+    const uint32_t bar_empty = bar_base + 8 * S;         // S: MMAs of the stage retired
     constexpr int NB = C::kAccBufs;
-    const uint32_t bar_acc_full = bar_base + 24 * S;          // NB
+    const uint32_t bar_acc_full = bar_base + 16 * S;          // NB
     const uint32_t bar_acc_empty = bar_acc_full + 8 * NB;     // NB
     const uint32_t bar_drain = bar_acc_empty + 8 * NB;        // 1
-    Ctl *ctl = reinterpret_cast<Ctl *>(gen_base + C::kOffBarriers + 24 * S + 16 * NB + 16);
+    Ctl *ctl = reinterpret_cast<Ctl *>(gen_base + C::kOffBarriers + 16 * S + 16 * NB + 16);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
-            // per operand-A slot in tensor-memory mode (4 decode warps); per stage otherwise, where the
-            // token copy completes on the same barrier (4 decode warps + the producer's arrival)
-            mbar_init(bar_dec + 8 * s, C::kATmem ? 4 : 5);
+            // four decode warps and the producer's arrival; the token copy completes on it too
+            mbar_init(bar_dec + 8 * s, 5);
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int b = 0; b < NB; ++b) {
@@ -551,7 +515,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         break;
                     }
                     const uint32_t stage = base + st * C::kStageBytes;
-                    const uint32_t tok_bar = C::kATmem ? bar_full + 8 * st : bar_dec + 8 * st;
+                    const uint32_t tok_bar = bar_dec + 8 * st;
                     mbar_arrive_expect_tx(tok_bar, C::kTokBytes);
                     tma_load_2d(stage + C::kTokOff, &tok_map, kb * kTileK, tt * TOK, tok_bar);
                     if (P.prefetch_codes) {
@@ -569,7 +533,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 // copies already issued must land before the CTA gives its memory back
                 const uint32_t first = it > (uint32_t)S ? it - S : 0u;
                 for (uint32_t j = first; j < it; ++j)
-                    wait_bounded((C::kATmem ? bar_full : bar_dec) + 8 * (j % S), (j / S) & 1u, ctl,
+                    wait_bounded(bar_dec + 8 * (j % S), (j / S) & 1u, ctl,
                                  P.sb, 11, kDrainLimitNs);
             }
         }
@@ -584,7 +548,6 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             const uint32_t a_lo0 = ((base & 0x3FFFFu) >> 4) | (1u << 16);
             const uint32_t b_lo0 = (((base + C::kTokOff) & 0x3FFFFu) >> 4) | (1u << 16);
             uint32_t st = 0, st_par = 0;                 // stage and its fill parity
-            uint32_t as = 0, as_par = 0;                 // operand-A slot and its parity
             uint32_t buf = 0, buf_par = 0;               // accumulator buffer and its parity
             bool ok = true;
             for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
@@ -599,11 +562,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         ok = false;
                         break;
                     }
-                    // decoded weights: per stage in shared memory, or per slot in tensor memory
-                    const uint32_t dslot = C::kATmem ? as : st;
-                    const uint32_t dpar = C::kATmem ? as_par : st_par;
-                    if (!wait_bounded(bar_dec + 8 * dslot, dpar, ctl, P.sb, 21) ||
-                        (C::kATmem && !wait_bounded(bar_full + 8 * st, st_par, ctl, P.sb, 23))) {
+                    // decoded weights and tokens of the stage
+                    if (!wait_bounded(bar_dec + 8 * st, st_par, ctl, P.sb, 21)) {
                         ok = false;
                         break;
                     }
@@ -612,15 +572,11 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     const uint32_t soff = st * (C::kStageBytes >> 4);
                     const uint64_t a_desc = ((uint64_t)kDescHi << 32) | (a_lo0 + soff);
                     const uint64_t b_desc = ((uint64_t)kDescHi << 32) | (b_lo0 + soff);
-                    const uint32_t a_tm = tmem_base + C::kAColBase + as * 32;
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
                         const uint32_t acc_flag = (!first || ks > 0) ? 1u : 0u;
-                        if (C::kATmem)
-                            tc_mma_i8_ts(d, a_tm + ks * 8, b_desc + (uint64_t)(ks * 2), idesc, acc_flag);
-                        else
-                            tc_mma_i8(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
-                                      acc_flag);
+                        tc_mma_i8(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
+                                  acc_flag);
                     }
                     tc_commit(bar_empty + 8 * st);
                     if (last) {
@@ -628,7 +584,6 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         if (++buf == (uint32_t)NB) { buf = 0; buf_par ^= 1u; }
                     }
                     if (++st == (uint32_t)S) { st = 0; st_par ^= 1u; }
-                    if (++as == (uint32_t)C::kASlots) { as = 0; as_par ^= 1u; }
                 }
             }
             // nothing issued may still be running when tensor memory is freed
@@ -642,9 +597,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         // so the fixed latency of one k-block (barrier wait, loads, proxy fence, arrive)
         // overlaps the table lookups of the other teams.
         const int dt = threadIdx.x - 32 * kFirstDecodeWarp;
-        // row r of the tile; with the operand in tensor memory a warp may only touch the lane
-        // quarter (warp index mod 4), so rows follow the warp index there
-        const int r = C::kATmem ? ((warp & 3) * 32 + lane) : (dt & 127);
+        const int r = dt & 127;                              // row of the tile
         const int team = dt >> 7;
         constexpr int T = C::kTeams;
         KbCursor cur;
@@ -673,32 +626,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             const uint32_t fill = cur.it / S;
             uint32_t t[4];
             build_tables(z, t);
-            if (C::kATmem) {
-                // The operand-A slot is free once the MMAs of the k-block that used it last
-                // (kASlots k-blocks ago) have retired: that is the stage barrier of that k-block.
-                const int aslot = cur.it % C::kASlots;
-                if (cur.it >= (uint32_t)C::kASlots) {
-                    const uint32_t j = cur.it - C::kASlots;
-                    ok = wait_bounded(bar_empty + 8 * (j % S), (j / S) & 1u, ctl, P.sb, 32);
-                }
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                uint32_t a[32];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const uint4 wq = w[q];
-                    decode8(wq.x, t, a[8 * q + 0], a[8 * q + 1]);
-                    decode8(wq.y, t, a[8 * q + 2], a[8 * q + 3]);
-                    decode8(wq.z, t, a[8 * q + 4], a[8 * q + 5]);
-                    decode8(wq.w, t, a[8 * q + 6], a[8 * q + 7]);
-                }
-                // lane = row, 32 columns of four INT8 each = the 128 k of this k-block
-                tc_st32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + C::kAColBase + aslot * 32, a);
-                tc_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_dec + 8 * aslot);
-            } else {
+            {
                 // the operand buffer is free once the MMAs of its last use have retired
                 ok = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
                 ok = __all_sync(0xffffffffu, ok);
