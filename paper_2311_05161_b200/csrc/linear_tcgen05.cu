@@ -775,16 +775,32 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     named_bar_sync(1, kEpiThreads);
                     if (is_last && n_ok) {
                         __threadfence();
-                        for (int j = 0; j < valid; ++j) {
-                            const int m = tok0 + j;
-                            int acc = 0;
-                            for (int ss = 0; ss < P.split_k; ++ss)
-                                acc += __ldcg(part + ((size_t)ss * P.m_pad + m) * P.L.n_pad + n);
-                            if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = acc;
-                            if (P.Y) {
-                                float x = rescale_channel(acc, s_tok[col0 + j], half_step);
-                                if (P.bias) x = __fadd_rn(x, bias_n);
-                                P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(x);
+                        // eight tokens at a time, so that many independent loads are in flight
+                        // (rows past the last token exist in the padded buffer and are ignored)
+                        for (int j0 = 0; j0 < valid; j0 += 8) {
+                            int acc[8];
+#pragma unroll
+                            for (int t = 0; t < 8; ++t) acc[t] = 0;
+#pragma unroll 2
+                            for (int ss = 0; ss < P.split_k; ++ss) {
+                                const int32_t *row =
+                                    part + ((size_t)ss * P.m_pad + tok0 + j0) * P.L.n_pad + n;
+#pragma unroll
+                                for (int t = 0; t < 8; ++t)
+                                    if (j0 + t < C::kColsPerThread)
+                                        acc[t] += __ldcg(row + (size_t)t * P.L.n_pad);
+                            }
+#pragma unroll
+                            for (int t = 0; t < 8; ++t) {
+                                const int j = j0 + t;
+                                if (j >= valid) break;
+                                const int m = tok0 + j;
+                                if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = acc[t];
+                                if (P.Y) {
+                                    float x = rescale_channel(acc[t], s_tok[col0 + j], half_step);
+                                    if (P.bias) x = __fadd_rn(x, bias_n);
+                                    P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(x);
+                                }
                             }
                         }
                     }
@@ -878,15 +894,29 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     named_bar_sync(1, kEpiThreads);
                     if (is_last && n_ok && P.Y) {
                         __threadfence();
-                        for (int j = 0; j < valid; ++j) {
-                            const int m = tok0 + j;
-                            float usm = 0.0f;
-                            for (int ss = 0; ss < P.split_k; ++ss)
-                                usm = __fadd_rn(
-                                    usm, __ldcg(part + ((size_t)ss * P.m_pad + m) * P.L.n_pad + n));
-                            float x = __fmul_rn(usm, s_tok[col0 + j]);
-                            if (P.bias) x = __fadd_rn(x, bias_n);
-                            P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(x);
+                        // eight tokens at a time (independent loads in flight); every token's
+                        // slices are still added in slice order
+                        for (int j0 = 0; j0 < valid; j0 += 8) {
+                            float usm[8];
+#pragma unroll
+                            for (int t = 0; t < 8; ++t) usm[t] = 0.0f;
+#pragma unroll 2
+                            for (int ss = 0; ss < P.split_k; ++ss) {
+                                const float *row =
+                                    part + ((size_t)ss * P.m_pad + tok0 + j0) * P.L.n_pad + n;
+#pragma unroll
+                                for (int t = 0; t < 8; ++t)
+                                    if (j0 + t < C::kColsPerThread)
+                                        usm[t] = __fadd_rn(usm[t], __ldcg(row + (size_t)t * P.L.n_pad));
+                            }
+#pragma unroll
+                            for (int t = 0; t < 8; ++t) {
+                                const int j = j0 + t;
+                                if (j >= valid) break;
+                                float x = __fmul_rn(usm[t], s_tok[col0 + j]);
+                                if (P.bias) x = __fadd_rn(x, bias_n);
+                                P.Y[(size_t)(tok0 + j) * P.L.N + n] = __float2bfloat16_rn(x);
+                            }
                         }
                     }
                 }
@@ -978,25 +1008,47 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     const bool grouped = L.group != 0;
     const int cap = grouped ? 128 : 256;
     int tok = opts ? opts->tok_tile : 0;
-    if (tok == 0) {
-        tok = 16;
-        while (tok < M && tok < cap) tok *= 2;
+    int split = opts ? opts->split_k : 0;
+    if (tok == 0 || split == 0) {
+        // Pick the token tile and the K split by a small cost model, in units of one k-block of
+        // one CTA (about 800 cycles whatever the token tile: the decode of the 128 x 128 weight
+        // tile dominates it).  Units are dealt round-robin to one persistent CTA per SM, so the
+        // job takes ceil(units / SMs) rounds of (k-blocks per unit + a fixed cost per unit for
+        // pipeline fill and epilogue); a split adds the partial tile's round trip per unit and,
+        // once at the end, the last slice's reduction (its loads go sixteen at a time).
+        const int sms = sm_count();
+        int tok_max = 16;
+        while (tok_max < M && tok_max < cap) tok_max *= 2;
+        double best = 0.0;
+        int best_tok = 0, best_split = 0;
+        const int t_first = tok ? tok : tok_max, t_last = tok ? tok : 16;
+        for (int t = t_first; t >= t_last; t /= 2) {
+            const long long tiles_t = (long long)((M + t - 1) / t) * L.n_tiles;
+            const int tokens = M < t ? M : t;
+            const int max_split = L.k_blocks / 2 > 16 ? 16 : (L.k_blocks / 2 > 0 ? L.k_blocks / 2 : 1);
+            for (int sp = 1; sp <= max_split; ++sp) {
+                if (split && sp != split) continue;
+                const int per = (L.k_blocks + sp - 1) / sp;
+                const int slices = (L.k_blocks + per - 1) / per;
+                if (slices != sp) continue;                  // the same plan as a smaller split
+                const long long units = tiles_t * slices;
+                const double rounds = (double)((units + sms - 1) / sms);
+                double cost = rounds * (per + 4.0 + (slices > 1 ? 1.0 : 0.0));
+                if (slices > 1) cost += 1.5 * tokens * slices / 16.0;
+                if (best_tok == 0 || cost < best * 0.999) {
+                    best = cost;
+                    best_tok = t;
+                    best_split = slices;
+                }
+            }
+        }
+        if (tok == 0) tok = best_tok ? best_tok : tok_max;
+        if (split == 0) split = best_split ? best_split : 1;
     }
     if (tok != 16 && tok != 32 && tok != 64 && tok != 128 && tok != 192 && tok != 256) return false;
     if (tok > cap) return false;
     const int tok_tiles = (M + tok - 1) / tok;
     const long long tiles = (long long)tok_tiles * L.n_tiles;
-    int split = opts ? opts->split_k : 0;
-    if (split == 0) {
-        split = 1;
-        const int sms = sm_count();
-        if (M <= 256 && tiles < sms) {
-            split = (int)((2LL * sms) / tiles);
-            const int max_split = L.k_blocks / 4 > 0 ? L.k_blocks / 4 : 1;   // >= 4 k-blocks each
-            if (split > max_split) split = max_split;
-            if (split < 1) split = 1;
-        }
-    }
     if (split < 1 || split > L.k_blocks) return false;
     const int kb_per = (L.k_blocks + split - 1) / split;
     split = (L.k_blocks + kb_per - 1) / kb_per;              // no empty slice
