@@ -18,22 +18,30 @@ from util import Problem, bf16_bits, check_y
 pytestmark = pytest.mark.gpu
 
 
+def first_shape(shapes, group, more_than):
+    """First (M, N, K) whose automatic plan needs more workspace than `more_than` bytes."""
+    for M, N, K in shapes:
+        if w4a8.linear_workspace_bytes(M, N, K, group) > more_than:
+            return M, N, K
+    raise AssertionError("no candidate shape has the wanted plan")
+
+
 @pytest.mark.parametrize("group", [0, 128])
 def test_static_scratch_entry_point_matches_linear_twice(group):
-    prob = Problem(1024, 384, 16, group, seed=123 + group)
+    # a shape whose automatic plan splits K: more scratch than the status block alone
+    M, N, K = first_shape([(16, 384, 1024), (16, 384, 4096), (16, 256, 8192)], group, 1024)
+    prob = Problem(K, N, M, group, seed=123 + group)
     d = prob.dev
     packed = w4a8.pack_weights(d["W"], d["s"], group)
     Xq, tok = w4a8.quantize_act(d["X"], d["inv_s"])
-    # the automatic plan for this shape splits K: more scratch than the status block alone
-    assert w4a8.linear_workspace_bytes(16, 384, 1024, group) > 1024
-    ws = w4a8.new_workspace(16, 384, 1024, group)
-    want = w4a8.linear(Xq, tok, packed, d["bias"], 384, group, ws)
+    ws = w4a8.new_workspace(M, N, K, group)
+    want = w4a8.linear(Xq, tok, packed, d["bias"], N, group, ws)
     w4a8.check_status(ws)
     want_bits = bf16_bits(want)
     check_y(prob, want_bits, exact=(group == 0))
     for call in range(2):
-        out = torch.full((16, 384), float("nan"), dtype=torch.bfloat16, device="cuda")
-        w4a8.linear_static(Xq, tok, packed, d["bias"], 384, group, out)
+        out = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        w4a8.linear_static(Xq, tok, packed, d["bias"], N, group, out)
         torch.cuda.synchronize()
         got = bf16_bits(out)
         assert np.array_equal(got, want_bits), f"call {call}: differs from w4a8_linear"
@@ -41,9 +49,8 @@ def test_static_scratch_entry_point_matches_linear_twice(group):
 
 
 def test_static_scratch_rejects_plans_beyond_its_size():
-    # M = 256 tokens on a narrow layer splits K eight ways: 32 MiB of partial tiles
-    M, N, K = 256, 4096, 4096
-    assert w4a8.linear_workspace_bytes(M, N, K, 0) > (8 << 20)
+    # a shape whose split-K partial tiles need more than the 8 MiB the library carries
+    M, N, K = first_shape([(128, 8192, 22016), (256, 4096, 4096), (128, 16384, 32768)], 0, 8 << 20)
     Xq = torch.zeros((M, K), dtype=torch.int8, device="cuda")
     tok = torch.zeros((M,), dtype=torch.float32, device="cuda")
     packed = torch.zeros(w4a8.packed_bytes(N, K, 0), dtype=torch.uint8, device="cuda")
