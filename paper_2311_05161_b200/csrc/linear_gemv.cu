@@ -86,10 +86,6 @@ linear_gemv_kernel(const GemvParams P)
     int8_t (*s_x)[kGemvMaxSteps * kGemvKb * kTileK] =
         reinterpret_cast<int8_t (*)[kGemvMaxSteps * kGemvKb * kTileK]>(gemv_smem + kGemvRingBytes);
     __shared__ int s_last;
-    if (!header_matches(P.blob, P.L)) {
-        if (threadIdx.x == 0) report_failure(P.sb, W4A8_ERR_BAD_BLOB, 3);
-        return;
-    }
     const int nt = blockIdx.x, slice = blockIdx.y, r = threadIdx.x;
     const int n = nt * kTileN + r;
     const int kb_first = slice * P.kb_per_slice;
@@ -120,6 +116,13 @@ linear_gemv_kernel(const GemvParams P)
     };
 #pragma unroll
     for (int s = 0; s < kGemvDepth; ++s) issue(s);
+    // The header is checked while the first codes are on their way (the copies stay inside
+    // the blob the caller described whatever the header says); nothing is written before it.
+    if (!header_matches(P.blob, P.L)) {
+        if (threadIdx.x == 0) report_failure(P.sb, W4A8_ERR_BAD_BLOB, 3);
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        return;
+    }
     // tokens of this K slice: MT rows of kb_count * 128 INT8
     constexpr int kRowChunks = kGemvMaxSteps * kGemvKb * (kTileK / 16);
     for (int i = r; i < MT * kRowChunks; i += 128) {
@@ -218,13 +221,15 @@ linear_gemv_kernel(const GemvParams P)
         if (GROUPED) {
             const float *part = reinterpret_cast<const float *>(P.partials);
             float u = 0.0f;
-            for (int s = 0; s < P.slices; ++s)
+#pragma unroll 8
+            for (int s = 0; s < P.slices; ++s)               // loads of eight slices in flight
                 u = __fadd_rn(u, __ldcg(part + ((size_t)s * P.M + m) * P.L.n_pad + n));
             tv = __fmul_rn(u, P.tok_scale ? P.tok_scale[m] : 0.0f);
         } else {
             const int32_t *part = reinterpret_cast<const int32_t *>(P.partials);
             int a = 0;
-            for (int s = 0; s < P.slices; ++s)
+#pragma unroll 8
+            for (int s = 0; s < P.slices; ++s)               // loads of eight slices in flight
                 a += __ldcg(part + ((size_t)s * P.M + m) * P.L.n_pad + n);
             if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = a;
             tv = rescale_channel(a, P.tok_scale ? P.tok_scale[m] : 0.0f,

@@ -447,10 +447,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     constexpr int S = C::kStages;
     extern __shared__ uint8_t smem_raw[];
 
-    if (!header_matches(P.blob, P.L)) {
-        if (threadIdx.x == 0) report_failure(P.sb, W4A8_ERR_BAD_BLOB, 2);
-        return;
-    }
+    // read now, looked at after the set-up below: the load's latency hides behind it
+    const bool blob_ok = header_matches(P.blob, P.L);
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
@@ -495,7 +493,10 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
 
     const int n_tiles = P.L.n_tiles, k_blocks = P.L.k_blocks;
 
-    if (warp == 0) {
+    if (!blob_ok) {
+        // not the blob the caller described: nothing is read or written, only the status
+        if (threadIdx.x == 0) report_failure(P.sb, W4A8_ERR_BAD_BLOB, 2);
+    } else if (warp == 0) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
             uint32_t it = 0;
