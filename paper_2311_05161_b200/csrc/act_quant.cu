@@ -67,6 +67,8 @@ act_quant_kernel(const __half *__restrict__ X, const float *__restrict__ inv_s, 
                  int8_t *__restrict__ Xq, float *__restrict__ tok_scale)
 {
     __shared__ float red[kActThreads / 32];
+    allow_dependents();
+    dependent_wait();                      // X may be the output of the kernel before
     const int m = blockIdx.x;
     const int tid = threadIdx.x;
     const int nvec = K >> 3;
@@ -135,15 +137,15 @@ cudaError_t launch_quantize_act(const __half *X, const float *inv_s, int M, int 
     const int nvec = K / 8;
     const int per_thread = (nvec + kActThreads - 1) / kActThreads;
     if (per_thread <= 1)
-        act_quant_kernel<1><<<M, kActThreads, 0, st>>>(X, inv_s, M, K, Xq, tok_scale);
+        launch_overlapped(act_quant_kernel<1>, dim3(M), dim3(kActThreads), 0, st, X, inv_s, M, K, Xq, tok_scale);
     else if (per_thread <= 2)
-        act_quant_kernel<2><<<M, kActThreads, 0, st>>>(X, inv_s, M, K, Xq, tok_scale);
+        launch_overlapped(act_quant_kernel<2>, dim3(M), dim3(kActThreads), 0, st, X, inv_s, M, K, Xq, tok_scale);
     else if (per_thread <= 4)
-        act_quant_kernel<4><<<M, kActThreads, 0, st>>>(X, inv_s, M, K, Xq, tok_scale);
+        launch_overlapped(act_quant_kernel<4>, dim3(M), dim3(kActThreads), 0, st, X, inv_s, M, K, Xq, tok_scale);
     else if (per_thread <= 8)
-        act_quant_kernel<8><<<M, kActThreads, 0, st>>>(X, inv_s, M, K, Xq, tok_scale);
+        launch_overlapped(act_quant_kernel<8>, dim3(M), dim3(kActThreads), 0, st, X, inv_s, M, K, Xq, tok_scale);
     else
-        act_quant_kernel<0><<<M, kActThreads, 0, st>>>(X, inv_s, M, K, Xq, tok_scale);
+        launch_overlapped(act_quant_kernel<0>, dim3(M), dim3(kActThreads), 0, st, X, inv_s, M, K, Xq, tok_scale);
     return cudaGetLastError();
 }
 

@@ -124,6 +124,43 @@ __device__ inline float add_bias(float t, const float *bias, int n)
 }
 
 // ---------------------------------------------------------------------------
+// ---------------------------------------------------------------------------
+// programmatic dependent launch
+// ---------------------------------------------------------------------------
+// The hot kernels (activation quantizer, both linear kernels) are launched so that one may
+// start while the kernel before it in the stream is still draining: launch latency, CTA
+// scheduling and each kernel's set-up then overlap the predecessor's tail.  The rule every
+// such kernel keeps: before dependent_wait() it touches no global memory except prefetch
+// hints; dependent_wait() returns once all earlier work in the stream is complete and visible.
+// Kernels launched the ordinary way (packing, the reference kernel) order as always.
+__device__ __forceinline__ void allow_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void dependent_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+#ifdef __CUDACC__
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                     cudaStream_t st, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // plan of the tensor-core kernel (shared by the workspace query and the launcher)
 // ---------------------------------------------------------------------------
 struct LinearPlan {

@@ -86,6 +86,7 @@ linear_gemv_kernel(const GemvParams P)
     int8_t (*s_x)[kGemvMaxSteps * kGemvKb * kTileK] =
         reinterpret_cast<int8_t (*)[kGemvMaxSteps * kGemvKb * kTileK]>(gemv_smem + kGemvRingBytes);
     __shared__ int s_last;
+    allow_dependents();
     const int nt = blockIdx.x, slice = blockIdx.y, r = threadIdx.x;
     const int n = nt * kTileN + r;
     const int kb_first = slice * P.kb_per_slice;
@@ -114,6 +115,9 @@ linear_gemv_kernel(const GemvParams P)
         }
         asm volatile("cp.async.commit_group;" ::: "memory");     // one group per step, even if empty
     };
+    // earlier work in the stream (the activation quantizer, a previous call's use of the
+    // workspace) is complete from here on
+    dependent_wait();
 #pragma unroll
     for (int s = 0; s < kGemvDepth; ++s) issue(s);
     // The header is checked while the first codes are on their way (the copies stay inside
@@ -246,7 +250,7 @@ void launch_gemv(dim3 grid, const GemvParams &P, cudaStream_t st)
     constexpr int smem = kGemvRingBytes + MT * kGemvMaxSteps * kGemvKb * kTileK;
     cudaFuncSetAttribute(linear_gemv_kernel<MT, GROUPED>,
                          cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    linear_gemv_kernel<MT, GROUPED><<<grid, 128, smem, st>>>(P);
+    launch_overlapped(linear_gemv_kernel<MT, GROUPED>, grid, dim3(128), smem, st, P);
 }
 
 }  // namespace

@@ -447,8 +447,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     constexpr int S = C::kStages;
     extern __shared__ uint8_t smem_raw[];
 
-    // read now, looked at after the set-up below: the load's latency hides behind it
-    const bool blob_ok = header_matches(P.blob, P.L);
+    allow_dependents();
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
@@ -490,6 +489,10 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    // Set-up is done; earlier work in the stream (the activation quantizer, a previous call's
+    // use of the workspace, the packing) is complete and visible from here on.
+    dependent_wait();
+    const bool blob_ok = header_matches(P.blob, P.L);
 
     const int n_tiles = P.L.n_tiles, k_blocks = P.L.k_blocks;
 
@@ -987,9 +990,10 @@ w4a8_status launch_dw(const Maps &maps, const Params &P, cudaStream_t st)
         cudaSuccess)
         return W4A8_ERR_CUDA;
     int grid = P.total_units < sm_count() ? P.total_units : sm_count();
-    kern<<<grid, C::kThreads, C::kSmemBytes, st>>>(maps.tok, C::kChunk == 32 ? maps.y32 : maps.y16,
-                                                   P);
-    return cudaGetLastError() == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+    const cudaError_t e =
+        launch_overlapped(kern, dim3(grid), dim3(C::kThreads), (size_t)C::kSmemBytes, st, maps.tok,
+                          C::kChunk == 32 ? maps.y32 : maps.y16, P);
+    return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
 
 template <int TOK, bool GROUPED>
