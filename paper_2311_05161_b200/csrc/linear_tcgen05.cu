@@ -253,25 +253,15 @@ __device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
     return r;
 }
-// Group mode turns every k-block's INT32 partial sums into FP32.  A partial is below 2^22 in
-// magnitude (128 products of at most 127 * 26), so the accumulator is not started at zero
-// but at the integer whose bits are the FP32 number 1.5 * 2^23: after the MMAs its bits read as
-// 1.5 * 2^23 + sum, exactly, and one FP32 subtraction gives float(sum) -- no conversion
-// instruction (an eighth of the FP32 rate) and no integer instruction on the pipe the decode
-// warps saturate.  The epilogue warps write that start value back after each read.
+// A group's INT32 partial sum is below 2^22 in magnitude (128 products of at most 127 * 26), so
+// its low 23 bits with bit 22 flipped, under the exponent of 2^23, are the FP32 number
+// 1.5 * 2^23 + sum: one logic instruction instead of a conversion, which runs at an eighth of
+// the FP32 rate.  Subtracting 1.5 * 2^23 afterwards is exact.
 constexpr uint32_t kMagicBits = 0x4B400000u;          // 1.5 * 2^23 = 12582912.0f
-__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&r)[8])
+__device__ __forceinline__ uint32_t biased_float_bits(uint32_t acc)
 {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr),
-        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
-        : "memory");
+    return (acc & 0x007FFFFFu) ^ kMagicBits;
 }
-__device__ __forceinline__ void tc_wait_st()
-{
-    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-}
-
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 {
     uint32_t d;
@@ -571,11 +561,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 for (int i = 0; i < nkb; ++i) {
                     const bool first = GROUPED || i == 0;
                     const bool last = GROUPED || i == nkb - 1;
-                    // per-channel: the buffer's previous unit has been read (a fresh barrier
-                    // passes); group mode: the buffer holds its start value again, which the
-                    // epilogue warps also announce once before the first use
-                    if (first && !wait_bounded(bar_acc_empty + 8 * buf,
-                                               GROUPED ? buf_par : (buf_par ^ 1u), ctl, P.sb, 20)) {
+                    if (first &&
+                        !wait_bounded(bar_acc_empty + 8 * buf, buf_par ^ 1u, ctl, P.sb, 20)) {
                         ok = false;
                         break;
                     }
@@ -591,7 +578,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     const uint64_t b_desc = ((uint64_t)kDescHi << 32) | (b_lo0 + soff);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
-                        const uint32_t acc_flag = (GROUPED || !first || ks > 0) ? 1u : 0u;
+                        const uint32_t acc_flag = (!first || ks > 0) ? 1u : 0u;
                         tc_mma_i8(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
                                   acc_flag);
                     }
@@ -711,23 +698,6 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             ++stores;
         };
 
-        uint32_t start8[8];                               // accumulator start value (group mode)
-#pragma unroll
-        for (int i = 0; i < 8; ++i) start8[i] = kMagicBits;
-        auto restart = [&](uint32_t buf) {
-            // this thread's share of accumulator buffer `buf` back to the start value
-#pragma unroll
-            for (int c = 0; c < C::kColsPerThread; c += 8)
-                tc_st8(tmem_base + lane_base + buf * TOK + col0 + c, start8);
-            tc_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
-        };
-        if (GROUPED) {
-            for (uint32_t b = 0; b < (uint32_t)NB; ++b) restart(b);
-        }
-
         for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
             const int s = u % P.split_k, rest = u / P.split_k;
             const int nt = rest % n_tiles, tt = rest / n_tiles;
@@ -840,10 +810,9 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     }
                 }
             } else {
-                // FP32 sums over the groups, two tokens per 64-bit register.  The accumulator
-                // bits read as 1.5 * 2^23 + partial (see kMagicBits), so each k-block costs one
-                // packed subtraction and one packed fused multiply-add per pair of tokens, with
-                // the roundings of fmaf(float(partial), step/2, sum)
+                // FP32 sums over the groups, two tokens per 64-bit register: each k-block adds
+                // float(partial) * step/2 with one packed add and one packed fused multiply-add
+                // per pair (same roundings as the scalar fmaf)
                 uint64_t usum2[C::kColsPerThread / 2];
 #pragma unroll
                 for (int j = 0; j < C::kColsPerThread / 2; ++j) usum2[j] = 0ull;
@@ -869,11 +838,15 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         const uint32_t taddr = tmem_base + lane_base + buf * TOK + col0 + c;
                         if (kAcc == 32) tc_ld32(taddr, v); else tc_ld16(taddr, v);
                         tc_wait_ld();
-                        // the partials are in registers: hand the buffer back, restarted
-                        if (c + kAcc >= C::kColsPerThread) restart(buf);
+                        if (c + kAcc >= C::kColsPerThread) {
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+                        }
 #pragma unroll
                         for (int j = 0; j < kAcc; j += 2) {
-                            const uint64_t biased = pack_f32x2(v[j], v[j + 1]);
+                            const uint64_t biased =
+                                pack_f32x2(biased_float_bits(v[j]), biased_float_bits(v[j + 1]));
                             usum2[(c + j) >> 1] =
                                 fma_f32x2(add_f32x2(biased, neg_magic2), h2, usum2[(c + j) >> 1]);
                         }
@@ -882,7 +855,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                             for (int j = 0; j < kAcc; ++j)
                                 if (c + j < valid)
                                     P.acc_out[((size_t)kb * P.M + tok0 + c + j) * P.L.N + n] =
-                                        (int)(v[j] - kMagicBits);
+                                        (int)v[j];
                         }
                     }
                 }
