@@ -29,6 +29,9 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 CONFIG = 2            # OPT-6.7B-shaped block
+# DRAM bytes per launch of the dominant kernel from one ncu capture of this command (see
+# profiles/); set to None whenever that kernel changes until the counters are taken again.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 55.1e6
 M_PREFILL = 2048
 M_DECODE = 1
 CPU_SAMPLE_TOKENS = 48
@@ -474,7 +477,12 @@ def main():
                      "peak_source": f"2 x {peaks['source']} sustained bf16 cuBLAS TFLOP/s",
                      "frac_of_nominal_4500": lin_tops / 4500.0,
                      "per_linear_ms": dict(zip([lay["label"] for lay in layers], lin_ms)),
-                     "traffic": None},
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                     "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum, mean over the "
+                                       "four launches of a step (profiles/bench_opt6.7b_block_launch_list.md)",
+                     "algorithmic_bytes_per_launch": sum(
+                         lay["N"] * lay["K"] // 2 + 5 * lay["N"] + M_PREFILL * lay["K"] + 4 * M_PREFILL
+                         + 2 * M_PREFILL * lay["N"] + 4 * lay["N"] for lay in layers) / len(layers)},
         "decode": {"metric": "w4a8_dint_linear_hbm_gbs", "value": dec_gbs, "unit": "GB/s", "M": M_DECODE,
                    "ms_per_step": ms_dec, "bytes_per_step": dec_bytes,
                    "frac_of_measured_copy": dec_gbs / peaks["hbm_gbs"],
