@@ -27,13 +27,15 @@ bool opts_ok(const w4a8_opts *o)
     return true;
 }
 
-// The weight-streaming kernel serves one to four tokens: by default there, or on request.
-bool use_gemv(int M, const w4a8_opts *o)
+// The weight-streaming kernel can serve one to four tokens (on request, any of them).  By
+// default it takes a single token, and two tokens on large matrices (64 MB of codes and more):
+// measured, the tensor-core kernel with its 16-token tile is as fast or faster everywhere else.
+bool use_gemv(int M, long long weights, const w4a8_opts *o)
 {
     const int path = o ? o->path : W4A8_PATH_AUTO;
     if (path == W4A8_PATH_GEMV) return true;
-    return path == W4A8_PATH_AUTO && M <= gemv_max_tokens() &&
-           !(o && (o->split_k || o->tok_tile || o->decode_warps));
+    if (path != W4A8_PATH_AUTO || (o && (o->split_k || o->tok_tile || o->decode_warps))) return false;
+    return M == 1 || (M == 2 && weights >= (128LL << 20));
 }
 
 w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *packed,
@@ -64,7 +66,7 @@ w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *
         return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
     }
     LinearPlan plan;
-    if (use_gemv(M, opts)) {
+    if (use_gemv(M, (long long)N * K, opts)) {
         gemv_plan(M, L, &plan);
         return launch_linear_gemv(Xq, tok_scale, blob, L, bias, M, static_cast<__nv_bfloat16 *>(Y),
                                   acc, static_cast<uint8_t *>(workspace), plan, st);
@@ -121,7 +123,7 @@ size_t w4a8_linear_workspace_bytes_ex(int M, int N, int K, int group_size, const
     if (!shape_ok(N, K, group_size) || M < 1 || !opts_ok(opts)) return 0;
     if (opts && opts->path == W4A8_PATH_SIMPLE) return sizeof(StatusBlock);
     LinearPlan plan;
-    if (use_gemv(M, opts)) {
+    if (use_gemv(M, (long long)N * K, opts)) {
         if (M > gemv_max_tokens()) return 0;
         gemv_plan(M, make_layout(N, K, group_size), &plan);
         return plan.workspace_bytes;
