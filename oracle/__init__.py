@@ -215,6 +215,64 @@ def linear_f64(Xq, tok_scale, codes, scales, zeros, bias=None, group: int = 0) -
     return Y
 
 
+def quantize_act_asym(X: np.ndarray, inv_s_in: np.ndarray | None = None):
+    """Asymmetric token-wise Min-Max activation quantizer (App. A.1).  X is [M, K] float16.
+
+    Returns (Q [M, K] uint8, tok_scale [M] float32, tok_zero [M] int32) with
+    x' ~ tok_scale * (Q - tok_zero).
+    """
+    X = _c(X, np.float16)
+    M, K = X.shape
+    if inv_s_in is not None:
+        inv_s_in = _c(inv_s_in, np.float32)
+        assert inv_s_in.shape == (K,)
+    Q = np.empty((M, K), dtype=np.uint8)
+    tok = np.empty((M,), dtype=np.float32)
+    zx = np.empty((M,), dtype=np.int32)
+    lib().oracle_quantize_act_asym(_p(X.view(np.uint16)),
+                                   _p(inv_s_in) if inv_s_in is not None else None,
+                                   ctypes.c_int(M), ctypes.c_int(K), _p(Q), _p(tok), _p(zx))
+    return Q, tok, zx
+
+
+def linear_asym_acc(Q, tok_zero, codes, zeros) -> np.ndarray:
+    """int64 sums [M, N] of (Q - tok_zero) times the doubled weight levels; per-channel weights."""
+    Q = _c(Q, np.uint8)
+    tok_zero = _c(tok_zero, np.int32)
+    codes = _c(codes, np.uint8)
+    zeros = _c(zeros, np.uint8)
+    M, K = Q.shape
+    N = codes.shape[0]
+    assert codes.shape == (N, K // 2) and zeros.shape == (1, N) and tok_zero.shape == (M,)
+    acc = np.empty((M, N), dtype=np.int64)
+    lib().oracle_linear_asym_acc_i64(_p(Q), _p(tok_zero), _p(codes), _p(zeros), ctypes.c_int(M),
+                                     ctypes.c_int(N), ctypes.c_int(K), _p(acc))
+    return acc
+
+
+def linear_asym(Q, tok_scale, tok_zero, codes, scales, zeros, bias=None, wide: bool = False):
+    """BF16 output bits [M, N] of the layer with asymmetric activations; with `wide` also the
+    unrounded binary64 values."""
+    Q = _c(Q, np.uint8)
+    tok_scale = _c(tok_scale, np.float32)
+    tok_zero = _c(tok_zero, np.int32)
+    codes = _c(codes, np.uint8)
+    zeros = _c(zeros, np.uint8)
+    scales = _c(scales, np.float32)
+    M, K = Q.shape
+    N = codes.shape[0]
+    assert codes.shape == (N, K // 2) and zeros.shape == (1, N) and scales.shape == (1, N)
+    if bias is not None:
+        bias = _c(bias, np.float32)
+    Y = np.empty((M, N), dtype=np.uint16)
+    W = np.empty((M, N), dtype=np.float64) if wide else None
+    lib().oracle_linear_asym(_p(Q), _p(tok_scale), _p(tok_zero), _p(codes), _p(scales), _p(zeros),
+                             _p(bias) if bias is not None else None, ctypes.c_int(M),
+                             ctypes.c_int(N), ctypes.c_int(K), _p(Y),
+                             _p(W) if wide else None)
+    return (Y, W) if wide else Y
+
+
 def bf16_bits_to_float(bits: np.ndarray) -> np.ndarray:
     """Widen BF16 bit patterns (uint16) to float32 values (exact)."""
     return (bits.astype(np.uint32) << 16).view(np.float32)

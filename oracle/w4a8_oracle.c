@@ -345,6 +345,101 @@ void oracle_linear_f64(const int8_t *Xq, const float *tok_scale,
 }
 
 /* ------------------------------------------------------------------------- */
+/* asymmetric token-wise activations (the paper's own activation quantizer)   */
+/* ------------------------------------------------------------------------- */
+
+/* App. A.1 quantizes activations token-wise with an asymmetric Min-Max quantizer.  The paper
+ * gives no formula; the reading here mirrors the weight side (range widened to contain
+ * zero, 2^8 - 1 steps) in binary32:
+ *   x'[k] = float(X[m][k]) * inv_s_in[k]
+ *   lo = min(0, min_k x'), hi = max(0, max_k x'), d = hi - lo
+ *   d == 0: all codes 0, zero-point 0, step 0
+ *   step = d / 255, r = 255 / d, zx = clamp(rint((-lo) * r), 0, 255)
+ *   Q[m][k] = clamp(rint(x'[k] * r) + zx, 0, 255)        so that x' ~ step * (Q - zx). */
+void oracle_quantize_act_asym(const uint16_t *X, const float *inv_s_in, int M, int K,
+                              uint8_t *Q, float *tok_scale, int32_t *tok_zero)
+{
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        float lo = 0.0f, hi = 0.0f;
+        for (int k = 0; k < K; ++k) {
+            float x = half_bits_to_float(X[(size_t)m * K + k]);
+            if (inv_s_in) x = x * inv_s_in[k];
+            if (x < lo) lo = x;
+            if (x > hi) hi = x;
+        }
+        const float d = hi - lo;
+        if (d == 0.0f) {
+            tok_scale[m] = 0.0f;
+            tok_zero[m] = 0;
+            for (int k = 0; k < K; ++k) Q[(size_t)m * K + k] = 0;
+            continue;
+        }
+        const float r = 255.0f / d;
+        tok_scale[m] = d / 255.0f;
+        const int zx = clampi(rint_to_int((-lo) * r), 0, 255);
+        tok_zero[m] = zx;
+        for (int k = 0; k < K; ++k) {
+            float x = half_bits_to_float(X[(size_t)m * K + k]);
+            if (inv_s_in) x = x * inv_s_in[k];
+            Q[(size_t)m * K + k] = (uint8_t)clampi(rint_to_int(x * r) + zx, 0, 255);
+        }
+    }
+}
+
+/* acc[m][n] = sum_k (Q[m][k] - zx[m]) * t2_{z[n]}[code[n][k]]: the contraction of the
+ * dequantized integers, per-output-channel weights (the paper's W4A8 setting), in 64-bit. */
+void oracle_linear_asym_acc_i64(const uint8_t *Q, const int32_t *tok_zero,
+                                const uint8_t *codes, const uint8_t *zeros, int M, int N,
+                                int K, int64_t *acc)
+{
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        int8_t t2[16];
+        oracle_dint_table2(zeros[n], 4, t2);
+        for (int m = 0; m < M; ++m) {
+            int64_t sum = 0;
+            for (int k = 0; k < K; ++k) {
+                const uint8_t byte = codes[(size_t)n * (K / 2) + k / 2];
+                const int code = (k & 1) ? (byte >> 4) : (byte & 15);
+                sum += (int64_t)((int)Q[(size_t)m * K + k] - tok_zero[m]) * (int64_t)t2[code];
+            }
+            acc[(size_t)m * N + n] = sum;
+        }
+    }
+}
+
+/* y = (float(acc) * tok_scale[m]) * (0.5f * s[n]) (+ bias[n]) -> BF16, as in oracle_linear;
+ * `wide` (may be NULL) receives the same value in binary64, unrounded. */
+void oracle_linear_asym(const uint8_t *Q, const float *tok_scale, const int32_t *tok_zero,
+                        const uint8_t *codes, const float *scales, const uint8_t *zeros,
+                        const float *bias, int M, int N, int K, uint16_t *Y, double *wide)
+{
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        int8_t t2[16];
+        oracle_dint_table2(zeros[n], 4, t2);
+        const float h = 0.5f * scales[n];
+        for (int m = 0; m < M; ++m) {
+            int32_t sum = 0;
+            for (int k = 0; k < K; ++k) {
+                const uint8_t byte = codes[(size_t)n * (K / 2) + k / 2];
+                const int code = (k & 1) ? (byte >> 4) : (byte & 15);
+                sum += ((int32_t)Q[(size_t)m * K + k] - tok_zero[m]) * (int32_t)t2[code];
+            }
+            float t = ((float)sum * tok_scale[m]) * h;
+            if (bias) t = t + bias[n];
+            if (Y) Y[(size_t)m * N + n] = float_to_bf16_bits(t);
+            if (wide) {
+                double w = (double)sum * (double)tok_scale[m] * (0.5 * (double)scales[n]);
+                if (bias) w += (double)bias[n];
+                wide[(size_t)m * N + n] = w;
+            }
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------- */
 /* threading of the outermost loops (sums are integer, so order-free)         */
 /* ------------------------------------------------------------------------- */
 
