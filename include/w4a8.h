@@ -152,6 +152,42 @@ w4a8_status w4a8_linear_static(const int8_t *Xq, const float *tok_scale, const v
                                const float *bias, int M, int N, int K, int group_size,
                                void *Y_bf16, void *stream);
 
+/* ---- asymmetric token-wise activations (the paper's own activation quantizer) ----
+ * Appendix A.1 quantizes activations token-wise with an asymmetric Min-Max quantizer; the
+ * three calls below are that variant of the path, for per-output-channel weights
+ * (group_size 0, the paper's W4A8 setting).
+ *
+ * Per token: x' = X * inv_s, lo = min(0, min x'), hi = max(0, max x'), d = hi - lo,
+ * tok_scale = d / 255, r = 255 / d, zx = clamp(rint(-lo * r), 0, 255),
+ * Q = clamp(rint(x' * r) + zx, 0, 255), so x' ~ tok_scale * (Q - zx); d = 0 gives scale 0.
+ * The unsigned code and its zero-point are stored shifted by 128 so that the INT8 tensor
+ * and CUDA-core paths take them unchanged:
+ *   Xq        out [M][K] INT8  = Q - 128
+ *   tok_scale out [M] FP32
+ *   tok_zero  out [M] INT32    = zx - 128                                               */
+w4a8_status w4a8_quantize_act_asym(const void *X_f16, const float *inv_s_in, int M, int K,
+                                   int8_t *Xq, float *tok_scale, int32_t *tok_zero,
+                                   void *stream);
+
+/* Row sums of the doubled weight levels, rowsum[g][n] = sum over k in group g of
+ * t2(code[n][k]) (INT32, [G][N]; G = 1 for per-channel weights): what a token's zero-point
+ * multiplies.  Offline, once per packed layer. */
+w4a8_status w4a8_weight_rowsum(const void *packed, int N, int K, int group_size,
+                               int32_t *rowsum, void *stream);
+
+/* The quantized matmul with asymmetric activations:
+ *   acc[m][n] = sum_k (Q[m][k] - zx[m]) * t2(code[n][k])
+ *             = sum_k Xq[m][k] * t2(code[n][k]) - tok_zero[m] * rowsum[n]          (INT32)
+ *   y = (float(acc) * tok_scale[m]) * (0.5 * step[n]) + bias[n]  ->  bfloat16.
+ * Xq, tok_scale, tok_zero as written by w4a8_quantize_act_asym; rowsum [N] as written by
+ * w4a8_weight_rowsum; packed with group_size 0.  Y_bf16 and acc ([M][N] INT32, the sums
+ * above) are outputs, either may be NULL but not both.  opts as in w4a8_linear_ex
+ * (NULL = automatic); workspace as for w4a8_linear_ex with the same opts. */
+w4a8_status w4a8_linear_asym(const int8_t *Xq, const float *tok_scale, const int32_t *tok_zero,
+                             const void *packed, const int32_t *rowsum, const float *bias,
+                             int M, int N, int K, void *Y_bf16, int32_t *acc, void *workspace,
+                             size_t workspace_bytes, void *stream, const w4a8_opts *opts);
+
 /* Test export: the INT32 accumulators of the contraction, acc [G][M][N], before any
  * rescale (Eq. 6 in units of step/2).  Uses the same kernels as w4a8_linear_ex. */
 w4a8_status w4a8_linear_acc_i32(const int8_t *Xq, const void *packed, int M, int N, int K,

@@ -9,5 +9,5 @@ from .binding import (  # noqa: F401
     EXPORTS, LIB_PATH, PATH_AUTO, PATH_GEMV, PATH_SIMPLE, PATH_TCGEN05, Opts, W4A8Error, check_status,
     dint4_table, lib, linear, linear_acc_i32, linear_static, linear_workspace_bytes, make_opts, new_workspace,
     pack_weights, packed_bytes, poll_status, quantize_act, unpack_codes, version,
-    workspace_init,
+    workspace_init, quantize_act_asym, weight_rowsum, linear_asym,
 )

@@ -27,6 +27,7 @@ EXPORTS = (
     "w4a8_linear_workspace_bytes", "w4a8_linear_workspace_bytes_ex", "w4a8_workspace_init",
     "w4a8_linear", "w4a8_linear_ex", "w4a8_linear_static", "w4a8_linear_acc_i32", "w4a8_unpack_codes",
     "w4a8_poll_status", "w4a8_dint4_table", "w4a8_version",
+    "w4a8_quantize_act_asym", "w4a8_weight_rowsum", "w4a8_linear_asym",
 )
 
 
@@ -67,6 +68,12 @@ def _load() -> ctypes.CDLL:
     lib.w4a8_linear_ex.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, vp, op]
     lib.w4a8_linear_static.restype = ci
     lib.w4a8_linear_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp]
+    lib.w4a8_quantize_act_asym.restype = ci
+    lib.w4a8_quantize_act_asym.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp]
+    lib.w4a8_weight_rowsum.restype = ci
+    lib.w4a8_weight_rowsum.argtypes = [vp, ci, ci, ci, vp, vp]
+    lib.w4a8_linear_asym.restype = ci
+    lib.w4a8_linear_asym.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, vp, vp, vp, sz, vp, op]
     lib.w4a8_linear_acc_i32.restype = ci
     lib.w4a8_linear_acc_i32.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, sz, vp, op]
     lib.w4a8_unpack_codes.restype = ci
@@ -191,6 +198,52 @@ def linear(Xq, tok_scale, packed, bias, N: int, group: int, workspace, opts: Opt
                                 ctypes.byref(opts))
     _check(st, "w4a8_linear")
     return out
+
+
+def quantize_act_asym(X, inv_s_in=None, out=None):
+    """Asymmetric token-wise quantizer: X [M, K] float16 (CUDA) ->
+    (Xq [M, K] int8 = code - 128, tok_scale [M] float32, tok_zero [M] int32 = zero-point - 128)."""
+    X = _dev(X, torch.float16, "X")
+    inv_s_in = _dev(inv_s_in, torch.float32, "inv_s_in")
+    M, K = X.shape
+    if out is None:
+        out = (torch.empty((M, K), dtype=torch.int8, device=X.device),
+               torch.empty((M,), dtype=torch.float32, device=X.device),
+               torch.empty((M,), dtype=torch.int32, device=X.device))
+    Xq, tok, zero = out
+    _check(lib.w4a8_quantize_act_asym(_ptr(X), _ptr(inv_s_in), M, K, _ptr(Xq), _ptr(tok),
+                                      _ptr(zero), _stream()), "w4a8_quantize_act_asym")
+    return Xq, tok, zero
+
+
+def weight_rowsum(packed, N: int, K: int, group: int = 0):
+    """Row sums of the doubled weight levels: int32 [G, N]."""
+    G = K // group if group else 1
+    out = torch.empty((G, N), dtype=torch.int32, device=packed.device)
+    _check(lib.w4a8_weight_rowsum(_ptr(packed), N, K, group, _ptr(out), _stream()),
+           "w4a8_weight_rowsum")
+    return out
+
+
+def linear_asym(Xq, tok_scale, tok_zero, packed, rowsum, bias, N: int, workspace,
+                opts: Opts | None = None, out=None, want_acc: bool = False):
+    """Quantized linear layer with asymmetric activations (per-channel weights): returns
+    Y [M, N] bfloat16, or (Y, acc [M, N] int32) with `want_acc`."""
+    Xq = _dev(Xq, torch.int8, "Xq")
+    tok_scale = _dev(tok_scale, torch.float32, "tok_scale")
+    tok_zero = _dev(tok_zero, torch.int32, "tok_zero")
+    rowsum = _dev(rowsum, torch.int32, "rowsum")
+    bias = _dev(bias, torch.float32, "bias")
+    M, K = Xq.shape
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=Xq.device)
+    acc = torch.empty((M, N), dtype=torch.int32, device=Xq.device) if want_acc else None
+    st = lib.w4a8_linear_asym(_ptr(Xq), _ptr(tok_scale), _ptr(tok_zero), _ptr(packed), _ptr(rowsum),
+                              _ptr(bias), M, N, K, _ptr(out), _ptr(acc), _ptr(workspace),
+                              workspace.numel(), _stream(),
+                              ctypes.byref(opts) if opts is not None else None)
+    _check(st, "w4a8_linear_asym")
+    return (out, acc) if want_acc else out
 
 
 def linear_static(Xq, tok_scale, packed, bias, N: int, group: int, out):

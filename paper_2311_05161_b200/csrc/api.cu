@@ -41,7 +41,7 @@ bool use_gemv(int M, long long weights, const w4a8_opts *o)
 w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *packed,
                           const float *bias, int M, int N, int K, int group, void *Y,
                           int32_t *acc, void *workspace, size_t workspace_bytes, void *stream,
-                          const w4a8_opts *opts)
+                          const w4a8_opts *opts, ZeroPoint zp = ZeroPoint())
 {
     if (!Xq || !packed || !workspace) return W4A8_ERR_NULL;
     if (!Y && !acc) return W4A8_ERR_NULL;
@@ -61,7 +61,7 @@ w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *
     if (opts && opts->path == W4A8_PATH_SIMPLE) {
         const cudaError_t e =
             launch_linear_simple(Xq, tok_scale, blob, L, bias, M, static_cast<__nv_bfloat16 *>(Y),
-                                 acc, static_cast<StatusBlock *>(workspace), st);
+                                 acc, static_cast<StatusBlock *>(workspace), st, zp);
         if (e == cudaErrorInvalidValue) return W4A8_ERR_SHAPE;
         return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
     }
@@ -69,11 +69,11 @@ w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *
     if (use_gemv(M, (long long)N * K, opts)) {
         gemv_plan(M, L, &plan);
         return launch_linear_gemv(Xq, tok_scale, blob, L, bias, M, static_cast<__nv_bfloat16 *>(Y),
-                                  acc, static_cast<uint8_t *>(workspace), plan, st);
+                                  acc, static_cast<uint8_t *>(workspace), plan, st, zp);
     }
     if (!make_plan(M, L, opts, &plan)) return W4A8_ERR_SHAPE;
     return launch_linear_tcgen05(Xq, tok_scale, blob, L, bias, M, static_cast<__nv_bfloat16 *>(Y),
-                                 acc, static_cast<uint8_t *>(workspace), plan, st);
+                                 acc, static_cast<uint8_t *>(workspace), plan, st, zp);
 }
 
 }  // namespace
@@ -173,6 +173,52 @@ w4a8_status w4a8_linear_acc_i32(const int8_t *Xq, const void *packed, int M, int
     if (!acc) return W4A8_ERR_NULL;
     return linear_common(Xq, nullptr, packed, nullptr, M, N, K, group_size, nullptr, acc,
                          workspace, workspace_bytes, stream, opts);
+}
+
+w4a8_status w4a8_quantize_act_asym(const void *X_f16, const float *inv_s_in, int M, int K,
+                                   int8_t *Xq, float *tok_scale, int32_t *tok_zero, void *stream)
+{
+    if (!X_f16 || !Xq || !tok_scale || !tok_zero) return W4A8_ERR_NULL;
+    if (M < 1 || K < 128 || K % 128 != 0 || K >= (1 << 19)) return W4A8_ERR_SHAPE;
+    if (!aligned(X_f16, 16) || !aligned(inv_s_in, 16) || !aligned(Xq, 16) ||
+        !aligned(tok_scale, 4) || !aligned(tok_zero, 4))
+        return W4A8_ERR_ALIGN;
+    const w4a8_status arch = check_arch();
+    if (arch != W4A8_OK) return arch;
+    const cudaError_t e =
+        launch_quantize_act_asym(static_cast<const __half *>(X_f16), inv_s_in, M, K, Xq, tok_scale,
+                                 tok_zero, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+w4a8_status w4a8_weight_rowsum(const void *packed, int N, int K, int group_size, int32_t *rowsum,
+                               void *stream)
+{
+    if (!packed || !rowsum) return W4A8_ERR_NULL;
+    if (!shape_ok(N, K, group_size)) return W4A8_ERR_SHAPE;
+    if (!aligned(packed, 256) || !aligned(rowsum, 4)) return W4A8_ERR_ALIGN;
+    const w4a8_status arch = check_arch();
+    if (arch != W4A8_OK) return arch;
+    const cudaError_t e =
+        launch_weight_rowsum(static_cast<const uint8_t *>(packed), make_layout(N, K, group_size),
+                             rowsum, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+w4a8_status w4a8_linear_asym(const int8_t *Xq, const float *tok_scale, const int32_t *tok_zero,
+                             const void *packed, const int32_t *rowsum, const float *bias, int M,
+                             int N, int K, void *Y_bf16, int32_t *acc, void *workspace,
+                             size_t workspace_bytes, void *stream, const w4a8_opts *opts)
+{
+    if (!tok_zero || !rowsum) return W4A8_ERR_NULL;
+    if (!aligned(tok_zero, 4) || !aligned(rowsum, 4)) return W4A8_ERR_ALIGN;
+    // (Q - zx) spans 255 where the symmetric INT8 spans 127: the INT32 bound on K halves
+    if ((long long)K * 255 * 26 >= (1LL << 31)) return W4A8_ERR_SHAPE;
+    ZeroPoint zp;
+    zp.tok_zero = tok_zero;
+    zp.rowsum = rowsum;
+    return linear_common(Xq, tok_scale, packed, bias, M, N, K, 0, Y_bf16, acc, workspace,
+                         workspace_bytes, stream, opts, zp);
 }
 
 w4a8_status w4a8_unpack_codes(const void *packed, int N, int K, int group_size, uint8_t *codes,

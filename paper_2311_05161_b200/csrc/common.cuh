@@ -172,6 +172,13 @@ struct LinearPlan {
     size_t off_counters, off_partials, workspace_bytes;
 };
 
+// Asymmetric activations: acc[m][n] -= tok_zero[m] * rowsum[n] before the rescale (both
+// pointers NULL for the symmetric path).
+struct ZeroPoint {
+    const int32_t *tok_zero = nullptr;   // [M]
+    const int32_t *rowsum = nullptr;     // [N]
+};
+
 // launchers (defined in the .cu files, called by api.cu)
 cudaError_t launch_pack(const __half *W, const float *s_in, const BlobLayout &L, float clip,
                         uint8_t *blob, cudaStream_t st);
@@ -179,21 +186,26 @@ cudaError_t launch_unpack(const uint8_t *blob, const BlobLayout &L, uint8_t *cod
                           float *scales, uint8_t *zeros, cudaStream_t st);
 cudaError_t launch_quantize_act(const __half *X, const float *inv_s, int M, int K, int8_t *Xq,
                                 float *tok_scale, cudaStream_t st);
+cudaError_t launch_quantize_act_asym(const __half *X, const float *inv_s, int M, int K, int8_t *Xq,
+                                     float *tok_scale, int32_t *tok_zero, cudaStream_t st);
+cudaError_t launch_weight_rowsum(const uint8_t *blob, const BlobLayout &L, int32_t *rowsum,
+                                 cudaStream_t st);
 cudaError_t launch_linear_simple(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
                                  const BlobLayout &L, const float *bias, int M,
                                  __nv_bfloat16 *Y, int32_t *acc, StatusBlock *sb,
-                                 cudaStream_t st);
+                                 cudaStream_t st, ZeroPoint zp = ZeroPoint());
 bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *plan);
 w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
                                   const BlobLayout &L, const float *bias, int M,
                                   __nv_bfloat16 *Y, int32_t *acc, uint8_t *workspace,
-                                  const LinearPlan &plan, cudaStream_t st);
+                                  const LinearPlan &plan, cudaStream_t st,
+                                  ZeroPoint zp = ZeroPoint());
 
 int gemv_max_tokens();
 void gemv_plan(int M, const BlobLayout &L, LinearPlan *plan);
 w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
                                const BlobLayout &L, const float *bias, int M, __nv_bfloat16 *Y,
                                int32_t *acc, uint8_t *workspace, const LinearPlan &plan,
-                               cudaStream_t st);
+                               cudaStream_t st, ZeroPoint zp = ZeroPoint());
 
 }  // namespace w4a8

@@ -74,6 +74,7 @@ struct GemvParams {
     void *partials;
     BlobLayout L;
     int M, slices, kb_per_slice;
+    ZeroPoint zp;
 };
 
 template <int MT, bool GROUPED>
@@ -235,6 +236,7 @@ linear_gemv_kernel(const GemvParams P)
 #pragma unroll 8
             for (int s = 0; s < P.slices; ++s)               // loads of eight slices in flight
                 a += __ldcg(part + ((size_t)s * P.M + m) * P.L.n_pad + n);
+            if (P.zp.tok_zero) a -= P.zp.tok_zero[m] * P.zp.rowsum[n];
             if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = a;
             tv = rescale_channel(a, P.tok_scale ? P.tok_scale[m] : 0.0f,
                                  __fmul_rn(0.5f, P.scales[n]));
@@ -284,7 +286,7 @@ void gemv_plan(int M, const BlobLayout &L, LinearPlan *plan)
 w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
                                const BlobLayout &L, const float *bias, int M, __nv_bfloat16 *Y,
                                int32_t *acc, uint8_t *workspace, const LinearPlan &plan,
-                               cudaStream_t st)
+                               cudaStream_t st, ZeroPoint zp)
 {
     if (M < 1 || M > kGemvMaxTokens) return W4A8_ERR_SHAPE;
     GemvParams P;
@@ -304,6 +306,7 @@ w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const u
     P.M = M;
     P.slices = plan.split_k;
     P.kb_per_slice = plan.kb_per_split;
+    P.zp = zp;
     if (P.slices > 65535) return W4A8_ERR_SHAPE;
     const dim3 grid(L.n_tiles, P.slices);
     const bool g = L.group != 0;

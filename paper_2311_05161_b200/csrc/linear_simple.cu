@@ -11,7 +11,7 @@ __global__ void __launch_bounds__(128)
 linear_simple_kernel(const int8_t *__restrict__ Xq, const float *__restrict__ tok_scale,
                      const uint8_t *__restrict__ blob, BlobLayout L,
                      const float *__restrict__ bias, int M, __nv_bfloat16 *__restrict__ Y,
-                     int32_t *__restrict__ acc_out, StatusBlock *sb)
+                     int32_t *__restrict__ acc_out, StatusBlock *sb, ZeroPoint zp)
 {
     if (!header_matches(blob, L)) {
         if (threadIdx.x == 0) report_failure(sb, W4A8_ERR_BAD_BLOB, 1);
@@ -51,6 +51,7 @@ linear_simple_kernel(const int8_t *__restrict__ Xq, const float *__restrict__ to
     if (grouped) {
         t = __fmul_rn(u, a);
     } else {
+        if (zp.tok_zero) acc -= zp.tok_zero[m] * zp.rowsum[n];
         if (acc_out) acc_out[(size_t)m * L.N + n] = acc;
         t = rescale_channel(acc, a, __fmul_rn(0.5f, scales[n]));
     }
@@ -62,11 +63,11 @@ linear_simple_kernel(const int8_t *__restrict__ Xq, const float *__restrict__ to
 cudaError_t launch_linear_simple(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
                                  const BlobLayout &L, const float *bias, int M,
                                  __nv_bfloat16 *Y, int32_t *acc, StatusBlock *sb,
-                                 cudaStream_t st)
+                                 cudaStream_t st, ZeroPoint zp)
 {
     if (M > 65535) return cudaErrorInvalidValue;
     dim3 grid(L.n_tiles, M);
-    linear_simple_kernel<<<grid, 128, 0, st>>>(Xq, tok_scale, blob, L, bias, M, Y, acc, sb);
+    linear_simple_kernel<<<grid, 128, 0, st>>>(Xq, tok_scale, blob, L, bias, M, Y, acc, sb, zp);
     return cudaGetLastError();
 }
 

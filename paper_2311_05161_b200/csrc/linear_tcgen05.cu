@@ -63,7 +63,8 @@ struct Cfg {
     static constexpr int kPrefetchAhead = 16;          // k-blocks of codes requested into L2
     // output staging: two buffers of kChunk tokens x 128 features BF16 per epilogue group
     static constexpr int kStagingBytes = kEpiGroups * kStageBufs * kChunk * kTileN * 2;
-    static constexpr int kTailBytes = kStagingBytes + 1024 /* token steps */ + 1024 /* barriers */;
+    static constexpr int kTailBytes =
+        kStagingBytes + 2048 /* token steps and zero-points */ + 1024 /* barriers */;
     static constexpr int kMaxStages = (232448 - 1024 - kTailBytes) / kStageBytes;
     static constexpr int kStages = kMaxStages > 9 ? 9 : kMaxStages;
     // accumulator buffers in tensor memory: two for per-channel weights (epilogue of one unit
@@ -75,7 +76,7 @@ struct Cfg {
                                      : kTmemNeed <= 256 ? 256 : 512;
     static constexpr int kOffStaging = kStages * kStageBytes;
     static constexpr int kOffTok = kOffStaging + kStagingBytes;
-    static constexpr int kOffBarriers = kOffTok + 1024;
+    static constexpr int kOffBarriers = kOffTok + 2048;
     static constexpr int kSmemBytes = kOffBarriers + 1024 + 1024 /* alignment slack */;
     static_assert(kStages >= 3, "pipeline depth");
     static_assert(kTmemNeed <= 512, "tensor memory budget");
@@ -97,6 +98,7 @@ struct Params {
     void *partials;
     BlobLayout L;
     int M, tok_tiles, m_pad, split_k, kb_per_split, total_units, prefetch_codes;
+    ZeroPoint zp;
 };
 
 // --------------------------------------------------------------------------- PTX wrappers
@@ -671,6 +673,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         const int group_bar = 2 + col_group;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         float *s_tok = reinterpret_cast<float *>(gen_base + C::kOffTok);
+        int *s_tz = reinterpret_cast<int *>(gen_base + C::kOffTok + 1024);   // tokens' zero-points
         __nv_bfloat16 *stg =
             reinterpret_cast<__nv_bfloat16 *>(gen_base + C::kOffStaging) +
             col_group * C::kStageBufs * C::kChunk * kTileN;
@@ -710,16 +713,22 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             valid = valid < 0 ? 0 : (valid > C::kColsPerThread ? C::kColsPerThread : valid);
             const float bias_n = (P.bias && n_ok) ? P.bias[n] : 0.0f;
 
-            if (P.Y) {
-                // token step sizes of this tile, shared by all epilogue threads
+            if (P.Y || P.zp.tok_zero) {
+                // token step sizes (and zero-points) of this tile, shared by all epilogue threads
                 named_bar_sync(1, kEpiThreads);
-                for (int i = et; i < TOK; i += kEpiThreads)
-                    s_tok[i] = (tt * TOK + i < P.M) ? __ldg(P.tok_scale + tt * TOK + i) : 0.0f;
+                for (int i = et; i < TOK; i += kEpiThreads) {
+                    const bool in = tt * TOK + i < P.M;
+                    s_tok[i] = (in && P.tok_scale) ? __ldg(P.tok_scale + tt * TOK + i) : 0.0f;
+                    s_tz[i] = (in && P.zp.tok_zero) ? __ldg(P.zp.tok_zero + tt * TOK + i) : 0;
+                }
                 named_bar_sync(1, kEpiThreads);
             }
 
             if (!GROUPED) {
                 const float half_step = __fmul_rn(0.5f, P.scales[n]);
+                // asymmetric activations: the token's zero-point times this row's level sum
+                // leaves the accumulator before the rescale (zero for the symmetric path)
+                const int row_sum = (P.zp.rowsum && n_ok) ? __ldg(P.zp.rowsum + n) : 0;
                 const uint32_t buf = phase % NB;
                 ok = wait_bounded_idle(bar_acc_full + 8 * buf, (phase / NB) & 1u, ctl, P.sb, 40);
                 ok = named_bar_and(1, kEpiThreads, ok);
@@ -740,6 +749,11 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
                     }
                     if (c >= valid) continue;             // uniform over the column group
+                    if (P.zp.tok_zero && P.split_k == 1) {
+#pragma unroll
+                        for (int j = 0; j < C::kChunk; ++j)
+                            v[j] = (uint32_t)((int)v[j] - s_tz[col0 + c + j] * row_sum);
+                    }
                     if (P.acc_out && P.split_k == 1 && n_ok) {
 #pragma unroll
                         for (int j = 0; j < C::kChunk; ++j)
@@ -799,6 +813,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                                 const int j = j0 + t;
                                 if (j >= valid) break;
                                 const int m = tok0 + j;
+                                acc[t] -= s_tz[col0 + j] * row_sum;
                                 if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = acc[t];
                                 if (P.Y) {
                                     float x = rescale_channel(acc[t], s_tok[col0 + j], half_step);
@@ -1077,7 +1092,7 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
 w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
                                   const BlobLayout &L, const float *bias, int M,
                                   __nv_bfloat16 *Y, int32_t *acc, uint8_t *workspace,
-                                  const LinearPlan &plan, cudaStream_t st)
+                                  const LinearPlan &plan, cudaStream_t st, ZeroPoint zp)
 {
     EncodeTiledFn enc = encode_tiled();
     if (!enc) return W4A8_ERR_CUDA;
@@ -1125,6 +1140,7 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     P.kb_per_split = plan.kb_per_split;
     P.total_units = plan.tok_tiles * L.n_tiles * plan.split_k;
     P.prefetch_codes = plan.tok_tiles == 1 ? 1 : 0;   // every code tile is read exactly once
+    P.zp = zp;
 
     const bool g = L.group != 0;
     switch (plan.tok_tile) {

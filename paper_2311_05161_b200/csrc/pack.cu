@@ -197,6 +197,32 @@ __global__ void unpack_kernel(const uint8_t *__restrict__ blob, BlobLayout L,
     }
 }
 
+// rowsum[g][n] = sum over the k of group g of t2(code[n][k]) (Eq. 6 in units of step/2): the
+// factor of a token's zero-point in the asymmetric-activation path.  One CTA per 128-row tile,
+// one thread per row; a warp reads 512 contiguous bytes per quarter tile.
+__global__ void __launch_bounds__(128)
+rowsum_kernel(const uint8_t *__restrict__ blob, BlobLayout L, int32_t *__restrict__ rowsum)
+{
+    const int nt = blockIdx.x, r = threadIdx.x;
+    const int n = nt * kTileN + r;
+    const uint8_t *zeros = blob + L.off_zeros;
+    const uint8_t *codes = blob + L.off_codes;
+    int z = zeros[n];
+    int sum = 0;
+    for (int kb = 0; kb < L.k_blocks; ++kb) {
+        if (L.group != 0) { z = zeros[(size_t)kb * L.n_pad + n]; sum = 0; }
+        const uint8_t *tile = codes + ((size_t)nt * L.k_blocks + kb) * kTileBytes;
+        for (int q = 0; q < 4; ++q) {
+            const uint4 w = *reinterpret_cast<const uint4 *>(tile + q * kQuarterBytes + r * 16);
+            const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sum += dint4_t2((words[i >> 3] >> (4 * (i & 7))) & 15, z);
+        }
+        if (L.group != 0 && n < L.N) rowsum[(size_t)kb * L.N + n] = sum;
+    }
+    if (L.group == 0 && n < L.N) rowsum[n] = sum;
+}
+
 }  // namespace
 
 cudaError_t launch_pack(const __half *W, const float *s_in, const BlobLayout &L, float clip,
@@ -216,6 +242,13 @@ cudaError_t launch_unpack(const uint8_t *blob, const BlobLayout &L, uint8_t *cod
     int blocks = (int)((total + 255) / 256);
     if (blocks > 148 * 16) blocks = 148 * 16;
     unpack_kernel<<<blocks, 256, 0, st>>>(blob, L, codes, scales, zeros);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_weight_rowsum(const uint8_t *blob, const BlobLayout &L, int32_t *rowsum,
+                                 cudaStream_t st)
+{
+    rowsum_kernel<<<L.n_tiles, 128, 0, st>>>(blob, L, rowsum);
     return cudaGetLastError();
 }
 
