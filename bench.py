@@ -338,6 +338,8 @@ def main():
         d["tok"] = torch.empty((M_PREFILL,), dtype=torch.float32, device=dev)
         d["Y"] = torch.empty((M_PREFILL, N), dtype=torch.bfloat16, device=dev)
         d["ws"] = w4a8.new_workspace(M_PREFILL, N, K, group)
+        d["tz"] = torch.empty((M_PREFILL,), dtype=torch.int32, device=dev)
+        d["rowsum"] = w4a8.weight_rowsum(d["packed"], N, K, group)[0].contiguous()
         d["K"], d["N"] = K, N
         d["X_host"] = torch.from_numpy(lay["X"]).pin_memory()
         d["Y_host"] = torch.empty((M_PREFILL, N), dtype=torch.bfloat16).pin_memory()
@@ -368,6 +370,13 @@ def main():
             w4a8.linear(d["Xq"], d["tok"], d["packed"], d["bias"], d["N"], group, d["ws"],
                         out=d["Y"])
             d["Y_host"].copy_(d["Y"], non_blocking=True)
+
+    def step_asym(it=None):
+        # the same block with the paper's asymmetric token-wise activation quantizer
+        for d in L:
+            w4a8.quantize_act_asym(d["X"], d["inv_s"], out=(d["Xq"], d["tok"], d["tz"]))
+            w4a8.linear_asym(d["Xq"], d["tok"], d["tz"], d["packed"], d["rowsum"], d["bias"],
+                             d["N"], d["ws"], out=d["Y"])
 
     def step_decode(it):
         for d in L:
@@ -419,6 +428,12 @@ def main():
     ms_e2e = timed(lambda it: step_e2e(), e2e_steps) / e2e_steps
     h2d = sum(d["X_host"].numel() * 2 for d in L)
     d2h = sum(d["Y_host"].numel() * 2 for d in L)
+
+    # ------------------------------------------------------------------ asymmetric activations
+    for _ in range(3):
+        step_asym()
+    asym_steps = max(3, min(args.steps, 50))
+    ms_asym = timed(step_asym, asym_steps) / asym_steps
 
     # ------------------------------------------------------------------ decode (M = 1)
     # The eight launches of a decode step take a few microseconds each: from Python they would
@@ -488,6 +503,10 @@ def main():
                    "frac_of_measured_copy": dec_gbs / peaks["hbm_gbs"],
                    "frac_of_nominal_8000": dec_gbs / 8000.0,
                    "note": "quantize_act + linear per shape, 3 rotating blob copies (> L2), CUDA graph replay"},
+        "asym": {"metric": "w4a8_dint_linear_tops", "value": replica_throughput(ops_per_step, world, ms_asym),
+                 "unit": "TOPS", "ms_per_step": ms_asym,
+                 "note": "same block and step with asymmetric token-wise activations "
+                         "(quantize_act_asym + linear_asym)"},
         "cpu_baseline": cpu,
     }
     print(json.dumps(line), flush=True)
