@@ -32,6 +32,7 @@ namespace {
 
 constexpr int kFirstDecodeWarp = 2;
 constexpr int kABytes = kTileN * kTileK;            // decoded INT8 tile, 16 KiB
+constexpr int kDefaultTeamWarps = 4;               // warps per decode team
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 // how long a waiting thread may stay suspended in hardware before it polls again (it is woken
 // at once when the barrier phase completes); keeps waiting warps out of the issue slots
@@ -40,7 +41,6 @@ constexpr unsigned long long kDrainLimitNs = 200000000ull;
 
 template <int TOK, bool GROUPED, int DW>
 struct Cfg {
-    static constexpr int kQuartersPerThread = 16 / DW;
     static constexpr int kFirstEpiWarp = kFirstDecodeWarp + DW;
     // epilogue warpgroups: group mode spreads the per-k-block FP32 accumulation over
     // 32 columns per thread (more warps in flight, fewer registers each)
@@ -54,7 +54,14 @@ struct Cfg {
     // Codes go from global memory straight into the decode threads' registers (shared-memory
     // bandwidth and capacity are the scarce resources); for weight-streaming shapes the
     // producer thread runs ahead with L2 prefetches of the code tiles.
-    static constexpr int kTeams = DW / 4;              // teams of 4 warps take k-blocks in turn
+    // Decode warps work in teams that take k-blocks in turn; a team of kTeamWarps warps splits
+    // the 128 x 128 tile into kTeamWarps / 4 column slices (a thread expands 64, 32 or 16 bytes
+    // of codes of one row).  Wider teams fill a stage sooner (the stage ring is short), narrower
+    // teams pay the per-k-block bookkeeping less often.
+    static constexpr int kTeamWarps = kDefaultTeamWarps <= DW ? kDefaultTeamWarps : DW;
+    static constexpr int kTeams = DW / kTeamWarps;
+    static constexpr int kQuartersPerThread = 16 / kTeamWarps;   // 32-k quarters of a row
+    static_assert(DW % kTeamWarps == 0 && kQuartersPerThread >= 1, "decode warps form whole teams");
     // One stage holds the decoded INT8 weights of a k-block (operand A, 16 KiB, written by the
     // decode warps) and the tokens of the same k-block (operand B, written by TMA).  Keeping
     // operand A in tensor memory instead was measured slower at every token tile.
@@ -466,8 +473,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
-            // four decode warps and the producer's arrival; the token copy completes on it too
-            mbar_init(bar_dec + 8 * s, 5);
+            // the warps of a decode team and the producer's arrival; the token copy completes on it too
+            mbar_init(bar_dec + 8 * s, C::kTeamWarps + 1);
             mbar_init(bar_empty + 8 * s, 1);
         }
         for (int b = 0; b < NB; ++b) {
@@ -599,33 +606,35 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         __syncwarp();
     } else if (warp < kFirstEpiWarp) {
         // ------------------------------------------------------------------ decode warps
-        // Four warps (one thread per feature row) form a team; teams take k-blocks in turn,
-        // so the fixed latency of one k-block (barrier wait, loads, proxy fence, arrive)
-        // overlaps the table lookups of the other teams.
+        // The warps of a team share a k-block (a thread takes one feature row and one column
+        // slice of it); teams take k-blocks in turn, so the fixed latency of one k-block (barrier
+        // wait, loads, proxy fence, arrive) overlaps the table lookups of the other teams.
         const int dt = threadIdx.x - 32 * kFirstDecodeWarp;
         const int r = dt & 127;                              // row of the tile
-        const int team = dt >> 7;
+        constexpr int QT = C::kQuartersPerThread;
+        const int q0 = ((dt >> 7) % (C::kTeamWarps / 4)) * QT;   // first 32-k quarter of this thread
+        const int team = dt / (32 * C::kTeamWarps);
         constexpr int T = C::kTeams;
         KbCursor cur;
         cur.start(blockIdx.x, gridDim.x, P.total_units, P.split_k, P.kb_per_split, k_blocks, n_tiles);
         cur.advance(team);
-        uint4 w[4];
+        uint4 w[QT];
         int z = 0;
-        auto fetch = [&](const KbCursor &c, uint4 (&dst)[4], int &zz) {
+        auto fetch = [&](const KbCursor &c, uint4 (&dst)[QT], int &zz) {
             const int nt = c.nt;
             const int n = nt * kTileN + r;
             zz = GROUPED ? P.zeros[(size_t)c.kb * P.L.n_pad + n] : P.zeros[n];
             const uint4 *src = reinterpret_cast<const uint4 *>(
                 P.codes + ((size_t)nt * k_blocks + c.kb) * kTileBytes + r * 16);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) dst[q] = ld_stream(src + q * (kQuarterBytes / 16));
+            for (int q = 0; q < QT; ++q) dst[q] = ld_stream(src + (q0 + q) * (kQuarterBytes / 16));
         };
         if (cur.valid()) fetch(cur, w, z);
         bool ok = true;
         while (cur.valid() && ok) {
             KbCursor nxt = cur;
             nxt.advance(T);
-            uint4 wn[4];
+            uint4 wn[QT];
             int zn = 0;
             if (nxt.valid()) fetch(nxt, wn, zn);                 // prefetch the team's next k-block
             const int st = cur.it % S;
@@ -641,22 +650,22 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 uint8_t *arow = stage + r * 128;
                 const int sw = r & 7;
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
+                for (int q = 0; q < QT; ++q) {
                     const uint4 wq = w[q];
                     uint4 c0, c1;
                     decode8(wq.x, t, c0.x, c0.y);
                     decode8(wq.y, t, c0.z, c0.w);
                     decode8(wq.z, t, c1.x, c1.y);
                     decode8(wq.w, t, c1.z, c1.w);
-                    *reinterpret_cast<uint4 *>(arow + (((2 * q) ^ sw) << 4)) = c0;
-                    *reinterpret_cast<uint4 *>(arow + (((2 * q + 1) ^ sw) << 4)) = c1;
+                    *reinterpret_cast<uint4 *>(arow + (((2 * (q0 + q)) ^ sw) << 4)) = c0;
+                    *reinterpret_cast<uint4 *>(arow + (((2 * (q0 + q) + 1) ^ sw) << 4)) = c1;
                 }
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_dec + 8 * st);
             }
 #pragma unroll
-            for (int q = 0; q < 4; ++q) w[q] = wn[q];
+            for (int q = 0; q < QT; ++q) w[q] = wn[q];
             z = zn;
             cur = nxt;
         }
