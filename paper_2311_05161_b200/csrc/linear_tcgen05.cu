@@ -58,7 +58,7 @@ struct Cfg {
     // the 128 x 128 tile into kTeamWarps / 4 column slices (a thread expands 64, 32 or 16 bytes
     // of codes of one row).  Wider teams fill a stage sooner (the stage ring is short), narrower
     // teams pay the per-k-block bookkeeping less often.
-    static constexpr int kTeamWarps = kDefaultTeamWarps <= DW ? kDefaultTeamWarps : DW;
+    static constexpr int kTeamWarps = (DW % kDefaultTeamWarps == 0) ? kDefaultTeamWarps : 4;
     static constexpr int kTeams = DW / kTeamWarps;
     static constexpr int kQuartersPerThread = 16 / kTeamWarps;   // 32-k quarters of a row
     static_assert(DW % kTeamWarps == 0 && kQuartersPerThread >= 1, "decode warps form whole teams");
