@@ -36,18 +36,6 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
     return r;
 }
 
-// Bits of fl(v + 1.5 * 2^23) for both lanes of a pair.  The adds are scalar on purpose: written
-// as a packed add behind the packed multiply, the two were contracted into one fused
-// multiply-add (one rounding), which rounds exact .5 products differently from the two-step
-// reference arithmetic.
-__device__ __forceinline__ void magic_round2(uint64_t v, uint32_t &lo, uint32_t &hi)
-{
-    uint32_t a, b;
-    unpair(v, a, b);
-    lo = __float_as_uint(__fadd_rn(__uint_as_float(a), 12582912.0f));
-    hi = __float_as_uint(__fadd_rn(__uint_as_float(b), 12582912.0f));
-}
-
 // Eight FP16 values -> four pairs of FP32, times the per-channel reciprocal scale when given.
 __device__ __forceinline__ void scaled8(const uint4 &v, const float *__restrict__ inv_s, int k0,
                                         uint64_t (&p)[4])
@@ -105,9 +93,10 @@ __device__ __forceinline__ uint32_t prmt_b(uint32_t a, uint32_t b, uint32_t sel)
 // which rounds to 127.
 __device__ __forceinline__ uint2 quantize8(const uint64_t (&p)[4], uint64_t rr)
 {
+    const uint64_t magic = pair(12582912.0f, 12582912.0f);
     uint32_t b[8];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) magic_round2(mul2(p[i], rr), b[2 * i], b[2 * i + 1]);
+    for (int i = 0; i < 4; ++i) unpair(add2(mul2(p[i], rr), magic), b[2 * i], b[2 * i + 1]);
     uint2 o;
     o.x = prmt_b(prmt_b(b[0], b[1], 0x0040u), prmt_b(b[2], b[3], 0x0040u), 0x5410u);
     o.y = prmt_b(prmt_b(b[4], b[5], 0x0040u), prmt_b(b[6], b[7], 0x0040u), 0x5410u);
@@ -229,10 +218,11 @@ __device__ __forceinline__ float2 block_min_max(float lo, float hi, float *smem)
 // zx can add up to one step outside 0..255).
 __device__ __forceinline__ uint2 quantize8_asym(const uint64_t (&p)[4], uint64_t rr, int shift)
 {
+    const uint64_t magic = pair(12582912.0f, 12582912.0f);
     uint32_t b[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        magic_round2(mul2(p[i], rr), b[2 * i], b[2 * i + 1]);
+        unpair(add2(mul2(p[i], rr), magic), b[2 * i], b[2 * i + 1]);
         b[2 * i] = (uint32_t)max(-128, min(127, (int)b[2 * i] + shift));
         b[2 * i + 1] = (uint32_t)max(-128, min(127, (int)b[2 * i + 1] + shift));
     }
