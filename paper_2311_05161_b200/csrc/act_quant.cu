@@ -10,72 +10,36 @@ namespace {
 
 constexpr int kActThreads = 256;
 
-// Pairs of FP32 values in 64-bit registers for the packed FP32 instructions (two lanes per
-// instruction, each lane rounded like the scalar instruction): the kernel is bound by its
-// instruction count, not by HBM, so the arithmetic is done two elements at a time.
-__device__ __forceinline__ uint64_t pair(float lo, float hi)
-{
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(__float_as_uint(lo)), "r"(__float_as_uint(hi)));
-    return r;
-}
-__device__ __forceinline__ void unpair(uint64_t v, uint32_t &lo, uint32_t &hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
-{
-    uint64_t r;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
-{
-    uint64_t r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-
-// Eight FP16 values -> four pairs of FP32, times the per-channel reciprocal scale when given.
 __device__ __forceinline__ void scaled8(const uint4 &v, const float *__restrict__ inv_s, int k0,
-                                        uint64_t (&p)[4])
+                                        float (&x)[8])
 {
     const __half2 *h2 = reinterpret_cast<const __half2 *>(&v);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const float2 f = __half22float2(h2[i]);
-        p[i] = pair(f.x, f.y);
+        x[2 * i] = f.x;
+        x[2 * i + 1] = f.y;
     }
     if (inv_s) {
         const float4 a = __ldg(reinterpret_cast<const float4 *>(inv_s + k0));
         const float4 b = __ldg(reinterpret_cast<const float4 *>(inv_s + k0 + 4));
-        p[0] = mul2(p[0], pair(a.x, a.y));
-        p[1] = mul2(p[1], pair(a.z, a.w));
-        p[2] = mul2(p[2], pair(b.x, b.y));
-        p[3] = mul2(p[3], pair(b.z, b.w));
+        x[0] = __fmul_rn(x[0], a.x); x[1] = __fmul_rn(x[1], a.y);
+        x[2] = __fmul_rn(x[2], a.z); x[3] = __fmul_rn(x[3], a.w);
+        x[4] = __fmul_rn(x[4], b.x); x[5] = __fmul_rn(x[5], b.y);
+        x[6] = __fmul_rn(x[6], b.z); x[7] = __fmul_rn(x[7], b.w);
     }
 }
 
-__device__ __forceinline__ float absmax8(const uint64_t (&p)[4], float amax)
+// rint(x * r) clamped to +-127, as the low byte of the result.  The product is rounded to
+// binary32 first (as in the reference arithmetic), then adding 1.5 * 2^23 rounds it to an
+// integer, half to even, and leaves that integer in the low mantissa bits (two's complement
+// in the low byte): two FP32 instructions instead of a float-to-int conversion, which the SM
+// issues at an eighth of the FP32 rate and which bounded this kernel.
+__device__ __forceinline__ uint32_t round_clamp_bits(float x, float r)
 {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        uint32_t lo, hi;
-        unpair(p[i], lo, hi);
-        amax = fmaxf(amax, fmaxf(fabsf(__uint_as_float(lo)), fabsf(__uint_as_float(hi))));
-    }
-    return amax;
-}
-
-__device__ __forceinline__ void minmax8(const uint64_t (&p)[4], float &mn, float &mx)
-{
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        uint32_t lo, hi;
-        unpair(p[i], lo, hi);
-        mn = fminf(mn, fminf(__uint_as_float(lo), __uint_as_float(hi)));
-        mx = fmaxf(mx, fmaxf(__uint_as_float(lo), __uint_as_float(hi)));
-    }
+    float p = __fmul_rn(x, r);
+    p = fminf(fmaxf(p, -127.0f), 127.0f);
+    return __float_as_uint(__fadd_rn(p, 12582912.0f));
 }
 
 __device__ __forceinline__ uint32_t prmt_b(uint32_t a, uint32_t b, uint32_t sel)
@@ -85,21 +49,19 @@ __device__ __forceinline__ uint32_t prmt_b(uint32_t a, uint32_t b, uint32_t sel)
     return d;
 }
 
-// rint(x * r) for eight values, as eight bytes.  The product is rounded to binary32 first (as
-// in the reference arithmetic); adding 1.5 * 2^23 then rounds it to an integer, half to even,
-// and leaves it in the low mantissa bits, two's complement in the low byte: two packed FP32
-// instructions per pair instead of float-to-int conversions (an eighth of the FP32 rate).
-// No clamp is needed: |x| <= amax and r = fl(127 / amax) give |x * r| <= 127 (1 + 2^-23),
-// which rounds to 127.
-__device__ __forceinline__ uint2 quantize8(const uint64_t (&p)[4], uint64_t rr)
+__device__ __forceinline__ uint32_t pack4(const float *x, float r)
 {
-    const uint64_t magic = pair(12582912.0f, 12582912.0f);
-    uint32_t b[8];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) unpair(add2(mul2(p[i], rr), magic), b[2 * i], b[2 * i + 1]);
+    const uint32_t a = round_clamp_bits(x[0], r), b = round_clamp_bits(x[1], r);
+    const uint32_t c = round_clamp_bits(x[2], r), d = round_clamp_bits(x[3], r);
+    // low bytes of a, b, c, d in that order
+    return prmt_b(prmt_b(a, b, 0x0040u), prmt_b(c, d, 0x0040u), 0x5410u);
+}
+
+__device__ __forceinline__ uint2 quantize8(const float (&x)[8], float r)
+{
     uint2 o;
-    o.x = prmt_b(prmt_b(b[0], b[1], 0x0040u), prmt_b(b[2], b[3], 0x0040u), 0x5410u);
-    o.y = prmt_b(prmt_b(b[4], b[5], 0x0040u), prmt_b(b[6], b[7], 0x0040u), 0x5410u);
+    o.x = pack4(x, r);
+    o.y = pack4(x + 4, r);
     return o;
 }
 
@@ -144,16 +106,18 @@ act_quant_kernel(const __half *__restrict__ X, const float *__restrict__ inv_s, 
         for (int i = 0; i < NR; ++i) {
             const int idx = tid + i * kActThreads;
             if (idx < nvec) {
-                uint64_t x[4];
+                float x[8];
                 scaled8(v[i], inv_s, idx * 8, x);
-                amax = absmax8(x, amax);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(x[e]));
             }
         }
     } else {
         for (int idx = tid; idx < nvec; idx += kActThreads) {
-            uint64_t x[4];
+            float x[8];
             scaled8(__ldg(row + idx), inv_s, idx * 8, x);
-            amax = absmax8(x, amax);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(x[e]));
         }
     }
     amax = block_max(amax, red);
@@ -163,23 +127,22 @@ act_quant_kernel(const __half *__restrict__ X, const float *__restrict__ inv_s, 
         return;
     }
     const float r = __fdiv_rn(127.0f, amax);
-    const uint64_t rr = pair(r, r);
     if (tid == 0) tok_scale[m] = __fdiv_rn(amax, 127.0f);
     if (NV > 0) {
 #pragma unroll
         for (int i = 0; i < NR; ++i) {
             const int idx = tid + i * kActThreads;
             if (idx < nvec) {
-                uint64_t x[4];
+                float x[8];
                 scaled8(v[i], inv_s, idx * 8, x);
-                out[idx] = quantize8(x, rr);
+                out[idx] = quantize8(x, r);
             }
         }
     } else {
         for (int idx = tid; idx < nvec; idx += kActThreads) {
-            uint64_t x[4];
+            float x[8];
             scaled8(__ldg(row + idx), inv_s, idx * 8, x);
-            out[idx] = quantize8(x, rr);
+            out[idx] = quantize8(x, r);
         }
     }
 }
@@ -212,23 +175,22 @@ __device__ __forceinline__ float2 block_min_max(float lo, float hi, float *smem)
     return make_float2(a, b);
 }
 
-// rint(x * r) + zx clamped to 0..255, minus 128, for eight values, as eight bytes: the packed
-// multiply and magic-number add as in quantize8, then `shift` = zx - 128 - bits(1.5 * 2^23) turns
-// the bits into the answer, which is clamped as an integer (the two roundings of rint(x * r) and
-// zx can add up to one step outside 0..255).
-__device__ __forceinline__ uint2 quantize8_asym(const uint64_t (&p)[4], uint64_t rr, int shift)
+// rint(x * r) + zx clamped to 0..255, minus 128, as the low byte of the result: the product
+// is rounded to binary32, adding 1.5 * 2^23 rounds it to an integer (half to even) in the low
+// mantissa bits, and `shift` = zx - 128 - bits(1.5 * 2^23) turns those bits into the answer.
+__device__ __forceinline__ uint32_t asym_bits(float x, float r, int shift)
 {
-    const uint64_t magic = pair(12582912.0f, 12582912.0f);
-    uint32_t b[8];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        unpair(add2(mul2(p[i], rr), magic), b[2 * i], b[2 * i + 1]);
-        b[2 * i] = (uint32_t)max(-128, min(127, (int)b[2 * i] + shift));
-        b[2 * i + 1] = (uint32_t)max(-128, min(127, (int)b[2 * i + 1] + shift));
-    }
+    const int q = (int)__float_as_uint(__fadd_rn(__fmul_rn(x, r), 12582912.0f)) + shift;
+    return (uint32_t)max(-128, min(127, q));
+}
+
+__device__ __forceinline__ uint2 quantize8_asym(const float (&x)[8], float r, int shift)
+{
     uint2 o;
-    o.x = prmt_b(prmt_b(b[0], b[1], 0x0040u), prmt_b(b[2], b[3], 0x0040u), 0x5410u);
-    o.y = prmt_b(prmt_b(b[4], b[5], 0x0040u), prmt_b(b[6], b[7], 0x0040u), 0x5410u);
+    o.x = prmt_b(prmt_b(asym_bits(x[0], r, shift), asym_bits(x[1], r, shift), 0x0040u),
+                 prmt_b(asym_bits(x[2], r, shift), asym_bits(x[3], r, shift), 0x0040u), 0x5410u);
+    o.y = prmt_b(prmt_b(asym_bits(x[4], r, shift), asym_bits(x[5], r, shift), 0x0040u),
+                 prmt_b(asym_bits(x[6], r, shift), asym_bits(x[7], r, shift), 0x0040u), 0x5410u);
     return o;
 }
 
@@ -260,16 +222,18 @@ act_quant_asym_kernel(const __half *__restrict__ X, const float *__restrict__ in
         for (int i = 0; i < NR; ++i) {
             const int idx = tid + i * kActThreads;
             if (idx < nvec) {
-                uint64_t x[4];
+                float x[8];
                 scaled8(v[i], inv_s, idx * 8, x);
-                minmax8(x, lo, hi);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { lo = fminf(lo, x[e]); hi = fmaxf(hi, x[e]); }
             }
         }
     } else {
         for (int idx = tid; idx < nvec; idx += kActThreads) {
-            uint64_t x[4];
+            float x[8];
             scaled8(__ldg(row + idx), inv_s, idx * 8, x);
-            minmax8(x, lo, hi);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { lo = fminf(lo, x[e]); hi = fmaxf(hi, x[e]); }
         }
     }
     const float2 mm = block_min_max(lo, hi, red);
@@ -284,22 +248,21 @@ act_quant_asym_kernel(const __half *__restrict__ X, const float *__restrict__ in
     const int zx = max(0, min(255, __float2int_rn(__fmul_rn(-mm.x, r))));
     if (tid == 0) { tok_scale[m] = __fdiv_rn(d, 255.0f); tok_zero[m] = zx - 128; }
     const int shift = zx - 128 - 0x4B400000;
-    const uint64_t rr = pair(r, r);
     if (NV > 0) {
 #pragma unroll
         for (int i = 0; i < NR; ++i) {
             const int idx = tid + i * kActThreads;
             if (idx < nvec) {
-                uint64_t x[4];
+                float x[8];
                 scaled8(v[i], inv_s, idx * 8, x);
-                out[idx] = quantize8_asym(x, rr, shift);
+                out[idx] = quantize8_asym(x, r, shift);
             }
         }
     } else {
         for (int idx = tid; idx < nvec; idx += kActThreads) {
-            uint64_t x[4];
+            float x[8];
             scaled8(__ldg(row + idx), inv_s, idx * 8, x);
-            out[idx] = quantize8_asym(x, rr, shift);
+            out[idx] = quantize8_asym(x, r, shift);
         }
     }
 }
