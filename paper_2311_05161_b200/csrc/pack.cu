@@ -198,18 +198,24 @@ __global__ void unpack_kernel(const uint8_t *__restrict__ blob, BlobLayout L,
 }
 
 // rowsum[g][n] = sum over the k of group g of t2(code[n][k]) (Eq. 6 in units of step/2): the
-// factor of a token's zero-point in the asymmetric-activation path.  One CTA per 128-row tile,
-// one thread per row; a warp reads 512 contiguous bytes per quarter tile.
+// factor of a token's zero-point in the asymmetric-activation path.  One CTA per 128-row tile
+// and K slice, one thread per row; a warp reads 512 contiguous bytes per quarter tile.
+// Per-channel weights: the slices add into rowsum[n] (zeroed by the launcher) with integer
+// atomics, so the result does not depend on their order.  Group mode: a slice is one k-block
+// and owns its entry.
 __global__ void __launch_bounds__(128)
-rowsum_kernel(const uint8_t *__restrict__ blob, BlobLayout L, int32_t *__restrict__ rowsum)
+rowsum_kernel(const uint8_t *__restrict__ blob, BlobLayout L, int kb_per_slice,
+              int32_t *__restrict__ rowsum)
 {
     const int nt = blockIdx.x, r = threadIdx.x;
     const int n = nt * kTileN + r;
     const uint8_t *zeros = blob + L.off_zeros;
     const uint8_t *codes = blob + L.off_codes;
+    const int kb0 = blockIdx.y * kb_per_slice;
+    const int kb1 = min(L.k_blocks, kb0 + kb_per_slice);
     int z = zeros[n];
     int sum = 0;
-    for (int kb = 0; kb < L.k_blocks; ++kb) {
+    for (int kb = kb0; kb < kb1; ++kb) {
         if (L.group != 0) { z = zeros[(size_t)kb * L.n_pad + n]; sum = 0; }
         const uint8_t *tile = codes + ((size_t)nt * L.k_blocks + kb) * kTileBytes;
         for (int q = 0; q < 4; ++q) {
@@ -220,7 +226,7 @@ rowsum_kernel(const uint8_t *__restrict__ blob, BlobLayout L, int32_t *__restric
         }
         if (L.group != 0 && n < L.N) rowsum[(size_t)kb * L.N + n] = sum;
     }
-    if (L.group == 0 && n < L.N) rowsum[n] = sum;
+    if (L.group == 0 && n < L.N) atomicAdd(rowsum + n, sum);
 }
 
 }  // namespace
@@ -248,7 +254,20 @@ cudaError_t launch_unpack(const uint8_t *blob, const BlobLayout &L, uint8_t *cod
 cudaError_t launch_weight_rowsum(const uint8_t *blob, const BlobLayout &L, int32_t *rowsum,
                                  cudaStream_t st)
 {
-    rowsum_kernel<<<L.n_tiles, 128, 0, st>>>(blob, L, rowsum);
+    // enough CTAs to fill the GPU: K slices of at least one k-block
+    int slices = 1;
+    if (L.group != 0) {
+        slices = L.k_blocks;
+    } else {
+        slices = (8 * 148 + L.n_tiles - 1) / L.n_tiles;
+        if (slices > L.k_blocks) slices = L.k_blocks;
+        if (cudaMemsetAsync(rowsum, 0, (size_t)L.N * sizeof(int32_t), st) != cudaSuccess)
+            return cudaGetLastError();
+    }
+    const int per = (L.k_blocks + slices - 1) / slices;
+    slices = (L.k_blocks + per - 1) / per;
+    if (slices > 65535) return cudaErrorInvalidValue;
+    rowsum_kernel<<<dim3(L.n_tiles, slices), 128, 0, st>>>(blob, L, per, rowsum);
     return cudaGetLastError();
 }
 
