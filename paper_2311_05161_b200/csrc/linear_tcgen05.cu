@@ -1062,7 +1062,11 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
                 if (slices != sp) continue;                  // the same plan as a smaller split
                 const long long units = tiles_t * slices;
                 const double rounds = (double)((units + sms - 1) / sms);
-                double cost = rounds * (per + 4.0 + (slices > 1 ? 1.0 : 0.0));
+                // a k-block costs a little more with a wide token tile (the MMAs), a unit costs
+                // its epilogue (by tile width) plus pipeline fill, a split unit its partial
+                // tile's round trip; constants fitted to measured mid-size shapes
+                const double kb_cost = 1.0 + 0.1 * t / 256.0;
+                double cost = rounds * (per * kb_cost + 2.0 + t / 64.0 + (slices > 1 ? 6.0 : 0.0));
                 if (slices > 1) cost += 1.5 * tokens * slices / 16.0;
                 if (best_tok == 0 || cost < best * 0.999) {
                     best = cost;
