@@ -273,6 +273,66 @@ def linear_asym(Q, tok_scale, tok_zero, codes, scales, zeros, bias=None, wide: b
     return (Y, W) if wide else Y
 
 
+# ---- special value s / 2^shift (App. A.5): shift = 1 is Eq. 5 / Eq. 6 --------------------
+
+def dint_quantize_fmt(x: float, s: float, z: int, shift: int, b: int = 4) -> int:
+    fn = lib().oracle_dint_quantize_fmt
+    fn.restype = ctypes.c_int
+    fn.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_int, ctypes.c_int, ctypes.c_int]
+    return int(fn(x, s, z, b, shift))
+
+
+def dint_dequantize_fmt(code: int, s: float, z: int, shift: int, b: int = 4) -> float:
+    fn = lib().oracle_dint_dequantize_fmt
+    fn.restype = ctypes.c_float
+    fn.argtypes = [ctypes.c_int, ctypes.c_float, ctypes.c_int, ctypes.c_int, ctypes.c_int]
+    return float(fn(code, s, z, b, shift))
+
+
+def dint_table_fmt(z: int, shift: int, b: int = 4) -> np.ndarray:
+    t = np.zeros(1 << b, dtype=np.int8)
+    lib().oracle_dint_table_fmt(ctypes.c_int(z), ctypes.c_int(b), ctypes.c_int(shift), _p(t))
+    return t
+
+
+def pack_weights_fmt(W, s_in, group: int, shift: int, clip: float = 1.0):
+    """pack_weights with the special value step / 2^shift."""
+    W = _c(W, np.float16)
+    N, K = W.shape
+    if s_in is not None:
+        s_in = _c(s_in, np.float32)
+    G = K // group if group else 1
+    codes = np.empty((N, K // 2), dtype=np.uint8)
+    scales = np.empty((G, N), dtype=np.float32)
+    zeros = np.empty((G, N), dtype=np.uint8)
+    lib().oracle_pack_weights_fmt(_p(W.view(np.uint16)), _p(s_in) if s_in is not None else None,
+                                  ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group),
+                                  ctypes.c_float(clip), ctypes.c_int(shift), _p(codes), _p(scales),
+                                  _p(zeros))
+    return codes, scales, zeros
+
+
+def linear_fmt(Xq, tok_scale, codes, scales, zeros, bias, group: int, shift: int):
+    """(acc int64 [G, M, N], Y bf16 bits [M, N], Y binary64 [M, N]) with levels in units of
+    step / 2^shift."""
+    Xq = _c(Xq, np.int8)
+    tok_scale = _c(tok_scale, np.float32)
+    codes = _c(codes, np.uint8)
+    zeros = _c(zeros, np.uint8)
+    scales = _c(scales, np.float32)
+    M, N, K, G = _shape(Xq, codes, zeros, group)
+    if bias is not None:
+        bias = _c(bias, np.float32)
+    acc = np.empty((G, M, N), dtype=np.int64)
+    Y = np.empty((M, N), dtype=np.uint16)
+    wide = np.empty((M, N), dtype=np.float64)
+    lib().oracle_linear_fmt(_p(Xq), _p(tok_scale), _p(codes), _p(scales), _p(zeros),
+                            _p(bias) if bias is not None else None, ctypes.c_int(M),
+                            ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group),
+                            ctypes.c_int(shift), _p(acc), _p(Y), _p(wide))
+    return acc, Y, wide
+
+
 def bf16_bits_to_float(bits: np.ndarray) -> np.ndarray:
     """Widen BF16 bit patterns (uint16) to float32 values (exact)."""
     return (bits.astype(np.uint32) << 16).view(np.float32)

@@ -440,6 +440,115 @@ void oracle_linear_asym(const uint8_t *Q, const float *tok_scale, const int32_t 
 }
 
 /* ------------------------------------------------------------------------- */
+/* other special values: c = s / 2^j (App. A.5 sweeps c/s = 0.5, 0.25, 0.125)  */
+/* ------------------------------------------------------------------------- */
+
+/* Section 4.2 asks for a special value that is the step size over a power of two; Eq. 5 and
+ * Eq. 6 are written for c = s/2 and the appendix gives no formulas for the others.  The
+ * reading here keeps Eq. 5's structure: a value goes to +-c when it lies between the midpoints
+ * of (0, c) and (c, s), i.e. c/2 < |x| <= (c + s)/2, with the same strictness as Eq. 5, and is
+ * rounded to the integer grid otherwise.  j = 1 reproduces Eq. 5 / Eq. 6 exactly. */
+int oracle_dint_quantize_fmt(float x, float s, int z, int b, int j)
+{
+    const int p = oracle_dint_p(b);
+    const float lower = ldexpf(s, -(j + 1));          /* c / 2 */
+    const float upper = 0.5f * s + lower;              /* (c + s) / 2 */
+    if (x > lower && x <= upper) return p + 1;
+    if (x < -lower && x >= -upper) return p + 2;
+    return clampi(rint_to_int(x / s) + z, 0, p);
+}
+
+float oracle_dint_dequantize_fmt(int code, float s, int z, int b, int j)
+{
+    const int p = oracle_dint_p(b);
+    if (code == p + 1) return ldexpf(s, -j);
+    if (code == p + 2) return -ldexpf(s, -j);
+    return (float)(code - z) * s;
+}
+
+/* Levels in units of c = s / 2^j: 2^j (code - z) for the integer levels, +1 and -1. */
+void oracle_dint_table_fmt(int z, int b, int j, int8_t *t)
+{
+    const int p = oracle_dint_p(b);
+    for (int c = 0; c <= p; ++c) t[c] = (int8_t)((c - z) * (1 << j));
+    t[p + 1] = 1;
+    t[p + 2] = -1;
+}
+
+/* oracle_pack_weights with the special value s / 2^j. */
+void oracle_pack_weights_fmt(const uint16_t *W, const float *s_in, int N, int K, int group,
+                             float clip, int j, uint8_t *codes, float *scales, uint8_t *zeros)
+{
+    const int glen = group ? group : K;
+    const int G = K / glen;
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        for (int g = 0; g < G; ++g) {
+            float lo = 0.0f, hi = 0.0f;
+            for (int k = g * glen; k < (g + 1) * glen; ++k) {
+                float w = half_bits_to_float(W[(size_t)n * K + k]);
+                if (s_in) w = w * s_in[k];
+                if (w < lo) lo = w;
+                if (w > hi) hi = w;
+            }
+            lo = lo * clip;
+            hi = hi * clip;
+            float s = (hi - lo) / 13.0f;
+            if (s == 0.0f) s = 1.0f;
+            const int z = clampi(rint_to_int((-lo) / s), 0, 13);
+            scales[(size_t)g * N + n] = s;
+            zeros[(size_t)g * N + n] = (uint8_t)z;
+            for (int k = g * glen; k < (g + 1) * glen; k += 2) {
+                float w0 = half_bits_to_float(W[(size_t)n * K + k]);
+                float w1 = half_bits_to_float(W[(size_t)n * K + k + 1]);
+                if (s_in) { w0 = w0 * s_in[k]; w1 = w1 * s_in[k + 1]; }
+                const int c0 = oracle_dint_quantize_fmt(w0, s, z, 4, j);
+                const int c1 = oracle_dint_quantize_fmt(w1, s, z, 4, j);
+                codes[(size_t)n * (K / 2) + k / 2] = (uint8_t)(c0 | (c1 << 4));
+            }
+        }
+    }
+}
+
+/* The layer with levels in units of s / 2^j: integer sums acc [G][M][N] (may be NULL), BF16
+ * output Y (may be NULL) in the evaluation order of oracle_linear with the level unit
+ * 2^-j * s in place of 0.5 * s, and the same value in binary64 (may be NULL). */
+void oracle_linear_fmt(const int8_t *Xq, const float *tok_scale, const uint8_t *codes,
+                       const float *scales, const uint8_t *zeros, const float *bias, int M,
+                       int N, int K, int group, int j, int64_t *acc, uint16_t *Y, double *wide)
+{
+    const int glen = group ? group : K;
+    const int G = K / glen;
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        for (int m = 0; m < M; ++m) {
+            float u = 0.0f, t = 0.0f;
+            double w = 0.0;
+            for (int g = 0; g < G; ++g) {
+                int8_t lv[16];
+                oracle_dint_table_fmt(zeros[(size_t)g * N + n], 4, j, lv);
+                int64_t sum = 0;
+                for (int k = g * glen; k < (g + 1) * glen; ++k) {
+                    const uint8_t byte = codes[(size_t)n * (K / 2) + k / 2];
+                    const int code = (k & 1) ? (byte >> 4) : (byte & 15);
+                    sum += (int64_t)Xq[(size_t)m * K + k] * (int64_t)lv[code];
+                }
+                if (acc) acc[((size_t)g * M + m) * N + n] = sum;
+                const float h = ldexpf(scales[(size_t)g * N + n], -j);
+                if (G == 1) t = ((float)(int32_t)sum * (tok_scale ? tok_scale[m] : 0.0f)) * h;
+                else u = fmaf((float)(int32_t)sum, h, u);
+                w += (double)sum * (double)h;
+            }
+            if (G != 1) t = u * (tok_scale ? tok_scale[m] : 0.0f);
+            w *= tok_scale ? (double)tok_scale[m] : 0.0;
+            if (bias) { t = t + bias[n]; w += (double)bias[n]; }
+            if (Y) Y[(size_t)m * N + n] = float_to_bf16_bits(t);
+            if (wide) wide[(size_t)m * N + n] = w;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------- */
 /* threading of the outermost loops (sums are integer, so order-free)         */
 /* ------------------------------------------------------------------------- */
 
