@@ -61,7 +61,9 @@ typedef struct {
     int split_k;     /* 0 = automatic; else number of K slices (tcgen05 path) */
     int tok_tile;    /* 0 = automatic; else tokens per tile: 16, 32, 64, 128 or 256 */
     int decode_warps;/* 0 = automatic; else warps that expand codes to INT8: 4, 8 or 16 */
-    int reserved[4]; /* must be zero */
+    int level_shift; /* special value of the blob = step / 2^level_shift: 0 or 1 (the paper's
+                        step/2), 2 or 3 (w4a8_pack_weights_fmt); must match the blob */
+    int reserved[3]; /* must be zero */
 } w4a8_opts;
 
 /* Bytes of the packed-weight blob for an [N][K] matrix; 0 if the shape is invalid.
@@ -84,6 +86,18 @@ size_t w4a8_packed_bytes(int N, int K, int group_size);
 w4a8_status w4a8_pack_weights(const void *W_f16, const float *s_in, int N, int K,
                               int group_size, float clip, void *packed,
                               size_t packed_bytes, void *stream);
+
+/* w4a8_pack_weights with another special value: c = step / 2^level_shift, level_shift 1 (the
+ * paper's step/2, Eq. 5 / Eq. 6), 2 or 3 (step/4, step/8: the sweep of Appendix A.5).  A
+ * value becomes +-c when c/2 < |x| <= (c + step)/2 (the midpoints towards 0 and towards
+ * +-step; Eq. 5's s/4 and 3s/4 for level_shift 1).  The levels are then integers in units of
+ * c: 2^level_shift (code - z), +1, -1, and the linear calls rescale by step / 2^level_shift.
+ * Linear calls on such a blob pass the same level_shift in their options: w4a8_linear_ex,
+ * w4a8_linear_acc_i32, w4a8_linear_asym; a mismatch is reported as W4A8_ERR_BAD_BLOB.
+ * K is limited so that K * 127 * 13 * 2^level_shift < 2^31. */
+w4a8_status w4a8_pack_weights_fmt(const void *W_f16, const float *s_in, int N, int K,
+                                  int group_size, float clip, int level_shift, void *packed,
+                                  size_t packed_bytes, void *stream);
 
 /* Activation side of Eq. 1, token-wise INT8 (Appendix A.1), every forward pass.
  *   X_f16     [M][K] IEEE binary16.
@@ -207,6 +221,9 @@ w4a8_status w4a8_poll_status(void *workspace, void *stream);
 /* Host: Eq. 6 in units of step/2 for zero-point z: out[code] = 2 (code - z) for
  * code <= 13, +1 for 14, -1 for 15.  `out` is a host array of 16. */
 void w4a8_dint4_table(int z, int8_t *out);
+
+/* Host: the same table in units of step / 2^level_shift: 2^level_shift (code - z), +1, -1. */
+void w4a8_dint4_table_fmt(int z, int level_shift, int8_t *out);
 
 /* Host: version string with static storage. */
 const char *w4a8_version(void);

@@ -28,6 +28,7 @@ EXPORTS = (
     "w4a8_linear", "w4a8_linear_ex", "w4a8_linear_static", "w4a8_linear_acc_i32", "w4a8_unpack_codes",
     "w4a8_poll_status", "w4a8_dint4_table", "w4a8_version",
     "w4a8_quantize_act_asym", "w4a8_weight_rowsum", "w4a8_linear_asym",
+    "w4a8_pack_weights_fmt", "w4a8_dint4_table_fmt",
 )
 
 
@@ -39,7 +40,8 @@ class W4A8Error(RuntimeError):
 
 class Opts(ctypes.Structure):
     _fields_ = [("path", ctypes.c_int), ("split_k", ctypes.c_int), ("tok_tile", ctypes.c_int),
-                ("decode_warps", ctypes.c_int), ("reserved", ctypes.c_int * 4)]
+                ("decode_warps", ctypes.c_int), ("level_shift", ctypes.c_int),
+                ("reserved", ctypes.c_int * 3)]
 
 
 def _load() -> ctypes.CDLL:
@@ -68,6 +70,8 @@ def _load() -> ctypes.CDLL:
     lib.w4a8_linear_ex.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, vp, op]
     lib.w4a8_linear_static.restype = ci
     lib.w4a8_linear_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp]
+    lib.w4a8_pack_weights_fmt.restype = ci
+    lib.w4a8_pack_weights_fmt.argtypes = [vp, vp, ci, ci, ci, cf, ci, vp, sz, vp]
     lib.w4a8_quantize_act_asym.restype = ci
     lib.w4a8_quantize_act_asym.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp]
     lib.w4a8_weight_rowsum.restype = ci
@@ -112,9 +116,10 @@ def _dev(t, dtype, what):
 
 
 def make_opts(path: int = PATH_AUTO, split_k: int = 0, tok_tile: int = 0,
-              decode_warps: int = 0) -> Opts:
+              decode_warps: int = 0, level_shift: int = 0) -> Opts:
     o = Opts()
     o.path, o.split_k, o.tok_tile, o.decode_warps = path, split_k, tok_tile, decode_warps
+    o.level_shift = level_shift
     return o
 
 
@@ -132,8 +137,9 @@ def packed_bytes(N: int, K: int, group: int = 0) -> int:
     return int(lib.w4a8_packed_bytes(N, K, group))
 
 
-def pack_weights(W, s_in=None, group: int = 0, clip: float = 1.0, out=None):
-    """W [N, K] float16 (CUDA) -> packed blob (uint8 CUDA tensor)."""
+def pack_weights(W, s_in=None, group: int = 0, clip: float = 1.0, out=None, level_shift: int = 1):
+    """W [N, K] float16 (CUDA) -> packed blob (uint8 CUDA tensor); special value
+    step / 2^level_shift."""
     W = _dev(W, torch.float16, "W")
     s_in = _dev(s_in, torch.float32, "s_in")
     N, K = W.shape
@@ -142,8 +148,8 @@ def pack_weights(W, s_in=None, group: int = 0, clip: float = 1.0, out=None):
         raise W4A8Error(2, "w4a8_packed_bytes")
     if out is None:
         out = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
-    _check(lib.w4a8_pack_weights(_ptr(W), _ptr(s_in), N, K, group, clip, _ptr(out),
-                                 out.numel(), _stream()), "w4a8_pack_weights")
+    _check(lib.w4a8_pack_weights_fmt(_ptr(W), _ptr(s_in), N, K, group, clip, level_shift, _ptr(out),
+                                     out.numel(), _stream()), "w4a8_pack_weights")
     return out
 
 

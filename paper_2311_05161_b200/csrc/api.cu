@@ -22,9 +22,19 @@ bool opts_ok(const w4a8_opts *o)
     if (!o) return true;
     if (o->path < W4A8_PATH_AUTO || o->path > W4A8_PATH_GEMV) return false;
     if (o->split_k < 0 || o->tok_tile < 0 || o->decode_warps < 0) return false;
-    for (int i = 0; i < 4; ++i)
+    if (o->level_shift < 0 || o->level_shift > 3) return false;
+    for (int i = 0; i < 3; ++i)
         if (o->reserved[i] != 0) return false;
     return true;
+}
+
+// special value = step / 2^shift; 0 in the options means the paper's 1
+int shift_of(const w4a8_opts *o) { return (o && o->level_shift) ? o->level_shift : 1; }
+
+// |level| <= 13 * 2^shift and |activation| <= amax: the INT32 sums must not overflow
+bool depth_ok(int K, int shift, int amax)
+{
+    return (long long)K * amax * (13LL << shift) < (1LL << 31);
 }
 
 // The weight-streaming kernel can serve one to four tokens (on request, any of them).  By
@@ -47,6 +57,7 @@ w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *
     if (!Y && !acc) return W4A8_ERR_NULL;
     if (Y && !tok_scale) return W4A8_ERR_NULL;
     if (!shape_ok(N, K, group) || M < 1 || !opts_ok(opts)) return W4A8_ERR_SHAPE;
+    if (!depth_ok(K, shift_of(opts), zp.tok_zero ? 255 : 127)) return W4A8_ERR_SHAPE;
     if (!aligned(Xq, 16) || !aligned(tok_scale, 4) || !aligned(bias, 4) || !aligned(Y, 16) ||
         !aligned(acc, 16) || !aligned(packed, 256) || !aligned(workspace, 256))
         return W4A8_ERR_ALIGN;
@@ -55,7 +66,7 @@ w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *
     if (workspace_bytes < need) return W4A8_ERR_BUFFER_TOO_SMALL;
     const w4a8_status arch = check_arch();
     if (arch != W4A8_OK) return arch;
-    const BlobLayout L = make_layout(N, K, group);
+    const BlobLayout L = make_layout(N, K, group, shift_of(opts));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint8_t *blob = static_cast<const uint8_t *>(packed);
     if (opts && opts->path == W4A8_PATH_SIMPLE) {
@@ -89,10 +100,19 @@ size_t w4a8_packed_bytes(int N, int K, int group_size)
 w4a8_status w4a8_pack_weights(const void *W_f16, const float *s_in, int N, int K, int group_size,
                               float clip, void *packed, size_t packed_bytes, void *stream)
 {
+    return w4a8_pack_weights_fmt(W_f16, s_in, N, K, group_size, clip, 1, packed, packed_bytes,
+                                 stream);
+}
+
+w4a8_status w4a8_pack_weights_fmt(const void *W_f16, const float *s_in, int N, int K,
+                                  int group_size, float clip, int level_shift, void *packed,
+                                  size_t packed_bytes, void *stream)
+{
     if (!W_f16 || !packed) return W4A8_ERR_NULL;
     if (!shape_ok(N, K, group_size) || !(clip > 0.0f && clip <= 1.0f)) return W4A8_ERR_SHAPE;
+    if (level_shift < 1 || level_shift > 3 || !depth_ok(K, level_shift, 127)) return W4A8_ERR_SHAPE;
     if (!aligned(W_f16, 16) || !aligned(s_in, 16) || !aligned(packed, 256)) return W4A8_ERR_ALIGN;
-    const BlobLayout L = make_layout(N, K, group_size);
+    const BlobLayout L = make_layout(N, K, group_size, level_shift);
     if (packed_bytes < L.total_bytes) return W4A8_ERR_BUFFER_TOO_SMALL;
     const w4a8_status arch = check_arch();
     if (arch != W4A8_OK) return arch;
@@ -212,8 +232,6 @@ w4a8_status w4a8_linear_asym(const int8_t *Xq, const float *tok_scale, const int
 {
     if (!tok_zero || !rowsum) return W4A8_ERR_NULL;
     if (!aligned(tok_zero, 4) || !aligned(rowsum, 4)) return W4A8_ERR_ALIGN;
-    // (Q - zx) spans 255 where the symmetric INT8 spans 127: the INT32 bound on K halves
-    if ((long long)K * 255 * 26 >= (1LL << 31)) return W4A8_ERR_SHAPE;
     ZeroPoint zp;
     zp.tok_zero = tok_zero;
     zp.rowsum = rowsum;
@@ -248,9 +266,11 @@ w4a8_status w4a8_poll_status(void *workspace, void *stream)
     return host[0] == W4A8_ERR_BAD_BLOB ? W4A8_ERR_BAD_BLOB : W4A8_ERR_TIMEOUT;
 }
 
-void w4a8_dint4_table(int z, int8_t *out)
+void w4a8_dint4_table(int z, int8_t *out) { w4a8_dint4_table_fmt(z, 1, out); }
+
+void w4a8_dint4_table_fmt(int z, int level_shift, int8_t *out)
 {
-    for (int c = 0; c < 16; ++c) out[c] = (int8_t)dint4_t2(c, z);
+    for (int c = 0; c < 16; ++c) out[c] = (int8_t)dint4_level(c, z, level_shift);
 }
 
 const char *w4a8_version(void) { return "w4a8-dint 0.1 (sm_100a)"; }

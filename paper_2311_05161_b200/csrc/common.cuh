@@ -27,7 +27,8 @@ constexpr uint32_t kBlobLayoutQuarterRow16 = 1u;
 struct BlobHeader {
     uint32_t magic, version, layout, group;
     int32_t N, K, G, n_tiles, k_blocks, n_pad;
-    uint32_t pad0[2];
+    uint32_t level_shift;   // special value = step / 2^level_shift; 0 (older blobs) means 1
+    uint32_t pad0;
     uint64_t off_scales, off_zeros, off_codes, total_bytes;
     float clip;
     uint32_t pad1[43];
@@ -36,14 +37,16 @@ static_assert(sizeof(BlobHeader) == kHeaderBytes, "blob header is 256 bytes");
 
 struct BlobLayout {
     int N, K, group, G, n_tiles, k_blocks, n_pad;
+    int shift;              // special value = step / 2^shift (1, 2 or 3); levels are in that unit
     size_t off_scales, off_zeros, off_codes, total_bytes;
 };
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-__host__ __device__ inline BlobLayout make_layout(int N, int K, int group)
+__host__ __device__ inline BlobLayout make_layout(int N, int K, int group, int shift = 1)
 {
     BlobLayout L;
+    L.shift = shift;
     L.N = N;
     L.K = K;
     L.group = group;
@@ -80,7 +83,8 @@ __device__ inline bool header_matches(const uint8_t *blob, const BlobLayout &L)
     const BlobHeader *h = reinterpret_cast<const BlobHeader *>(blob);
     return h->magic == kBlobMagic && h->version == kBlobVersion &&
            h->layout == kBlobLayoutQuarterRow16 && h->N == L.N && h->K == L.K &&
-           h->group == (uint32_t)L.group;
+           h->group == (uint32_t)L.group &&
+           (h->level_shift == 0u ? 1u : h->level_shift) == (uint32_t)L.shift;
 }
 
 // ---------------------------------------------------------------------------
@@ -103,11 +107,45 @@ __device__ inline void report_failure(StatusBlock *sb, int status, int where)
 }
 
 // ---------------------------------------------------------------------------
-// dINT4 decode in units of step/2 (Eq. 6 doubled)
+// dINT4 decode (Eq. 6) in units of the special value c = step / 2^shift, so that every
+// level is an integer: 2^shift (code - z) for the integer levels, +1 for c1, -1 for c2.
+// shift = 1 is the paper's c = step / 2; App. A.5 also tries step / 4 and step / 8.
 // ---------------------------------------------------------------------------
-__host__ __device__ inline int dint4_t2(int code, int z)
+__host__ __device__ inline int dint4_level(int code, int z, int shift)
 {
-    return code <= 13 ? 2 * (code - z) : (code == 14 ? 1 : -1);
+    return code <= 13 ? (code - z) * (1 << shift) : (code == 14 ? 1 : -1);
+}
+// the unit itself as a factor of the step: 2^-shift, exact
+__host__ __device__ inline float level_unit(int shift)
+{
+    return shift == 1 ? 0.5f : (shift == 2 ? 0.25f : 0.125f);
+}
+// Byte tables of the levels for the permute-based decode: table word w, byte i holds the level
+// of code 4 w + i.  A thread builds them as (base[w] - z * zmul) ^ 0x80808080 (bytes carry a
+// 0x80 offset so that the subtraction never borrows); base and zmul depend on the shift only.
+struct LevelTables {
+    uint32_t base[4];
+    uint32_t zmul;
+};
+inline LevelTables make_level_tables(int shift)
+{
+    const uint32_t m = 1u << shift;
+    LevelTables t;
+    t.base[0] = 0x80808080u + m * 0x03020100u;
+    t.base[1] = 0x80808080u + m * 0x07060504u;
+    t.base[2] = 0x80808080u + m * 0x0B0A0908u;
+    t.base[3] = 0x00008080u + m * 0x00000D0Cu;
+    t.zmul = m * 0x01010101u;
+    return t;
+}
+__device__ __forceinline__ void build_level_tables(int z, const LevelTables &lt, uint32_t (&t)[4])
+{
+    const uint32_t zz = (uint32_t)z * lt.zmul;
+    t[0] = (lt.base[0] - zz) ^ 0x80808080u;
+    t[1] = (lt.base[1] - zz) ^ 0x80808080u;
+    t[2] = (lt.base[2] - zz) ^ 0x80808080u;
+    // codes 12 and 13, then the two special values +1 and -1
+    t[3] = (((lt.base[3] - (zz & 0xFFFFu)) ^ 0x00008080u) & 0xFFFFu) | 0xFF010000u;
 }
 
 // ---------------------------------------------------------------------------

@@ -28,15 +28,6 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
     return d;
 }
 
-__device__ __forceinline__ void build_tables(int z, uint32_t (&t)[4])
-{
-    const uint32_t zz = (uint32_t)(2 * z) * 0x01010101u;
-    t[0] = ((0x86848280u) - zz) ^ 0x80808080u;
-    t[1] = ((0x8E8C8A88u) - zz) ^ 0x80808080u;
-    t[2] = ((0x96949290u) - zz) ^ 0x80808080u;
-    t[3] = ((((0x00009A98u) - (zz & 0xFFFFu)) ^ 0x00008080u) & 0xFFFFu) | 0xFF010000u;
-}
-
 __device__ __forceinline__ void decode8(uint32_t w, const uint32_t (&t)[4], uint32_t &o0,
                                         uint32_t &o1)
 {
@@ -75,6 +66,8 @@ struct GemvParams {
     BlobLayout L;
     int M, slices, kb_per_slice;
     ZeroPoint zp;
+    LevelTables lt;
+    float unit;          // level unit as a factor of the step: 2^-shift
 };
 
 template <int MT, bool GROUPED>
@@ -144,7 +137,7 @@ linear_gemv_kernel(const GemvParams P)
 #pragma unroll
     for (int m = 0; m < MT; ++m) { acc[m] = 0; usum[m] = 0.0f; }
     uint32_t t[4];
-    if (!GROUPED) build_tables(P.zeros[n], t);
+    if (!GROUPED) build_level_tables(P.zeros[n], P.lt, t);
 #pragma unroll 1
     for (int step = 0; step < steps; ++step) {
         // the group of this step is the oldest of kGemvDepth outstanding ones
@@ -162,7 +155,7 @@ linear_gemv_kernel(const GemvParams P)
             if (kl < kb_count) {
                 const int kb = kb_first + kl;
                 if (GROUPED) {
-                    build_tables(P.zeros[(size_t)kb * P.L.n_pad + n], t);
+                    build_level_tables(P.zeros[(size_t)kb * P.L.n_pad + n], P.lt, t);
 #pragma unroll
                     for (int m = 0; m < MT; ++m) acc[m] = 0;
                 }
@@ -183,7 +176,7 @@ linear_gemv_kernel(const GemvParams P)
                     }
                 }
                 if (GROUPED) {
-                    const float h = __fmul_rn(0.5f, P.scales[(size_t)kb * P.L.n_pad + n]);
+                    const float h = __fmul_rn(P.unit, P.scales[(size_t)kb * P.L.n_pad + n]);
 #pragma unroll
                     for (int m = 0; m < MT; ++m) {
                         usum[m] = fmaf((float)acc[m], h, usum[m]);
@@ -239,7 +232,7 @@ linear_gemv_kernel(const GemvParams P)
             if (P.zp.tok_zero) a -= P.zp.tok_zero[m] * P.zp.rowsum[n];
             if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = a;
             tv = rescale_channel(a, P.tok_scale ? P.tok_scale[m] : 0.0f,
-                                 __fmul_rn(0.5f, P.scales[n]));
+                                 __fmul_rn(P.unit, P.scales[n]));
         }
         if (P.bias) tv = __fadd_rn(tv, bias_n);
         if (P.Y) P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(tv);
@@ -307,6 +300,8 @@ w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const u
     P.slices = plan.split_k;
     P.kb_per_slice = plan.kb_per_split;
     P.zp = zp;
+    P.lt = make_level_tables(L.shift);
+    P.unit = level_unit(L.shift);
     if (P.slices > 65535) return W4A8_ERR_SHAPE;
     const dim3 grid(L.n_tiles, P.slices);
     const bool g = L.group != 0;

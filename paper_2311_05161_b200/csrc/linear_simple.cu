@@ -37,12 +37,12 @@ linear_simple_kernel(const int8_t *__restrict__ Xq, const float *__restrict__ to
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
                 const int code = (words[i >> 3] >> (4 * (i & 7))) & 15;
-                acc += (int32_t)xk[i] * dint4_t2(code, z);
+                acc += (int32_t)xk[i] * dint4_level(code, z, L.shift);
             }
         }
         if (grouped && n < L.N) {
             if (acc_out) acc_out[((size_t)kb * M + m) * L.N + n] = acc;
-            u = fmaf((float)acc, __fmul_rn(0.5f, scales[(size_t)kb * L.n_pad + n]), u);
+            u = fmaf((float)acc, __fmul_rn(level_unit(L.shift), scales[(size_t)kb * L.n_pad + n]), u);
         }
     }
     if (n >= L.N) return;
@@ -53,7 +53,7 @@ linear_simple_kernel(const int8_t *__restrict__ Xq, const float *__restrict__ to
     } else {
         if (zp.tok_zero) acc -= zp.tok_zero[m] * zp.rowsum[n];
         if (acc_out) acc_out[(size_t)m * L.N + n] = acc;
-        t = rescale_channel(acc, a, __fmul_rn(0.5f, scales[n]));
+        t = rescale_channel(acc, a, __fmul_rn(level_unit(L.shift), scales[n]));
     }
     if (Y) Y[(size_t)m * L.N + n] = __float2bfloat16_rn(add_bias(t, bias, n));
 }

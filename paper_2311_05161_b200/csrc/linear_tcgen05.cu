@@ -106,6 +106,8 @@ struct Params {
     BlobLayout L;
     int M, tok_tiles, m_pad, split_k, kb_per_split, total_units, prefetch_codes;
     ZeroPoint zp;
+    LevelTables lt;
+    float unit;          // level unit as a factor of the step: 2^-shift
 };
 
 // --------------------------------------------------------------------------- PTX wrappers
@@ -419,18 +421,6 @@ __device__ __forceinline__ uint4 ld_stream(const uint4 *p)
 }
 
 // --------------------------------------------------------------------------- decode
-// Byte tables of Eq. 6 in units of step/2 for zero-point z: t[c / 4] byte c % 4 holds
-// 2 (c - z) for c <= 13, +1 for c = 14, -1 for c = 15.
-__device__ __forceinline__ void build_tables(int z, uint32_t (&t)[4])
-{
-    const uint32_t zz = (uint32_t)(2 * z) * 0x01010101u;
-    // per byte: (0x80 + 2c) - 2z never borrows; the XOR removes the 0x80 again
-    t[0] = ((0x86848280u) - zz) ^ 0x80808080u;
-    t[1] = ((0x8E8C8A88u) - zz) ^ 0x80808080u;
-    t[2] = ((0x96949290u) - zz) ^ 0x80808080u;
-    t[3] = ((((0x00009A98u) - (zz & 0xFFFFu)) ^ 0x00008080u) & 0xFFFFu) | 0xFF010000u;
-}
-
 // Eight codes (nibble i = code of k0 + i) -> eight INT8 values, bytes in k order.
 __device__ __forceinline__ void decode8(uint32_t w, const uint32_t (&t)[4], uint32_t &o0,
                                         uint32_t &o1)
@@ -640,7 +630,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             const int st = cur.it % S;
             const uint32_t fill = cur.it / S;
             uint32_t t[4];
-            build_tables(z, t);
+            build_level_tables(z, P.lt, t);
             {
                 // the operand buffer is free once the MMAs of its last use have retired
                 ok = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
@@ -734,7 +724,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             }
 
             if (!GROUPED) {
-                const float half_step = __fmul_rn(0.5f, P.scales[n]);
+                const float half_step = __fmul_rn(P.unit, P.scales[n]);
                 // asymmetric activations: the token's zero-point times this row's level sum
                 // leaves the accumulator before the rescale (zero for the symmetric path)
                 const int row_sum = (P.zp.rowsum && n_ok) ? __ldg(P.zp.rowsum + n) : 0;
@@ -847,7 +837,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 float step_next = P.scales[(size_t)kb0 * P.L.n_pad + n];
                 constexpr int kAcc = 16;          // columns per tensor-memory load while accumulating
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    const uint32_t h_bits = __float_as_uint(__fmul_rn(0.5f, step_next));
+                    const uint32_t h_bits = __float_as_uint(__fmul_rn(P.unit, step_next));
                     const uint64_t h2 = pack_f32x2(h_bits, h_bits);
                     if (kb + 1 < kb1) step_next = P.scales[(size_t)(kb + 1) * P.L.n_pad + n];
                     const uint32_t buf = phase % NB;
@@ -1154,6 +1144,8 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     P.total_units = plan.tok_tiles * L.n_tiles * plan.split_k;
     P.prefetch_codes = plan.tok_tiles == 1 ? 1 : 0;   // every code tile is read exactly once
     P.zp = zp;
+    P.lt = make_level_tables(L.shift);
+    P.unit = level_unit(L.shift);
 
     const bool g = L.group != 0;
     switch (plan.tok_tile) {

@@ -8,7 +8,14 @@ namespace {
 
 constexpr int kPackThreads = 256;
 
-// Eq. 5 for b = 4: codes 0..13 integer levels, 14 = c1 (+s/2), 15 = c2 (-s/2).
+// Eq. 5 for b = 4: codes 0..13 integer levels, 14 = c1 (+c), 15 = c2 (-c), c = s / 2^shift.
+// A value is special between the midpoints of (0, c) and (c, s): `lower` = c / 2,
+// `upper` = (c + s) / 2, i.e. s/4 and 3s/4 for the paper's c = s/2.
+__device__ __forceinline__ void special_band(float s, int shift, float &lower, float &upper)
+{
+    lower = __fmul_rn(0.5f * level_unit(shift), s);
+    upper = shift == 1 ? __fmul_rn(0.75f, s) : __fadd_rn(__fmul_rn(0.5f, s), lower);
+}
 __device__ __forceinline__ uint32_t dint4_quantize(float x, float s, int z, float quarter,
                                                    float threeq)
 {
@@ -52,6 +59,7 @@ __device__ __forceinline__ void write_header(uint8_t *blob, const BlobLayout &L,
     h.off_scales = L.off_scales; h.off_zeros = L.off_zeros;
     h.off_codes = L.off_codes; h.total_bytes = L.total_bytes;
     h.clip = clip;
+    h.level_shift = (uint32_t)L.shift;
     *reinterpret_cast<BlobHeader *>(blob) = h;
 }
 
@@ -109,7 +117,8 @@ pack_rows_kernel(const __half *__restrict__ W, const float *__restrict__ s_in, B
     __syncthreads();
     const float s = s_step;
     const int z = s_zero;
-    const float quarter = __fmul_rn(0.25f, s), threeq = __fmul_rn(0.75f, s);
+    float quarter, threeq;
+    special_band(s, L.shift, quarter, threeq);
     for (int k0 = tid * 8; k0 < L.K; k0 += kPackThreads * 8) {
         uint32_t word = 0;
         if (real) {
@@ -164,7 +173,8 @@ pack_groups_kernel(const __half *__restrict__ W, const float *__restrict__ s_in,
             scales[(size_t)g * L.n_pad + n] = s;
             zeros[(size_t)g * L.n_pad + n] = (uint8_t)z;
         }
-        const float quarter = __fmul_rn(0.25f, s), threeq = __fmul_rn(0.75f, s);
+        float quarter, threeq;
+        special_band(s, L.shift, quarter, threeq);
         uint32_t half_word = 0;
 #pragma unroll
         for (int i = 0; i < 4; ++i)
@@ -211,6 +221,9 @@ rowsum_kernel(const uint8_t *__restrict__ blob, BlobLayout L, int kb_per_slice,
     const int n = nt * kTileN + r;
     const uint8_t *zeros = blob + L.off_zeros;
     const uint8_t *codes = blob + L.off_codes;
+    // the unit of the levels is the blob's own (0 in the header of an older blob means 1)
+    const uint32_t hs = reinterpret_cast<const BlobHeader *>(blob)->level_shift;
+    const int shift = hs == 0u ? 1 : (int)hs;
     const int kb0 = blockIdx.y * kb_per_slice;
     const int kb1 = min(L.k_blocks, kb0 + kb_per_slice);
     int z = zeros[n];
@@ -222,7 +235,7 @@ rowsum_kernel(const uint8_t *__restrict__ blob, BlobLayout L, int kb_per_slice,
             const uint4 w = *reinterpret_cast<const uint4 *>(tile + q * kQuarterBytes + r * 16);
             const uint32_t words[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-            for (int i = 0; i < 32; ++i) sum += dint4_t2((words[i >> 3] >> (4 * (i & 7))) & 15, z);
+            for (int i = 0; i < 32; ++i) sum += dint4_level((words[i >> 3] >> (4 * (i & 7))) & 15, z, shift);
         }
         if (L.group != 0 && n < L.N) rowsum[(size_t)kb * L.N + n] = sum;
     }
