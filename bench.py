@@ -458,6 +458,26 @@ def main():
     asym_steps = max(3, min(args.steps, 50))
     ms_asym = timed(step_asym, asym_steps) / asym_steps
 
+    # ------------------------------------------------------------------ special value step / 4
+    fmt_opts = w4a8.make_opts(level_shift=2)
+    for d, lay in zip(L, layers):
+        W = torch.from_numpy(lay["W"]).to(dev)
+        d["packed_fmt"] = w4a8.pack_weights(W, d["s"], group, level_shift=2)
+        del W
+
+    def step_fmt(it=None):
+        for d in L:
+            w4a8.quantize_act(d["X"], d["inv_s"], out=(d["Xq"], d["tok"]))
+            w4a8.linear(d["Xq"], d["tok"], d["packed_fmt"], d["bias"], d["N"], group, d["ws"],
+                        fmt_opts, out=d["Y"])
+
+    for _ in range(3):
+        step_fmt()
+    ms_fmt = timed(step_fmt, asym_steps) / asym_steps
+    for d in L:
+        w4a8.check_status(d["ws"])
+        del d["packed_fmt"]
+
     # ------------------------------------------------------------------ decode (M = 1)
     # The eight launches of a decode step take a few microseconds each: from Python they would
     # be launch-bound, so the steps are captured once into a CUDA graph and the replay is timed.
@@ -530,6 +550,11 @@ def main():
                  "unit": "TOPS", "ms_per_step": ms_asym,
                  "note": "same block and step with asymmetric token-wise activations "
                          "(quantize_act_asym + linear_asym)"},
+        "special_value_quarter_step": {"metric": "w4a8_dint_linear_tops",
+                                       "value": replica_throughput(ops_per_step, world, ms_fmt),
+                                       "unit": "TOPS", "ms_per_step": ms_fmt,
+                                       "note": "same block and step with weights packed for the special "
+                                               "value step/4 (pack_weights_fmt, level_shift 2)"},
         "cpu_baseline": cpu,
     }
     print(json.dumps(line), flush=True)
