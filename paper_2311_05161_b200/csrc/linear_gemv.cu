@@ -239,6 +239,159 @@ linear_gemv_kernel(const GemvParams P)
     }
 }
 
+// ---------------------------------------------------------------------------
+// Row-slab variant: one CTA owns 32 output rows over the whole of K.
+// ---------------------------------------------------------------------------
+// The K split happens inside the CTA (warp w takes k-blocks w, w + W, ...), the warps' sums meet
+// in shared memory, and the CTA writes its 32 outputs itself: no partial sums in global memory,
+// no atomic counter, no second phase.  For a weight stream of a few tens of megabytes that
+// second phase and its round trips are a third of the launch.  A lane owns one row: per k-block
+// it reads 4 x 16 bytes (a warp reads 4 x 512 contiguous bytes), two k-blocks ahead in registers.
+constexpr int kRowsPerCta = 32;
+constexpr int kRowSlabMaxTokenBytes = 96 * 1024;
+constexpr bool kUseRowSlabs = true;
+
+template <int MT, bool GROUPED, int W>
+__global__ void __launch_bounds__(32 * W)
+linear_gemv_rows_kernel(const GemvParams P)
+{
+    extern __shared__ __align__(16) uint8_t rows_smem[];
+    int8_t *s_x = reinterpret_cast<int8_t *>(rows_smem);                       // [MT][K]
+    int32_t *s_red = reinterpret_cast<int32_t *>(rows_smem + (size_t)MT * P.L.K);   // [W][MT][32]
+    allow_dependents();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nt = blockIdx.x >> 2, slab = blockIdx.x & 3;
+    const int r = slab * kRowsPerCta + lane;                  // row inside the 128-row tile
+    const int n = nt * kTileN + r;
+    const int k_blocks = P.L.k_blocks;
+    const uint8_t *src = P.codes + (size_t)nt * k_blocks * kTileBytes + r * 16;
+    auto fetch = [&](int kb, uint4 (&dst)[4]) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            dst[q] = ld_stream(reinterpret_cast<const uint4 *>(src + (size_t)kb * kTileBytes +
+                                                               q * kQuarterBytes));
+    };
+    // earlier work in the stream (the activation quantizer) is complete from here on
+    dependent_wait();
+    uint4 wa[4], wb[4];
+    int kb = warp;
+    if (kb < k_blocks) fetch(kb, wa);
+    if (kb + W < k_blocks) fetch(kb + W, wb);
+    // the tokens, whole rows, for all warps
+    {
+        const int chunks = P.L.K / 16;
+        for (int i = threadIdx.x; i < MT * chunks; i += 32 * W) {
+            const int m = i / chunks, c = i - m * chunks;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (m < P.M) v = __ldg(reinterpret_cast<const uint4 *>(P.Xq + (size_t)m * P.L.K) + c);
+            reinterpret_cast<uint4 *>(s_x + (size_t)m * P.L.K)[c] = v;
+        }
+    }
+    const bool blob_ok = header_matches(P.blob, P.L);
+    __syncthreads();
+    if (!blob_ok) {
+        if (threadIdx.x == 0) report_failure(P.sb, W4A8_ERR_BAD_BLOB, 4);
+        return;
+    }
+    int acc[MT];
+    float usum[MT];
+#pragma unroll
+    for (int m = 0; m < MT; ++m) { acc[m] = 0; usum[m] = 0.0f; }
+    uint32_t t[4];
+    if (!GROUPED) build_level_tables(P.zeros[n], P.lt, t);
+    auto consume = [&](int kbi, const uint4 (&w)[4]) {
+        if (GROUPED) {
+            build_level_tables(P.zeros[(size_t)kbi * P.L.n_pad + n], P.lt, t);
+#pragma unroll
+            for (int m = 0; m < MT; ++m) acc[m] = 0;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t words[4] = {w[q].x, w[q].y, w[q].z, w[q].w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t d0, d1;
+                decode8(words[i], t, d0, d1);
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    const uint2 x = *reinterpret_cast<const uint2 *>(
+                        s_x + (size_t)m * P.L.K + kbi * kTileK + q * 32 + i * 8);
+                    acc[m] = __dp4a((int)d0, (int)x.x, acc[m]);
+                    acc[m] = __dp4a((int)d1, (int)x.y, acc[m]);
+                }
+            }
+        }
+        if (GROUPED) {
+            const float h = __fmul_rn(P.unit, P.scales[(size_t)kbi * P.L.n_pad + n]);
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                usum[m] = fmaf((float)acc[m], h, usum[m]);
+                if (P.acc_out && m < P.M && n < P.L.N)
+                    P.acc_out[((size_t)kbi * P.M + m) * P.L.N + n] = acc[m];
+            }
+        }
+    };
+    // two register sets alternate; each is refilled right after it has been consumed
+    for (; kb < k_blocks; kb += 2 * W) {
+        consume(kb, wa);
+        if (kb + 2 * W < k_blocks) fetch(kb + 2 * W, wa);
+        if (kb + W < k_blocks) {
+            consume(kb + W, wb);
+            if (kb + 3 * W < k_blocks) fetch(kb + 3 * W, wb);
+        }
+    }
+#pragma unroll
+    for (int m = 0; m < MT; ++m)
+        s_red[(warp * MT + m) * 32 + lane] = GROUPED ? (int32_t)__float_as_int(usum[m]) : acc[m];
+    __syncthreads();
+    if (warp != 0 || n >= P.L.N) return;
+    const float bias_n = P.bias ? P.bias[n] : 0.0f;
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+        if (m >= P.M) break;
+        float tv;
+        if (GROUPED) {
+            float u = 0.0f;
+            for (int w = 0; w < W; ++w) u = __fadd_rn(u, __int_as_float(s_red[(w * MT + m) * 32 + lane]));
+            tv = __fmul_rn(u, P.tok_scale ? P.tok_scale[m] : 0.0f);
+        } else {
+            int a = 0;
+            for (int w = 0; w < W; ++w) a += s_red[(w * MT + m) * 32 + lane];
+            if (P.zp.tok_zero) a -= P.zp.tok_zero[m] * P.zp.rowsum[n];
+            if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = a;
+            tv = rescale_channel(a, P.tok_scale ? P.tok_scale[m] : 0.0f,
+                                 __fmul_rn(P.unit, P.scales[n]));
+        }
+        if (P.bias) tv = __fadd_rn(tv, bias_n);
+        if (P.Y) P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(tv);
+    }
+}
+
+template <int MT, bool GROUPED, int W>
+void launch_rows(const GemvParams &P, cudaStream_t st)
+{
+    const int smem = MT * P.L.K + W * MT * 32 * 4;
+    cudaFuncSetAttribute(linear_gemv_rows_kernel<MT, GROUPED, W>,
+                         cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    launch_overlapped(linear_gemv_rows_kernel<MT, GROUPED, W>, dim3(P.L.n_tiles * 4), dim3(32 * W),
+                      (size_t)smem, st, P);
+}
+
+template <int MT, bool GROUPED>
+void launch_rows_w(const GemvParams &P, cudaStream_t st)
+{
+    if (P.L.k_blocks >= 32) launch_rows<MT, GROUPED, 16>(P, st);
+    else if (P.L.k_blocks >= 16) launch_rows<MT, GROUPED, 8>(P, st);
+    else launch_rows<MT, GROUPED, 4>(P, st);
+}
+
+// enough row slabs to occupy the GPU, and the tokens fit in shared memory
+inline bool row_slabs_fit(int M, const BlobLayout &L)
+{
+    const int mt = M == 1 ? 1 : (M == 2 ? 2 : 4);
+    return kUseRowSlabs && L.n_tiles * 4 >= 96 && (size_t)mt * L.K <= (size_t)kRowSlabMaxTokenBytes;
+}
+
 template <int MT, bool GROUPED>
 void launch_gemv(dim3 grid, const GemvParams &P, cudaStream_t st)
 {
@@ -305,6 +458,12 @@ w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const u
     if (P.slices > 65535) return W4A8_ERR_SHAPE;
     const dim3 grid(L.n_tiles, P.slices);
     const bool g = L.group != 0;
+    if (row_slabs_fit(M, L)) {
+        if (M == 1) { if (g) launch_rows_w<1, true>(P, st); else launch_rows_w<1, false>(P, st); }
+        else if (M == 2) { if (g) launch_rows_w<2, true>(P, st); else launch_rows_w<2, false>(P, st); }
+        else { if (g) launch_rows_w<4, true>(P, st); else launch_rows_w<4, false>(P, st); }
+        return cudaGetLastError() == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+    }
     if (M == 1) {
         if (g) launch_gemv<1, true>(grid, P, st);
         else launch_gemv<1, false>(grid, P, st);

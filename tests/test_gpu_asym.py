@@ -125,6 +125,14 @@ def test_gemv_path(M):
     check(lay, Y, acc)
 
 
+@pytest.mark.parametrize("M", [1, 2])
+def test_gemv_row_slab_kernel(M):
+    K, N = 2560, 3080
+    lay = make(K, N, M, seed=45 + M)
+    Y, acc = run(lay, K, N, M, w4a8.make_opts(w4a8.PATH_GEMV))
+    check(lay, Y, acc)
+
+
 @pytest.mark.parametrize("M", [1, 3, 16, 100, 300])
 def test_automatic_plan(M):
     K, N = 1024, 640
