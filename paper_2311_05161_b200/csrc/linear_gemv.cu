@@ -389,7 +389,11 @@ void launch_rows_w(const GemvParams &P, cudaStream_t st)
 inline bool row_slabs_fit(int M, const BlobLayout &L)
 {
     const int mt = M == 1 ? 1 : (M == 2 ? 2 : 4);
-    return kUseRowSlabs && L.n_tiles * 4 >= 96 && (size_t)mt * L.K <= (size_t)kRowSlabMaxTokenBytes;
+    const int slabs = L.n_tiles * 4;
+    // fewer slabs than SMs and a long K: each CTA would stream too much alone (measured on
+    // 16384 -> 4096: the two-phase kernel is faster there)
+    if (slabs < 148 && L.k_blocks > 96) return false;
+    return kUseRowSlabs && slabs >= 96 && (size_t)mt * L.K <= (size_t)kRowSlabMaxTokenBytes;
 }
 
 template <int MT, bool GROUPED>
