@@ -204,7 +204,10 @@ def run_case(args):
     tok_tile = vals[4] if len(vals) > 4 else 0
     split_k = vals[5] if len(vals) > 5 else 0
     dw = vals[6] if len(vals) > 6 else 0
-    opts = w4a8.make_opts(w4a8.PATH_TCGEN05, split_k, tok_tile, dw) if (tok_tile or split_k or dw) else None
+    if tok_tile < 0:            # the weight-streaming kernel on request; dw = warps of a row-slab CTA
+        opts = w4a8.make_opts(w4a8.PATH_GEMV, 0, 0, dw)
+    else:
+        opts = w4a8.make_opts(w4a8.PATH_TCGEN05, split_k, tok_tile, dw) if (tok_tile or split_k or dw) else None
     torch.cuda.set_device(0)
     peaks = read_peaks()
     lay = synth.make_layer(K, N, M, seed=7, dist="normal", outliers=0.001, mult=60.0)
@@ -298,6 +301,7 @@ def main():
                     help="--case only: time with per-launch events, no CUDA graph replay")
     ap.add_argument("--case", default=None,
                     help="K,N,M,group[,tok_tile[,split_k[,decode_warps]]]: time one linear shape instead of "
+                         "(tok_tile -1: the weight-streaming kernel, decode_warps = warps per CTA) "
                          "the block (profiling and sweeps); prints its own JSON line")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -350,6 +354,7 @@ def main():
         d["tok1"] = torch.empty((M_DECODE,), dtype=torch.float32, device=dev)
         d["Y1"] = torch.empty((M_DECODE, N), dtype=torch.bfloat16, device=dev)
         d["ws1"] = w4a8.new_workspace(M_DECODE, N, K, group)
+        d["wsf"] = w4a8.new_quantize_linear_workspace(M_DECODE, N, K, group)
         L.append(d)
     ops_per_step = sum(2 * M_PREFILL * d["K"] * d["N"] for d in L)
 
@@ -401,6 +406,12 @@ def main():
             w4a8.quantize_act(d["X1"], d["inv_s"], out=(d["Xq1"], d["tok1"]))
             w4a8.linear(d["Xq1"], d["tok1"], d["packed_rot"][it % 3], d["bias"], d["N"], group,
                         d["ws1"], out=d["Y1"])
+
+    def step_decode_fused(it):
+        # the same decode step with the quantizer inside the weight-streaming kernel: one launch per linear
+        for d in L:
+            w4a8.quantize_linear(d["X1"], d["inv_s"], d["packed_rot"][it % 3], d["bias"], d["N"], group,
+                                 d["wsf"], out=d["Y1"])
 
     def barrier():
         if world > 1:
@@ -481,26 +492,32 @@ def main():
     # ------------------------------------------------------------------ decode (M = 1)
     # The eight launches of a decode step take a few microseconds each: from Python they would
     # be launch-bound, so the steps are captured once into a CUDA graph and the replay is timed.
-    for it in range(6):
-        step_decode(it)
     dec_steps = 60
-    torch.cuda.synchronize()
-    graph = torch.cuda.CUDAGraph()
-    side = torch.cuda.Stream()
-    side.wait_stream(torch.cuda.current_stream())
-    with torch.cuda.stream(side):
-        with torch.cuda.graph(graph, stream=side):
-            for it in range(dec_steps):
-                step_decode(it)
-    torch.cuda.synchronize()
-    graph.replay()
-    ms_dec = timed(lambda it: graph.replay(), 3) / (3 * dec_steps)
+
+    def graph_ms(step_fn):
+        for it in range(6):
+            step_fn(it)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                for it in range(dec_steps):
+                    step_fn(it)
+        torch.cuda.synchronize()
+        graph.replay()
+        return timed(lambda it: graph.replay(), 3) / (3 * dec_steps)
+
+    ms_dec = graph_ms(step_decode)
+    ms_dec_fused = graph_ms(step_decode_fused)
     dec_bytes = sum(d["K"] * d["N"] // 2 + 5 * d["N"] + M_DECODE * (d["K"] + 4) + 2 * M_DECODE * d["N"]
                     + 4 * d["N"] for d in L)
     dec_gbs = dec_bytes / (ms_dec * 1e-3) / 1e9
     for d in L:
         w4a8.check_status(d["ws"])
         w4a8.check_status(d["ws1"])
+        w4a8.check_status(d["wsf"])
 
     if rank != 0:
         if world > 1:
@@ -545,7 +562,12 @@ def main():
                    "ms_per_step": ms_dec, "bytes_per_step": dec_bytes,
                    "frac_of_measured_copy": dec_gbs / peaks["hbm_gbs"],
                    "frac_of_nominal_8000": dec_gbs / 8000.0,
-                   "note": "quantize_act + linear per shape, 3 rotating blob copies (> L2), CUDA graph replay"},
+                   "note": "quantize_act + linear per shape, 3 rotating blob copies (> L2), CUDA graph replay",
+                   "one_launch": {"value": dec_bytes / (ms_dec_fused * 1e-3) / 1e9, "unit": "GB/s",
+                                  "ms_per_step": ms_dec_fused,
+                                  "frac_of_measured_copy": dec_bytes / (ms_dec_fused * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                  "note": "the same step through quantize_linear: the quantizer runs inside "
+                                          "the weight-streaming kernel, one launch per linear"}},
         "asym": {"metric": "w4a8_dint_linear_tops", "value": replica_throughput(ops_per_step, world, ms_asym),
                  "unit": "TOPS", "ms_per_step": ms_asym,
                  "note": "same block and step with asymmetric token-wise activations "

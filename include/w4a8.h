@@ -60,7 +60,8 @@ typedef struct {
     int path;        /* w4a8_path */
     int split_k;     /* 0 = automatic; else number of K slices (tcgen05 path) */
     int tok_tile;    /* 0 = automatic; else tokens per tile: 16, 32, 64, 128 or 256 */
-    int decode_warps;/* 0 = automatic; else warps that expand codes to INT8: 4, 8 or 16 */
+    int decode_warps;/* 0 = automatic; else warps that expand codes to INT8: 4, 8 or 16 (with
+                        W4A8_PATH_GEMV: the warps of a CTA that owns a slab of rows) */
     int level_shift; /* special value of the blob = step / 2^level_shift: 0 or 1 (the paper's
                         step/2), 2 or 3 (w4a8_pack_weights_fmt); must match the blob */
     int reserved[3]; /* must be zero */
@@ -143,6 +144,27 @@ w4a8_status w4a8_linear_ex(const int8_t *Xq, const float *tok_scale, const void 
                            const float *bias, int M, int N, int K, int group_size,
                            void *Y_bf16, void *workspace, size_t workspace_bytes,
                            void *stream, const w4a8_opts *opts);
+
+/* Decode form of the whole of Eq. 1 for one to four tokens: the token-wise activation
+ * quantizer (Appendix A.1, as in w4a8_quantize_act) and the quantized matmul with the Eq. 6
+ * dequantization (as in w4a8_linear) in ONE launch.  With so few tokens the layer is a single
+ * scan of the packed weights, and a separate quantizer launch costs as much as a good part of
+ * that scan; here every CTA of the weight-streaming kernel quantizes the tokens itself
+ * (M * K elements, read from L2) while its first codes are on their way.
+ *   X_f16     [M][K] IEEE binary16, 1 <= M <= 4 (else W4A8_ERR_SHAPE).
+ *   inv_s_in  [K] FP32 reciprocal of the Eq. 1 scale, or NULL.
+ *   packed    as written by w4a8_pack_weights (special value step/2) for N, K, group_size.
+ *   bias      [N] FP32 or NULL.   Y_bf16  out [M][N] bfloat16.
+ *   workspace >= w4a8_quantize_linear_workspace_bytes(M, N, K, group_size) bytes, zero-filled
+ *             once (w4a8_workspace_init); same rules as for w4a8_linear.
+ * The result has the very bits of w4a8_quantize_act followed by w4a8_linear on the same
+ * inputs; the INT8 tokens and their steps are not written anywhere.  Kernel-side failures
+ * are reported by w4a8_poll_status. */
+size_t w4a8_quantize_linear_workspace_bytes(int M, int N, int K, int group_size);
+w4a8_status w4a8_quantize_linear(const void *X_f16, const float *inv_s_in, const void *packed,
+                                 const float *bias, int M, int N, int K, int group_size,
+                                 void *Y_bf16, void *workspace, size_t workspace_bytes,
+                                 void *stream);
 
 /* w4a8_linear for callers that must not allocate device memory and therefore have no
  * workspace to pass: code running after a host framework has claimed the whole device for

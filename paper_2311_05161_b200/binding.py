@@ -29,6 +29,7 @@ EXPORTS = (
     "w4a8_poll_status", "w4a8_dint4_table", "w4a8_version",
     "w4a8_quantize_act_asym", "w4a8_weight_rowsum", "w4a8_linear_asym",
     "w4a8_pack_weights_fmt", "w4a8_dint4_table_fmt",
+    "w4a8_quantize_linear", "w4a8_quantize_linear_workspace_bytes",
 )
 
 
@@ -70,6 +71,10 @@ def _load() -> ctypes.CDLL:
     lib.w4a8_linear_ex.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, vp, op]
     lib.w4a8_linear_static.restype = ci
     lib.w4a8_linear_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp]
+    lib.w4a8_quantize_linear_workspace_bytes.restype = sz
+    lib.w4a8_quantize_linear_workspace_bytes.argtypes = [ci, ci, ci, ci]
+    lib.w4a8_quantize_linear.restype = ci
+    lib.w4a8_quantize_linear.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, vp]
     lib.w4a8_pack_weights_fmt.restype = ci
     lib.w4a8_pack_weights_fmt.argtypes = [vp, vp, ci, ci, ci, cf, ci, vp, sz, vp]
     lib.w4a8_quantize_act_asym.restype = ci
@@ -203,6 +208,34 @@ def linear(Xq, tok_scale, packed, bias, N: int, group: int, workspace, opts: Opt
                                 group, _ptr(out), _ptr(workspace), workspace.numel(), _stream(),
                                 ctypes.byref(opts))
     _check(st, "w4a8_linear")
+    return out
+
+
+def quantize_linear_workspace_bytes(M: int, N: int, K: int, group: int = 0) -> int:
+    return int(lib.w4a8_quantize_linear_workspace_bytes(M, N, K, group))
+
+
+def new_quantize_linear_workspace(M: int, N: int, K: int, group: int = 0, device="cuda"):
+    nbytes = quantize_linear_workspace_bytes(M, N, K, group)
+    if nbytes == 0:
+        raise W4A8Error(2, "w4a8_quantize_linear_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    workspace_init(ws)
+    return ws
+
+
+def quantize_linear(X, inv_s_in, packed, bias, N: int, group: int, workspace, out=None):
+    """Decode form, one to four tokens: activation quantizer and quantized linear layer in one
+    launch.  X [M, K] float16 (CUDA) -> Y [M, N] bfloat16."""
+    X = _dev(X, torch.float16, "X")
+    inv_s_in = _dev(inv_s_in, torch.float32, "inv_s_in")
+    bias = _dev(bias, torch.float32, "bias")
+    M, K = X.shape
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
+    _check(lib.w4a8_quantize_linear(_ptr(X), _ptr(inv_s_in), _ptr(packed), _ptr(bias), M, N, K,
+                                    group, _ptr(out), _ptr(workspace), workspace.numel(),
+                                    _stream()), "w4a8_quantize_linear")
     return out
 
 

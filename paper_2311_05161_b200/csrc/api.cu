@@ -79,6 +79,10 @@ w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *
     LinearPlan plan;
     if (use_gemv(M, (long long)N * K, opts)) {
         gemv_plan(M, L, &plan);
+        // on request, the warps of a CTA of the row-slab variant (else chosen by the length of K)
+        const int dw = opts ? opts->decode_warps : 0;
+        if (dw != 0 && dw != 4 && dw != 8 && dw != 16) return W4A8_ERR_SHAPE;
+        plan.decode_warps = dw;
         return launch_linear_gemv(Xq, tok_scale, blob, L, bias, M, static_cast<__nv_bfloat16 *>(Y),
                                   acc, static_cast<uint8_t *>(workspace), plan, st, zp);
     }
@@ -184,6 +188,38 @@ w4a8_status w4a8_linear_ex(const int8_t *Xq, const float *tok_scale, const void 
     if (!Y_bf16) return W4A8_ERR_NULL;
     return linear_common(Xq, tok_scale, packed, bias, M, N, K, group_size, Y_bf16, nullptr,
                          workspace, workspace_bytes, stream, opts);
+}
+
+size_t w4a8_quantize_linear_workspace_bytes(int M, int N, int K, int group_size)
+{
+    if (!shape_ok(N, K, group_size) || M < 1 || M > gemv_max_tokens()) return 0;
+    LinearPlan plan;
+    gemv_plan(M, make_layout(N, K, group_size), &plan);
+    return plan.workspace_bytes;
+}
+
+w4a8_status w4a8_quantize_linear(const void *X_f16, const float *inv_s_in, const void *packed,
+                                 const float *bias, int M, int N, int K, int group_size,
+                                 void *Y_bf16, void *workspace, size_t workspace_bytes,
+                                 void *stream)
+{
+    if (!X_f16 || !packed || !Y_bf16 || !workspace) return W4A8_ERR_NULL;
+    if (!shape_ok(N, K, group_size) || M < 1 || M > gemv_max_tokens()) return W4A8_ERR_SHAPE;
+    if (!depth_ok(K, 1, 127)) return W4A8_ERR_SHAPE;
+    if (!aligned(X_f16, 16) || !aligned(inv_s_in, 16) || !aligned(bias, 4) ||
+        !aligned(Y_bf16, 16) || !aligned(packed, 256) || !aligned(workspace, 256))
+        return W4A8_ERR_ALIGN;
+    const BlobLayout L = make_layout(N, K, group_size);
+    LinearPlan plan;
+    gemv_plan(M, L, &plan);
+    if (workspace_bytes < plan.workspace_bytes) return W4A8_ERR_BUFFER_TOO_SMALL;
+    const w4a8_status arch = check_arch();
+    if (arch != W4A8_OK) return arch;
+    return launch_linear_gemv(nullptr, nullptr, static_cast<const uint8_t *>(packed), L, bias, M,
+                              static_cast<__nv_bfloat16 *>(Y_bf16), nullptr,
+                              static_cast<uint8_t *>(workspace), plan,
+                              static_cast<cudaStream_t>(stream), ZeroPoint(),
+                              static_cast<const __half *>(X_f16), inv_s_in);
 }
 
 w4a8_status w4a8_linear_acc_i32(const int8_t *Xq, const void *packed, int M, int N, int K,

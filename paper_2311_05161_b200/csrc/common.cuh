@@ -244,6 +244,7 @@ void gemv_plan(int M, const BlobLayout &L, LinearPlan *plan);
 w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
                                const BlobLayout &L, const float *bias, int M, __nv_bfloat16 *Y,
                                int32_t *acc, uint8_t *workspace, const LinearPlan &plan,
-                               cudaStream_t st, ZeroPoint zp = ZeroPoint());
+                               cudaStream_t st, ZeroPoint zp = ZeroPoint(),
+                               const __half *X = nullptr, const float *inv_s = nullptr);
 
 }  // namespace w4a8

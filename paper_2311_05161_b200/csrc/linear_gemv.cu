@@ -10,6 +10,7 @@
 // tile to finish (an atomic counter, nobody waits) adds them in slice order and applies the
 // FP32 rescale, so results do not depend on scheduling.
 #include "common.cuh"
+#include "quant_math.cuh"
 
 namespace w4a8 {
 
@@ -57,6 +58,10 @@ struct GemvParams {
     const uint8_t *zeros;
     const int8_t *Xq;
     const float *tok_scale;
+    // Fused form (X != NULL): the tokens arrive as FP16 with the Eq. 1 reciprocal scale and
+    // every CTA quantizes them itself (Xq and tok_scale are then unused).
+    const __half *X;
+    const float *inv_s;
     const float *bias;
     __nv_bfloat16 *Y;
     int32_t *acc_out;
@@ -70,6 +75,53 @@ struct GemvParams {
     float unit;          // level unit as a factor of the step: 2^-shift
 };
 
+
+// Token-wise absmax of the scaled tokens over the whole of K (activation side of Eq. 1), by
+// all threads of the CTA; the result is the same in every thread.  `red` holds warps x MT
+// floats.  Same arithmetic, element by element, as the stand-alone quantizer kernel.
+template <int MT>
+__device__ __forceinline__ void cta_token_absmax(const __half *X, const float *inv_s, int M, int K,
+                                                 float *red, float (&amax)[MT])
+{
+    const int nvec = K >> 3, nthr = blockDim.x, warps = nthr >> 5;
+#pragma unroll
+    for (int m = 0; m < MT; ++m) amax[m] = 0.0f;
+#pragma unroll 2
+    for (int c = threadIdx.x; c < nvec; c += nthr) {
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+            if (m < M) {
+                float x[8];
+                scaled8(__ldg(reinterpret_cast<const uint4 *>(X + (size_t)m * K) + c), inv_s, c * 8, x);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) amax[m] = fmaxf(amax[m], fabsf(x[e]));
+            }
+    }
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) amax[m] = fmaxf(amax[m], __shfl_xor_sync(0xffffffffu, amax[m], o));
+        if ((threadIdx.x & 31) == 0) red[(threadIdx.x >> 5) * MT + m] = amax[m];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+        float a = red[m];
+        for (int w = 1; w < warps; ++w) a = fmaxf(a, red[w * MT + m]);
+        amax[m] = a;
+    }
+}
+
+// Eight scaled elements of token m starting at feature 8 c, rounded to INT8 with the token's
+// factor r = 127 / amax (0 for an all-zero token, whose codes are all zero).
+__device__ __forceinline__ uint2 quantize_vec8(const __half *X, const float *inv_s, int K, int m,
+                                               int c, float r)
+{
+    float x[8];
+    scaled8(__ldg(reinterpret_cast<const uint4 *>(X + (size_t)m * K) + c), inv_s, c * 8, x);
+    return quantize8(x, r);
+}
+
 template <int MT, bool GROUPED>
 __global__ void __launch_bounds__(128, 6)
 linear_gemv_kernel(const GemvParams P)
@@ -80,6 +132,8 @@ linear_gemv_kernel(const GemvParams P)
     int8_t (*s_x)[kGemvMaxSteps * kGemvKb * kTileK] =
         reinterpret_cast<int8_t (*)[kGemvMaxSteps * kGemvKb * kTileK]>(gemv_smem + kGemvRingBytes);
     __shared__ int s_last;
+    __shared__ float s_amax[4 * MT];
+    __shared__ float s_tok[MT];          // token steps (read or, in the fused form, computed here)
     allow_dependents();
     const int nt = blockIdx.x, slice = blockIdx.y, r = threadIdx.x;
     const int n = nt * kTileN + r;
@@ -122,13 +176,36 @@ linear_gemv_kernel(const GemvParams P)
         return;
     }
     // tokens of this K slice: MT rows of kb_count * 128 INT8
-    constexpr int kRowChunks = kGemvMaxSteps * kGemvKb * (kTileK / 16);
-    for (int i = r; i < MT * kRowChunks; i += 128) {
-        const int m = i / kRowChunks, c = i % kRowChunks;
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (m < P.M && c < kb_count * (kTileK / 16))
-            v = __ldg(reinterpret_cast<const uint4 *>(P.Xq + (size_t)m * P.L.K + kb_first * kTileK) + c);
-        reinterpret_cast<uint4 *>(&s_x[m][0])[c] = v;
+    if (P.X) {
+        // fused form: the absmax needs the whole token, the codes only this slice
+        float amax[MT];
+        cta_token_absmax<MT>(P.X, P.inv_s, P.M, P.L.K, s_amax, amax);
+        float rq[MT];
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            rq[m] = amax[m] > 0.0f ? __fdiv_rn(127.0f, amax[m]) : 0.0f;
+            if (r == 0) s_tok[m] = amax[m] > 0.0f ? __fdiv_rn(amax[m], 127.0f) : 0.0f;
+        }
+        constexpr int kRowVecs = kGemvMaxSteps * kGemvKb * (kTileK / 8);
+        for (int c = r; c < kRowVecs; c += 128) {
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                uint2 v = make_uint2(0u, 0u);
+                if (m < P.M && c < kb_count * (kTileK / 8))
+                    v = quantize_vec8(P.X, P.inv_s, P.L.K, m, kb_first * (kTileK / 8) + c, rq[m]);
+                reinterpret_cast<uint2 *>(&s_x[m][0])[c] = v;
+            }
+        }
+    } else {
+        if (r < MT) s_tok[r] = (P.tok_scale && r < P.M) ? P.tok_scale[r] : 0.0f;
+        constexpr int kRowChunks = kGemvMaxSteps * kGemvKb * (kTileK / 16);
+        for (int i = r; i < MT * kRowChunks; i += 128) {
+            const int m = i / kRowChunks, c = i % kRowChunks;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (m < P.M && c < kb_count * (kTileK / 16))
+                v = __ldg(reinterpret_cast<const uint4 *>(P.Xq + (size_t)m * P.L.K + kb_first * kTileK) + c);
+            reinterpret_cast<uint4 *>(&s_x[m][0])[c] = v;
+        }
     }
     __syncthreads();
 
@@ -222,7 +299,7 @@ linear_gemv_kernel(const GemvParams P)
 #pragma unroll 8
             for (int s = 0; s < P.slices; ++s)               // loads of eight slices in flight
                 u = __fadd_rn(u, __ldcg(part + ((size_t)s * P.M + m) * P.L.n_pad + n));
-            tv = __fmul_rn(u, P.tok_scale ? P.tok_scale[m] : 0.0f);
+            tv = __fmul_rn(u, s_tok[m]);
         } else {
             const int32_t *part = reinterpret_cast<const int32_t *>(P.partials);
             int a = 0;
@@ -231,8 +308,7 @@ linear_gemv_kernel(const GemvParams P)
                 a += __ldcg(part + ((size_t)s * P.M + m) * P.L.n_pad + n);
             if (P.zp.tok_zero) a -= P.zp.tok_zero[m] * P.zp.rowsum[n];
             if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = a;
-            tv = rescale_channel(a, P.tok_scale ? P.tok_scale[m] : 0.0f,
-                                 __fmul_rn(P.unit, P.scales[n]));
+            tv = rescale_channel(a, s_tok[m], __fmul_rn(P.unit, P.scales[n]));
         }
         if (P.bias) tv = __fadd_rn(tv, bias_n);
         if (P.Y) P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(tv);
@@ -258,6 +334,7 @@ linear_gemv_rows_kernel(const GemvParams P)
     extern __shared__ __align__(16) uint8_t rows_smem[];
     int8_t *s_x = reinterpret_cast<int8_t *>(rows_smem);                       // [MT][K]
     int32_t *s_red = reinterpret_cast<int32_t *>(rows_smem + (size_t)MT * P.L.K);   // [W][MT][32]
+    __shared__ float s_tok[MT];          // token steps (read or, in the fused form, computed here)
     allow_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nt = blockIdx.x >> 2, slab = blockIdx.x & 3;
@@ -278,7 +355,28 @@ linear_gemv_rows_kernel(const GemvParams P)
     if (kb < k_blocks) fetch(kb, wa);
     if (kb + W < k_blocks) fetch(kb + W, wb);
     // the tokens, whole rows, for all warps
-    {
+    if (P.X) {
+        // fused form: quantize the tokens here (the codes of the first k-blocks are on their way)
+        float amax[MT];
+        cta_token_absmax<MT>(P.X, P.inv_s, P.M, P.L.K, reinterpret_cast<float *>(s_red), amax);
+        float rq[MT];
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            rq[m] = amax[m] > 0.0f ? __fdiv_rn(127.0f, amax[m]) : 0.0f;
+            if (threadIdx.x == 0) s_tok[m] = amax[m] > 0.0f ? __fdiv_rn(amax[m], 127.0f) : 0.0f;
+        }
+        const int nvec = P.L.K / 8;
+        for (int c = threadIdx.x; c < nvec; c += 32 * W) {
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                uint2 v = make_uint2(0u, 0u);
+                if (m < P.M) v = quantize_vec8(P.X, P.inv_s, P.L.K, m, c, rq[m]);
+                reinterpret_cast<uint2 *>(s_x + (size_t)m * P.L.K)[c] = v;
+            }
+        }
+    } else {
+        if (threadIdx.x < MT)
+            s_tok[threadIdx.x] = (P.tok_scale && (int)threadIdx.x < P.M) ? P.tok_scale[threadIdx.x] : 0.0f;
         const int chunks = P.L.K / 16;
         for (int i = threadIdx.x; i < MT * chunks; i += 32 * W) {
             const int m = i / chunks, c = i - m * chunks;
@@ -353,14 +451,13 @@ linear_gemv_rows_kernel(const GemvParams P)
         if (GROUPED) {
             float u = 0.0f;
             for (int w = 0; w < W; ++w) u = __fadd_rn(u, __int_as_float(s_red[(w * MT + m) * 32 + lane]));
-            tv = __fmul_rn(u, P.tok_scale ? P.tok_scale[m] : 0.0f);
+            tv = __fmul_rn(u, s_tok[m]);
         } else {
             int a = 0;
             for (int w = 0; w < W; ++w) a += s_red[(w * MT + m) * 32 + lane];
             if (P.zp.tok_zero) a -= P.zp.tok_zero[m] * P.zp.rowsum[n];
             if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = a;
-            tv = rescale_channel(a, P.tok_scale ? P.tok_scale[m] : 0.0f,
-                                 __fmul_rn(P.unit, P.scales[n]));
+            tv = rescale_channel(a, s_tok[m], __fmul_rn(P.unit, P.scales[n]));
         }
         if (P.bias) tv = __fadd_rn(tv, bias_n);
         if (P.Y) P.Y[(size_t)m * P.L.N + n] = __float2bfloat16_rn(tv);
@@ -378,10 +475,19 @@ void launch_rows(const GemvParams &P, cudaStream_t st)
 }
 
 template <int MT, bool GROUPED>
-void launch_rows_w(const GemvParams &P, cudaStream_t st)
+void launch_rows_w(const GemvParams &P, cudaStream_t st, int warps)
 {
-    if (P.L.k_blocks >= 32) launch_rows<MT, GROUPED, 16>(P, st);
-    else if (P.L.k_blocks >= 16) launch_rows<MT, GROUPED, 8>(P, st);
+    if (warps == 0) {
+        // As many warps per CTA as keep the whole grid resident at once (32 warps of 64 registers
+        // per SM, 148 SMs): a second wave of CTAs repeats the start-up latency.  Measured on
+        // 4096 -> 16384: 13.9 us with 16 warps (1.7 waves), 11.6 us with 8 (all resident).
+        const int slabs = P.L.n_tiles * 4, resident_warps = 148 * 32;
+        if (slabs * 16 <= resident_warps && P.L.k_blocks >= 32) warps = 16;
+        else if (slabs * 8 <= resident_warps && P.L.k_blocks >= 16) warps = 8;
+        else warps = P.L.k_blocks >= 64 ? 8 : 4;
+    }
+    if (warps == 16) launch_rows<MT, GROUPED, 16>(P, st);
+    else if (warps == 8) launch_rows<MT, GROUPED, 8>(P, st);
     else launch_rows<MT, GROUPED, 4>(P, st);
 }
 
@@ -436,10 +542,12 @@ void gemv_plan(int M, const BlobLayout &L, LinearPlan *plan)
 w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
                                const BlobLayout &L, const float *bias, int M, __nv_bfloat16 *Y,
                                int32_t *acc, uint8_t *workspace, const LinearPlan &plan,
-                               cudaStream_t st, ZeroPoint zp)
+                               cudaStream_t st, ZeroPoint zp, const __half *X, const float *inv_s)
 {
     if (M < 1 || M > kGemvMaxTokens) return W4A8_ERR_SHAPE;
     GemvParams P;
+    P.X = X;
+    P.inv_s = inv_s;
     P.blob = blob;
     P.codes = blob + L.off_codes;
     P.scales = reinterpret_cast<const float *>(blob + L.off_scales);
@@ -463,9 +571,10 @@ w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const u
     const dim3 grid(L.n_tiles, P.slices);
     const bool g = L.group != 0;
     if (row_slabs_fit(M, L)) {
-        if (M == 1) { if (g) launch_rows_w<1, true>(P, st); else launch_rows_w<1, false>(P, st); }
-        else if (M == 2) { if (g) launch_rows_w<2, true>(P, st); else launch_rows_w<2, false>(P, st); }
-        else { if (g) launch_rows_w<4, true>(P, st); else launch_rows_w<4, false>(P, st); }
+        const int w = plan.decode_warps;
+        if (M == 1) { if (g) launch_rows_w<1, true>(P, st, w); else launch_rows_w<1, false>(P, st, w); }
+        else if (M == 2) { if (g) launch_rows_w<2, true>(P, st, w); else launch_rows_w<2, false>(P, st, w); }
+        else { if (g) launch_rows_w<4, true>(P, st, w); else launch_rows_w<4, false>(P, st, w); }
         return cudaGetLastError() == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
     }
     if (M == 1) {
