@@ -51,6 +51,72 @@ __device__ __forceinline__ uint4 ld_stream(const uint4 *p)
     return v;
 }
 
+// Cheaper expansion for special values step/2 and step/4.  The levels are stored with an offset
+// `off` = 13 * 2^shift, so every table byte lies in [0, 2 off] <= 104 and has its top bit clear.
+// A permute whose selector nibble has bit 3 set returns the selected byte's sign spread over the
+// byte, which is zero for such a table.  So the raw code nibbles pick from the table of codes
+// 0..7 and give 0 for codes 8..15, the nibbles with bit 3 flipped do the opposite on the table
+// of codes 8..15, and the two results go to dp4a as they are (one of them is zero in every
+// byte): no mask, no select.  The sums then carry off * (sum of the tokens' INT8 values over the
+// k-block), which is subtracted per k-block from a small table of those sums.  Integer
+// arithmetic modulo 2^32 throughout, so the result is exact whenever the true sum fits.
+__device__ __forceinline__ void build_offset_tables(int z, const LevelTables &lt, int shift,
+                                                    uint32_t (&t)[4])
+{
+    const uint32_t off = 13u << shift;
+    const uint32_t kc = (128u - off) * 0x01010101u;      // the tables' 0x80 bias minus the offset
+    const uint32_t zz = (uint32_t)z * lt.zmul;
+    t[0] = lt.base[0] - zz - kc;
+    t[1] = lt.base[1] - zz - kc;
+    t[2] = lt.base[2] - zz - kc;
+    // codes 12 and 13, then the two special values +1 and -1
+    t[3] = ((lt.base[3] - (zz & 0xFFFFu) - (kc & 0xFFFFu)) & 0xFFFFu) | ((off + 1u) << 16) |
+           ((off - 1u) << 24);
+}
+
+// One k-block (128 input features) of one output row against MT tokens: w = the row's 64 bytes
+// of codes, xk = the tokens' INT8 values of this k-block (token stride in bytes).
+template <int MT>
+__device__ __forceinline__ void block_dot_offset(const uint4 (&w)[4], const uint32_t (&t)[4],
+                                                 const int8_t *xk, size_t token_stride,
+                                                 int (&acc)[MT])
+{
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const uint32_t words[4] = {w[q].x, w[q].y, w[q].z, w[q].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t wv = words[i], wx = wv ^ 0x88888888u;
+            const uint32_t a0 = prmt(t[0], t[1], wv), b0 = prmt(t[2], t[3], wx);
+            const uint32_t a1 = prmt(t[0], t[1], wv >> 16), b1 = prmt(t[2], t[3], wx >> 16);
+            if (MT == 1) {
+                const uint2 x = *reinterpret_cast<const uint2 *>(xk + q * 32 + i * 8);
+                acc[0] = __dp4a((int)a0, (int)x.x, acc[0]);
+                acc[0] = __dp4a((int)b0, (int)x.x, acc[0]);
+                acc[0] = __dp4a((int)a1, (int)x.y, acc[0]);
+                acc[0] = __dp4a((int)b1, (int)x.y, acc[0]);
+            } else {
+                const uint32_t d0 = a0 | b0, d1 = a1 | b1;
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    const uint2 x = *reinterpret_cast<const uint2 *>(xk + m * token_stride + q * 32 + i * 8);
+                    acc[m] = __dp4a((int)d0, (int)x.x, acc[m]);
+                    acc[m] = __dp4a((int)d1, (int)x.y, acc[m]);
+                }
+            }
+        }
+    }
+}
+
+// Sum of the 128 INT8 values at xk, by one warp; every lane gets it.
+__device__ __forceinline__ int warp_sum128(const int8_t *xk)
+{
+    int s = __dp4a(0x01010101, reinterpret_cast<const int *>(xk)[threadIdx.x & 31], 0);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    return s;
+}
+
 struct GemvParams {
     const uint8_t *blob;
     const uint8_t *codes;
@@ -134,6 +200,7 @@ linear_gemv_kernel(const GemvParams P)
     __shared__ int s_last;
     __shared__ float s_amax[4 * MT];
     __shared__ float s_tok[MT];          // token steps (read or, in the fused form, computed here)
+    __shared__ int s_sum[MT][kGemvMaxSteps * kGemvKb];   // sums of the tokens' values per k-block
     allow_dependents();
     const int nt = blockIdx.x, slice = blockIdx.y, r = threadIdx.x;
     const int n = nt * kTileN + r;
@@ -208,13 +275,27 @@ linear_gemv_kernel(const GemvParams P)
         }
     }
     __syncthreads();
+    // offset-table expansion (see build_offset_tables) for special values step/2 and step/4
+    const bool offset_tables = P.L.shift <= 2;
+    const int off = 13 << P.L.shift;
+    if (offset_tables) {
+        for (int i = r >> 5; i < MT * kb_count; i += 4) {
+            const int m = i / kb_count, kl = i - m * kb_count;
+            const int sum = warp_sum128(&s_x[m][kl * kTileK]);
+            if ((r & 31) == 0) s_sum[m][kl] = sum;
+        }
+        __syncthreads();
+    }
 
     int acc[MT];
     float usum[MT];
 #pragma unroll
     for (int m = 0; m < MT; ++m) { acc[m] = 0; usum[m] = 0.0f; }
     uint32_t t[4];
-    if (!GROUPED) build_level_tables(P.zeros[n], P.lt, t);
+    if (!GROUPED) {
+        if (offset_tables) build_offset_tables(P.zeros[n], P.lt, P.L.shift, t);
+        else build_level_tables(P.zeros[n], P.lt, t);
+    }
 #pragma unroll 1
     for (int step = 0; step < steps; ++step) {
         // the group of this step is the oldest of kGemvDepth outstanding ones
@@ -232,23 +313,31 @@ linear_gemv_kernel(const GemvParams P)
             if (kl < kb_count) {
                 const int kb = kb_first + kl;
                 if (GROUPED) {
-                    build_level_tables(P.zeros[(size_t)kb * P.L.n_pad + n], P.lt, t);
+                    const int z = P.zeros[(size_t)kb * P.L.n_pad + n];
+                    if (offset_tables) build_offset_tables(z, P.lt, P.L.shift, t);
+                    else build_level_tables(z, P.lt, t);
 #pragma unroll
                     for (int m = 0; m < MT; ++m) acc[m] = 0;
                 }
+                if (offset_tables) {
+                    block_dot_offset<MT>(w[b], t, &s_x[0][kl * kTileK], sizeof(s_x[0]), acc);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const uint32_t words[4] = {w[b][q].x, w[b][q].y, w[b][q].z, w[b][q].w};
+                    for (int m = 0; m < MT; ++m) acc[m] = (int)((uint32_t)acc[m] - (uint32_t)off * (uint32_t)s_sum[m][kl]);
+                } else {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint32_t d0, d1;
-                        decode8(words[i], t, d0, d1);
+                    for (int q = 0; q < 4; ++q) {
+                        const uint32_t words[4] = {w[b][q].x, w[b][q].y, w[b][q].z, w[b][q].w};
 #pragma unroll
-                        for (int m = 0; m < MT; ++m) {
-                            const uint2 x = *reinterpret_cast<const uint2 *>(
-                                &s_x[m][kl * kTileK + q * 32 + i * 8]);
-                            acc[m] = __dp4a((int)d0, (int)x.x, acc[m]);
-                            acc[m] = __dp4a((int)d1, (int)x.y, acc[m]);
+                        for (int i = 0; i < 4; ++i) {
+                            uint32_t d0, d1;
+                            decode8(words[i], t, d0, d1);
+#pragma unroll
+                            for (int m = 0; m < MT; ++m) {
+                                const uint2 x = *reinterpret_cast<const uint2 *>(
+                                    &s_x[m][kl * kTileK + q * 32 + i * 8]);
+                                acc[m] = __dp4a((int)d0, (int)x.x, acc[m]);
+                                acc[m] = __dp4a((int)d1, (int)x.y, acc[m]);
+                            }
                         }
                     }
                 }
@@ -334,6 +423,7 @@ linear_gemv_rows_kernel(const GemvParams P)
     extern __shared__ __align__(16) uint8_t rows_smem[];
     int8_t *s_x = reinterpret_cast<int8_t *>(rows_smem);                       // [MT][K]
     int32_t *s_red = reinterpret_cast<int32_t *>(rows_smem + (size_t)MT * P.L.K);   // [W][MT][32]
+    int *s_sum = s_red + W * MT * 32;     // [MT][k_blocks] sums of the tokens' values per k-block
     __shared__ float s_tok[MT];          // token steps (read or, in the fused form, computed here)
     allow_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -391,31 +481,56 @@ linear_gemv_rows_kernel(const GemvParams P)
         if (threadIdx.x == 0) report_failure(P.sb, W4A8_ERR_BAD_BLOB, 4);
         return;
     }
+    // offset-table expansion (see build_offset_tables) for special values step/2 and step/4;
+    // a warp sums the token values of its own k-blocks (written and read by the same warp)
+    const bool offset_tables = P.L.shift <= 2;
+    const int off = 13 << P.L.shift;
+    if (offset_tables) {
+        for (int kbi = warp; kbi < k_blocks; kbi += W)
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                const int sum = warp_sum128(s_x + (size_t)m * P.L.K + kbi * kTileK);
+                if (lane == 0) s_sum[m * k_blocks + kbi] = sum;
+            }
+        __syncwarp();
+    }
     int acc[MT];
     float usum[MT];
 #pragma unroll
     for (int m = 0; m < MT; ++m) { acc[m] = 0; usum[m] = 0.0f; }
     uint32_t t[4];
-    if (!GROUPED) build_level_tables(P.zeros[n], P.lt, t);
+    if (!GROUPED) {
+        if (offset_tables) build_offset_tables(P.zeros[n], P.lt, P.L.shift, t);
+        else build_level_tables(P.zeros[n], P.lt, t);
+    }
     auto consume = [&](int kbi, const uint4 (&w)[4]) {
         if (GROUPED) {
-            build_level_tables(P.zeros[(size_t)kbi * P.L.n_pad + n], P.lt, t);
+            const int z = P.zeros[(size_t)kbi * P.L.n_pad + n];
+            if (offset_tables) build_offset_tables(z, P.lt, P.L.shift, t);
+            else build_level_tables(z, P.lt, t);
 #pragma unroll
             for (int m = 0; m < MT; ++m) acc[m] = 0;
         }
+        if (offset_tables) {
+            block_dot_offset<MT>(w, t, s_x + kbi * kTileK, (size_t)P.L.K, acc);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const uint32_t words[4] = {w[q].x, w[q].y, w[q].z, w[q].w};
+            for (int m = 0; m < MT; ++m)
+                acc[m] = (int)((uint32_t)acc[m] - (uint32_t)off * (uint32_t)s_sum[m * k_blocks + kbi]);
+        } else {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint32_t d0, d1;
-                decode8(words[i], t, d0, d1);
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t words[4] = {w[q].x, w[q].y, w[q].z, w[q].w};
 #pragma unroll
-                for (int m = 0; m < MT; ++m) {
-                    const uint2 x = *reinterpret_cast<const uint2 *>(
-                        s_x + (size_t)m * P.L.K + kbi * kTileK + q * 32 + i * 8);
-                    acc[m] = __dp4a((int)d0, (int)x.x, acc[m]);
-                    acc[m] = __dp4a((int)d1, (int)x.y, acc[m]);
+                for (int i = 0; i < 4; ++i) {
+                    uint32_t d0, d1;
+                    decode8(words[i], t, d0, d1);
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) {
+                        const uint2 x = *reinterpret_cast<const uint2 *>(
+                            s_x + (size_t)m * P.L.K + kbi * kTileK + q * 32 + i * 8);
+                        acc[m] = __dp4a((int)d0, (int)x.x, acc[m]);
+                        acc[m] = __dp4a((int)d1, (int)x.y, acc[m]);
+                    }
                 }
             }
         }
@@ -467,7 +582,7 @@ linear_gemv_rows_kernel(const GemvParams P)
 template <int MT, bool GROUPED, int W>
 void launch_rows(const GemvParams &P, cudaStream_t st)
 {
-    const int smem = MT * P.L.K + W * MT * 32 * 4;
+    const int smem = MT * P.L.K + W * MT * 32 * 4 + MT * P.L.k_blocks * 4;
     cudaFuncSetAttribute(linear_gemv_rows_kernel<MT, GROUPED, W>,
                          cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     launch_overlapped(linear_gemv_rows_kernel<MT, GROUPED, W>, dim3(P.L.n_tiles * 4), dim3(32 * W),

@@ -112,3 +112,35 @@ def test_asymmetric_activations_with_other_special_values(shift):
     t = (t + lay["bias"][None, :]).astype(np.float32)
     want = torch.from_numpy(t).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     assert np.array_equal(bf16_bits(Y), want)
+
+
+@pytest.mark.parametrize("shift", [1, 2, 3])
+@pytest.mark.parametrize("N,M", [(200, 1), (200, 3), (3080, 1), (3080, 2), (3080, 4)])
+def test_weight_streaming_kernels_every_zero_point(shift, N, M):
+    """Rows built so that output row n gets zero-point n mod 14: both weight-streaming kernels
+    (K-sliced for N = 200, row slabs for N = 3080) expand every code under every zero-point,
+    with the offset tables (step/2, step/4) and with the plain ones (step/8)."""
+    K = 1280
+    rng = np.random.default_rng(900 + shift + N + M)
+    z = np.arange(N) % 14
+    W = rng.integers(0, 14, size=(N, K)) - z[:, None]                 # integer levels -z .. 13-z
+    W = W + rng.choice([0.0, 0.5, -0.5, 0.3, -0.3], size=(N, K)) * (np.abs(W) < 1)   # near zero: specials
+    W[:, 0] = -z
+    W[:, 1] = 13 - z
+    W = (W * 2.0 ** -6).astype(np.float16)
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    codes, scales, zeros = oracle.pack_weights_fmt(W, None, 0, shift)
+    assert np.array_equal(zeros[0], z)
+    assert len(np.unique(codes & 15)) == 16
+    d = {"W": to_dev(W), "X": to_dev(X)}
+    packed = w4a8.pack_weights(d["W"], None, 0, level_shift=shift)
+    opts = w4a8.make_opts(w4a8.PATH_GEMV, level_shift=shift)
+    Xq, tok = w4a8.quantize_act(d["X"], None)
+    ws = w4a8.new_workspace(M, N, K, 0, opts)
+    Y = w4a8.linear(Xq, tok, packed, None, N, 0, ws, opts)
+    acc = w4a8.linear_acc_i32(Xq, packed, N, 0, ws, opts)
+    w4a8.check_status(ws)
+    oXq, otok = oracle.quantize_act(X, None)
+    want_acc, want_Y, _ = oracle.linear_fmt(oXq, otok, codes, scales, zeros, None, 0, shift)
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), want_acc)
+    assert np.array_equal(bf16_bits(Y), want_Y)
