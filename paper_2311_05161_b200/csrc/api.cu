@@ -81,7 +81,7 @@ w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *
         gemv_plan(M, L, &plan);
         // on request, the warps of a CTA of the row-slab variant (else chosen by the length of K)
         const int dw = opts ? opts->decode_warps : 0;
-        if (dw != 0 && dw != 4 && dw != 8 && dw != 16) return W4A8_ERR_SHAPE;
+        if (dw != 0 && dw != 4 && dw != 8 && dw != 16 && dw != 32) return W4A8_ERR_SHAPE;
         plan.decode_warps = dw;
         return launch_linear_gemv(Xq, tok_scale, blob, L, bias, M, static_cast<__nv_bfloat16 *>(Y),
                                   acc, static_cast<uint8_t *>(workspace), plan, st, zp);

@@ -9,6 +9,12 @@
 // held in shared memory.  K slices leave partial sums in the workspace; the last slice of a row
 // tile to finish (an atomic counter, nobody waits) adds them in slice order and applies the
 // FP32 rescale, so results do not depend on scheduling.
+//
+// Wide layers take the row-slab variant further down instead (a CTA owns 32 rows over all of K,
+// its warps split the k-blocks, nothing goes through global memory).  Both kernels expand the
+// codes with the offset tables described at build_offset_tables (the 16-lane logic pipe that
+// runs the permutes is what bounds them, not HBM), and both can quantize their one to four
+// FP16 tokens themselves (w4a8_quantize_linear), which saves the quantizer's launch.
 #include "common.cuh"
 #include "quant_math.cuh"
 
@@ -597,24 +603,32 @@ void launch_rows_w(const GemvParams &P, cudaStream_t st, int warps)
         // per SM, 148 SMs): a second wave of CTAs repeats the start-up latency.  Measured on
         // 4096 -> 16384: 13.9 us with 16 warps (1.7 waves), 11.6 us with 8 (all resident).
         const int slabs = P.L.n_tiles * 4, resident_warps = 148 * 32;
-        if (slabs * 16 <= resident_warps && P.L.k_blocks >= 32) warps = 16;
+        if (MT <= 2 && slabs * 32 <= resident_warps && P.L.k_blocks >= 32) warps = 32;
+        else if (slabs * 16 <= resident_warps && P.L.k_blocks >= 32) warps = 16;
         else if (slabs * 8 <= resident_warps && P.L.k_blocks >= 16) warps = 8;
         else warps = P.L.k_blocks >= 64 ? 8 : 4;
     }
-    if (warps == 16) launch_rows<MT, GROUPED, 16>(P, st);
+    if (warps == 32) {
+        // 1024 threads leave 64 registers each: enough for one or two tokens only
+        if constexpr (MT <= 2) launch_rows<MT, GROUPED, 32>(P, st);
+        else launch_rows<MT, GROUPED, 16>(P, st);
+    } else if (warps == 16) launch_rows<MT, GROUPED, 16>(P, st);
     else if (warps == 8) launch_rows<MT, GROUPED, 8>(P, st);
     else launch_rows<MT, GROUPED, 4>(P, st);
 }
 
 // enough row slabs to occupy the GPU, and the tokens fit in shared memory
-inline bool row_slabs_fit(int M, const BlobLayout &L)
+inline bool row_slabs_fit(int M, const BlobLayout &L, bool requested)
 {
     const int mt = M == 1 ? 1 : (M == 2 ? 2 : 4);
     const int slabs = L.n_tiles * 4;
-    // fewer slabs than SMs and a long K: each CTA would stream too much alone (measured on
-    // 16384 -> 4096: the two-phase kernel is faster there)
-    if (slabs < 148 && L.k_blocks > 96) return false;
-    return kUseRowSlabs && slabs >= 96 && (size_t)mt * L.K <= (size_t)kRowSlabMaxTokenBytes;
+    if ((size_t)mt * L.K > (size_t)kRowSlabMaxTokenBytes) return false;
+    if (requested) return true;              // the caller named the warps of a row-slab CTA
+    // Fewer slabs than SMs and a long K: with four tokens a CTA has at most 16 warps and would
+    // stream too much alone (the K-sliced kernel is faster there); with one or two tokens a CTA
+    // of 32 warps keeps enough in flight (16384 -> 4096, one token: 11.6 us against 15.0 us).
+    if (mt > 2 && slabs < 148 && L.k_blocks > 96) return false;
+    return kUseRowSlabs && slabs >= 96;
 }
 
 template <int MT, bool GROUPED>
@@ -685,7 +699,7 @@ w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const u
     if (P.slices > 65535) return W4A8_ERR_SHAPE;
     const dim3 grid(L.n_tiles, P.slices);
     const bool g = L.group != 0;
-    if (row_slabs_fit(M, L)) {
+    if (row_slabs_fit(M, L, plan.decode_warps != 0)) {
         const int w = plan.decode_warps;
         if (M == 1) { if (g) launch_rows_w<1, true>(P, st, w); else launch_rows_w<1, false>(P, st, w); }
         else if (M == 2) { if (g) launch_rows_w<2, true>(P, st, w); else launch_rows_w<2, false>(P, st, w); }

@@ -151,5 +151,18 @@ def test_gemv_row_slab_kernel(M, K, group):
         check_y(prob, Y, exact=(group == 0))
 
 
+@pytest.mark.parametrize("group", [0, 128])
+@pytest.mark.parametrize("warps", [4, 8, 16, 32])
+def test_gemv_row_slab_kernel_with_requested_warps(warps, group):
+    """Naming the warps of a row-slab CTA selects that kernel whatever the shape: ten k-blocks,
+    so CTAs of 16 and 32 warps have warps without work; N = 200 leaves a ragged last tile."""
+    M = 2 if warps == 32 else 3
+    prob = Problem(1280, 200, M, group, seed=400 + warps + group, dist="laplace", outliers=0.01, mult=20.0)
+    opts = w4a8.make_opts(w4a8.PATH_GEMV, decode_warps=warps)
+    Y, acc = run_linear(prob, opts)
+    assert np.array_equal(acc, prob.oracle_acc())
+    check_y(prob, Y, exact=(group == 0))
+
+
 def test_gemv_path_rejects_more_than_four_tokens():
     assert w4a8.linear_workspace_bytes(5, 256, 256, 0, w4a8.make_opts(w4a8.PATH_GEMV)) == 0
