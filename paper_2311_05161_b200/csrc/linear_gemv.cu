@@ -444,6 +444,17 @@ linear_gemv_rows_kernel(const GemvParams P)
             dst[q] = ld_stream(reinterpret_cast<const uint4 *>(src + (size_t)kb * kTileBytes +
                                                                q * kQuarterBytes));
     };
+    // Before the wait only prefetch hints are allowed: ask L2 for this warp's first two
+    // k-blocks (its 32 rows x 16 bytes x 4 quarters each = sixteen 128-byte lines per k-block, one
+    // line per lane), so that their HBM round trip overlaps the tail of the kernel before.
+    {
+        const int kbp = warp + (lane >> 4) * W;
+        if (kbp < k_blocks) {
+            const uint8_t *line = P.codes + ((size_t)nt * k_blocks + kbp) * kTileBytes +
+                                  ((lane >> 2) & 3) * kQuarterBytes + slab * (kRowsPerCta * 16) + (lane & 3) * 128;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
+        }
+    }
     // earlier work in the stream (the activation quantizer) is complete from here on
     dependent_wait();
     uint4 wa[4], wb[4];
