@@ -31,7 +31,7 @@ sys.path.insert(0, ROOT)
 CONFIG = 2            # OPT-6.7B-shaped block
 # DRAM bytes per launch of the dominant kernel from one ncu capture of this command (see
 # profiles/); set to None whenever that kernel changes until the counters are taken again.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 54.5e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 54.7e6
 M_PREFILL = 2048
 M_DECODE = 1
 CPU_SAMPLE_TOKENS = 48

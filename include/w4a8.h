@@ -171,8 +171,11 @@ w4a8_status w4a8_quantize_linear(const void *X_f16, const float *inv_s_in, const
  * its own pool (a cudaMalloc there fails or stalls the device), plug-ins whose host forbids
  * allocation once serving has started, and real-time loops that may not risk the implicit
  * synchronisation of an allocation.  The paper has no counterpart of this call; it is
- * w4a8_linear with the same kernel, the same automatic plan and the same results, and it
- * calls no allocating routine.
+ * w4a8_linear on the tensor-core kernel with its automatic plan (also for one or two
+ * tokens, where w4a8_linear would pick the weight-streaming kernel), and it calls no
+ * allocating routine.  Per-channel results have the bits of w4a8_linear; group-128 results
+ * too wherever w4a8_linear runs the same kernel (three tokens and more), else they agree
+ * within the FP32 reordering allowance of the group sums.
  *   The scratch is an 8 MiB array inside the library image (each GPU that loads the
  *   library holds it until the process ends).  Shapes whose plan needs more than that
  *   (large split-K cases; w4a8_linear_workspace_bytes tells) return

@@ -236,6 +236,15 @@ linear_gemv_kernel(const GemvParams P)
         }
         asm volatile("cp.async.commit_group;" ::: "memory");     // one group per step, even if empty
     };
+    // Before the wait only prefetch hints are allowed: ask L2 for the codes of the first
+    // kGemvDepth steps (contiguous tiles of this row tile), so that their HBM round trip overlaps
+    // the tail of the kernel before.
+    {
+        const int ahead = min(kb_count, kGemvDepth * kGemvKb) * (kTileBytes / 128);
+        const uint8_t *first = P.codes + ((size_t)nt * P.L.k_blocks + kb_first) * kTileBytes;
+        for (int i = r; i < ahead; i += 128)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(first + (size_t)i * 128));
+    }
     // earlier work in the stream (the activation quantizer, a previous call's use of the
     // workspace) is complete from here on
     dependent_wait();
@@ -447,14 +456,16 @@ linear_gemv_rows_kernel(const GemvParams P)
     // Before the wait only prefetch hints are allowed: ask L2 for this warp's first two
     // k-blocks (its 32 rows x 16 bytes x 4 quarters each = sixteen 128-byte lines per k-block, one
     // line per lane), so that their HBM round trip overlaps the tail of the kernel before.
-    {
-        const int kbp = warp + (lane >> 4) * W;
+    // (Hints further ahead inside the main loop were measured slower on the large shapes.)
+    auto prefetch_pair = [&](int kb0) {      // k-blocks kb0 and kb0 + W of this warp
+        const int kbp = kb0 + (lane >> 4) * W;
         if (kbp < k_blocks) {
             const uint8_t *line = P.codes + ((size_t)nt * k_blocks + kbp) * kTileBytes +
                                   ((lane >> 2) & 3) * kQuarterBytes + slab * (kRowsPerCta * 16) + (lane & 3) * 128;
             asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
         }
-    }
+    };
+    prefetch_pair(warp);
     // earlier work in the stream (the activation quantizer) is complete from here on
     dependent_wait();
     uint4 wa[4], wb[4];
