@@ -53,7 +53,7 @@ typedef enum {
     W4A8_PATH_AUTO = 0,
     W4A8_PATH_SIMPLE = 1,   /* one thread per output, CUDA cores: slow cross-check */
     W4A8_PATH_TCGEN05 = 2,  /* TMA + in-register dINT decode + tcgen05 kind::i8 MMA */
-    W4A8_PATH_GEMV = 3      /* weight-streaming CUDA-core kernel, M <= 4 tokens (AUTO picks it there) */
+    W4A8_PATH_GEMV = 3      /* weight-streaming CUDA-core kernel, M <= 4 tokens (AUTO picks it for M <= 2) */
 } w4a8_path;
 
 typedef struct {
