@@ -519,6 +519,38 @@ def main():
         w4a8.check_status(d["ws1"])
         w4a8.check_status(d["wsf"])
 
+    # ------------------------------------------------------------------ decode, one large layer
+    # OPT-66B-shaped fc1 (9216 -> 36864, 170 MB of codes) at M = 1: the weight stream without the
+    # fixed cost that dominates the 8-34 MB layers of the block above.  Two blob copies (> L2).
+    from paper_2311_05161_b200 import synth
+    for d in L:
+        for k in ("packed_rot", "packed", "X", "Xq", "Y", "X_host", "Y_host"):
+            d.pop(k, None)
+    torch.cuda.empty_cache()
+    big = synth.workload_layer(4, 0, M_DECODE)
+    bK, bN = big["W"].shape[1], big["W"].shape[0]
+    bd = {k: torch.from_numpy(big[k]).to(dev) for k in ("W", "X", "s", "inv_s", "bias")}
+    bpacked = [w4a8.pack_weights(bd["W"], bd["s"], 0)]
+    del bd["W"]
+    bpacked.append(bpacked[0].clone())
+    bws = w4a8.new_workspace(M_DECODE, bN, bK, 0)
+    bY = torch.empty((M_DECODE, bN), dtype=torch.bfloat16, device=dev)
+    bXq = torch.empty((M_DECODE, bK), dtype=torch.int8, device=dev)
+    btok = torch.empty((M_DECODE,), dtype=torch.float32, device=dev)
+
+    def step_big(it):
+        # two calls: on a matrix this large every CTA of the one-launch form would repeat the
+        # quantizer for several waves of CTAs (measured 38 us against 35 us)
+        w4a8.quantize_act(bd["X"], bd["inv_s"], out=(bXq, btok))
+        w4a8.linear(bXq, btok, bpacked[it % 2], bd["bias"], bN, 0, bws, out=bY)
+
+    dec_steps = 40
+    ms_big = graph_ms(step_big)
+    w4a8.check_status(bws)
+    big_bytes = bK * bN // 2 + 5 * bN + M_DECODE * (bK + 4) + 2 * M_DECODE * bN + 4 * bN   # as for the block above
+    big_gbs = big_bytes / (ms_big * 1e-3) / 1e9
+    del bpacked, big
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -567,7 +599,13 @@ def main():
                                   "ms_per_step": ms_dec_fused,
                                   "frac_of_measured_copy": dec_bytes / (ms_dec_fused * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                   "note": "the same step through quantize_linear: the quantizer runs inside "
-                                          "the weight-streaming kernel, one launch per linear"}},
+                                          "the weight-streaming kernel, one launch per linear"},
+                   "large_layer": {"workload": "opt-66b fc1 9216->36864, M=1, per-channel dINT4 (quantize_act + linear)",
+                                   "value": big_gbs, "unit": "GB/s", "ms_per_step": ms_big,
+                                   "bytes_per_step": big_bytes,
+                                   "frac_of_measured_copy": big_gbs / peaks["hbm_gbs"],
+                                   "frac_of_nominal_8000": big_gbs / 8000.0,
+                                   "note": "2 rotating blob copies (> L2), CUDA graph replay"}},
         "asym": {"metric": "w4a8_dint_linear_tops", "value": replica_throughput(ops_per_step, world, ms_asym),
                  "unit": "TOPS", "ms_per_step": ms_asym,
                  "note": "same block and step with asymmetric token-wise activations "

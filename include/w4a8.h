@@ -157,6 +157,9 @@ w4a8_status w4a8_linear_ex(const int8_t *Xq, const float *tok_scale, const void 
  *   bias      [N] FP32 or NULL.   Y_bf16  out [M][N] bfloat16.
  *   workspace >= w4a8_quantize_linear_workspace_bytes(M, N, K, group_size) bytes, zero-filled
  *             once (w4a8_workspace_init); same rules as for w4a8_linear.
+ * It pays on layers of a few tens of megabytes of codes (the OPT-6.7B-shaped block: 45 -> 42 us
+ * per step); on a matrix of 170 MB, whose CTAs come in several waves that each repeat the
+ * quantizer, the two calls are faster (35 against 38 us).
  * The result has the very bits of w4a8_quantize_act followed by w4a8_linear on the same
  * inputs; the INT8 tokens and their steps are not written anywhere.  Kernel-side failures
  * are reported by w4a8_poll_status. */
