@@ -158,10 +158,11 @@ w4a8_status w4a8_linear_ex(const int8_t *Xq, const float *tok_scale, const void 
  *   workspace >= w4a8_quantize_linear_workspace_bytes(M, N, K, group_size) bytes, zero-filled
  *             once (w4a8_workspace_init); same rules as for w4a8_linear.
  * It pays on layers of a few tens of megabytes of codes (the OPT-6.7B-shaped block: 45 -> 42 us
- * per step); on a matrix of 170 MB, whose CTAs come in several waves that each repeat the
- * quantizer, the two calls are faster (35 against 38 us).
+ * per step).  On a matrix so large that its CTAs come in several waves (170 MB of codes), each
+ * wave would repeat the quantizer; there the call runs the quantizer as a launch of its own in
+ * front, into the tail of the workspace (same results, two launches).
  * The result has the very bits of w4a8_quantize_act followed by w4a8_linear on the same
- * inputs; the INT8 tokens and their steps are not written anywhere.  Kernel-side failures
+ * inputs; the INT8 tokens and their steps are not returned.  Kernel-side failures
  * are reported by w4a8_poll_status. */
 size_t w4a8_quantize_linear_workspace_bytes(int M, int N, int K, int group_size);
 w4a8_status w4a8_quantize_linear(const void *X_f16, const float *inv_s_in, const void *packed,

@@ -197,7 +197,9 @@ size_t w4a8_quantize_linear_workspace_bytes(int M, int N, int K, int group_size)
     if (!shape_ok(N, K, group_size) || M < 1 || M > gemv_max_tokens()) return 0;
     LinearPlan plan;
     gemv_plan(M, make_layout(N, K, group_size), &plan);
-    return plan.workspace_bytes;
+    // behind the kernel's own scratch: room for the INT8 tokens and their steps, used when the
+    // quantizer runs as a launch of its own (see gemv_quantize_inside)
+    return align_up(plan.workspace_bytes, 256) + align_up((size_t)M * K, 256) + 256;
 }
 
 w4a8_status w4a8_quantize_linear(const void *X_f16, const float *inv_s_in, const void *packed,
@@ -214,9 +216,23 @@ w4a8_status w4a8_quantize_linear(const void *X_f16, const float *inv_s_in, const
     const BlobLayout L = make_layout(N, K, group_size);
     LinearPlan plan;
     gemv_plan(M, L, &plan);
-    if (workspace_bytes < plan.workspace_bytes) return W4A8_ERR_BUFFER_TOO_SMALL;
+    if (workspace_bytes < w4a8_quantize_linear_workspace_bytes(M, N, K, group_size))
+        return W4A8_ERR_BUFFER_TOO_SMALL;
     const w4a8_status arch = check_arch();
     if (arch != W4A8_OK) return arch;
+    if (!gemv_quantize_inside(M, L)) {
+        // several waves of CTAs: quantize once, in front, into the tail of the workspace
+        uint8_t *ws = static_cast<uint8_t *>(workspace);
+        int8_t *Xq = reinterpret_cast<int8_t *>(ws + align_up(plan.workspace_bytes, 256));
+        float *tok = reinterpret_cast<float *>(ws + align_up(plan.workspace_bytes, 256) +
+                                               align_up((size_t)M * K, 256));
+        if (launch_quantize_act(static_cast<const __half *>(X_f16), inv_s_in, M, K, Xq, tok,
+                                static_cast<cudaStream_t>(stream)) != cudaSuccess)
+            return W4A8_ERR_CUDA;
+        return launch_linear_gemv(Xq, tok, static_cast<const uint8_t *>(packed), L, bias, M,
+                                  static_cast<__nv_bfloat16 *>(Y_bf16), nullptr, ws, plan,
+                                  static_cast<cudaStream_t>(stream));
+    }
     return launch_linear_gemv(nullptr, nullptr, static_cast<const uint8_t *>(packed), L, bias, M,
                               static_cast<__nv_bfloat16 *>(Y_bf16), nullptr,
                               static_cast<uint8_t *>(workspace), plan,

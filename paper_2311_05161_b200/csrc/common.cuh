@@ -240,6 +240,7 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
                                   ZeroPoint zp = ZeroPoint());
 
 int gemv_max_tokens();
+bool gemv_quantize_inside(int M, const BlobLayout &L);
 void gemv_plan(int M, const BlobLayout &L, LinearPlan *plan);
 w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
                                const BlobLayout &L, const float *bias, int M, __nv_bfloat16 *Y,

@@ -617,19 +617,23 @@ void launch_rows(const GemvParams &P, cudaStream_t st)
                       (size_t)smem, st, P);
 }
 
+// As many warps per row-slab CTA as keep the whole grid resident at once (32 warps of 64
+// registers per SM, 148 SMs): a second wave of CTAs repeats the start-up latency.  Measured on
+// 4096 -> 16384: 13.9 us with 16 warps (1.7 waves), 11.6 us with 8 (all resident).
+constexpr int kResidentWarps = 148 * 32;
+inline int row_slab_warps(int mt, const BlobLayout &L)
+{
+    const int slabs = L.n_tiles * 4;
+    if (mt <= 2 && slabs * 32 <= kResidentWarps && L.k_blocks >= 32) return 32;
+    if (slabs * 16 <= kResidentWarps && L.k_blocks >= 32) return 16;
+    if (slabs * 8 <= kResidentWarps && L.k_blocks >= 16) return 8;
+    return L.k_blocks >= 64 ? 8 : 4;
+}
+
 template <int MT, bool GROUPED>
 void launch_rows_w(const GemvParams &P, cudaStream_t st, int warps)
 {
-    if (warps == 0) {
-        // As many warps per CTA as keep the whole grid resident at once (32 warps of 64 registers
-        // per SM, 148 SMs): a second wave of CTAs repeats the start-up latency.  Measured on
-        // 4096 -> 16384: 13.9 us with 16 warps (1.7 waves), 11.6 us with 8 (all resident).
-        const int slabs = P.L.n_tiles * 4, resident_warps = 148 * 32;
-        if (MT <= 2 && slabs * 32 <= resident_warps && P.L.k_blocks >= 32) warps = 32;
-        else if (slabs * 16 <= resident_warps && P.L.k_blocks >= 32) warps = 16;
-        else if (slabs * 8 <= resident_warps && P.L.k_blocks >= 16) warps = 8;
-        else warps = P.L.k_blocks >= 64 ? 8 : 4;
-    }
+    if (warps == 0) warps = row_slab_warps(MT, P.L);
     if (warps == 32) {
         // 1024 threads leave 64 registers each: enough for one or two tokens only
         if constexpr (MT <= 2) launch_rows<MT, GROUPED, 32>(P, st);
@@ -665,6 +669,17 @@ void launch_gemv(dim3 grid, const GemvParams &P, cudaStream_t st)
 }  // namespace
 
 int gemv_max_tokens() { return kGemvMaxTokens; }
+
+// Whether the one-launch decode form should quantize the tokens inside the weight-streaming
+// kernel: yes while the grid is resident at once (every CTA repeats the quantizer once); on a
+// matrix whose row slabs come in several waves each wave would repeat it, and a quantizer launch
+// of its own in front is faster (9216 -> 36864, one token: 35 against 38 us).
+bool gemv_quantize_inside(int M, const BlobLayout &L)
+{
+    if (!row_slabs_fit(M, L, false)) return true;        // the K-sliced grid is sized to be resident
+    const int mt = M == 1 ? 1 : (M == 2 ? 2 : 4);
+    return L.n_tiles * 4 * row_slab_warps(mt, L) <= kResidentWarps;
+}
 
 // Workspace of the GEMV path: status block, one counter per row tile, partial sums
 // [slices][M][n_pad] (4 bytes each).

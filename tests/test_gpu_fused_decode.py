@@ -80,6 +80,16 @@ def test_fused_decode_full_size_decode_shapes_sampled_rows():
         check_y(prob, Y[:, rows], exact=True)
 
 
+def test_fused_decode_quantizer_in_front_on_very_wide_layers():
+    """N = 38016 gives 1188 row slabs of four warps: more than are resident at once, so the call
+    runs the quantizer as a launch of its own into the tail of the workspace.  Same bits."""
+    prob = Problem(256, 38016, 2, 0, seed=77)
+    packed = w4a8.pack_weights(prob.dev["W"], prob.dev["s"], 0)
+    Y = run_fused(prob, packed)
+    check_y(prob, Y, exact=True)
+    assert np.array_equal(Y, run_two_calls(prob, packed))
+
+
 def test_fused_decode_rejects_bad_arguments():
     assert binding.quantize_linear_workspace_bytes(5, 256, 256, 0) == 0
     assert binding.quantize_linear_workspace_bytes(1, 256, 200, 0) == 0
