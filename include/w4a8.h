@@ -59,12 +59,17 @@ typedef enum {
 typedef struct {
     int path;        /* w4a8_path */
     int split_k;     /* 0 = automatic; else number of K slices (tcgen05 path) */
-    int tok_tile;    /* 0 = automatic; else tokens per tile: 16, 32, 64, 128 or 256 */
-    int decode_warps;/* 0 = automatic; else warps that expand codes to INT8: 4, 8 or 16 (with
-                        W4A8_PATH_GEMV: the warps of a CTA that owns a slab of rows) */
+    int tok_tile;    /* 0 = automatic; else tokens per tile: 16, 32, 64, 128, 192 or 256 */
+    int decode_warps;/* 0 = automatic; else warps that expand codes to INT8: 4, 8, 12 or 16 (with
+                        W4A8_PATH_GEMV: the warps of a CTA that owns a slab of rows: 4, 8, 16
+                        or 32) */
     int level_shift; /* special value of the blob = step / 2^level_shift: 0 or 1 (the paper's
                         step/2), 2 or 3 (w4a8_pack_weights_fmt); must match the blob */
-    int reserved[3]; /* must be zero */
+    int cluster;     /* 0 = automatic; else CTAs per thread-block cluster of the tensor-core kernel:
+                        1, or 2 (token tiles of 128 and more): the two CTAs work on two token
+                        tiles of the same weight rows and each expands half of every code tile
+                        for both */
+    int reserved[2]; /* must be zero */
 } w4a8_opts;
 
 /* Bytes of the packed-weight blob for an [N][K] matrix; 0 if the shape is invalid.
@@ -117,6 +122,17 @@ w4a8_status w4a8_quantize_act(const void *X_f16, const float *inv_s_in, int M, i
 size_t w4a8_linear_workspace_bytes(int M, int N, int K, int group_size);
 size_t w4a8_linear_workspace_bytes_ex(int M, int N, int K, int group_size,
                                       const w4a8_opts *opts);
+
+/* Host: which kernel and tiling w4a8_linear_ex would run for this shape and these options
+ * (NULL = automatic, i.e. what w4a8_linear runs), without touching a device.  `out` is a host
+ * array of 5: out[0] = w4a8_path; out[1] = tokens per tile (tensor-core kernel, else 0);
+ * out[2] = K slices; out[3] = warps that expand codes (tensor-core kernel) or warps of a
+ * row-slab CTA (weight-streaming kernel; 0 = its K-sliced variant); out[4] = CTAs per cluster.
+ * The plan follows the SM
+ * count of the current device (148 when there is none).  Eq. 1 fixes the result, not the plan:
+ * this call only reports the choice, e.g. where the weight-streaming kernel hands over to the
+ * tensor-core kernel as M grows. */
+w4a8_status w4a8_linear_plan(int M, int N, int K, int group_size, const w4a8_opts *opts, int *out);
 
 /* Zero-fill a workspace (enqueued on `stream`). */
 w4a8_status w4a8_workspace_init(void *workspace, size_t workspace_bytes, void *stream);

@@ -10,5 +10,5 @@ from .binding import (  # noqa: F401
     dint4_table, lib, linear, linear_acc_i32, linear_static, linear_workspace_bytes, make_opts, new_workspace,
     pack_weights, packed_bytes, poll_status, quantize_act, unpack_codes, version,
     workspace_init, quantize_act_asym, weight_rowsum, linear_asym,
-    quantize_linear, quantize_linear_workspace_bytes, new_quantize_linear_workspace,
+    quantize_linear, quantize_linear_workspace_bytes, new_quantize_linear_workspace, linear_plan,
 )

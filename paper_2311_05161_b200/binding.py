@@ -29,7 +29,7 @@ EXPORTS = (
     "w4a8_poll_status", "w4a8_dint4_table", "w4a8_version",
     "w4a8_quantize_act_asym", "w4a8_weight_rowsum", "w4a8_linear_asym",
     "w4a8_pack_weights_fmt", "w4a8_dint4_table_fmt",
-    "w4a8_quantize_linear", "w4a8_quantize_linear_workspace_bytes",
+    "w4a8_quantize_linear", "w4a8_quantize_linear_workspace_bytes", "w4a8_linear_plan",
 )
 
 
@@ -42,7 +42,7 @@ class W4A8Error(RuntimeError):
 class Opts(ctypes.Structure):
     _fields_ = [("path", ctypes.c_int), ("split_k", ctypes.c_int), ("tok_tile", ctypes.c_int),
                 ("decode_warps", ctypes.c_int), ("level_shift", ctypes.c_int),
-                ("reserved", ctypes.c_int * 3)]
+                ("cluster", ctypes.c_int), ("reserved", ctypes.c_int * 2)]
 
 
 def _load() -> ctypes.CDLL:
@@ -63,6 +63,8 @@ def _load() -> ctypes.CDLL:
     lib.w4a8_linear_workspace_bytes.argtypes = [ci, ci, ci, ci]
     lib.w4a8_linear_workspace_bytes_ex.restype = sz
     lib.w4a8_linear_workspace_bytes_ex.argtypes = [ci, ci, ci, ci, op]
+    lib.w4a8_linear_plan.restype = ci
+    lib.w4a8_linear_plan.argtypes = [ci, ci, ci, ci, op, vp]
     lib.w4a8_workspace_init.restype = ci
     lib.w4a8_workspace_init.argtypes = [vp, sz, vp]
     lib.w4a8_linear.restype = ci
@@ -121,10 +123,11 @@ def _dev(t, dtype, what):
 
 
 def make_opts(path: int = PATH_AUTO, split_k: int = 0, tok_tile: int = 0,
-              decode_warps: int = 0, level_shift: int = 0) -> Opts:
+              decode_warps: int = 0, level_shift: int = 0, cluster: int = 0) -> Opts:
     o = Opts()
     o.path, o.split_k, o.tok_tile, o.decode_warps = path, split_k, tok_tile, decode_warps
     o.level_shift = level_shift
+    o.cluster = cluster
     return o
 
 
@@ -176,6 +179,16 @@ def linear_workspace_bytes(M: int, N: int, K: int, group: int = 0, opts: Opts | 
     if opts is None:
         return int(lib.w4a8_linear_workspace_bytes(M, N, K, group))
     return int(lib.w4a8_linear_workspace_bytes_ex(M, N, K, group, ctypes.byref(opts)))
+
+
+def linear_plan(M: int, N: int, K: int, group: int = 0, opts: Opts | None = None) -> dict:
+    """What w4a8_linear(_ex) would run for this shape: kernel, token tile, K slices, warps."""
+    out = (ctypes.c_int * 5)()
+    _check(lib.w4a8_linear_plan(M, N, K, group, ctypes.byref(opts) if opts is not None else None,
+                                out), "w4a8_linear_plan")
+    names = {PATH_SIMPLE: "simple", PATH_TCGEN05: "tcgen05", PATH_GEMV: "weight-streaming"}
+    return {"kernel": names.get(out[0], str(out[0])), "tok_tile": out[1], "split_k": out[2],
+            "warps": out[3], "cluster": out[4]}
 
 
 def workspace_init(ws):

@@ -426,7 +426,8 @@ cudaError_t launch_quantize_act(const __half *X, const float *inv_s, int M, int 
         // (64 registers per thread: 1024 threads per SM)
         const int threads = ((nvec + 1) / 2 + 31) / 32 * 32;
         const int per_sm = 1024 / threads > 0 ? 1024 / threads : 1;
-        const int grid = M < 148 * per_sm ? M : 148 * per_sm;
+        const int sms = device_sms();
+        const int grid = M < sms * per_sm ? M : sms * per_sm;
         if (inv_s)
             launch_overlapped(act_quant_stream_kernel<true>, dim3(grid), dim3(threads), 0, st, X, inv_s, M, K, Xq, tok_scale);
         else
@@ -458,7 +459,8 @@ cudaError_t launch_quantize_act_asym(const __half *X, const float *inv_s, int M,
     if (nvec <= 2048) {
         const int threads = ((nvec + 1) / 2 + 31) / 32 * 32;
         const int per_sm = 1024 / threads > 0 ? 1024 / threads : 1;
-        const int ctas = M < 148 * per_sm ? M : 148 * per_sm;
+        const int sms = device_sms();
+        const int ctas = M < sms * per_sm ? M : sms * per_sm;
         if (inv_s)
             launch_overlapped(act_quant_asym_stream_kernel<true>, dim3(ctas), dim3(threads), 0, st, X, inv_s, M, K, Xq, tok_scale, tok_zero);
         else

@@ -3,6 +3,20 @@
 
 using namespace w4a8;
 
+namespace w4a8 {
+
+int device_sms()
+{
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+        return v;
+    cudaGetLastError();          // no device: not an error for the host-only queries
+    return 148;
+}
+
+}  // namespace w4a8
+
 namespace {
 
 inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -23,7 +37,8 @@ bool opts_ok(const w4a8_opts *o)
     if (o->path < W4A8_PATH_AUTO || o->path > W4A8_PATH_GEMV) return false;
     if (o->split_k < 0 || o->tok_tile < 0 || o->decode_warps < 0) return false;
     if (o->level_shift < 0 || o->level_shift > 3) return false;
-    for (int i = 0; i < 3; ++i)
+    if (o->cluster < 0 || o->cluster > 2) return false;
+    for (int i = 0; i < 2; ++i)
         if (o->reserved[i] != 0) return false;
     return true;
 }
@@ -41,12 +56,12 @@ bool depth_ok(int K, int shift, int amax)
 // default it takes one and two tokens: measured, it is as fast or faster there on every shape
 // (two tokens: 5.0 against 9.3 us on 4096 -> 4096, 13.2 against 17.7 us on 16384 -> 4096, equal on
 // 9216 -> 36864), and the tensor-core kernel with its 16-token tile wins from four tokens on.
-bool use_gemv(int M, long long weights, const w4a8_opts *o)
+bool use_gemv(int M, const w4a8_opts *o)
 {
     const int path = o ? o->path : W4A8_PATH_AUTO;
     if (path == W4A8_PATH_GEMV) return true;
-    if (path != W4A8_PATH_AUTO || (o && (o->split_k || o->tok_tile || o->decode_warps))) return false;
-    (void)weights;
+    if (path != W4A8_PATH_AUTO || (o && (o->split_k || o->tok_tile || o->decode_warps || o->cluster)))
+        return false;
     return M <= 2;
 }
 
@@ -79,7 +94,7 @@ w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *
         return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
     }
     LinearPlan plan;
-    if (use_gemv(M, (long long)N * K, opts)) {
+    if (use_gemv(M, opts)) {
         gemv_plan(M, L, &plan);
         // on request, the warps of a CTA of the row-slab variant (else chosen by the length of K)
         const int dw = opts ? opts->decode_warps : 0;
@@ -149,7 +164,7 @@ size_t w4a8_linear_workspace_bytes_ex(int M, int N, int K, int group_size, const
     if (!shape_ok(N, K, group_size) || M < 1 || !opts_ok(opts)) return 0;
     if (opts && opts->path == W4A8_PATH_SIMPLE) return sizeof(StatusBlock);
     LinearPlan plan;
-    if (use_gemv(M, (long long)N * K, opts)) {
+    if (use_gemv(M, opts)) {
         if (M > gemv_max_tokens()) return 0;
         gemv_plan(M, make_layout(N, K, group_size), &plan);
         return plan.workspace_bytes;
@@ -161,6 +176,36 @@ size_t w4a8_linear_workspace_bytes_ex(int M, int N, int K, int group_size, const
 size_t w4a8_linear_workspace_bytes(int M, int N, int K, int group_size)
 {
     return w4a8_linear_workspace_bytes_ex(M, N, K, group_size, nullptr);
+}
+
+w4a8_status w4a8_linear_plan(int M, int N, int K, int group_size, const w4a8_opts *opts, int *out)
+{
+    if (!out) return W4A8_ERR_NULL;
+    if (!shape_ok(N, K, group_size) || M < 1 || !opts_ok(opts)) return W4A8_ERR_SHAPE;
+    const BlobLayout L = make_layout(N, K, group_size, shift_of(opts));
+    out[0] = out[1] = out[2] = out[3] = 0;
+    out[4] = 1;
+    if (opts && opts->path == W4A8_PATH_SIMPLE) {
+        out[0] = W4A8_PATH_SIMPLE;
+        return W4A8_OK;
+    }
+    LinearPlan plan;
+    if (use_gemv(M, opts)) {
+        if (M > gemv_max_tokens()) return W4A8_ERR_SHAPE;
+        gemv_plan(M, L, &plan);
+        const int warps = gemv_row_slab_warps(M, L, opts ? opts->decode_warps : 0);
+        out[0] = W4A8_PATH_GEMV;
+        out[2] = warps ? 1 : plan.split_k;
+        out[3] = warps;
+        return W4A8_OK;
+    }
+    if (!make_plan(M, L, opts, &plan)) return W4A8_ERR_SHAPE;
+    out[0] = W4A8_PATH_TCGEN05;
+    out[1] = plan.tok_tile;
+    out[2] = plan.split_k;
+    out[3] = plan.decode_warps;
+    out[4] = plan.cluster;
+    return W4A8_OK;
 }
 
 w4a8_status w4a8_workspace_init(void *workspace, size_t workspace_bytes, void *stream)

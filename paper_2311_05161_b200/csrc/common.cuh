@@ -182,20 +182,34 @@ __device__ __forceinline__ void dependent_wait()
 
 #ifdef __CUDACC__
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
-                                     cudaStream_t st, Args &&...args)
+inline cudaError_t launch_overlapped_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block,
+                                             size_t smem, cudaStream_t st, int cluster,
+                                             Args &&...args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (cluster > 1) {                  // thread-block clusters of `cluster` CTAs along x
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)cluster;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
+    cfg.attrs = attr;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                     cudaStream_t st, Args &&...args)
+{
+    return launch_overlapped_cluster(kernel, grid, block, smem, st, 1, static_cast<Args &&>(args)...);
 }
 #endif
 
@@ -206,6 +220,7 @@ struct LinearPlan {
     int tok_tiles;    // ceil(M / tok_tile)
     int split_k;      // K slices (1 = none)
     int decode_warps; // warps converting codes to INT8: 4, 8 or 16
+    int cluster;      // CTAs per cluster: 1, or 2 (each CTA expands half of every code tile for both)
     int kb_per_split; // k-blocks per slice (last slice may be shorter)
     size_t off_counters, off_partials, workspace_bytes;
 };
@@ -216,6 +231,10 @@ struct ZeroPoint {
     const int32_t *tok_zero = nullptr;   // [M]
     const int32_t *rowsum = nullptr;     // [N]
 };
+
+// SM count of the current device (asked on every call: a process may drive several devices;
+// 148, a B200, when no device answers, so that the size queries work without one)
+int device_sms();
 
 // launchers (defined in the .cu files, called by api.cu)
 cudaError_t launch_pack(const __half *W, const float *s_in, const BlobLayout &L, float clip,
@@ -241,6 +260,8 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
 
 int gemv_max_tokens();
 bool gemv_quantize_inside(int M, const BlobLayout &L);
+// warps of a row-slab CTA for this shape, 0 when the K-sliced variant runs instead
+int gemv_row_slab_warps(int M, const BlobLayout &L, int requested_warps);
 void gemv_plan(int M, const BlobLayout &L, LinearPlan *plan);
 w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
                                const BlobLayout &L, const float *bias, int M, __nv_bfloat16 *Y,

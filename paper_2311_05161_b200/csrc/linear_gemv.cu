@@ -429,7 +429,6 @@ linear_gemv_kernel(const GemvParams P)
 // it reads 4 x 16 bytes (a warp reads 4 x 512 contiguous bytes), two k-blocks ahead in registers.
 constexpr int kRowsPerCta = 32;
 constexpr int kRowSlabMaxTokenBytes = 96 * 1024;
-constexpr bool kUseRowSlabs = true;
 
 template <int MT, bool GROUPED, int W>
 __global__ void __launch_bounds__(32 * W)
@@ -618,12 +617,13 @@ void launch_rows(const GemvParams &P, cudaStream_t st)
 }
 
 // As many warps per row-slab CTA as keep the whole grid resident at once (32 warps of 64
-// registers per SM, 148 SMs): a second wave of CTAs repeats the start-up latency.  Measured on
+// registers per SM on every SM): a second wave of CTAs repeats the start-up latency.  Measured on
 // 4096 -> 16384: 13.9 us with 16 warps (1.7 waves), 11.6 us with 8 (all resident).
-constexpr int kResidentWarps = 148 * 32;
+inline int resident_warps() { return device_sms() * 32; }
 inline int row_slab_warps(int mt, const BlobLayout &L)
 {
     const int slabs = L.n_tiles * 4;
+    const int kResidentWarps = resident_warps();
     if (mt <= 2 && slabs * 32 <= kResidentWarps && L.k_blocks >= 32) return 32;
     if (slabs * 16 <= kResidentWarps && L.k_blocks >= 32) return 16;
     if (slabs * 8 <= kResidentWarps && L.k_blocks >= 16) return 8;
@@ -653,8 +653,8 @@ inline bool row_slabs_fit(int M, const BlobLayout &L, bool requested)
     // Fewer slabs than SMs and a long K: with four tokens a CTA has at most 16 warps and would
     // stream too much alone (the K-sliced kernel is faster there); with one or two tokens a CTA
     // of 32 warps keeps enough in flight (16384 -> 4096, one token: 11.6 us against 15.0 us).
-    if (mt > 2 && slabs < 148 && L.k_blocks > 96) return false;
-    return kUseRowSlabs && slabs >= 96;
+    if (mt > 2 && slabs < device_sms() && L.k_blocks > 96) return false;
+    return slabs >= 96;
 }
 
 template <int MT, bool GROUPED>
@@ -670,6 +670,15 @@ void launch_gemv(dim3 grid, const GemvParams &P, cudaStream_t st)
 
 int gemv_max_tokens() { return kGemvMaxTokens; }
 
+int gemv_row_slab_warps(int M, const BlobLayout &L, int requested_warps)
+{
+    if (!row_slabs_fit(M, L, requested_warps != 0)) return 0;
+    const int mt = M == 1 ? 1 : (M == 2 ? 2 : 4);
+    int w = requested_warps ? requested_warps : row_slab_warps(mt, L);
+    if (w == 32 && mt > 2) w = 16;
+    return w;
+}
+
 // Whether the one-launch decode form should quantize the tokens inside the weight-streaming
 // kernel: yes while the grid is resident at once (every CTA repeats the quantizer once); on a
 // matrix whose row slabs come in several waves each wave would repeat it, and a quantizer launch
@@ -678,7 +687,7 @@ bool gemv_quantize_inside(int M, const BlobLayout &L)
 {
     if (!row_slabs_fit(M, L, false)) return true;        // the K-sliced grid is sized to be resident
     const int mt = M == 1 ? 1 : (M == 2 ? 2 : 4);
-    return L.n_tiles * 4 * row_slab_warps(mt, L) <= kResidentWarps;
+    return L.n_tiles * 4 * row_slab_warps(mt, L) <= resident_warps();
 }
 
 // Workspace of the GEMV path: status block, one counter per row tile, partial sums
@@ -687,7 +696,7 @@ void gemv_plan(int M, const BlobLayout &L, LinearPlan *plan)
 {
     // K slices so that the grid fills, but does not exceed, six CTAs per SM when it can;
     // a slice is between 2 and 16 k-blocks
-    const int target_ctas = 148 * 6;
+    const int target_ctas = device_sms() * 6;
     int slices = target_ctas / L.n_tiles;
     if (slices < 1) slices = 1;
     int per = (L.k_blocks + slices - 1) / slices;

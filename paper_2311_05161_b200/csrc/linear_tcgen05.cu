@@ -24,6 +24,8 @@
 // roles poll, and the CTA drains its copies, frees tensor memory and returns.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "common.cuh"
 
 namespace w4a8 {
@@ -31,6 +33,7 @@ namespace w4a8 {
 namespace {
 
 constexpr int kFirstDecodeWarp = 2;
+constexpr int kMaxDevices = 64;
 constexpr int kABytes = kTileN * kTileK;            // decoded INT8 tile, 16 KiB
 constexpr int kDefaultTeamWarps = 4;               // warps per decode team
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -39,7 +42,7 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 constexpr uint32_t kSuspendHintNs = 20000u;
 constexpr unsigned long long kDrainLimitNs = 200000000ull;
 
-template <int TOK, bool GROUPED, int DW>
+template <int TOK, bool GROUPED, int DW, int CL>
 struct Cfg {
     static constexpr int kFirstEpiWarp = kFirstDecodeWarp + DW;
     // epilogue warpgroups: group mode spreads the per-k-block FP32 accumulation over
@@ -60,8 +63,14 @@ struct Cfg {
     // teams pay the per-k-block bookkeeping less often.
     static constexpr int kTeamWarps = (DW % kDefaultTeamWarps == 0) ? kDefaultTeamWarps : 4;
     static constexpr int kTeams = DW / kTeamWarps;
-    static constexpr int kQuartersPerThread = 16 / kTeamWarps;   // 32-k quarters of a row
-    static_assert(DW % kTeamWarps == 0 && kQuartersPerThread >= 1, "decode warps form whole teams");
+    // The CTAs of a cluster (CL = 1 or 2) work on the same row tile and k-block at the same time,
+    // each on its own token tile.  Each expands 128 / CL of the tile's rows and writes them into
+    // every CTA's stage (its own and, through distributed shared memory, its peer's), so the
+    // table lookups per MMA halve with CL = 2.
+    static constexpr int kRowsPerCta = kTileN / CL;
+    static constexpr int kQuartersPerThread = 4 / CL;            // 32-k quarters of a row per thread
+    static_assert(CL == 1 || CL == 2, "cluster of one or two CTAs");
+    static_assert(DW % kTeamWarps == 0 && kTeamWarps == 4, "decode warps form whole teams of four");
     // One stage holds the decoded INT8 weights of a k-block (operand A, 16 KiB, written by the
     // decode warps) and the tokens of the same k-block (operand B, written by TMA).  Keeping
     // operand A in tensor memory instead was measured slower at every token tile.
@@ -146,6 +155,53 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
+// The same test with cluster-scope acquire: the peer CTA's stores into this CTA's shared memory,
+// released by its arrival, are visible afterwards.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, const uint4 &v)
+{
+    asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y),
+                 "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_in_cluster)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_in_cluster)
+                 : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_all()
+{
+    asm volatile("fence.proxy.async;" ::: "memory");
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,
                                             uint32_t bar)
 {
@@ -153,15 +209,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
         "[%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
         "l"(map), "r"(bar), "r"(x), "r"(y)
-        : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes,
-                                          uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
-            "r"(dst),
-        "l"(src), "r"(bytes), "r"(bar)
         : "memory");
 }
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y)
@@ -197,6 +244,15 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::
                      "r"(bar)
                  : "memory");
+}
+// The same arrival on the barrier at this offset in every CTA of `mask`.
+__device__ __forceinline__ void tc_commit_multicast(uint32_t bar, uint16_t mask)
+{
+    asm volatile(
+        "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::
+            "r"(bar),
+        "h"(mask)
+        : "memory");
 }
 __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
                                           uint32_t idesc, uint32_t accumulate)
@@ -298,16 +354,9 @@ __device__ __forceinline__ bool named_bar_and(int id, int threads, bool pred)
     return out != 0;
 }
 
-// Shared-memory matrix descriptor of a K-major operand tile with 128-byte rows and
-// 128-byte swizzle: 8-row groups are 1024 bytes apart; `addr` may be advanced by 32 bytes
-// per 32-deep MMA step inside the swizzle span.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
-{
-    const uint32_t lo = ((addr & 0x3FFFFu) >> 4) | (1u << 16);
-    const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
-    return ((uint64_t)hi << 32) | lo;
-}
-
+// Shared-memory matrix descriptors (built in the MMA thread): K-major operand tile with 128-byte
+// rows and 128-byte swizzle, 8-row groups 1024 bytes apart; the start address advances by 32
+// bytes per 32-deep MMA step inside the swizzle span.
 // Instruction descriptor: signed 8-bit A and B, both K-major, INT32 accumulate, M = 128.
 __host__ __device__ constexpr uint32_t instr_desc_i8(int n)
 {
@@ -321,15 +370,19 @@ struct Ctl {
     uint32_t tmem_base;
 };
 
+template <bool CLUSTER_ACQUIRE = false>
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Ctl *ctl,
                                              StatusBlock *sb, int where,
                                              unsigned long long limit = kWaitLimitNs)
 {
-    if (mbar_try_wait(bar, parity)) return true;
+    auto test = [&]() {
+        return CLUSTER_ACQUIRE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity);
+    };
+    if (test()) return true;
     // the timer is slow to read: it is only consulted after many failed polls
     unsigned long long t0 = 0;
     for (uint32_t i = 1;; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (test()) return true;
         if ((i & 63u) == 0u) {
             if (ctl->abort) return false;
             if (t0 == 0) {
@@ -436,12 +489,12 @@ __device__ __forceinline__ void decode8(uint32_t w, const uint32_t (&t)[4], uint
 }
 
 // --------------------------------------------------------------------------- the kernel
-template <int TOK, bool GROUPED, int DW>
-__global__ void __launch_bounds__(Cfg<TOK, GROUPED, DW>::kThreads, 1)
+template <int TOK, bool GROUPED, int DW, int CL>
+__global__ void __launch_bounds__(Cfg<TOK, GROUPED, DW, CL>::kThreads, 1)
 linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                       const __grid_constant__ CUtensorMap y_map, const Params P)
 {
-    using C = Cfg<TOK, GROUPED, DW>;
+    using C = Cfg<TOK, GROUPED, DW, CL>;
     constexpr int kFirstEpiWarp = C::kFirstEpiWarp;
     constexpr int S = C::kStages;
     extern __shared__ uint8_t smem_raw[];
@@ -460,12 +513,18 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     Ctl *ctl = reinterpret_cast<Ctl *>(gen_base + C::kOffBarriers + 16 * S + 16 * NB + 16);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // Units (token-tile group, row tile, K slice) are dealt round-robin to the clusters; CTA
+    // `rank` of a cluster takes token tile CL * group + rank of the unit.
+    const uint32_t rank = CL > 1 ? cluster_ctarank() : 0u;
+    const int unit0 = (int)blockIdx.x / CL, unit_step = (int)gridDim.x / CL;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
-            // the warps of a decode team and the producer's arrival; the token copy completes on it too
-            mbar_init(bar_dec + 8 * s, C::kTeamWarps + 1);
-            mbar_init(bar_empty + 8 * s, 1);
+            // the warps of a decode team in every CTA of the cluster and the producer's arrival;
+            // the token copy completes on it too
+            mbar_init(bar_dec + 8 * s, C::kTeamWarps * CL + 1);
+            // the MMA threads of all CTAs of the cluster: they all read rows this CTA wrote
+            mbar_init(bar_empty + 8 * s, CL);
         }
         for (int b = 0; b < NB; ++b) {
             mbar_init(bar_acc_full + 8 * b, 1);
@@ -486,6 +545,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     }
     tc_fence_before();
     __syncthreads();
+    // no CTA may touch a peer's barriers or stages before the peer has set them up
+    if (CL > 1) cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     // Set-up is done; earlier work in the stream (the activation quantizer, a previous call's
@@ -504,10 +565,10 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             uint32_t it = 0;
             bool ok = true;
             KbCursor pf;
-            pf.start(blockIdx.x, gridDim.x, P.total_units, P.split_k, P.kb_per_split, k_blocks, n_tiles);
-            for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
+            pf.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, n_tiles);
+            for (int u = unit0; u < P.total_units && ok; u += unit_step) {
                 const int s = u % P.split_k, rest = u / P.split_k;
-                const int tt = rest / n_tiles;
+                const int tt = (rest / n_tiles) * CL + (int)rank;
                 const int kb0 = s * P.kb_per_split;
                 const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
@@ -553,7 +614,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             uint32_t st = 0, st_par = 0;                 // stage and its fill parity
             uint32_t buf = 0, buf_par = 0;               // accumulator buffer and its parity
             bool ok = true;
-            for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
+            for (int u = unit0; u < P.total_units && ok; u += unit_step) {
                 const int s = u % P.split_k;
                 const int kb0 = s * P.kb_per_split;
                 const int nkb = min(k_blocks, kb0 + P.kb_per_split) - kb0;
@@ -566,7 +627,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         break;
                     }
                     // decoded weights and tokens of the stage
-                    if (!wait_bounded(bar_dec + 8 * st, st_par, ctl, P.sb, 21)) {
+                    if (!wait_bounded<(CL > 1)>(bar_dec + 8 * st, st_par, ctl, P.sb, 21)) {
                         ok = false;
                         break;
                     }
@@ -581,7 +642,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         tc_mma_i8(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
                                   acc_flag);
                     }
-                    tc_commit(bar_empty + 8 * st);
+                    if (CL > 1) tc_commit_multicast(bar_empty + 8 * st, (uint16_t)((1u << CL) - 1u));
+                    else tc_commit(bar_empty + 8 * st);
                     if (last) {
                         tc_commit(bar_acc_full + 8 * buf);
                         if (++buf == (uint32_t)NB) { buf = 0; buf_par ^= 1u; }
@@ -600,13 +662,16 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         // slice of it); teams take k-blocks in turn, so the fixed latency of one k-block (barrier
         // wait, loads, proxy fence, arrive) overlaps the table lookups of the other teams.
         const int dt = threadIdx.x - 32 * kFirstDecodeWarp;
-        const int r = dt & 127;                              // row of the tile
         constexpr int QT = C::kQuartersPerThread;
-        const int q0 = ((dt >> 7) % (C::kTeamWarps / 4)) * QT;   // first 32-k quarter of this thread
+        // this CTA's share of the tile's rows; with two CTAs a thread takes half a row
+        const int r = (int)rank * C::kRowsPerCta + (dt & (C::kRowsPerCta - 1));
+        const int q0 = ((dt & 127) / C::kRowsPerCta) * QT;   // first 32-k quarter of this thread
         const int team = dt / (32 * C::kTeamWarps);
         constexpr int T = C::kTeams;
+        // the same stage and barrier in the peer CTA
+        const uint32_t peer = rank ^ 1u;
         KbCursor cur;
-        cur.start(blockIdx.x, gridDim.x, P.total_units, P.split_k, P.kb_per_split, k_blocks, n_tiles);
+        cur.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, n_tiles);
         cur.advance(team);
         uint4 w[QT];
         int z = 0;
@@ -647,12 +712,21 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     decode8(wq.y, t, c0.z, c0.w);
                     decode8(wq.z, t, c1.x, c1.y);
                     decode8(wq.w, t, c1.z, c1.w);
-                    *reinterpret_cast<uint4 *>(arow + (((2 * (q0 + q)) ^ sw) << 4)) = c0;
-                    *reinterpret_cast<uint4 *>(arow + (((2 * (q0 + q) + 1) ^ sw) << 4)) = c1;
+                    const int o0 = ((2 * (q0 + q)) ^ sw) << 4, o1 = ((2 * (q0 + q) + 1) ^ sw) << 4;
+                    *reinterpret_cast<uint4 *>(arow + o0) = c0;
+                    *reinterpret_cast<uint4 *>(arow + o1) = c1;
+                    if (CL > 1) {
+                        const uint32_t prow = map_to_cta(smem_u32(arow), peer);
+                        st_cluster_v4(prow + o0, c0);
+                        st_cluster_v4(prow + o1, c1);
+                    }
                 }
-                fence_proxy_async();
+                if (CL > 1) fence_proxy_async_all(); else fence_proxy_async();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_dec + 8 * st);
+                if (lane == 0) {
+                    mbar_arrive(bar_dec + 8 * st);
+                    if (CL > 1) mbar_arrive_cluster(map_to_cta(bar_dec + 8 * st, peer));
+                }
             }
 #pragma unroll
             for (int q = 0; q < QT; ++q) w[q] = wn[q];
@@ -700,9 +774,9 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             ++stores;
         };
 
-        for (int u = blockIdx.x; u < P.total_units && ok; u += gridDim.x) {
+        for (int u = unit0; u < P.total_units && ok; u += unit_step) {
             const int s = u % P.split_k, rest = u / P.split_k;
-            const int nt = rest % n_tiles, tt = rest / n_tiles;
+            const int nt = rest % n_tiles, tt = (rest / n_tiles) * CL + (int)rank;
             const int kb0 = s * P.kb_per_split;
             const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
             const int n = nt * kTileN + f;
@@ -947,6 +1021,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     // ---------------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
+    // a peer may still write this CTA's stages or arrive on its barriers until it is done too
+    if (CL > 1) cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
@@ -977,46 +1053,80 @@ EncodeTiledFn encode_tiled()
     return fn;
 }
 
-int sm_count()
-{
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-            n = v;
-        else
-            return 148;
-    }
-    return n;
-}
-
 struct Maps {
     CUtensorMap tok, y16, y32;      // activations; output with 16- and 32-token boxes
 };
 
-template <int TOK, bool GROUPED, int DW>
-w4a8_status launch_dw(const Maps &maps, const Params &P, cudaStream_t st)
+// Clusters of CL CTAs of this kernel that the current device can hold at once (one CTA per
+// SM); asked once per kernel instance and device.
+template <int TOK, bool GROUPED, int DW, int CL>
+int resident_clusters()
 {
-    using C = Cfg<TOK, GROUPED, DW>;
-    auto kern = linear_tcgen05_kernel<TOK, GROUPED, DW>;
+    using C = Cfg<TOK, GROUPED, DW, CL>;
+    static std::atomic<int> cached[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    int n = cached[dev].load(std::memory_order_acquire);
+    if (n > 0) return n;
+    auto kern = linear_tcgen05_kernel<TOK, GROUPED, DW, CL>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) !=
         cudaSuccess)
-        return W4A8_ERR_CUDA;
-    int grid = P.total_units < sm_count() ? P.total_units : sm_count();
+        return 0;
+    if (CL == 1) {
+        n = device_sms();
+    } else {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(CL * device_sms());
+        cfg.blockDim = dim3(C::kThreads);
+        cfg.dynamicSmemBytes = C::kSmemBytes;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = CL;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) {
+            cudaGetLastError();
+            return 0;
+        }
+    }
+    cached[dev].store(n, std::memory_order_release);
+    return n;
+}
+
+template <int TOK, bool GROUPED, int DW, int CL>
+w4a8_status launch_cl(const Maps &maps, const Params &P, cudaStream_t st)
+{
+    using C = Cfg<TOK, GROUPED, DW, CL>;
+    auto kern = linear_tcgen05_kernel<TOK, GROUPED, DW, CL>;
+    const int resident = resident_clusters<TOK, GROUPED, DW, CL>();   // also sizes the kernel's shared memory
+    if (resident < 1) return W4A8_ERR_CUDA;
+    const int clusters = P.total_units < resident ? P.total_units : resident;
     const cudaError_t e =
-        launch_overlapped(kern, dim3(grid), dim3(C::kThreads), (size_t)C::kSmemBytes, st, maps.tok,
-                          C::kChunk == 32 ? maps.y32 : maps.y16, P);
+        launch_overlapped_cluster(kern, dim3(clusters * CL), dim3(C::kThreads), (size_t)C::kSmemBytes, st, CL,
+                          maps.tok, C::kChunk == 32 ? maps.y32 : maps.y16, P);
     return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
 
-template <int TOK, bool GROUPED>
-w4a8_status launch_one(const Maps &maps, const Params &P, int dw, cudaStream_t st)
+template <int TOK, bool GROUPED, int DW>
+w4a8_status launch_dw(const Maps &maps, const Params &P, int cluster, cudaStream_t st)
 {
-    if (dw == 4) return launch_dw<TOK, GROUPED, 4>(maps, P, st);
-    if (dw == 8) return launch_dw<TOK, GROUPED, 8>(maps, P, st);
-    if (dw == 12 && !GROUPED) return launch_dw<TOK, false, 12>(maps, P, st);
-    if (dw == 16 && !GROUPED) return launch_dw<TOK, false, 16>(maps, P, st);
+    // two-CTA clusters exist for the wide token tiles: narrow ones serve few tokens
+    if constexpr (TOK >= 128) {
+        if (cluster == 2) return launch_cl<TOK, GROUPED, DW, 2>(maps, P, st);
+    }
+    if (cluster == 1) return launch_cl<TOK, GROUPED, DW, 1>(maps, P, st);
+    return W4A8_ERR_SHAPE;
+}
+
+template <int TOK, bool GROUPED>
+w4a8_status launch_one(const Maps &maps, const Params &P, int dw, int cluster, cudaStream_t st)
+{
+    if (dw == 4) return launch_dw<TOK, GROUPED, 4>(maps, P, cluster, st);
+    if (dw == 8) return launch_dw<TOK, GROUPED, 8>(maps, P, cluster, st);
+    if (dw == 12 && !GROUPED) return launch_dw<TOK, false, 12>(maps, P, cluster, st);
+    if (dw == 16 && !GROUPED) return launch_dw<TOK, false, 16>(maps, P, cluster, st);
     return W4A8_ERR_SHAPE;
 }
 
@@ -1035,7 +1145,7 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
         // job takes ceil(units / SMs) rounds of (k-blocks per unit + a fixed cost per unit for
         // pipeline fill and epilogue); a split adds the partial tile's round trip per unit and,
         // once at the end, the last slice's reduction (its loads go sixteen at a time).
-        const int sms = sm_count();
+        const int sms = device_sms();
         int tok_max = 16;
         while (tok_max < M && tok_max < cap) tok_max *= 2;
         double best = 0.0;
@@ -1071,7 +1181,14 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     if (tok != 16 && tok != 32 && tok != 64 && tok != 128 && tok != 192 && tok != 256) return false;
     if (tok > cap) return false;
     const int tok_tiles = (M + tok - 1) / tok;
-    const long long tiles = (long long)tok_tiles * L.n_tiles;
+    // Two-CTA clusters (each CTA expands half of the code tile for both) when there are at least
+    // two wide token tiles to pair; an odd last tile is paired with an empty one.
+    int cluster = opts ? opts->cluster : 0;
+    if (cluster == 0) cluster = (tok >= 128 && tok_tiles >= 2 && !grouped) ? 2 : 1;
+    if (cluster != 1 && !(cluster == 2 && tok >= 128)) return false;
+    const int tok_groups = (tok_tiles + cluster - 1) / cluster;
+    // one counter per (token tile, row tile), empty partner tiles included
+    const long long tiles = (long long)tok_groups * cluster * L.n_tiles;
     if (split < 1 || split > L.k_blocks) return false;
     const int kb_per = (L.k_blocks + split - 1) / split;
     split = (L.k_blocks + kb_per - 1) / kb_per;              // no empty slice
@@ -1080,6 +1197,7 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     if (dw == 0) dw = grouped ? 8 : 16;
     if (dw != 4 && dw != 8 && !((dw == 12 || dw == 16) && !grouped)) return false;
     plan->decode_warps = dw;
+    plan->cluster = cluster;
     plan->tok_tile = tok;
     plan->tok_tiles = tok_tiles;
     plan->split_k = split;
@@ -1141,7 +1259,7 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     P.m_pad = plan.tok_tiles * plan.tok_tile;
     P.split_k = plan.split_k;
     P.kb_per_split = plan.kb_per_split;
-    P.total_units = plan.tok_tiles * L.n_tiles * plan.split_k;
+    P.total_units = (plan.tok_tiles + plan.cluster - 1) / plan.cluster * L.n_tiles * plan.split_k;
     P.prefetch_codes = plan.tok_tiles == 1 ? 1 : 0;   // every code tile is read exactly once
     P.zp = zp;
     P.lt = make_level_tables(L.shift);
@@ -1149,12 +1267,12 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
 
     const bool g = L.group != 0;
     switch (plan.tok_tile) {
-    case 16: return g ? launch_one<16, true>(maps, P, plan.decode_warps, st) : launch_one<16, false>(maps, P, plan.decode_warps, st);
-    case 32: return g ? launch_one<32, true>(maps, P, plan.decode_warps, st) : launch_one<32, false>(maps, P, plan.decode_warps, st);
-    case 64: return g ? launch_one<64, true>(maps, P, plan.decode_warps, st) : launch_one<64, false>(maps, P, plan.decode_warps, st);
-    case 128: return g ? launch_one<128, true>(maps, P, plan.decode_warps, st) : launch_one<128, false>(maps, P, plan.decode_warps, st);
-    case 192: return g ? W4A8_ERR_SHAPE : launch_one<192, false>(maps, P, plan.decode_warps, st);
-    case 256: return g ? W4A8_ERR_SHAPE : launch_one<256, false>(maps, P, plan.decode_warps, st);
+    case 16: return g ? launch_one<16, true>(maps, P, plan.decode_warps, plan.cluster, st) : launch_one<16, false>(maps, P, plan.decode_warps, plan.cluster, st);
+    case 32: return g ? launch_one<32, true>(maps, P, plan.decode_warps, plan.cluster, st) : launch_one<32, false>(maps, P, plan.decode_warps, plan.cluster, st);
+    case 64: return g ? launch_one<64, true>(maps, P, plan.decode_warps, plan.cluster, st) : launch_one<64, false>(maps, P, plan.decode_warps, plan.cluster, st);
+    case 128: return g ? launch_one<128, true>(maps, P, plan.decode_warps, plan.cluster, st) : launch_one<128, false>(maps, P, plan.decode_warps, plan.cluster, st);
+    case 192: return g ? W4A8_ERR_SHAPE : launch_one<192, false>(maps, P, plan.decode_warps, plan.cluster, st);
+    case 256: return g ? W4A8_ERR_SHAPE : launch_one<256, false>(maps, P, plan.decode_warps, plan.cluster, st);
     }
     return W4A8_ERR_SHAPE;
 }

@@ -259,7 +259,8 @@ cudaError_t launch_unpack(const uint8_t *blob, const BlobLayout &L, uint8_t *cod
 {
     const size_t total = (size_t)L.N * L.K / 2;
     int blocks = (int)((total + 255) / 256);
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    const int cap = device_sms() * 16;
+    if (blocks > cap) blocks = cap;
     unpack_kernel<<<blocks, 256, 0, st>>>(blob, L, codes, scales, zeros);
     return cudaGetLastError();
 }
@@ -272,7 +273,7 @@ cudaError_t launch_weight_rowsum(const uint8_t *blob, const BlobLayout &L, int32
     if (L.group != 0) {
         slices = L.k_blocks;
     } else {
-        slices = (8 * 148 + L.n_tiles - 1) / L.n_tiles;
+        slices = (8 * device_sms() + L.n_tiles - 1) / L.n_tiles;
         if (slices > L.k_blocks) slices = L.k_blocks;
         if (cudaMemsetAsync(rowsum, 0, (size_t)L.N * sizeof(int32_t), st) != cudaSuccess)
             return cudaGetLastError();

@@ -70,15 +70,21 @@ def outlier_channels(K: int, spec, seed: int) -> np.ndarray:
     return np.sort(rng.permutation(K)[: n_outliers(K, spec)])
 
 
-def make_weights(N: int, K: int, seed: int) -> np.ndarray:
-    """[N, K] float16, normal with standard deviation 0.02."""
+def make_weights(N: int, K: int, seed: int, n_rows: int | None = None) -> np.ndarray:
+    """[N, K] float16, normal with standard deviation 0.02.  With `n_rows` only the first
+    n_rows rows are drawn (the same values the full matrix has there)."""
     rng = np.random.Generator(np.random.PCG64([seed, 1]))
-    out = np.empty((N, K), dtype=np.float16)
+    n_out = N if n_rows is None else min(N, n_rows)
+    out = np.empty((n_out, K), dtype=np.float16)
     rows = max(1, (1 << 24) // K)
-    for r0 in range(0, N, rows):
-        r1 = min(N, r0 + rows)
-        out[r0:r1] = (rng.standard_normal((r1 - r0, K), dtype=np.float32)
-                      * np.float32(0.02)).astype(np.float16)
+    buf = np.empty((rows, K), dtype=np.float32)
+    for r0 in range(0, n_out, rows):
+        r1 = min(N, r0 + rows)          # chunk boundaries follow the full matrix
+        chunk = buf[: r1 - r0]
+        rng.standard_normal(out=chunk, dtype=np.float32)
+        np.multiply(chunk, np.float32(0.02), out=chunk)
+        keep = min(r1, n_out) - r0
+        out[r0:r0 + keep] = chunk[:keep]
     return out
 
 
@@ -114,8 +120,15 @@ def make_channel_scales(X: np.ndarray, W: np.ndarray):
     multiplies by s, the activation side by the binary32 reciprocal.
     Returns (s [K] float32, inv_s [K] float32).
     """
-    ax = np.abs(X.astype(np.float32)).max(axis=0)
-    aw = np.abs(W.astype(np.float32)).max(axis=0)
+    def col_absmax(A):
+        m = np.zeros(A.shape[1], dtype=np.float32)
+        rows = max(1, (1 << 24) // A.shape[1])
+        for r0 in range(0, A.shape[0], rows):
+            np.maximum(m, np.abs(A[r0:r0 + rows]).max(axis=0).astype(np.float32), out=m)
+        return m
+
+    ax = col_absmax(X)
+    aw = col_absmax(W)
     with np.errstate(divide="ignore", invalid="ignore"):
         s = np.sqrt(ax / aw)
     s = np.where(np.isfinite(s), s, 1.0)

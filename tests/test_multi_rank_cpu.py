@@ -59,3 +59,34 @@ def test_reference_arm_prints_on_rank_0_only():
                         "--gpus", "2", "--steps", "1", "--warmup", "0"], env=env,
                        capture_output=True, text=True, timeout=300)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_gpus_flag_is_honoured():
+    """--gpus N decides the launch: alone for one GPU, as a rank of a launcher whose world size
+    agrees, by starting the ranks itself when no launcher did; a disagreeing launcher is an error."""
+    import pytest
+
+    import bench
+    assert bench.launch_mode(1, {}) == "single"
+    assert bench.launch_mode(1, {"WORLD_SIZE": "1"}) == "single"
+    assert bench.launch_mode(4, {"WORLD_SIZE": "4"}) == "rank"
+    assert bench.launch_mode(2, {}) == "spawn"
+    with pytest.raises(SystemExit):
+        bench.launch_mode(8, {"WORLD_SIZE": "2"})
+    with pytest.raises(SystemExit):
+        bench.launch_mode(1, {"WORLD_SIZE": "2"})
+    with pytest.raises(SystemExit):
+        bench.launch_mode(0, {})
+    cmd = bench.spawn_command(2, ["--gpus", "2", "--steps", "3"], 29511)
+    assert "torch.distributed.run" in cmd and "--nproc-per-node=2" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-4:] == ["--gpus", "2", "--steps", "3"]
+
+
+def test_reference_arm_does_not_need_the_cuda_library():
+    """The CPU-only arm draws its inputs without importing the package that loads libw4a8.so."""
+    code = ("import sys, bench; s = bench.load_synth(); "
+            "assert s.WORKLOADS[4].shapes[0][:2] == (9216, 36864); "
+            "assert 'paper_2311_05161_b200' not in sys.modules")
+    r = subprocess.run([sys.executable, "-c", code], cwd=ROOT, capture_output=True, text=True, timeout=120)
+    assert r.returncode == 0, r.stderr
