@@ -395,6 +395,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-legs", action="store_true",
                     help="only the headline workload (resident and host-buffer timings)")
+    ap.add_argument("--plan", default=None,
+                    help="tok_tile,split_k,decode_warps,cluster for the tensor-core kernel of the headline "
+                         "instead of the library's own choice (sweeps)")
     ap.add_argument("--no-graph", action="store_true",
                     help="--case only: time with per-launch events, no CUDA graph replay")
     ap.add_argument("--case", default=None,
@@ -449,7 +452,12 @@ def main():
         barrier()
         return max_over_ranks(e0.elapsed_time(e1), world, dev)
 
-    def device_block(layers, M, rot=1, host_buffers=False, asym=False):
+    plan_opts = None
+    if args.plan:
+        pt, ps, pd, pc = [int(v) for v in args.plan.split(",")]
+        plan_opts = w4a8.make_opts(w4a8.PATH_TCGEN05, ps, pt, pd, cluster=pc)
+
+    def device_block(layers, M, rot=1, host_buffers=False, asym=False, opts=None):
         """Device tensors of a list of layers: packed weights (rot rotating copies), inputs,
         outputs, workspaces."""
         L = []
@@ -462,8 +470,8 @@ def main():
             d["Xq"] = torch.empty((M, K), dtype=torch.int8, device=dev)
             d["tok"] = torch.empty((M,), dtype=torch.float32, device=dev)
             d["Y"] = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
-            d["ws"] = w4a8.new_workspace(M, N, K, group)
-            d.update(K=K, N=N, M=M, group=group, label=lay["label"])
+            d["ws"] = w4a8.new_workspace(M, N, K, group, opts)
+            d.update(K=K, N=N, M=M, group=group, label=lay["label"], opts=opts)
             if host_buffers:
                 d["X_host"] = torch.from_numpy(lay["X"]).pin_memory()
                 d["Y_host"] = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
@@ -479,7 +487,7 @@ def main():
             if record is not None:
                 record[i][0].record()
             w4a8.linear(d["Xq"], d["tok"], d["packed_rot"][it % len(d["packed_rot"])], d["bias"],
-                        d["N"], d["group"], d["ws"], out=d["Y"])
+                        d["N"], d["group"], d["ws"], d["opts"], out=d["Y"])
             if record is not None:
                 record[i][1].record()
 
@@ -540,7 +548,7 @@ def main():
 
     # ------------------------------------------------------------------ headline: set-up (untimed)
     layers = host_layers(synth, HEADLINE_CONFIG, HEADLINE_SHAPES, M_PREFILL)
-    L = device_block(layers, M_PREFILL, host_buffers=True)
+    L = device_block(layers, M_PREFILL, host_buffers=True, opts=plan_opts)
     ops_per_pass = sum(2 * M_PREFILL * d["K"] * d["N"] for d in L)
 
     # ------------------------------------------------------------------ headline: resident inputs
@@ -573,7 +581,7 @@ def main():
             main_stream.wait_event(ev_down[i])       # the previous pass's download has read Y
             w4a8.quantize_act(d["X"], d["inv_s"], out=(d["Xq"], d["tok"]))
             w4a8.linear(d["Xq"], d["tok"], d["packed"], d["bias"], d["N"], d["group"], d["ws"],
-                        out=d["Y"])
+                        d["opts"], out=d["Y"])
             ev_done[i].record(main_stream)
             with torch.cuda.stream(s_down):
                 s_down.wait_event(ev_done[i])
@@ -791,6 +799,7 @@ def main():
                    "pass": "4 x (quantize_act + linear); weights packed once before timing",
                    "passes_per_step": passes, "ms_per_pass": ms_pass, "timed_region_s": region_s,
                    "l2": "inputs larger than L2 (about 1.3 GB touched per pass)",
+                   "plan": w4a8.linear_plan(M_PREFILL, layers[2]["N"], layers[2]["K"], layers[2]["group"], plan_opts),
                    "parallelism": "replicas" if world > 1 else "single"},
         "clocks": clocks,
         "e2e": {"value": replica_throughput(ops_per_pass, world, ms_e2e), "unit": "TOPS",

@@ -44,6 +44,7 @@ constexpr unsigned long long kDrainLimitNs = 200000000ull;
 
 template <int TOK, bool GROUPED, int DW, int CL>
 struct Cfg {
+    // warps in a row: producer, MMA issuer, DW decode warps, epilogue warps
     static constexpr int kFirstEpiWarp = kFirstDecodeWarp + DW;
     // epilogue warpgroups: group mode spreads the per-k-block FP32 accumulation over
     // 32 columns per thread (more warps in flight, fewer registers each)
@@ -51,6 +52,9 @@ struct Cfg {
     static constexpr int kStageBufs = GROUPED ? 1 : 2;      // output staging buffers per group
     static constexpr int kEpiWarps = 4 * kEpiGroups;
     static constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
+    // With at most 512 threads a thread has the registers to expand its codes before the stage
+    // they go to is free (its raw codes, the next k-block's raw codes and the expanded levels).
+    static constexpr bool kExpandAhead = kThreads <= 512;
     static constexpr int kColsPerThread = TOK / kEpiGroups;
     static constexpr int kChunk = kColsPerThread >= 32 ? 32 : 16;
     static constexpr int kTokBytes = TOK * kTileK;
@@ -64,9 +68,9 @@ struct Cfg {
     static constexpr int kTeamWarps = (DW % kDefaultTeamWarps == 0) ? kDefaultTeamWarps : 4;
     static constexpr int kTeams = DW / kTeamWarps;
     // The CTAs of a cluster (CL = 1 or 2) work on the same row tile and k-block at the same time,
-    // each on its own token tile.  Each expands 128 / CL of the tile's rows and writes them into
-    // every CTA's stage (its own and, through distributed shared memory, its peer's), so the
-    // table lookups per MMA halve with CL = 2.
+    // each on its own token tile.  With CL = 2 each expands 64 of the tile's 128 rows into its own
+    // stage and sends them to its peer's stage with a bulk copy through distributed shared memory
+    // that completes on the peer's barrier, so the table lookups per MMA halve.
     static constexpr int kRowsPerCta = kTileN / CL;
     static constexpr int kQuartersPerThread = 4 / CL;            // 32-k quarters of a row per thread
     static_assert(CL == 1 || CL == 2, "cluster of one or two CTAs");
@@ -155,20 +159,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// The same test with cluster-scope acquire: the peer CTA's stores into this CTA's shared memory,
-// released by its arrival, are visible afterwards.
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
-        : "memory");
-    return ok != 0;
-}
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {
     uint32_t r;
@@ -182,25 +172,21 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void st_cluster_v4(uint32_t addr, const uint4 &v)
+// Copy `bytes` (a multiple of 16) of this CTA's shared memory into a peer CTA's shared memory;
+// the bytes count towards the transaction count of the peer's barrier `bar_in_cluster`.
+__device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_in_cluster, uint32_t src, uint32_t bytes,
+                                                 uint32_t bar_in_cluster)
 {
-    asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y),
-                 "r"(v.z), "r"(v.w)
-                 : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_in_cluster)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_in_cluster)
-                 : "memory");
+    asm volatile(
+        "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
+            "r"(dst_in_cluster),
+        "r"(src), "r"(bytes), "r"(bar_in_cluster)
+        : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void fence_proxy_async_all()
-{
-    asm volatile("fence.proxy.async;" ::: "memory");
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,
                                             uint32_t bar)
@@ -320,14 +306,19 @@ __device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
     return r;
 }
-// A group's INT32 partial sum is below 2^22 in magnitude (128 products of at most 127 * 26), so
-// its low 23 bits with bit 22 flipped, under the exponent of 2^23, are the FP32 number
-// 1.5 * 2^23 + sum: one logic instruction instead of a conversion, which runs at an eighth of
-// the FP32 rate.  Subtracting 1.5 * 2^23 afterwards is exact.
+// A group's INT32 partial sum is below 2^22 in magnitude (128 products of at most 127 * 104), so
+// adding it, as an integer, to the bit pattern of 1.5 * 2^23 gives the FP32 number 1.5 * 2^23 + sum:
+// no conversion instruction (an eighth of the FP32 rate).  The add is written as a multiply-add
+// by a register that holds 1, which runs on the FMA pipe: the 16-lane logic pipe is what the
+// decode warps need.  Subtracting 1.5 * 2^23 afterwards is exact.  (Accumulators that start from
+// that bit pattern, refilled with tcgen05.st after every read, were measured slower: the refill
+// sits in the hand-over chain.)
 constexpr uint32_t kMagicBits = 0x4B400000u;          // 1.5 * 2^23 = 12582912.0f
-__device__ __forceinline__ uint32_t biased_float_bits(uint32_t acc)
+__device__ __forceinline__ uint32_t biased_float_bits(uint32_t acc, uint32_t one)
 {
-    return (acc & 0x007FFFFFu) ^ kMagicBits;
+    uint32_t r;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(acc), "r"(one), "r"(kMagicBits));
+    return r;
 }
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 {
@@ -370,19 +361,15 @@ struct Ctl {
     uint32_t tmem_base;
 };
 
-template <bool CLUSTER_ACQUIRE = false>
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Ctl *ctl,
                                              StatusBlock *sb, int where,
                                              unsigned long long limit = kWaitLimitNs)
 {
-    auto test = [&]() {
-        return CLUSTER_ACQUIRE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity);
-    };
-    if (test()) return true;
+    if (mbar_try_wait(bar, parity)) return true;
     // the timer is slow to read: it is only consulted after many failed polls
     unsigned long long t0 = 0;
     for (uint32_t i = 1;; ++i) {
-        if (test()) return true;
+        if (mbar_try_wait(bar, parity)) return true;
         if ((i & 63u) == 0u) {
             if (ctl->abort) return false;
             if (t0 == 0) {
@@ -513,6 +500,13 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     Ctl *ctl = reinterpret_cast<Ctl *>(gen_base + C::kOffBarriers + 16 * S + 16 * NB + 16);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // role of this warp and its index inside the role
+    enum { kProducer, kMma, kDecode, kEpilogue };
+    int role, role_idx = 0;
+    if (warp == 0) role = kProducer;
+    else if (warp == 1) role = kMma;
+    else if (warp < kFirstEpiWarp) { role = kDecode; role_idx = warp - kFirstDecodeWarp; }
+    else { role = kEpilogue; role_idx = warp - kFirstEpiWarp; }
     // Units (token-tile group, row tile, K slice) are dealt round-robin to the clusters; CTA
     // `rank` of a cluster takes token tile CL * group + rank of the unit.
     const uint32_t rank = CL > 1 ? cluster_ctarank() : 0u;
@@ -520,9 +514,9 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
-            // the warps of a decode team in every CTA of the cluster and the producer's arrival;
-            // the token copy completes on it too
-            mbar_init(bar_dec + 8 * s, C::kTeamWarps * CL + 1);
+            // the warps of a decode team and the producer's arrival; the token copy and, in a
+            // cluster, the peer's half of the expanded rows complete on it too
+            mbar_init(bar_dec + 8 * s, C::kTeamWarps + 1);
             // the MMA threads of all CTAs of the cluster: they all read rows this CTA wrote
             mbar_init(bar_empty + 8 * s, CL);
         }
@@ -536,7 +530,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
-    if (warp == 1) {
+    if (role == kMma) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                          smem_u32(&ctl->tmem_base)),
                      "r"((uint32_t)C::kTmemCols)
@@ -559,7 +553,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     if (!blob_ok) {
         // not the blob the caller described: nothing is read or written, only the status
         if (threadIdx.x == 0) report_failure(P.sb, W4A8_ERR_BAD_BLOB, 2);
-    } else if (warp == 0) {
+    } else if (role == kProducer) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
             uint32_t it = 0;
@@ -580,7 +574,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     }
                     const uint32_t stage = base + st * C::kStageBytes;
                     const uint32_t tok_bar = bar_dec + 8 * st;
-                    mbar_arrive_expect_tx(tok_bar, C::kTokBytes);
+                    mbar_arrive_expect_tx(tok_bar, C::kTokBytes + (CL > 1 ? kABytes / CL : 0));
                     tma_load_2d(stage + C::kTokOff, &tok_map, kb * kTileK, tt * TOK, tok_bar);
                     if (P.prefetch_codes) {
                         // keep the code stream kPrefetchAhead k-blocks ahead of the decode warps
@@ -602,7 +596,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             }
         }
         __syncwarp();
-    } else if (warp == 1) {
+    } else if (role == kMma) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             // This loop is the serial spine of the kernel (one thread, once per k-block): all
@@ -627,7 +621,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         break;
                     }
                     // decoded weights and tokens of the stage
-                    if (!wait_bounded<(CL > 1)>(bar_dec + 8 * st, st_par, ctl, P.sb, 21)) {
+                    if (!wait_bounded(bar_dec + 8 * st, st_par, ctl, P.sb, 21)) {
                         ok = false;
                         break;
                     }
@@ -656,16 +650,19 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             wait_bounded(bar_drain, 0u, ctl, P.sb, 22, ok ? kWaitLimitNs : kDrainLimitNs);
         }
         __syncwarp();
-    } else if (warp < kFirstEpiWarp) {
+    } else if (role == kDecode) {
         // ------------------------------------------------------------------ decode warps
         // The warps of a team share a k-block (a thread takes one feature row and one column
         // slice of it); teams take k-blocks in turn, so the fixed latency of one k-block (barrier
         // wait, loads, proxy fence, arrive) overlaps the table lookups of the other teams.
-        const int dt = threadIdx.x - 32 * kFirstDecodeWarp;
+        const int dt = role_idx * 32 + lane;
         constexpr int QT = C::kQuartersPerThread;
-        // this CTA's share of the tile's rows; with two CTAs a thread takes half a row
-        const int r = (int)rank * C::kRowsPerCta + (dt & (C::kRowsPerCta - 1));
-        const int q0 = ((dt & 127) / C::kRowsPerCta) * QT;   // first 32-k quarter of this thread
+        // One thread per row of the tile; in a cluster this CTA takes 64 of the rows, a warp 16 of
+        // them, and a thread half a row, so that a warp's rows are one contiguous 2 KiB piece of
+        // the stage.
+        const int r = CL == 1 ? (dt & 127)
+                              : (int)rank * C::kRowsPerCta + ((dt >> 5) & 3) * 16 + (lane & 15);
+        const int q0 = CL == 1 ? 0 : (lane >> 4) * QT;       // first 32-k quarter of this thread
         const int team = dt / (32 * C::kTeamWarps);
         constexpr int T = C::kTeams;
         // the same stage and barrier in the peer CTA
@@ -696,36 +693,49 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             const uint32_t fill = cur.it / S;
             uint32_t t[4];
             build_level_tables(z, P.lt, t);
+            uint4 lv[2 * QT];                    // the thread's INT8 levels, 16 per register quad
+            auto expand = [&]() {
+#pragma unroll
+                for (int q = 0; q < QT; ++q) {
+                    const uint4 wq = w[q];
+                    decode8(wq.x, t, lv[2 * q].x, lv[2 * q].y);
+                    decode8(wq.y, t, lv[2 * q].z, lv[2 * q].w);
+                    decode8(wq.z, t, lv[2 * q + 1].x, lv[2 * q + 1].y);
+                    decode8(wq.w, t, lv[2 * q + 1].z, lv[2 * q + 1].w);
+                }
+            };
+            if (C::kExpandAhead) {
+                // The levels are ready in registers before the stage is: only the stores stand
+                // between the moment the stage is free and the moment its operands are in place.
+                expand();
+#pragma unroll
+                for (int q = 0; q < 2 * QT; ++q)
+                    asm volatile("" : "+r"(lv[q].x), "+r"(lv[q].y), "+r"(lv[q].z), "+r"(lv[q].w));
+            }
             {
                 // the operand buffer is free once the MMAs of its last use have retired
                 ok = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+                if (!C::kExpandAhead) expand();
                 uint8_t *stage = gen_base + st * C::kStageBytes;
                 uint8_t *arow = stage + r * 128;
                 const int sw = r & 7;
 #pragma unroll
                 for (int q = 0; q < QT; ++q) {
-                    const uint4 wq = w[q];
-                    uint4 c0, c1;
-                    decode8(wq.x, t, c0.x, c0.y);
-                    decode8(wq.y, t, c0.z, c0.w);
-                    decode8(wq.z, t, c1.x, c1.y);
-                    decode8(wq.w, t, c1.z, c1.w);
-                    const int o0 = ((2 * (q0 + q)) ^ sw) << 4, o1 = ((2 * (q0 + q) + 1) ^ sw) << 4;
-                    *reinterpret_cast<uint4 *>(arow + o0) = c0;
-                    *reinterpret_cast<uint4 *>(arow + o1) = c1;
-                    if (CL > 1) {
-                        const uint32_t prow = map_to_cta(smem_u32(arow), peer);
-                        st_cluster_v4(prow + o0, c0);
-                        st_cluster_v4(prow + o1, c1);
-                    }
+                    *reinterpret_cast<uint4 *>(arow + (((2 * (q0 + q)) ^ sw) << 4)) = lv[2 * q];
+                    *reinterpret_cast<uint4 *>(arow + (((2 * (q0 + q) + 1) ^ sw) << 4)) = lv[2 * q + 1];
                 }
-                if (CL > 1) fence_proxy_async_all(); else fence_proxy_async();
+                fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive(bar_dec + 8 * st);
-                    if (CL > 1) mbar_arrive_cluster(map_to_cta(bar_dec + 8 * st, peer));
+                    if (CL > 1) {
+                        // this warp's 16 rows, now complete in the local stage, go to the peer
+                        const uint32_t piece = base + st * C::kStageBytes + (uint32_t)(r * 128);
+                        bulk_copy_to_cta(map_to_cta(piece, peer), piece, 16 * 128,
+                                         map_to_cta(bar_dec + 8 * st, peer));
+                    }
                 }
             }
 #pragma unroll
@@ -733,15 +743,15 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             z = zn;
             cur = nxt;
         }
-    } else {
+    } else if (role == kEpilogue) {
         // ------------------------------------------------------------------ epilogue warps
-        const int ew = warp - kFirstEpiWarp;
+        const int ew = role_idx;
         const int quarter = warp & 3;                     // tensor-memory lane quarter
         const int col_group = ew >> 2;                    // which share of the columns
         const int col0 = col_group * C::kColsPerThread;
         const int f = quarter * 32 + lane;                // feature row inside the tile
         constexpr int kEpiThreads = 32 * C::kEpiWarps;
-        const int et = threadIdx.x - 32 * kFirstEpiWarp;
+        const int et = ew * 32 + lane;
         const bool elected = et == col_group * 128;       // issues this group's bulk stores
         const int group_bar = 2 + col_group;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
@@ -904,6 +914,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 uint64_t usum2[C::kColsPerThread / 2];
 #pragma unroll
                 for (int j = 0; j < C::kColsPerThread / 2; ++j) usum2[j] = 0ull;
+                uint32_t one = 1u;                       // opaque to the compiler: see biased_float_bits
+                asm volatile("" : "+r"(one));
                 const uint32_t neg_magic = __float_as_uint(-12582912.0f);
                 const uint64_t neg_magic2 = pack_f32x2(neg_magic, neg_magic);
                 // the next group's step is loaded one k-block ahead and only touched when used,
@@ -924,7 +936,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     for (int c = 0; c < C::kColsPerThread; c += kAcc) {
                         uint32_t v[32];
                         const uint32_t taddr = tmem_base + lane_base + buf * TOK + col0 + c;
-                        if (kAcc == 32) tc_ld32(taddr, v); else tc_ld16(taddr, v);
+                        tc_ld16(taddr, v);
                         tc_wait_ld();
                         if (c + kAcc >= C::kColsPerThread) {
                             tc_fence_before();
@@ -934,7 +946,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
 #pragma unroll
                         for (int j = 0; j < kAcc; j += 2) {
                             const uint64_t biased =
-                                pack_f32x2(biased_float_bits(v[j]), biased_float_bits(v[j + 1]));
+                                pack_f32x2(biased_float_bits(v[j], one), biased_float_bits(v[j + 1], one));
                             usum2[(c + j) >> 1] =
                                 fma_f32x2(add_f32x2(biased, neg_magic2), h2, usum2[(c + j) >> 1]);
                         }
@@ -1023,7 +1035,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     __syncthreads();
     // a peer may still write this CTA's stages or arrive on its barriers until it is done too
     if (CL > 1) cluster_sync_all();
-    if (warp == 1) {
+    if (role == kMma) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                      "r"((uint32_t)C::kTmemCols)
@@ -1181,10 +1193,13 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     if (tok != 16 && tok != 32 && tok != 64 && tok != 128 && tok != 192 && tok != 256) return false;
     if (tok > cap) return false;
     const int tok_tiles = (M + tok - 1) / tok;
-    // Two-CTA clusters (each CTA expands half of the code tile for both) when there are at least
-    // two wide token tiles to pair; an odd last tile is paired with an empty one.
+    // Two-CTA clusters (each CTA expands half of the code tile for both; an odd last token tile
+    // is paired with an empty one) are there on request.  Measured on 9216 -> 36864 at 2048 tokens
+    // they halve the table lookups and run at a higher clock under the power cap (1590 against
+    // 1370 MHz), but the hand-over between the two CTAs lengthens the per-k-block chain more than
+    // that gains (2200 against 2380 TOPS sustained), so the automatic plan stays with one CTA.
     int cluster = opts ? opts->cluster : 0;
-    if (cluster == 0) cluster = (tok >= 128 && tok_tiles >= 2 && !grouped) ? 2 : 1;
+    if (cluster == 0) cluster = 1;
     if (cluster != 1 && !(cluster == 2 && tok >= 128)) return false;
     const int tok_groups = (tok_tiles + cluster - 1) / cluster;
     // one counter per (token tile, row tile), empty partner tiles included

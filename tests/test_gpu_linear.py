@@ -40,11 +40,9 @@ def test_tcgen05_config1(group):
     check_y(prob, Y, exact=(group == 0))
 
 
-@pytest.mark.parametrize("group", [0, 128])
-@pytest.mark.parametrize("tok_tile", [16, 32, 64, 128, 192, 256])
+@pytest.mark.parametrize("tok_tile,group", [(t, g) for g in (0, 128) for t in (16, 32, 64, 128, 192, 256)
+                                            if not (g and t > 128)])   # group mode tiles at most 128 tokens
 def test_tcgen05_token_tiles_and_ragged_edges(tok_tile, group):
-    if group and tok_tile > 128:
-        pytest.skip("group mode tiles at most 128 tokens")
     # M spans several token tiles with a ragged tail; N = 200 is not a multiple of 128
     M = tok_tile * 2 + 5
     prob = Problem(1024, 200, M, group, seed=tok_tile + group, dist="laplace", outliers=0.01,
@@ -166,3 +164,39 @@ def test_gemv_row_slab_kernel_with_requested_warps(warps, group):
 
 def test_gemv_path_rejects_more_than_four_tokens():
     assert w4a8.linear_workspace_bytes(5, 256, 256, 0, w4a8.make_opts(w4a8.PATH_GEMV)) == 0
+
+
+@pytest.mark.parametrize("tok_tile", [128, 192, 256])
+def test_tcgen05_two_cta_clusters(tok_tile):
+    """Two CTAs of a cluster share the expansion of every code tile (each writes half of the rows
+    into both CTAs' stages).  Three token tiles: the last one is paired with an empty tile; N = 200
+    leaves a ragged row tile.  The one-CTA form of the same plan gives the same bits."""
+    M = tok_tile * 2 + 5
+    prob = Problem(1024, 200, M, 0, seed=700 + tok_tile, dist="laplace", outliers=0.01, mult=20.0)
+    packed = w4a8.pack_weights(prob.dev["W"], prob.dev["s"], 0)
+    Y2, acc2 = run_linear(prob, w4a8.make_opts(w4a8.PATH_TCGEN05, tok_tile=tok_tile, cluster=2), packed)
+    Y1, acc1 = run_linear(prob, w4a8.make_opts(w4a8.PATH_TCGEN05, tok_tile=tok_tile, cluster=1), packed)
+    assert np.array_equal(acc2, prob.oracle_acc())
+    assert np.array_equal(acc1, acc2) and np.array_equal(Y1, Y2)
+    check_y(prob, Y2, exact=True)
+
+
+def test_tcgen05_two_cta_clusters_many_units_and_split_k():
+    # more units than clusters (every cluster walks several units, stages and accumulators wrap),
+    # then a K split on top (partial tiles, last-arriver reduction, an empty partner tile)
+    prob = Problem(1536, 128 * 44, 300, 0, seed=711)
+    packed = w4a8.pack_weights(prob.dev["W"], prob.dev["s"], 0)
+    want = prob.oracle_acc()
+    for split in (1, 3):
+        opts = w4a8.make_opts(w4a8.PATH_TCGEN05, split_k=split, tok_tile=128, cluster=2)
+        for _ in range(2):
+            Y, acc = run_linear(prob, opts, packed)
+            assert np.array_equal(acc, want)
+            check_y(prob, Y, exact=True)
+
+
+def test_cluster_option_is_validated():
+    assert w4a8.linear_workspace_bytes(300, 256, 256, 0, w4a8.make_opts(tok_tile=64, cluster=2)) == 0
+    assert w4a8.linear_workspace_bytes(300, 256, 256, 0, w4a8.make_opts(tok_tile=128, cluster=3)) == 0
+    assert w4a8.linear_plan(2048, 4096, 4096, 0)["cluster"] == 1
+    assert w4a8.linear_plan(2048, 4096, 4096, 0, w4a8.make_opts(tok_tile=256, cluster=2))["cluster"] == 2
