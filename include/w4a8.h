@@ -20,7 +20,8 @@
  *   - Base pointers must be 16-byte aligned, `packed` and `workspace` 256-byte aligned.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All work
  *     is enqueued on it; no call synchronizes the device except w4a8_poll_status.
- *   - The library allocates no device memory and keeps no device state between calls.
+ *   - The library allocates no device memory and keeps no device state between calls (the one
+ *     exception is the fixed scratch array of w4a8_linear_static, see there).
  *   - Every call validates its arguments first and launches nothing when validation
  *     fails.  Inputs holding NaN or Inf are a precondition violation.
  *   - There is no CPU or other-architecture fallback: a device that is not compute
@@ -69,7 +70,13 @@ typedef struct {
                         1, or 2 (token tiles of 128 and more): the two CTAs work on two token
                         tiles of the same weight rows and each expands half of every code tile
                         for both */
-    int reserved[2]; /* must be zero */
+    int debug_wait_ms;   /* test hook, 0 = off: limit of every bounded wait inside the tensor-core
+                            kernel in milliseconds (normally 2 s) */
+    int debug_skip_load; /* test hook, 0 = off: the copy thread of every CTA leaves out the token
+                            load of its k-block number debug_skip_load - 1, so that a wait runs
+                            out and the kernel reports W4A8_ERR_TIMEOUT.  Both hooks are refused
+                            (W4A8_ERR_SHAPE) unless the library was built with W4A8_DEBUG_HOOKS,
+                            and only w4a8_linear_ex with W4A8_PATH_TCGEN05 takes them */
 } w4a8_opts;
 
 /* Bytes of the packed-weight blob for an [N][K] matrix; 0 if the shape is invalid.
@@ -116,7 +123,8 @@ w4a8_status w4a8_quantize_act(const void *X_f16, const float *inv_s_in, int M, i
 
 /* Scratch bytes w4a8_linear needs for this shape (always >= 256: the first 256 bytes
  * hold the status block read by w4a8_poll_status).  The caller zero-fills the workspace
- * once after allocating it (w4a8_workspace_init); calls leave it ready for reuse.  Calls
+ * once after allocating it (w4a8_workspace_init); calls that end without a reported failure
+ * leave it ready for reuse (after a failure: see w4a8_poll_status).  Calls
  * that may overlap on the device need separate workspaces.  The _ex form answers for
  * explicit options (NULL = automatic); 0 means the shape or the options are invalid. */
 size_t w4a8_linear_workspace_bytes(int M, int N, int K, int group_size);
@@ -260,7 +268,10 @@ w4a8_status w4a8_unpack_codes(const void *packed, int N, int K, int group_size,
                               uint8_t *codes, float *scales, uint8_t *zeros, void *stream);
 
 /* Synchronizes `stream`, then reads and clears the status block of `workspace`:
- * W4A8_OK, W4A8_ERR_TIMEOUT or W4A8_ERR_BAD_BLOB (first failure since the last poll). */
+ * W4A8_OK, W4A8_ERR_TIMEOUT or W4A8_ERR_BAD_BLOB (first failure since the last poll).
+ * A kernel that gave up (W4A8_ERR_TIMEOUT) may leave split-K tile counters behind in the
+ * workspace: run w4a8_workspace_init on it before the next call, else a later split-K call can
+ * reduce partial tiles too early.  The output of a call that reported a failure is undefined. */
 w4a8_status w4a8_poll_status(void *workspace, void *stream);
 
 /* Host: Eq. 6 in units of step/2 for zero-point z: out[code] = 2 (code - z) for

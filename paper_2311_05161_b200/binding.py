@@ -42,7 +42,7 @@ class W4A8Error(RuntimeError):
 class Opts(ctypes.Structure):
     _fields_ = [("path", ctypes.c_int), ("split_k", ctypes.c_int), ("tok_tile", ctypes.c_int),
                 ("decode_warps", ctypes.c_int), ("level_shift", ctypes.c_int),
-                ("cluster", ctypes.c_int), ("reserved", ctypes.c_int * 2)]
+                ("cluster", ctypes.c_int), ("debug_wait_ms", ctypes.c_int), ("debug_skip_load", ctypes.c_int)]
 
 
 def _load() -> ctypes.CDLL:
@@ -123,11 +123,13 @@ def _dev(t, dtype, what):
 
 
 def make_opts(path: int = PATH_AUTO, split_k: int = 0, tok_tile: int = 0,
-              decode_warps: int = 0, level_shift: int = 0, cluster: int = 0) -> Opts:
+              decode_warps: int = 0, level_shift: int = 0, cluster: int = 0,
+              debug_wait_ms: int = 0, debug_skip_load: int = 0) -> Opts:
     o = Opts()
     o.path, o.split_k, o.tok_tile, o.decode_warps = path, split_k, tok_tile, decode_warps
     o.level_shift = level_shift
     o.cluster = cluster
+    o.debug_wait_ms, o.debug_skip_load = debug_wait_ms, debug_skip_load
     return o
 
 
@@ -312,12 +314,12 @@ def linear_static(Xq, tok_scale, packed, bias, N: int, group: int, out):
     return out
 
 
-def linear_acc_i32(Xq, packed, N: int, group: int, workspace, opts: Opts | None = None):
+def linear_acc_i32(Xq, packed, N: int, group: int, workspace, opts: Opts | None = None, out=None):
     """INT32 accumulators [G, M, N] of the contraction (test export)."""
     Xq = _dev(Xq, torch.int8, "Xq")
     M, K = Xq.shape
     G = K // group if group else 1
-    acc = torch.empty((G, M, N), dtype=torch.int32, device=Xq.device)
+    acc = out if out is not None else torch.empty((G, M, N), dtype=torch.int32, device=Xq.device)
     _check(lib.w4a8_linear_acc_i32(_ptr(Xq), _ptr(packed), M, N, K, group, _ptr(acc),
                                    _ptr(workspace), workspace.numel(), _stream(),
                                    ctypes.byref(opts) if opts is not None else None),

@@ -38,8 +38,12 @@ bool opts_ok(const w4a8_opts *o)
     if (o->split_k < 0 || o->tok_tile < 0 || o->decode_warps < 0) return false;
     if (o->level_shift < 0 || o->level_shift > 3) return false;
     if (o->cluster < 0 || o->cluster > 2) return false;
-    for (int i = 0; i < 2; ++i)
-        if (o->reserved[i] != 0) return false;
+#ifdef W4A8_DEBUG_HOOKS
+    if (o->debug_wait_ms < 0 || o->debug_wait_ms > 2000 || o->debug_skip_load < 0) return false;
+    if ((o->debug_wait_ms || o->debug_skip_load) && o->path != W4A8_PATH_TCGEN05) return false;
+#else
+    if (o->debug_wait_ms != 0 || o->debug_skip_load != 0) return false;
+#endif
     return true;
 }
 

@@ -121,6 +121,9 @@ struct Params {
     ZeroPoint zp;
     LevelTables lt;
     float unit;          // level unit as a factor of the step: 2^-shift
+    unsigned long long wait_ns, drain_ns;   // limits of the bounded waits
+    int skip_load;       // test hook: every producer leaves out the token load of its k-block
+                         // number skip_load - 1 (0 = none), so that a wait runs out
 };
 
 // --------------------------------------------------------------------------- PTX wrappers
@@ -359,11 +362,13 @@ struct Ctl {
     volatile int abort;
     int is_last;
     uint32_t tmem_base;
+    unsigned long long wait_ns, drain_ns;      // limits of an ordinary wait and of a drain wait
 };
 
+// `draining`: the CTA has given up and only waits for what it has in flight (copies, MMAs):
+// such a wait does not end because of the abort flag, and it has the shorter limit.
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Ctl *ctl,
-                                             StatusBlock *sb, int where,
-                                             unsigned long long limit = kWaitLimitNs)
+                                             StatusBlock *sb, int where, bool draining = false)
 {
     if (mbar_try_wait(bar, parity)) return true;
     // the timer is slow to read: it is only consulted after many failed polls
@@ -371,10 +376,10 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Ctl 
     for (uint32_t i = 1;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 63u) == 0u) {
-            if (ctl->abort) return false;
+            if (ctl->abort && !draining) return false;
             if (t0 == 0) {
                 t0 = global_ns();
-            } else if (global_ns() - t0 > limit) {
+            } else if (global_ns() - t0 > (draining ? ctl->drain_ns : ctl->wait_ns)) {
                 ctl->abort = 1;
                 report_failure(sb, W4A8_ERR_TIMEOUT, where);
                 return false;
@@ -398,7 +403,7 @@ __device__ __forceinline__ bool wait_bounded_idle(uint32_t bar, uint32_t parity,
             if (ctl->abort) return false;
             if (t0 == 0) {
                 t0 = global_ns();
-            } else if (global_ns() - t0 > kWaitLimitNs) {
+            } else if (global_ns() - t0 > ctl->wait_ns) {
                 ctl->abort = 1;
                 report_failure(sb, W4A8_ERR_TIMEOUT, where);
                 return false;
@@ -527,6 +532,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         mbar_init(bar_drain, 1);
         ctl->abort = 0;
         ctl->is_last = 0;
+        ctl->wait_ns = P.wait_ns;
+        ctl->drain_ns = P.drain_ns;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
@@ -572,6 +579,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         ok = false;
                         break;
                     }
+                    if (P.skip_load != 0 && it == (uint32_t)(P.skip_load - 1)) continue;
                     const uint32_t stage = base + st * C::kStageBytes;
                     const uint32_t tok_bar = bar_dec + 8 * st;
                     mbar_arrive_expect_tx(tok_bar, C::kTokBytes + (CL > 1 ? kABytes / CL : 0));
@@ -591,8 +599,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 // copies already issued must land before the CTA gives its memory back
                 const uint32_t first = it > (uint32_t)S ? it - S : 0u;
                 for (uint32_t j = first; j < it; ++j)
-                    wait_bounded(bar_dec + 8 * (j % S), (j / S) & 1u, ctl,
-                                 P.sb, 11, kDrainLimitNs);
+                    wait_bounded(bar_dec + 8 * (j % S), (j / S) & 1u, ctl, P.sb, 11, true);
             }
         }
         __syncwarp();
@@ -647,7 +654,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             }
             // nothing issued may still be running when tensor memory is freed
             tc_commit(bar_drain);
-            wait_bounded(bar_drain, 0u, ctl, P.sb, 22, ok ? kWaitLimitNs : kDrainLimitNs);
+            wait_bounded(bar_drain, 0u, ctl, P.sb, 22, !ok);
         }
         __syncwarp();
     } else if (role == kDecode) {
@@ -1213,6 +1220,8 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     if (dw != 4 && dw != 8 && !((dw == 12 || dw == 16) && !grouped)) return false;
     plan->decode_warps = dw;
     plan->cluster = cluster;
+    plan->debug_wait_ms = opts ? opts->debug_wait_ms : 0;
+    plan->debug_skip_load = opts ? opts->debug_skip_load : 0;
     plan->tok_tile = tok;
     plan->tok_tiles = tok_tiles;
     plan->split_k = split;
@@ -1279,6 +1288,9 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     P.zp = zp;
     P.lt = make_level_tables(L.shift);
     P.unit = level_unit(L.shift);
+    P.wait_ns = plan.debug_wait_ms > 0 ? (unsigned long long)plan.debug_wait_ms * 1000000ull : kWaitLimitNs;
+    P.drain_ns = plan.debug_wait_ms > 0 ? P.wait_ns : kDrainLimitNs;
+    P.skip_load = plan.debug_skip_load;
 
     const bool g = L.group != 0;
     switch (plan.tok_tile) {

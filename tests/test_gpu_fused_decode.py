@@ -9,7 +9,7 @@ import torch
 import oracle
 import paper_2311_05161_b200 as w4a8
 from paper_2311_05161_b200 import binding
-from util import Problem, bf16_bits, check_y
+from util import Guarded, Problem, bf16_bits, check_y, guarded_workspace
 
 pytestmark = pytest.mark.gpu
 
@@ -18,11 +18,16 @@ def run_fused(prob, packed, X=None, inv_s=None):
     d = prob.dev
     X = d["X"] if X is None else X
     inv_s = d["inv_s"] if inv_s is None else inv_s
-    ws = binding.new_quantize_linear_workspace(prob.M, prob.N, prob.K, prob.group)
+    # workspace (the quantizer may use its tail) and output between patterned margins
+    gws = guarded_workspace(binding.quantize_linear_workspace_bytes(prob.M, prob.N, prob.K, prob.group))
+    gY = Guarded((prob.M, prob.N), torch.bfloat16)
+    ws = gws.t
     out = []
     for _ in range(2):                       # the second call reuses the self-cleaned workspace
-        Y = binding.quantize_linear(X, inv_s, packed, d["bias"], prob.N, prob.group, ws)
+        Y = binding.quantize_linear(X, inv_s, packed, d["bias"], prob.N, prob.group, ws, out=gY.t)
         w4a8.check_status(ws)
+        gws.check("workspace")
+        gY.check("Y")
         out.append(bf16_bits(Y))
     assert np.array_equal(out[0], out[1])
     return out[0]

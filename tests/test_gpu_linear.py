@@ -7,7 +7,7 @@ import torch
 
 import oracle
 import paper_2311_05161_b200 as w4a8
-from util import Problem, bf16_bits, check_y
+from util import Guarded, Problem, bf16_bits, check_y, guarded_workspace
 
 pytestmark = pytest.mark.gpu
 
@@ -16,11 +16,17 @@ def run_linear(prob, opts=None, packed=None, want_acc=True):
     d = prob.dev
     if packed is None:
         packed = w4a8.pack_weights(d["W"], d["s"], prob.group)
-    Xq, tok = w4a8.quantize_act(d["X"], d["inv_s"])
-    ws = w4a8.new_workspace(prob.M, prob.N, prob.K, prob.group, opts)
-    Y = w4a8.linear(Xq, tok, packed, d["bias"], prob.N, prob.group, ws, opts)
-    acc = w4a8.linear_acc_i32(Xq, packed, prob.N, prob.group, ws, opts) if want_acc else None
-    w4a8.check_status(ws)
+    # every output and the workspace sit between patterned margins that must stay untouched
+    G = prob.K // prob.group if prob.group else 1
+    gXq, gtok = Guarded((prob.M, prob.K), torch.int8), Guarded((prob.M,), torch.float32)
+    gY, gacc = Guarded((prob.M, prob.N), torch.bfloat16), Guarded((G, prob.M, prob.N), torch.int32)
+    gws = guarded_workspace(w4a8.linear_workspace_bytes(prob.M, prob.N, prob.K, prob.group, opts))
+    Xq, tok = w4a8.quantize_act(d["X"], d["inv_s"], out=(gXq.t, gtok.t))
+    Y = w4a8.linear(Xq, tok, packed, d["bias"], prob.N, prob.group, gws.t, opts, out=gY.t)
+    acc = w4a8.linear_acc_i32(Xq, packed, prob.N, prob.group, gws.t, opts, out=gacc.t) if want_acc else None
+    w4a8.check_status(gws.t)
+    for g, what in ((gXq, "Xq"), (gtok, "tok_scale"), (gY, "Y"), (gacc, "acc"), (gws, "workspace")):
+        g.check(what)
     return bf16_bits(Y), (acc.cpu().numpy() if want_acc else None)
 
 

@@ -41,11 +41,34 @@ def test_static_scratch_entry_point_matches_linear_twice(group):
     check_y(prob, want_bits, exact=(group == 0))
     for call in range(2):
         out = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        torch.cuda.synchronize()
+        free_before, held_before = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
         w4a8.linear_static(Xq, tok, packed, d["bias"], N, group, out)
         torch.cuda.synchronize()
+        if call == 1:       # (the first call on a device may load the kernel's code)
+            assert torch.cuda.mem_get_info()[0] == free_before, "the call took device memory"
+        assert torch.cuda.memory_allocated() == held_before
         got = bf16_bits(out)
         assert np.array_equal(got, want_bits), f"call {call}: differs from w4a8_linear"
         check_y(prob, got, exact=(group == 0))
+
+
+def test_static_scratch_entry_point_with_two_tokens():
+    # two tokens: w4a8_linear picks the weight-streaming kernel here, the workspace-free call
+    # the tensor-core kernel; per-channel results have the same bits either way
+    prob = Problem(1024, 384, 2, 0, seed=321)
+    d = prob.dev
+    packed = w4a8.pack_weights(d["W"], d["s"], 0)
+    Xq, tok = w4a8.quantize_act(d["X"], d["inv_s"])
+    ws = w4a8.new_workspace(2, 384, 1024, 0)
+    want_bits = bf16_bits(w4a8.linear(Xq, tok, packed, d["bias"], 384, 0, ws))
+    w4a8.check_status(ws)
+    for call in range(2):
+        out = torch.full((2, 384), float("nan"), dtype=torch.bfloat16, device="cuda")
+        w4a8.linear_static(Xq, tok, packed, d["bias"], 384, 0, out)
+        torch.cuda.synchronize()
+        assert np.array_equal(bf16_bits(out), want_bits), f"call {call}"
+        check_y(prob, bf16_bits(out), exact=True)
 
 
 def test_static_scratch_rejects_plans_beyond_its_size():

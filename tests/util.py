@@ -73,3 +73,29 @@ def check_y(prob, Y, exact):
     # and never more than one BF16 step from the binary32-order oracle value
     ref = oracle.bf16_bits_to_float(want).astype(np.float64)
     assert np.all(np.abs(got - ref) <= 2 * bf16_ulp(y64) + tol)
+
+
+class Guarded:
+    """A device tensor in the middle of a larger allocation whose margins hold a byte pattern:
+    a kernel that writes outside the tensor it was given changes a margin."""
+    MARGIN = 8192
+    PATTERN = 0xA5
+
+    def __init__(self, shape, dtype):
+        shape = tuple(int(x) for x in shape)
+        self.nbytes = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        body = (self.nbytes + 255) // 256 * 256
+        self.raw = torch.full((2 * self.MARGIN + body,), self.PATTERN, dtype=torch.uint8, device="cuda")
+        self.t = self.raw[self.MARGIN:self.MARGIN + self.nbytes].view(dtype).view(shape)
+
+    def check(self, what=""):
+        lo = self.raw[:self.MARGIN]
+        hi = self.raw[self.MARGIN + self.nbytes:]
+        assert bool((lo == self.PATTERN).all()), f"{what}: bytes before the buffer were written"
+        assert bool((hi == self.PATTERN).all()), f"{what}: bytes behind the buffer were written"
+
+
+def guarded_workspace(nbytes):
+    g = Guarded((nbytes,), torch.uint8)
+    w4a8.workspace_init(g.t)
+    return g
