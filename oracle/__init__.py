@@ -159,6 +159,29 @@ def quantize_act(X: np.ndarray, inv_s_in: np.ndarray | None = None):
     return Xq, tok
 
 
+def norm_quantize_act(X: np.ndarray, weight: np.ndarray, bias: np.ndarray | None = None,
+                      kind: str = "rms", eps: float = 1e-5):
+    """Token-wise INT8 quantizer behind an RMSNorm ("rms") or LayerNorm ("layer") whose weight
+    and bias carry the reciprocal Eq. 1 scale (Fig. 1(a), Section 3.1).  X is [M, K] float16.
+
+    Returns (Xq [M, K] int8, tok_scale [M] float32).
+    """
+    X = _c(X, np.float16)
+    M, K = X.shape
+    weight = _c(weight, np.float32)
+    assert weight.shape == (K,)
+    if bias is not None:
+        bias = _c(bias, np.float32)
+        assert bias.shape == (K,)
+    Xq = np.empty((M, K), dtype=np.int8)
+    tok = np.empty((M,), dtype=np.float32)
+    lib().oracle_norm_quantize_act(_p(X.view(np.uint16)), _p(weight),
+                                   _p(bias) if bias is not None else None,
+                                   ctypes.c_int({"rms": 0, "layer": 1}[kind]), ctypes.c_float(eps),
+                                   ctypes.c_int(M), ctypes.c_int(K), _p(Xq), _p(tok))
+    return Xq, tok
+
+
 def _shape(Xq, codes, zeros, group):
     M, K = Xq.shape
     N = codes.shape[0]

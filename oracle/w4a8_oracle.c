@@ -552,6 +552,70 @@ void oracle_linear_fmt(const int8_t *Xq, const float *tok_scale, const uint8_t *
 /* threading of the outermost loops (sums are integer, so order-free)         */
 /* ------------------------------------------------------------------------- */
 
+/* ---------------------------------------------------------------------------
+ * Activation side of Eq. 1 with the scale diag(s)^-1 merged into the
+ * normalisation in front of the matmul (Fig. 1(a), Section 3.1): the layer's
+ * input is norm(X), the normalisation's weight (and bias) already carry 1/s,
+ * and the token-wise INT8 quantizer (Appendix A.1) follows at once.
+ *
+ * kind 0, RMSNorm:    ms = (sum_k x_k^2) / K,  r = 1 / sqrt(ms + eps),
+ *                     x'_k = (x_k * r) * w_k
+ * kind 1, LayerNorm:  mu = (sum_k x_k) / K,  var = (sum_k (x_k - mu)^2) / K,
+ *                     r = 1 / sqrt(var + eps),  x'_k = ((x_k - mu) * r) * w_k + b_k
+ *
+ * Precision (the paper gives none; this is the reading): the statistics (the
+ * sums, mu, ms, var, r) are binary64, summed in ascending k; r and x_k - mu
+ * are then rounded once to binary32 and everything per element is binary32,
+ * one rounded operation per written operation.  Then the symmetric absmax
+ * quantizer exactly as in oracle_quantize_act.
+ * ------------------------------------------------------------------------- */
+void oracle_norm_quantize_act(const uint16_t *X, const float *w, const float *b, int kind,
+                              float eps, int M, int K, int8_t *Xq, float *tok_scale)
+{
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        const uint16_t *row = X + (size_t)m * K;
+        double mu = 0.0;
+        if (kind == 1) {
+            double sum = 0.0;
+            for (int k = 0; k < K; ++k) sum += (double)half_bits_to_float(row[k]);
+            mu = sum / (double)K;
+        }
+        double ss = 0.0;
+        for (int k = 0; k < K; ++k) {
+            const double d = (double)half_bits_to_float(row[k]) - mu;
+            ss += d * d;
+        }
+        const float r = (float)(1.0 / sqrt(ss / (double)K + (double)eps));
+        float amax = 0.0f;
+        for (int pass = 0; pass < 2; ++pass) {
+            float q_r = 0.0f;
+            if (pass == 1) {
+                if (amax == 0.0f) {
+                    tok_scale[m] = 0.0f;
+                    for (int k = 0; k < K; ++k) Xq[(size_t)m * K + k] = 0;
+                    break;
+                }
+                q_r = 127.0f / amax;
+                tok_scale[m] = amax / 127.0f;
+            }
+            for (int k = 0; k < K; ++k) {
+                const float d = (float)((double)half_bits_to_float(row[k]) - mu);
+                float x = d * r;
+                x = x * w[k];
+                if (b) x = x + b[k];
+                if (pass == 0) {
+                    const float a = fabsf(x);
+                    if (a > amax) amax = a;
+                } else {
+                    Xq[(size_t)m * K + k] = (int8_t)clampi(rint_to_int(x * q_r), -127, 127);
+                }
+            }
+        }
+    }
+}
+
+
 void oracle_set_threads(int n)
 {
 #ifdef _OPENMP
