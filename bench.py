@@ -740,6 +740,27 @@ def main():
                             "frac_of_measured_copy": big1["frac_of_measured_copy"],
                             "frac_of_nominal_8000": big1["frac_of_nominal_8000"],
                             "note": "2 rotating blob copies (> L2), CUDA graph replay"}}
+        # the activation quantizer with the normalisation in front of it fused in (the Eq. 1 scale
+        # lives in the normalisation's weight): one pass over X instead of norm + quantizer
+        nq = {}
+        for name, K in (("hidden_4096", 4096), ("hidden_16384", 16384)):
+            d = next(x for x in L2 if x["K"] == K)
+            gamma = (1.0 / d["s"]).contiguous()
+            beta = torch.zeros_like(gamma)
+            for kind, code, bias_t in (("rms", w4a8.NORM_RMS, None), ("layer", w4a8.NORM_LAYER, beta)):
+                fn = lambda it, d=d, code=code, bias_t=bias_t: w4a8.norm_quantize_act(
+                    d["X"], gamma, bias_t, code, 1e-5, out=(d["Xq"], d["tok"]))
+                ms_n = graph_ms(fn, 20)
+                gbs = (3.0 * M_PREFILL * K + 4 * M_PREFILL) / (ms_n * 1e-3) / 1e9
+                nq[f"{name}_{kind}"] = {"ms": ms_n, "gbs": gbs, "frac_of_measured_copy": gbs / peaks["hbm_gbs"]}
+            ms_p = graph_ms(lambda it, d=d: w4a8.quantize_act(d["X"], d["inv_s"], out=(d["Xq"], d["tok"])), 20)
+            gbs = (3.0 * M_PREFILL * K + 4 * M_PREFILL) / (ms_p * 1e-3) / 1e9
+            nq[f"{name}_plain_quantizer"] = {"ms": ms_p, "gbs": gbs, "frac_of_measured_copy": gbs / peaks["hbm_gbs"]}
+        legs["norm_fused_act_quant"] = {
+            "metric": "hbm_gbs", "unit": "GB/s", "tokens": M_PREFILL, **nq,
+            "note": "w4a8_norm_quantize_act (RMSNorm; LayerNorm with bias) against w4a8_quantize_act, "
+                    "3 bytes per element, CUDA graph replay of 20 launches on the same tensor (L2-warm "
+                    "for 4096, larger than L2 with its output for 16384)"}
         for d in L2:
             d.clear()
         del L2, layers2

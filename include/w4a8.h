@@ -121,6 +121,24 @@ w4a8_status w4a8_pack_weights_fmt(const void *W_f16, const float *s_in, int N, i
 w4a8_status w4a8_quantize_act(const void *X_f16, const float *inv_s_in, int M, int K,
                               int8_t *Xq, float *tok_scale, void *stream);
 
+/* The activation side of Eq. 1 where it lives in a decoder layer: inside the normalisation in
+ * front of the matmul (Fig. 1(a), Section 3.1 - the reciprocal scale diag(s)^-1 is merged into
+ * the normalisation's weight and bias), followed at once by the token-wise INT8 quantizer
+ * (Appendix A.1).  One pass over X: the normalised FP16 tensor is never written.
+ *   X_f16        [M][K] IEEE binary16, the layer input before the normalisation.
+ *   norm_weight  [K] FP32, the normalisation's weight times the reciprocal Eq. 1 scale.
+ *   norm_bias    [K] FP32 likewise, or NULL.
+ *   norm_kind    W4A8_NORM_RMS:   x' = (x / sqrt(mean(x^2) + eps)) * weight (+ bias)
+ *                W4A8_NORM_LAYER: x' = ((x - mean(x)) / sqrt(var(x) + eps)) * weight (+ bias)
+ *   eps          > 0.   K <= 16384 (the hidden sizes a normalisation sees).
+ *   Xq, tok_scale  out, as from w4a8_quantize_act applied to x'.
+ * Precision: the token statistics (sums, mean, variance, reciprocal root) in binary64, rounded
+ * once to binary32; everything per element in binary32, one rounding per operation. */
+typedef enum { W4A8_NORM_RMS = 0, W4A8_NORM_LAYER = 1 } w4a8_norm;
+w4a8_status w4a8_norm_quantize_act(const void *X_f16, const float *norm_weight,
+                                   const float *norm_bias, int norm_kind, float eps, int M, int K,
+                                   int8_t *Xq, float *tok_scale, void *stream);
+
 /* Scratch bytes w4a8_linear needs for this shape (always >= 256: the first 256 bytes
  * hold the status block read by w4a8_poll_status).  The caller zero-fills the workspace
  * once after allocating it (w4a8_workspace_init); calls that end without a reported failure

@@ -558,16 +558,18 @@ void oracle_linear_fmt(const int8_t *Xq, const float *tok_scale, const uint8_t *
  * input is norm(X), the normalisation's weight (and bias) already carry 1/s,
  * and the token-wise INT8 quantizer (Appendix A.1) follows at once.
  *
- * kind 0, RMSNorm:    ms = (sum_k x_k^2) / K,  r = 1 / sqrt(ms + eps),
- *                     x'_k = (x_k * r) * w_k
- * kind 1, LayerNorm:  mu = (sum_k x_k) / K,  var = (sum_k (x_k - mu)^2) / K,
- *                     r = 1 / sqrt(var + eps),  x'_k = ((x_k - mu) * r) * w_k + b_k
+ * kind 0, RMSNorm:    d_k = x_k,        ms = (sum_k d_k^2) / K
+ * kind 1, LayerNorm:  d_k = x_k - mu,   mu = (sum_k x_k) / K,  ms = (sum_k d_k^2) / K
+ * both:               r = 1 / sqrt(ms + eps),  x'_k = (d_k * r) * w_k (+ b_k)
  *
- * Precision (the paper gives none; this is the reading): the statistics (the
- * sums, mu, ms, var, r) are binary64, summed in ascending k; r and x_k - mu
- * are then rounded once to binary32 and everything per element is binary32,
- * one rounded operation per written operation.  Then the symmetric absmax
- * quantizer exactly as in oracle_quantize_act.
+ * Precision (the paper gives none; this is the reading): a sum over the K
+ * features is taken in binary32 inside each run of 8 consecutive features
+ * (ascending k; the squares enter by fmaf, and a binary16 value squared is
+ * exact in binary32), and the K / 8 partial sums are added in binary64
+ * (ascending); mu, ms and r are binary64, mu and r are rounded once to
+ * binary32, and everything per element (x - mu, the products, the bias) is
+ * binary32, one rounded operation per written operation.  Then the symmetric
+ * absmax quantizer exactly as in oracle_quantize_act.  K % 8 == 0.
  * ------------------------------------------------------------------------- */
 void oracle_norm_quantize_act(const uint16_t *X, const float *w, const float *b, int kind,
                               float eps, int M, int K, int8_t *Xq, float *tok_scale)
@@ -575,16 +577,25 @@ void oracle_norm_quantize_act(const uint16_t *X, const float *w, const float *b,
 #pragma omp parallel for schedule(static)
     for (int m = 0; m < M; ++m) {
         const uint16_t *row = X + (size_t)m * K;
-        double mu = 0.0;
+        float mu32 = 0.0f;
         if (kind == 1) {
             double sum = 0.0;
-            for (int k = 0; k < K; ++k) sum += (double)half_bits_to_float(row[k]);
-            mu = sum / (double)K;
+            for (int g = 0; g < K; g += 8) {
+                float part = 0.0f;
+                for (int k = g; k < g + 8; ++k) part = part + half_bits_to_float(row[k]);
+                sum += (double)part;
+            }
+            mu32 = (float)(sum / (double)K);
         }
         double ss = 0.0;
-        for (int k = 0; k < K; ++k) {
-            const double d = (double)half_bits_to_float(row[k]) - mu;
-            ss += d * d;
+        for (int g = 0; g < K; g += 8) {
+            float part = 0.0f;
+            for (int k = g; k < g + 8; ++k) {
+                const float d = kind == 1 ? half_bits_to_float(row[k]) - mu32
+                                          : half_bits_to_float(row[k]);
+                part = fmaf(d, d, part);
+            }
+            ss += (double)part;
         }
         const float r = (float)(1.0 / sqrt(ss / (double)K + (double)eps));
         float amax = 0.0f;
@@ -600,8 +611,9 @@ void oracle_norm_quantize_act(const uint16_t *X, const float *w, const float *b,
                 tok_scale[m] = amax / 127.0f;
             }
             for (int k = 0; k < K; ++k) {
-                const float d = (float)((double)half_bits_to_float(row[k]) - mu);
-                float x = d * r;
+                float x = half_bits_to_float(row[k]);
+                if (kind == 1) x = x - mu32;
+                x = x * r;
                 x = x * w[k];
                 if (b) x = x + b[k];
                 if (pass == 0) {
@@ -614,7 +626,6 @@ void oracle_norm_quantize_act(const uint16_t *X, const float *w, const float *b,
         }
     }
 }
-
 
 void oracle_set_threads(int n)
 {

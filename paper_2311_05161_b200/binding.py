@@ -29,7 +29,7 @@ EXPORTS = (
     "w4a8_poll_status", "w4a8_dint4_table", "w4a8_version",
     "w4a8_quantize_act_asym", "w4a8_weight_rowsum", "w4a8_linear_asym",
     "w4a8_pack_weights_fmt", "w4a8_dint4_table_fmt",
-    "w4a8_quantize_linear", "w4a8_quantize_linear_workspace_bytes", "w4a8_linear_plan",
+    "w4a8_quantize_linear", "w4a8_quantize_linear_workspace_bytes", "w4a8_linear_plan", "w4a8_norm_quantize_act",
 )
 
 
@@ -59,6 +59,8 @@ def _load() -> ctypes.CDLL:
     lib.w4a8_pack_weights.argtypes = [vp, vp, ci, ci, ci, cf, vp, sz, vp]
     lib.w4a8_quantize_act.restype = ci
     lib.w4a8_quantize_act.argtypes = [vp, vp, ci, ci, vp, vp, vp]
+    lib.w4a8_norm_quantize_act.restype = ci
+    lib.w4a8_norm_quantize_act.argtypes = [vp, vp, vp, ci, cf, ci, ci, vp, vp, vp]
     lib.w4a8_linear_workspace_bytes.restype = sz
     lib.w4a8_linear_workspace_bytes.argtypes = [ci, ci, ci, ci]
     lib.w4a8_linear_workspace_bytes_ex.restype = sz
@@ -174,6 +176,25 @@ def quantize_act(X, inv_s_in=None, out=None):
     Xq, tok = out
     _check(lib.w4a8_quantize_act(_ptr(X), _ptr(inv_s_in), M, K, _ptr(Xq), _ptr(tok), _stream()),
            "w4a8_quantize_act")
+    return Xq, tok
+
+
+NORM_RMS, NORM_LAYER = 0, 1
+
+
+def norm_quantize_act(X, norm_weight, norm_bias=None, kind: int = NORM_RMS, eps: float = 1e-5, out=None):
+    """RMSNorm / LayerNorm (weight and bias carry the reciprocal Eq. 1 scale) and the token-wise
+    INT8 quantizer in one pass: X [M, K] float16 (CUDA) -> (Xq [M, K] int8, tok_scale [M] float32)."""
+    X = _dev(X, torch.float16, "X")
+    norm_weight = _dev(norm_weight, torch.float32, "norm_weight")
+    norm_bias = _dev(norm_bias, torch.float32, "norm_bias")
+    M, K = X.shape
+    if out is None:
+        out = (torch.empty((M, K), dtype=torch.int8, device=X.device),
+               torch.empty((M,), dtype=torch.float32, device=X.device))
+    Xq, tok = out
+    _check(lib.w4a8_norm_quantize_act(_ptr(X), _ptr(norm_weight), _ptr(norm_bias), kind, eps, M, K,
+                                      _ptr(Xq), _ptr(tok), _stream()), "w4a8_norm_quantize_act")
     return Xq, tok
 
 

@@ -163,6 +163,25 @@ w4a8_status w4a8_quantize_act(const void *X_f16, const float *inv_s_in, int M, i
     return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
 
+w4a8_status w4a8_norm_quantize_act(const void *X_f16, const float *norm_weight,
+                                   const float *norm_bias, int norm_kind, float eps, int M, int K,
+                                   int8_t *Xq, float *tok_scale, void *stream)
+{
+    if (!X_f16 || !norm_weight || !Xq || !tok_scale) return W4A8_ERR_NULL;
+    if (M < 1 || K < 128 || K % 128 != 0 || K > 16384) return W4A8_ERR_SHAPE;
+    if (norm_kind != W4A8_NORM_RMS && norm_kind != W4A8_NORM_LAYER) return W4A8_ERR_SHAPE;
+    if (!(eps > 0.0f)) return W4A8_ERR_SHAPE;
+    if (!aligned(X_f16, 16) || !aligned(norm_weight, 16) || !aligned(norm_bias, 16) ||
+        !aligned(Xq, 16) || !aligned(tok_scale, 4))
+        return W4A8_ERR_ALIGN;
+    const w4a8_status arch = check_arch();
+    if (arch != W4A8_OK) return arch;
+    const cudaError_t e = launch_norm_quantize_act(
+        static_cast<const __half *>(X_f16), norm_weight, norm_bias, norm_kind == W4A8_NORM_LAYER, eps,
+        M, K, Xq, tok_scale, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
 size_t w4a8_linear_workspace_bytes_ex(int M, int N, int K, int group_size, const w4a8_opts *opts)
 {
     if (!shape_ok(N, K, group_size) || M < 1 || !opts_ok(opts)) return 0;

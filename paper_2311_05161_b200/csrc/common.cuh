@@ -246,6 +246,9 @@ cudaError_t launch_quantize_act(const __half *X, const float *inv_s, int M, int 
                                 float *tok_scale, cudaStream_t st);
 cudaError_t launch_quantize_act_asym(const __half *X, const float *inv_s, int M, int K, int8_t *Xq,
                                      float *tok_scale, int32_t *tok_zero, cudaStream_t st);
+cudaError_t launch_norm_quantize_act(const __half *X, const float *weight, const float *bias,
+                                     int layer_norm, float eps, int M, int K, int8_t *Xq,
+                                     float *tok_scale, cudaStream_t st);
 cudaError_t launch_weight_rowsum(const uint8_t *blob, const BlobLayout &L, int32_t *rowsum,
                                  cudaStream_t st);
 cudaError_t launch_linear_simple(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,

@@ -84,7 +84,9 @@ def test_layer_norm_ignores_a_common_offset_and_rms_norm_does_not():
     w = np.ones(K, dtype=np.float32)
     a = oracle.norm_quantize_act(X0, w, None, "layer", 1e-5)
     b = oracle.norm_quantize_act(X1, w, None, "layer", 1e-5)
-    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    # (the mean is rounded to binary32 once, so the invariance holds to rounding, not to the bit)
+    assert np.abs(a[0].astype(int) - b[0].astype(int)).max() <= 1
+    assert np.mean(a[0] != b[0]) < 0.01 and np.allclose(a[1], b[1], rtol=1e-5)
     c = oracle.norm_quantize_act(X1, w, None, "rms", 1e-5)
     assert not np.array_equal(a[0], c[0])
 
