@@ -356,6 +356,44 @@ def linear_fmt(Xq, tok_scale, codes, scales, zeros, bias, group: int, shift: int
     return acc, Y, wide
 
 
+def pack_weights_bits(W, s_in, group: int, bits: int, shift: int = 1, clip: float = 1.0):
+    """pack_weights for the b-bit format (b = 3: integer codes 0..5, code 6 = +c, code 7 = -c),
+    special value step / 2^shift.  Codes come two per byte whatever the width."""
+    W = _c(W, np.float16)
+    N, K = W.shape
+    if s_in is not None:
+        s_in = _c(s_in, np.float32)
+    G = K // group if group else 1
+    codes = np.empty((N, K // 2), dtype=np.uint8)
+    scales = np.empty((G, N), dtype=np.float32)
+    zeros = np.empty((G, N), dtype=np.uint8)
+    lib().oracle_pack_weights_bits(_p(W.view(np.uint16)), _p(s_in) if s_in is not None else None,
+                                   ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group),
+                                   ctypes.c_float(clip), ctypes.c_int(bits), ctypes.c_int(shift),
+                                   _p(codes), _p(scales), _p(zeros))
+    return codes, scales, zeros
+
+
+def linear_bits(Xq, tok_scale, codes, scales, zeros, bias, group: int, bits: int, shift: int = 1):
+    """(acc int64 [G, M, N], Y bf16 bits [M, N], Y binary64 [M, N]) for b-bit codes."""
+    Xq = _c(Xq, np.int8)
+    tok_scale = _c(tok_scale, np.float32)
+    codes = _c(codes, np.uint8)
+    zeros = _c(zeros, np.uint8)
+    scales = _c(scales, np.float32)
+    M, N, K, G = _shape(Xq, codes, zeros, group)
+    if bias is not None:
+        bias = _c(bias, np.float32)
+    acc = np.empty((G, M, N), dtype=np.int64)
+    Y = np.empty((M, N), dtype=np.uint16)
+    wide = np.empty((M, N), dtype=np.float64)
+    lib().oracle_linear_bits(_p(Xq), _p(tok_scale), _p(codes), _p(scales), _p(zeros),
+                             _p(bias) if bias is not None else None, ctypes.c_int(M),
+                             ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group),
+                             ctypes.c_int(bits), ctypes.c_int(shift), _p(acc), _p(Y), _p(wide))
+    return acc, Y, wide
+
+
 def bf16_bits_to_float(bits: np.ndarray) -> np.ndarray:
     """Widen BF16 bit patterns (uint16) to float32 values (exact)."""
     return (bits.astype(np.uint32) << 16).view(np.float32)

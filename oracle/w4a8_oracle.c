@@ -475,10 +475,14 @@ void oracle_dint_table_fmt(int z, int b, int j, int8_t *t)
     t[p + 2] = -1;
 }
 
-/* oracle_pack_weights with the special value s / 2^j. */
-void oracle_pack_weights_fmt(const uint16_t *W, const float *s_in, int N, int K, int group,
-                             float clip, int j, uint8_t *codes, float *scales, uint8_t *zeros)
+/* oracle_pack_weights for the b-bit format (p = 2^b - 3 uniform steps, Section 4.2; b = 4 in
+ * the paper's main results, b = 3 in Tables 10-11) with the special value s / 2^j.  Codes are
+ * stored two per byte whatever b is (a 3-bit code occupies the low bits of its nibble). */
+void oracle_pack_weights_bits(const uint16_t *W, const float *s_in, int N, int K, int group,
+                              float clip, int b, int j, uint8_t *codes, float *scales,
+                              uint8_t *zeros)
 {
+    const int p = oracle_dint_p(b);
     const int glen = group ? group : K;
     const int G = K / glen;
 #pragma omp parallel for schedule(static)
@@ -493,29 +497,37 @@ void oracle_pack_weights_fmt(const uint16_t *W, const float *s_in, int N, int K,
             }
             lo = lo * clip;
             hi = hi * clip;
-            float s = (hi - lo) / 13.0f;
+            float s = (hi - lo) / (float)p;
             if (s == 0.0f) s = 1.0f;
-            const int z = clampi(rint_to_int((-lo) / s), 0, 13);
+            const int z = clampi(rint_to_int((-lo) / s), 0, p);
             scales[(size_t)g * N + n] = s;
             zeros[(size_t)g * N + n] = (uint8_t)z;
             for (int k = g * glen; k < (g + 1) * glen; k += 2) {
                 float w0 = half_bits_to_float(W[(size_t)n * K + k]);
                 float w1 = half_bits_to_float(W[(size_t)n * K + k + 1]);
                 if (s_in) { w0 = w0 * s_in[k]; w1 = w1 * s_in[k + 1]; }
-                const int c0 = oracle_dint_quantize_fmt(w0, s, z, 4, j);
-                const int c1 = oracle_dint_quantize_fmt(w1, s, z, 4, j);
+                const int c0 = oracle_dint_quantize_fmt(w0, s, z, b, j);
+                const int c1 = oracle_dint_quantize_fmt(w1, s, z, b, j);
                 codes[(size_t)n * (K / 2) + k / 2] = (uint8_t)(c0 | (c1 << 4));
             }
         }
     }
 }
 
+/* oracle_pack_weights with the special value s / 2^j (4-bit format). */
+void oracle_pack_weights_fmt(const uint16_t *W, const float *s_in, int N, int K, int group,
+                             float clip, int j, uint8_t *codes, float *scales, uint8_t *zeros)
+{
+    oracle_pack_weights_bits(W, s_in, N, K, group, clip, 4, j, codes, scales, zeros);
+}
+
 /* The layer with levels in units of s / 2^j: integer sums acc [G][M][N] (may be NULL), BF16
  * output Y (may be NULL) in the evaluation order of oracle_linear with the level unit
  * 2^-j * s in place of 0.5 * s, and the same value in binary64 (may be NULL). */
-void oracle_linear_fmt(const int8_t *Xq, const float *tok_scale, const uint8_t *codes,
-                       const float *scales, const uint8_t *zeros, const float *bias, int M,
-                       int N, int K, int group, int j, int64_t *acc, uint16_t *Y, double *wide)
+void oracle_linear_bits(const int8_t *Xq, const float *tok_scale, const uint8_t *codes,
+                        const float *scales, const uint8_t *zeros, const float *bias, int M,
+                        int N, int K, int group, int b, int j, int64_t *acc, uint16_t *Y,
+                        double *wide)
 {
     const int glen = group ? group : K;
     const int G = K / glen;
@@ -526,7 +538,7 @@ void oracle_linear_fmt(const int8_t *Xq, const float *tok_scale, const uint8_t *
             double w = 0.0;
             for (int g = 0; g < G; ++g) {
                 int8_t lv[16];
-                oracle_dint_table_fmt(zeros[(size_t)g * N + n], 4, j, lv);
+                oracle_dint_table_fmt(zeros[(size_t)g * N + n], b, j, lv);
                 int64_t sum = 0;
                 for (int k = g * glen; k < (g + 1) * glen; ++k) {
                     const uint8_t byte = codes[(size_t)n * (K / 2) + k / 2];
@@ -548,9 +560,12 @@ void oracle_linear_fmt(const int8_t *Xq, const float *tok_scale, const uint8_t *
     }
 }
 
-/* ------------------------------------------------------------------------- */
-/* threading of the outermost loops (sums are integer, so order-free)         */
-/* ------------------------------------------------------------------------- */
+void oracle_linear_fmt(const int8_t *Xq, const float *tok_scale, const uint8_t *codes,
+                       const float *scales, const uint8_t *zeros, const float *bias, int M,
+                       int N, int K, int group, int j, int64_t *acc, uint16_t *Y, double *wide)
+{
+    oracle_linear_bits(Xq, tok_scale, codes, scales, zeros, bias, M, N, K, group, 4, j, acc, Y, wide);
+}
 
 /* ---------------------------------------------------------------------------
  * Activation side of Eq. 1 with the scale diag(s)^-1 merged into the
@@ -627,6 +642,9 @@ void oracle_norm_quantize_act(const uint16_t *X, const float *w, const float *b,
     }
 }
 
+/* ------------------------------------------------------------------------- */
+/* threading of the outermost loops (sums are integer, so order-free)         */
+/* ------------------------------------------------------------------------- */
 void oracle_set_threads(int n)
 {
 #ifdef _OPENMP
