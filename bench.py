@@ -698,6 +698,50 @@ def main():
             w4a8.check_status(d["ws"])
             del d["packed_fmt"]
 
+        # 3-bit dINT (p = 5 steps; Tables 10-11): the same block from 0.375-byte-per-weight blobs
+        opts3 = w4a8.make_opts(bits=3)
+        for d, lay in zip(L2, layers2):
+            W = torch.from_numpy(lay["W"]).to(dev)
+            d["packed3"] = [w4a8.pack_weights(W, d["s"], d["group"], bits=3)]
+            d["packed3"] += [d["packed3"][0].clone() for _ in range(2)]
+            d["ws3"] = w4a8.new_workspace(M_PREFILL, d["N"], d["K"], d["group"], opts3)
+            d["ws3_1"] = w4a8.new_workspace(1, d["N"], d["K"], d["group"], opts3)
+            del W
+
+        def pass_dint3(it=None):
+            for d in L2:
+                w4a8.quantize_act(d["X"], d["inv_s"], out=(d["Xq"], d["tok"]))
+                w4a8.linear(d["Xq"], d["tok"], d["packed3"][0], d["bias"], d["N"], d["group"], d["ws3"],
+                            opts3, out=d["Y"])
+        for _ in range(3):
+            pass_dint3()
+        ms_d3 = timed(pass_dint3, 100) / 100
+        Xq1 = {id(d): torch.empty((1, d["K"]), dtype=torch.int8, device=dev) for d in L2}
+        tok1 = torch.empty((1,), dtype=torch.float32, device=dev)
+        Y1 = {id(d): torch.empty((1, d["N"]), dtype=torch.bfloat16, device=dev) for d in L2}
+
+        def step_dint3_decode(it):
+            for d in L2:
+                w4a8.quantize_act(d["X"][:1], d["inv_s"], out=(Xq1[id(d)], tok1))
+                w4a8.linear(Xq1[id(d)], tok1, d["packed3"][it % 3], d["bias"], d["N"], d["group"],
+                            d["ws3_1"], opts3, out=Y1[id(d)])
+        ms_d3_dec = graph_ms(step_dint3_decode, 60)
+        bytes3 = sum(3 * d["K"] * d["N"] // 8 + 5 * d["N"] + d["K"] + 4 + 2 * d["N"] + 4 * d["N"] for d in L2)
+        for d in L2:
+            w4a8.check_status(d["ws3"])
+            w4a8.check_status(d["ws3_1"])
+            for k in ("packed3", "ws3", "ws3_1"):
+                del d[k]
+        legs["dint3"] = {
+            "workload": "opt-6.7b block linears, 3-bit dINT weights (0.375 byte per weight), per-channel",
+            "prefill": {"metric": "w4a8_dint_linear_tops", "M": M_PREFILL,
+                        "value": ops2 / (ms_d3 * 1e-3) / 1e12, "unit": "TOPS", "ms_per_pass": ms_d3},
+            "decode": {"metric": "w4a8_dint_linear_hbm_gbs", "M": 1, "value": bytes3 / (ms_d3_dec * 1e-3) / 1e9,
+                       "unit": "GB/s", "ms_per_step": ms_d3_dec, "bytes_per_step": bytes3,
+                       "frac_of_measured_copy": bytes3 / (ms_d3_dec * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                       "note": "tensor-core kernel with a 16-token tile (the weight-streaming kernels "
+                               "read 4-bit tiles only), 3 rotating blob copies, CUDA graph replay"}}
+
         # decode, M = 1: eight launches of a few microseconds per step, timed from a CUDA graph
         for d in L2:
             d["X1"] = d["X"][:1].contiguous()

@@ -77,6 +77,10 @@ typedef struct {
                             out and the kernel reports W4A8_ERR_TIMEOUT.  Both hooks are refused
                             (W4A8_ERR_SHAPE) unless the library was built with W4A8_DEBUG_HOOKS,
                             and only w4a8_linear_ex with W4A8_PATH_TCGEN05 takes them */
+    int bits;        /* code width of the blob: 0 or 4 (dINT4), or 3 (dINT3, packed by
+                        w4a8_pack_weights_bits); must match the blob.  3-bit blobs run on the
+                        tensor-core kernel (any M) or the simple kernel, with symmetric activations */
+    int reserved;    /* must be zero */
 } w4a8_opts;
 
 /* Bytes of the packed-weight blob for an [N][K] matrix; 0 if the shape is invalid.
@@ -111,6 +115,20 @@ w4a8_status w4a8_pack_weights(const void *W_f16, const float *s_in, int N, int K
 w4a8_status w4a8_pack_weights_fmt(const void *W_f16, const float *s_in, int N, int K,
                                   int group_size, float clip, int level_shift, void *packed,
                                   size_t packed_bytes, void *stream);
+
+/* The same quantizer for the b-bit dINT format of Section 4.2 with b = 3 or 4: p = 2^b - 3
+ * uniform steps, integer codes 0..p, code p + 1 = +c, code p + 2 = -c (b = 3, the format of
+ * Tables 10-11: codes 0..5, 6 = +c, 7 = -c; step = range / 5, zero-point 0..5).  A 3-bit blob
+ * has the layout of the 4-bit one except for its code tiles: 6144 bytes per 128 x 128 tile
+ * (0.375 byte per weight); per 32-k quarter and row three 32-bit words hold 32 codes - nibble j
+ * of word w carries the code of k = 8 w + j in its low three bits, and the spare top bits of
+ * the nibbles j of words 0, 1, 2 are bits 0, 1, 2 of the code of k = 24 + j; word w of row r of
+ * quarter q is at byte q * 1536 + w * 512 + r * 4 of the tile.
+ * Linear calls on a 3-bit blob name bits = 3 (and the level_shift) in their options. */
+size_t w4a8_packed_bytes_bits(int N, int K, int group_size, int bits);
+w4a8_status w4a8_pack_weights_bits(const void *W_f16, const float *s_in, int N, int K,
+                                   int group_size, float clip, int bits, int level_shift,
+                                   void *packed, size_t packed_bytes, void *stream);
 
 /* Activation side of Eq. 1, token-wise INT8 (Appendix A.1), every forward pass.
  *   X_f16     [M][K] IEEE binary16.
@@ -285,6 +303,11 @@ w4a8_status w4a8_linear_acc_i32(const int8_t *Xq, const void *packed, int M, int
 w4a8_status w4a8_unpack_codes(const void *packed, int N, int K, int group_size,
                               uint8_t *codes, float *scales, uint8_t *zeros, void *stream);
 
+/* w4a8_unpack_codes for a blob of `bits`-bit codes (3 or 4); codes come two per byte either way
+ * (a 3-bit code in the low bits of its nibble). */
+w4a8_status w4a8_unpack_codes_bits(const void *packed, int N, int K, int group_size, int bits,
+                                   uint8_t *codes, float *scales, uint8_t *zeros, void *stream);
+
 /* Synchronizes `stream`, then reads and clears the status block of `workspace`:
  * W4A8_OK, W4A8_ERR_TIMEOUT or W4A8_ERR_BAD_BLOB (first failure since the last poll).
  * A kernel that gave up (W4A8_ERR_TIMEOUT) may leave split-K tile counters behind in the
@@ -298,6 +321,10 @@ void w4a8_dint4_table(int z, int8_t *out);
 
 /* Host: the same table in units of step / 2^level_shift: 2^level_shift (code - z), +1, -1. */
 void w4a8_dint4_table_fmt(int z, int level_shift, int8_t *out);
+
+/* Host: the table for `bits`-bit codes (3 or 4): 2^level_shift (code - z) for the integer codes
+ * 0..p, +1 for code p + 1, -1 for code p + 2; entries past 2^bits are zero.  `out` holds 16. */
+void w4a8_dint_table_bits(int z, int bits, int level_shift, int8_t *out);
 
 /* Host: version string with static storage. */
 const char *w4a8_version(void);

@@ -11,5 +11,5 @@ from .binding import (  # noqa: F401
     pack_weights, packed_bytes, poll_status, quantize_act, unpack_codes, version,
     workspace_init, quantize_act_asym, weight_rowsum, linear_asym,
     quantize_linear, quantize_linear_workspace_bytes, new_quantize_linear_workspace, linear_plan,
-    norm_quantize_act, NORM_RMS, NORM_LAYER,
+    norm_quantize_act, NORM_RMS, NORM_LAYER, dint_table,
 )

@@ -30,6 +30,7 @@ EXPORTS = (
     "w4a8_quantize_act_asym", "w4a8_weight_rowsum", "w4a8_linear_asym",
     "w4a8_pack_weights_fmt", "w4a8_dint4_table_fmt",
     "w4a8_quantize_linear", "w4a8_quantize_linear_workspace_bytes", "w4a8_linear_plan", "w4a8_norm_quantize_act",
+    "w4a8_packed_bytes_bits", "w4a8_pack_weights_bits", "w4a8_unpack_codes_bits", "w4a8_dint_table_bits",
 )
 
 
@@ -42,7 +43,8 @@ class W4A8Error(RuntimeError):
 class Opts(ctypes.Structure):
     _fields_ = [("path", ctypes.c_int), ("split_k", ctypes.c_int), ("tok_tile", ctypes.c_int),
                 ("decode_warps", ctypes.c_int), ("level_shift", ctypes.c_int),
-                ("cluster", ctypes.c_int), ("debug_wait_ms", ctypes.c_int), ("debug_skip_load", ctypes.c_int)]
+                ("cluster", ctypes.c_int), ("debug_wait_ms", ctypes.c_int), ("debug_skip_load", ctypes.c_int),
+                ("bits", ctypes.c_int), ("reserved", ctypes.c_int)]
 
 
 def _load() -> ctypes.CDLL:
@@ -79,6 +81,14 @@ def _load() -> ctypes.CDLL:
     lib.w4a8_quantize_linear_workspace_bytes.argtypes = [ci, ci, ci, ci]
     lib.w4a8_quantize_linear.restype = ci
     lib.w4a8_quantize_linear.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, vp]
+    lib.w4a8_packed_bytes_bits.restype = sz
+    lib.w4a8_packed_bytes_bits.argtypes = [ci, ci, ci, ci]
+    lib.w4a8_pack_weights_bits.restype = ci
+    lib.w4a8_pack_weights_bits.argtypes = [vp, vp, ci, ci, ci, cf, ci, ci, vp, sz, vp]
+    lib.w4a8_unpack_codes_bits.restype = ci
+    lib.w4a8_unpack_codes_bits.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp]
+    lib.w4a8_dint_table_bits.restype = None
+    lib.w4a8_dint_table_bits.argtypes = [ci, ci, ci, vp]
     lib.w4a8_pack_weights_fmt.restype = ci
     lib.w4a8_pack_weights_fmt.argtypes = [vp, vp, ci, ci, ci, cf, ci, vp, sz, vp]
     lib.w4a8_quantize_act_asym.restype = ci
@@ -126,12 +136,13 @@ def _dev(t, dtype, what):
 
 def make_opts(path: int = PATH_AUTO, split_k: int = 0, tok_tile: int = 0,
               decode_warps: int = 0, level_shift: int = 0, cluster: int = 0,
-              debug_wait_ms: int = 0, debug_skip_load: int = 0) -> Opts:
+              debug_wait_ms: int = 0, debug_skip_load: int = 0, bits: int = 0) -> Opts:
     o = Opts()
     o.path, o.split_k, o.tok_tile, o.decode_warps = path, split_k, tok_tile, decode_warps
     o.level_shift = level_shift
     o.cluster = cluster
     o.debug_wait_ms, o.debug_skip_load = debug_wait_ms, debug_skip_load
+    o.bits = bits
     return o
 
 
@@ -145,23 +156,30 @@ def dint4_table(z: int):
     return list(buf)
 
 
-def packed_bytes(N: int, K: int, group: int = 0) -> int:
-    return int(lib.w4a8_packed_bytes(N, K, group))
+def packed_bytes(N: int, K: int, group: int = 0, bits: int = 4) -> int:
+    return int(lib.w4a8_packed_bytes_bits(N, K, group, bits))
 
 
-def pack_weights(W, s_in=None, group: int = 0, clip: float = 1.0, out=None, level_shift: int = 1):
-    """W [N, K] float16 (CUDA) -> packed blob (uint8 CUDA tensor); special value
-    step / 2^level_shift."""
+def dint_table(z: int, bits: int = 4, level_shift: int = 1):
+    buf = (ctypes.c_int8 * 16)()
+    lib.w4a8_dint_table_bits(z, bits, level_shift, buf)
+    return list(buf)[: 1 << bits]
+
+
+def pack_weights(W, s_in=None, group: int = 0, clip: float = 1.0, out=None, level_shift: int = 1,
+                 bits: int = 4):
+    """W [N, K] float16 (CUDA) -> packed blob (uint8 CUDA tensor); `bits`-bit dINT codes,
+    special value step / 2^level_shift."""
     W = _dev(W, torch.float16, "W")
     s_in = _dev(s_in, torch.float32, "s_in")
     N, K = W.shape
-    nbytes = packed_bytes(N, K, group)
+    nbytes = packed_bytes(N, K, group, bits)
     if nbytes == 0:
         raise W4A8Error(2, "w4a8_packed_bytes")
     if out is None:
         out = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
-    _check(lib.w4a8_pack_weights_fmt(_ptr(W), _ptr(s_in), N, K, group, clip, level_shift, _ptr(out),
-                                     out.numel(), _stream()), "w4a8_pack_weights")
+    _check(lib.w4a8_pack_weights_bits(_ptr(W), _ptr(s_in), N, K, group, clip, bits, level_shift,
+                                      _ptr(out), out.numel(), _stream()), "w4a8_pack_weights")
     return out
 
 
@@ -348,14 +366,14 @@ def linear_acc_i32(Xq, packed, N: int, group: int, workspace, opts: Opts | None 
     return acc
 
 
-def unpack_codes(packed, N: int, K: int, group: int = 0):
+def unpack_codes(packed, N: int, K: int, group: int = 0, bits: int = 4):
     """Blob -> (codes [N, K/2] uint8, scales [G, N] float32, zeros [G, N] uint8)."""
     G = K // group if group else 1
     codes = torch.empty((N, K // 2), dtype=torch.uint8, device=packed.device)
     scales = torch.empty((G, N), dtype=torch.float32, device=packed.device)
     zeros = torch.empty((G, N), dtype=torch.uint8, device=packed.device)
-    _check(lib.w4a8_unpack_codes(_ptr(packed), N, K, group, _ptr(codes), _ptr(scales),
-                                 _ptr(zeros), _stream()), "w4a8_unpack_codes")
+    _check(lib.w4a8_unpack_codes_bits(_ptr(packed), N, K, group, bits, _ptr(codes), _ptr(scales),
+                                      _ptr(zeros), _stream()), "w4a8_unpack_codes")
     return codes, scales, zeros
 
 

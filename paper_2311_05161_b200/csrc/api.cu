@@ -38,6 +38,8 @@ bool opts_ok(const w4a8_opts *o)
     if (o->split_k < 0 || o->tok_tile < 0 || o->decode_warps < 0) return false;
     if (o->level_shift < 0 || o->level_shift > 3) return false;
     if (o->cluster < 0 || o->cluster > 2) return false;
+    if (o->reserved != 0 || (o->bits != 0 && !bits_ok(o->bits))) return false;
+    if (o->bits == 3 && (o->path == W4A8_PATH_GEMV || o->cluster == 2)) return false;
 #ifdef W4A8_DEBUG_HOOKS
     if (o->debug_wait_ms < 0 || o->debug_wait_ms > 2000 || o->debug_skip_load < 0) return false;
     if ((o->debug_wait_ms || o->debug_skip_load) && o->path != W4A8_PATH_TCGEN05) return false;
@@ -49,6 +51,7 @@ bool opts_ok(const w4a8_opts *o)
 
 // special value = step / 2^shift; 0 in the options means the paper's 1
 int shift_of(const w4a8_opts *o) { return (o && o->level_shift) ? o->level_shift : 1; }
+int bits_of(const w4a8_opts *o) { return (o && o->bits) ? o->bits : 4; }
 
 // |level| <= 13 * 2^shift and |activation| <= amax: the INT32 sums must not overflow
 bool depth_ok(int K, int shift, int amax)
@@ -64,6 +67,7 @@ bool use_gemv(int M, const w4a8_opts *o)
 {
     const int path = o ? o->path : W4A8_PATH_AUTO;
     if (path == W4A8_PATH_GEMV) return true;
+    if (bits_of(o) == 3) return false;       // the weight-streaming kernels read 4-bit tiles
     if (path != W4A8_PATH_AUTO || (o && (o->split_k || o->tok_tile || o->decode_warps || o->cluster)))
         return false;
     return M <= 2;
@@ -87,7 +91,8 @@ w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *
     if (workspace_bytes < need) return W4A8_ERR_BUFFER_TOO_SMALL;
     const w4a8_status arch = check_arch();
     if (arch != W4A8_OK) return arch;
-    const BlobLayout L = make_layout(N, K, group, shift_of(opts));
+    const BlobLayout L = make_layout(N, K, group, shift_of(opts), bits_of(opts));
+    if (L.bits == 3 && zp.tok_zero) return W4A8_ERR_SHAPE;      // no row sums for 3-bit tiles
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint8_t *blob = static_cast<const uint8_t *>(packed);
     if (opts && opts->path == W4A8_PATH_SIMPLE) {
@@ -133,11 +138,25 @@ w4a8_status w4a8_pack_weights_fmt(const void *W_f16, const float *s_in, int N, i
                                   int group_size, float clip, int level_shift, void *packed,
                                   size_t packed_bytes, void *stream)
 {
+    return w4a8_pack_weights_bits(W_f16, s_in, N, K, group_size, clip, 4, level_shift, packed,
+                                  packed_bytes, stream);
+}
+
+size_t w4a8_packed_bytes_bits(int N, int K, int group_size, int bits)
+{
+    if (!shape_ok(N, K, group_size) || !bits_ok(bits)) return 0;
+    return make_layout(N, K, group_size, 1, bits).total_bytes;
+}
+
+w4a8_status w4a8_pack_weights_bits(const void *W_f16, const float *s_in, int N, int K,
+                                   int group_size, float clip, int bits, int level_shift,
+                                   void *packed, size_t packed_bytes, void *stream)
+{
     if (!W_f16 || !packed) return W4A8_ERR_NULL;
-    if (!shape_ok(N, K, group_size) || !(clip > 0.0f && clip <= 1.0f)) return W4A8_ERR_SHAPE;
+    if (!shape_ok(N, K, group_size) || !(clip > 0.0f && clip <= 1.0f) || !bits_ok(bits)) return W4A8_ERR_SHAPE;
     if (level_shift < 1 || level_shift > 3 || !depth_ok(K, level_shift, 127)) return W4A8_ERR_SHAPE;
     if (!aligned(W_f16, 16) || !aligned(s_in, 16) || !aligned(packed, 256)) return W4A8_ERR_ALIGN;
-    const BlobLayout L = make_layout(N, K, group_size, level_shift);
+    const BlobLayout L = make_layout(N, K, group_size, level_shift, bits);
     if (packed_bytes < L.total_bytes) return W4A8_ERR_BUFFER_TOO_SMALL;
     const w4a8_status arch = check_arch();
     if (arch != W4A8_OK) return arch;
@@ -192,7 +211,7 @@ size_t w4a8_linear_workspace_bytes_ex(int M, int N, int K, int group_size, const
         gemv_plan(M, make_layout(N, K, group_size), &plan);
         return plan.workspace_bytes;
     }
-    if (!make_plan(M, make_layout(N, K, group_size), opts, &plan)) return 0;
+    if (!make_plan(M, make_layout(N, K, group_size, shift_of(opts), bits_of(opts)), opts, &plan)) return 0;
     return plan.workspace_bytes;
 }
 
@@ -205,7 +224,7 @@ w4a8_status w4a8_linear_plan(int M, int N, int K, int group_size, const w4a8_opt
 {
     if (!out) return W4A8_ERR_NULL;
     if (!shape_ok(N, K, group_size) || M < 1 || !opts_ok(opts)) return W4A8_ERR_SHAPE;
-    const BlobLayout L = make_layout(N, K, group_size, shift_of(opts));
+    const BlobLayout L = make_layout(N, K, group_size, shift_of(opts), bits_of(opts));
     out[0] = out[1] = out[2] = out[3] = 0;
     out[4] = 1;
     if (opts && opts->path == W4A8_PATH_SIMPLE) {
@@ -364,13 +383,19 @@ w4a8_status w4a8_linear_asym(const int8_t *Xq, const float *tok_scale, const int
 w4a8_status w4a8_unpack_codes(const void *packed, int N, int K, int group_size, uint8_t *codes,
                               float *scales, uint8_t *zeros, void *stream)
 {
+    return w4a8_unpack_codes_bits(packed, N, K, group_size, 4, codes, scales, zeros, stream);
+}
+
+w4a8_status w4a8_unpack_codes_bits(const void *packed, int N, int K, int group_size, int bits,
+                                   uint8_t *codes, float *scales, uint8_t *zeros, void *stream)
+{
     if (!packed || !codes || !scales || !zeros) return W4A8_ERR_NULL;
-    if (!shape_ok(N, K, group_size)) return W4A8_ERR_SHAPE;
+    if (!shape_ok(N, K, group_size) || !bits_ok(bits)) return W4A8_ERR_SHAPE;
     if (!aligned(packed, 256) || !aligned(scales, 4)) return W4A8_ERR_ALIGN;
     const w4a8_status arch = check_arch();
     if (arch != W4A8_OK) return arch;
     const cudaError_t e =
-        launch_unpack(static_cast<const uint8_t *>(packed), make_layout(N, K, group_size), codes,
+        launch_unpack(static_cast<const uint8_t *>(packed), make_layout(N, K, group_size, 1, bits), codes,
                       scales, zeros, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
@@ -393,6 +418,11 @@ void w4a8_dint4_table(int z, int8_t *out) { w4a8_dint4_table_fmt(z, 1, out); }
 void w4a8_dint4_table_fmt(int z, int level_shift, int8_t *out)
 {
     for (int c = 0; c < 16; ++c) out[c] = (int8_t)dint4_level(c, z, level_shift);
+}
+
+void w4a8_dint_table_bits(int z, int bits, int level_shift, int8_t *out)
+{
+    for (int c = 0; c < 16; ++c) out[c] = c < (1 << bits) ? (int8_t)dint_level(c, z, level_shift, bits) : 0;
 }
 
 const char *w4a8_version(void) { return "w4a8-dint 0.1 (sm_100a)"; }

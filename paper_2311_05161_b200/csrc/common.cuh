@@ -17,8 +17,15 @@ namespace w4a8 {
 // ---------------------------------------------------------------------------
 constexpr int kTileN = 128;        // output rows per code tile
 constexpr int kTileK = 128;        // input features per code tile (= one quantization group)
-constexpr int kTileBytes = 8192;   // 128 x 128 nibbles
+constexpr int kTileBytes = 8192;   // 128 x 128 nibbles (4-bit codes)
 constexpr int kQuarterBytes = 2048;
+// 3-bit codes (dINT3): a tile is 128 x 128 x 3 bits.  Per 32-k quarter and row three 32-bit
+// words hold 32 codes: nibble j of word w (w = 0, 1, 2) carries in its low three bits the code
+// of k = 8 w + j, and the three spare top bits of the nibbles j of words 0, 1, 2 are bits 0,
+// 1, 2 of the code of k = 24 + j.  Word w of row r of quarter q sits at byte
+// q * 1536 + w * 512 + r * 4, so a warp reads 128 contiguous bytes per word.
+constexpr int kTileBytes3 = 6144;
+constexpr int kQuarterBytes3 = 1536;
 constexpr int kHeaderBytes = 256;
 constexpr uint32_t kBlobMagic = 0x38413457u;   // "W4A8"
 constexpr uint32_t kBlobVersion = 1u;
@@ -28,7 +35,7 @@ struct BlobHeader {
     uint32_t magic, version, layout, group;
     int32_t N, K, G, n_tiles, k_blocks, n_pad;
     uint32_t level_shift;   // special value = step / 2^level_shift; 0 (older blobs) means 1
-    uint32_t pad0;
+    uint32_t bits;          // code width: 3 or 4; 0 (older blobs) means 4
     uint64_t off_scales, off_zeros, off_codes, total_bytes;
     float clip;
     uint32_t pad1[43];
@@ -38,15 +45,20 @@ static_assert(sizeof(BlobHeader) == kHeaderBytes, "blob header is 256 bytes");
 struct BlobLayout {
     int N, K, group, G, n_tiles, k_blocks, n_pad;
     int shift;              // special value = step / 2^shift (1, 2 or 3); levels are in that unit
+    int bits;               // code width b: 4 (p = 13 integer steps) or 3 (p = 5)
+    int tile_bytes;         // bytes of one 128 x 128 code tile: 8192 or 6144
     size_t off_scales, off_zeros, off_codes, total_bytes;
 };
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-__host__ __device__ inline BlobLayout make_layout(int N, int K, int group, int shift = 1)
+__host__ __device__ inline BlobLayout make_layout(int N, int K, int group, int shift = 1,
+                                                  int bits = 4)
 {
     BlobLayout L;
     L.shift = shift;
+    L.bits = bits;
+    L.tile_bytes = bits == 3 ? kTileBytes3 : kTileBytes;
     L.N = N;
     L.K = K;
     L.group = group;
@@ -57,7 +69,7 @@ __host__ __device__ inline BlobLayout make_layout(int N, int K, int group, int s
     L.off_scales = kHeaderBytes;
     L.off_zeros = align_up(L.off_scales + (size_t)L.G * L.n_pad * sizeof(float), 256);
     L.off_codes = align_up(L.off_zeros + (size_t)L.G * L.n_pad, 256);
-    L.total_bytes = L.off_codes + (size_t)L.n_tiles * L.k_blocks * kTileBytes;
+    L.total_bytes = L.off_codes + (size_t)L.n_tiles * L.k_blocks * L.tile_bytes;
     return L;
 }
 
@@ -69,6 +81,8 @@ __host__ __device__ inline size_t code_byte_offset(const BlobLayout &L, int n, i
     const int q = kk / 32, j = (kk % 32) / 2;
     return ((size_t)nt * L.k_blocks + kb) * kTileBytes + (size_t)q * kQuarterBytes + r * 16 + j;
 }
+
+inline bool bits_ok(int bits) { return bits == 3 || bits == 4; }
 
 inline bool shape_ok(int N, int K, int group)
 {
@@ -84,7 +98,25 @@ __device__ inline bool header_matches(const uint8_t *blob, const BlobLayout &L)
     return h->magic == kBlobMagic && h->version == kBlobVersion &&
            h->layout == kBlobLayoutQuarterRow16 && h->N == L.N && h->K == L.K &&
            h->group == (uint32_t)L.group &&
-           (h->level_shift == 0u ? 1u : h->level_shift) == (uint32_t)L.shift;
+           (h->level_shift == 0u ? 1u : h->level_shift) == (uint32_t)L.shift &&
+           (h->bits == 0u ? 4u : h->bits) == (uint32_t)L.bits;
+}
+
+// The 3-bit code of k = 32 q + i of a row from the row's three words of quarter q.
+__host__ __device__ inline int code3_of(uint32_t w0, uint32_t w1, uint32_t w2, int i)
+{
+    if (i < 24) {
+        const uint32_t w = i < 8 ? w0 : (i < 16 ? w1 : w2);
+        return (int)((w >> (4 * (i & 7))) & 7u);
+    }
+    const int sh = 4 * (i - 24) + 3;
+    return (int)(((w0 >> sh) & 1u) | (((w1 >> sh) & 1u) << 1) | (((w2 >> sh) & 1u) << 2));
+}
+// Byte offset, inside the code section, of word w of the 3-bit codes of row n, quarter (kb, q).
+__host__ __device__ inline size_t code3_word_offset(const BlobLayout &L, int n, int kb, int q, int w)
+{
+    const int nt = n / kTileN, r = n % kTileN;
+    return ((size_t)nt * L.k_blocks + kb) * kTileBytes3 + (size_t)q * kQuarterBytes3 + w * 512 + r * 4;
 }
 
 // ---------------------------------------------------------------------------
@@ -115,6 +147,12 @@ __host__ __device__ inline int dint4_level(int code, int z, int shift)
 {
     return code <= 13 ? (code - z) * (1 << shift) : (code == 14 ? 1 : -1);
 }
+// the same for b-bit codes: integer codes 0..p, p + 1 = +c, p + 2 = -c, p = 2^b - 3
+__host__ __device__ inline int dint_level(int code, int z, int shift, int bits)
+{
+    const int p = (1 << bits) - 3;
+    return code <= p ? (code - z) * (1 << shift) : (code == p + 1 ? 1 : -1);
+}
 // the unit itself as a factor of the step: 2^-shift, exact
 __host__ __device__ inline float level_unit(int shift)
 {
@@ -137,6 +175,14 @@ inline LevelTables make_level_tables(int shift)
     t.base[3] = 0x00008080u + m * 0x00000D0Cu;
     t.zmul = m * 0x01010101u;
     return t;
+}
+// 3-bit codes: eight levels in two words (codes 0..3, then 4, 5, +1, -1).
+__device__ __forceinline__ void build_level_tables3(int z, int shift, uint32_t (&t)[2])
+{
+    const uint32_t m = 1u << shift;
+    const uint32_t zz = (uint32_t)z * m * 0x01010101u;
+    t[0] = ((0x80808080u + m * 0x03020100u) - zz) ^ 0x80808080u;
+    t[1] = ((((0x00008080u + m * 0x00000504u) - (zz & 0xFFFFu)) ^ 0x00008080u) & 0xFFFFu) | 0xFF010000u;
 }
 __device__ __forceinline__ void build_level_tables(int z, const LevelTables &lt, uint32_t (&t)[4])
 {

@@ -29,8 +29,16 @@ linear_simple_kernel(const int8_t *__restrict__ Xq, const float *__restrict__ to
     float u = 0.0f;
     for (int kb = 0; kb < L.k_blocks; ++kb) {
         if (grouped) { z = zeros[(size_t)kb * L.n_pad + n]; acc = 0; }
-        const uint8_t *tile = codes + ((size_t)nt * L.k_blocks + kb) * kTileBytes;
+        const uint8_t *tile = codes + ((size_t)nt * L.k_blocks + kb) * L.tile_bytes;
         for (int q = 0; q < 4; ++q) {
+            if (L.bits == 3) {
+                const uint32_t *w3 = reinterpret_cast<const uint32_t *>(tile + q * kQuarterBytes3 + r * 4);
+                const uint32_t w0 = w3[0], w1 = w3[128], w2 = w3[256];
+                const int8_t *xk = x + kb * kTileK + q * 32;
+                for (int i = 0; i < 32; ++i)
+                    acc += (int32_t)xk[i] * dint_level(code3_of(w0, w1, w2, i), z, L.shift, 3);
+                continue;
+            }
             const uint4 w = *reinterpret_cast<const uint4 *>(tile + q * kQuarterBytes + r * 16);
             const uint32_t words[4] = {w.x, w.y, w.z, w.w};
             const int8_t *xk = x + kb * kTileK + q * 32;

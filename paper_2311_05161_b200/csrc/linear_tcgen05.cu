@@ -481,7 +481,7 @@ __device__ __forceinline__ void decode8(uint32_t w, const uint32_t (&t)[4], uint
 }
 
 // --------------------------------------------------------------------------- the kernel
-template <int TOK, bool GROUPED, int DW, int CL>
+template <int TOK, bool GROUPED, int DW, int CL, int BITS>
 __global__ void __launch_bounds__(Cfg<TOK, GROUPED, DW, CL>::kThreads, 1)
 linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                       const __grid_constant__ CUtensorMap y_map, const Params P)
@@ -588,8 +588,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         // keep the code stream kPrefetchAhead k-blocks ahead of the decode warps
                         while (pf.valid() && pf.it < it + C::kPrefetchAhead) {
                             const int pnt = pf.nt;
-                            prefetch_l2(P.codes + ((size_t)pnt * k_blocks + pf.kb) * kTileBytes,
-                                        kTileBytes);
+                            prefetch_l2(P.codes + ((size_t)pnt * k_blocks + pf.kb) * (BITS == 3 ? kTileBytes3 : kTileBytes),
+                                        BITS == 3 ? kTileBytes3 : kTileBytes);
                             pf.advance(1);
                         }
                     }
@@ -677,6 +677,67 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         KbCursor cur;
         cur.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, n_tiles);
         cur.advance(team);
+        if constexpr (BITS == 3) {
+            // 3-bit codes: twelve words per row and k-block (three per 32-k quarter, each read
+            // as 128 contiguous bytes by a warp); the selector nibbles of eight codes are the
+            // words with their top bits cleared, the fourth selector of a quarter is put
+            // together from those top bits; one byte permute on the two table words yields four
+            // levels.  One thread per row (no clusters in this mode).
+            static_assert(CL == 1, "3-bit codes: one CTA per cluster");
+            uint32_t w3[12];
+            int z3 = 0;
+            auto fetch3 = [&](const KbCursor &c, uint32_t (&dst)[12], int &zz) {
+                const int n = c.nt * kTileN + r;
+                zz = GROUPED ? P.zeros[(size_t)c.kb * P.L.n_pad + n] : P.zeros[n];
+                const uint32_t *src = reinterpret_cast<const uint32_t *>(
+                    P.codes + ((size_t)c.nt * k_blocks + c.kb) * kTileBytes3 + r * 4);
+#pragma unroll
+                for (int i = 0; i < 12; ++i) {
+                    uint32_t v;
+                    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(src + i * 128));
+                    dst[i] = v;
+                }
+            };
+            if (cur.valid()) fetch3(cur, w3, z3);
+            bool ok3 = true;
+            while (cur.valid() && ok3) {
+                KbCursor nxt = cur;
+                nxt.advance(C::kTeams);
+                uint32_t wn3[12];
+                int zn3 = 0;
+                if (nxt.valid()) fetch3(nxt, wn3, zn3);
+                const int st = cur.it % S;
+                const uint32_t fill = cur.it / S;
+                uint32_t t3[2];
+                build_level_tables3(z3, P.L.shift, t3);
+                ok3 = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
+                ok3 = __all_sync(0xffffffffu, ok3);
+                if (!ok3) break;
+                uint8_t *arow = gen_base + st * C::kStageBytes + r * 128;
+                const int sw = r & 7;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t a = w3[3 * q], b = w3[3 * q + 1], c = w3[3 * q + 2];
+                    const uint32_t s0 = a & 0x77777777u, s1 = b & 0x77777777u, s2 = c & 0x77777777u;
+                    const uint32_t s3 = ((a >> 3) & 0x11111111u) | ((b >> 2) & 0x22222222u) |
+                                        ((c >> 1) & 0x44444444u);
+                    uint4 c0, c1;
+                    c0.x = prmt(t3[0], t3[1], s0); c0.y = prmt(t3[0], t3[1], s0 >> 16);
+                    c0.z = prmt(t3[0], t3[1], s1); c0.w = prmt(t3[0], t3[1], s1 >> 16);
+                    c1.x = prmt(t3[0], t3[1], s2); c1.y = prmt(t3[0], t3[1], s2 >> 16);
+                    c1.z = prmt(t3[0], t3[1], s3); c1.w = prmt(t3[0], t3[1], s3 >> 16);
+                    *reinterpret_cast<uint4 *>(arow + (((2 * q) ^ sw) << 4)) = c0;
+                    *reinterpret_cast<uint4 *>(arow + (((2 * q + 1) ^ sw) << 4)) = c1;
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_dec + 8 * st);
+#pragma unroll
+                for (int i = 0; i < 12; ++i) w3[i] = wn3[i];
+                z3 = zn3;
+                cur = nxt;
+            }
+        } else {
         uint4 w[QT];
         int z = 0;
         auto fetch = [&](const KbCursor &c, uint4 (&dst)[QT], int &zz) {
@@ -750,6 +811,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             z = zn;
             cur = nxt;
         }
+        }   // 4-bit codes
     } else if (role == kEpilogue) {
         // ------------------------------------------------------------------ epilogue warps
         const int ew = role_idx;
@@ -1078,7 +1140,7 @@ struct Maps {
 
 // Clusters of CL CTAs of this kernel that the current device can hold at once (one CTA per
 // SM); asked once per kernel instance and device.
-template <int TOK, bool GROUPED, int DW, int CL>
+template <int TOK, bool GROUPED, int DW, int CL, int BITS>
 int resident_clusters()
 {
     using C = Cfg<TOK, GROUPED, DW, CL>;
@@ -1087,7 +1149,7 @@ int resident_clusters()
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
     int n = cached[dev].load(std::memory_order_acquire);
     if (n > 0) return n;
-    auto kern = linear_tcgen05_kernel<TOK, GROUPED, DW, CL>;
+    auto kern = linear_tcgen05_kernel<TOK, GROUPED, DW, CL, BITS>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) !=
         cudaSuccess)
         return 0;
@@ -1114,12 +1176,12 @@ int resident_clusters()
     return n;
 }
 
-template <int TOK, bool GROUPED, int DW, int CL>
+template <int TOK, bool GROUPED, int DW, int CL, int BITS = 4>
 w4a8_status launch_cl(const Maps &maps, const Params &P, cudaStream_t st)
 {
     using C = Cfg<TOK, GROUPED, DW, CL>;
-    auto kern = linear_tcgen05_kernel<TOK, GROUPED, DW, CL>;
-    const int resident = resident_clusters<TOK, GROUPED, DW, CL>();   // also sizes the kernel's shared memory
+    auto kern = linear_tcgen05_kernel<TOK, GROUPED, DW, CL, BITS>;
+    const int resident = resident_clusters<TOK, GROUPED, DW, CL, BITS>();   // also sizes the kernel's shared memory
     if (resident < 1) return W4A8_ERR_CUDA;
     const int clusters = P.total_units < resident ? P.total_units : resident;
     const cudaError_t e =
@@ -1142,6 +1204,8 @@ w4a8_status launch_dw(const Maps &maps, const Params &P, int cluster, cudaStream
 template <int TOK, bool GROUPED>
 w4a8_status launch_one(const Maps &maps, const Params &P, int dw, int cluster, cudaStream_t st)
 {
+    // 3-bit codes: eight decode warps, no clusters (make_plan picks nothing else)
+    if (P.L.bits == 3) return dw == 8 && cluster == 1 ? launch_cl<TOK, GROUPED, 8, 1, 3>(maps, P, st) : W4A8_ERR_SHAPE;
     if (dw == 4) return launch_dw<TOK, GROUPED, 4>(maps, P, cluster, st);
     if (dw == 8) return launch_dw<TOK, GROUPED, 8>(maps, P, cluster, st);
     if (dw == 12 && !GROUPED) return launch_dw<TOK, false, 12>(maps, P, cluster, st);
@@ -1216,7 +1280,8 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     split = (L.k_blocks + kb_per - 1) / kb_per;              // no empty slice
     if (tiles * split > 0x7fffffffLL) return false;
     int dw = opts ? opts->decode_warps : 0;
-    if (dw == 0) dw = grouped ? 8 : 16;
+    if (dw == 0) dw = (grouped || L.bits == 3) ? 8 : 16;
+    if (L.bits == 3 && (dw != 8 || cluster != 1)) return false;
     if (dw != 4 && dw != 8 && !((dw == 12 || dw == 16) && !grouped)) return false;
     plan->decode_warps = dw;
     plan->cluster = cluster;

@@ -28,16 +28,30 @@ __device__ __forceinline__ uint32_t dint4_quantize(float x, float s, int z, floa
     return (uint32_t)q;
 }
 
-__device__ __forceinline__ void step_and_zero(float lo, float hi, float clip, float &s, int &z)
+// step = range / p and zero-point for p uniform steps (p = 13 for 4-bit codes, 5 for 3-bit)
+__device__ __forceinline__ void step_and_zero(float lo, float hi, float clip, float &s, int &z,
+                                              int p = 13)
 {
     lo = __fmul_rn(lo, clip);
     hi = __fmul_rn(hi, clip);
-    s = __fdiv_rn(__fsub_rn(hi, lo), 13.0f);
+    s = __fdiv_rn(__fsub_rn(hi, lo), (float)p);
     if (s == 0.0f) s = 1.0f;
     float r = rintf(__fdiv_rn(-lo, s));
     r = fminf(fmaxf(r, -1048576.0f), 1048576.0f);
     z = (int)r;
-    z = z < 0 ? 0 : (z > 13 ? 13 : z);
+    z = z < 0 ? 0 : (z > p ? p : z);
+}
+
+// Eq. 5 for b = 3: codes 0..5 integer levels, 6 = c1 (+c), 7 = c2 (-c)
+__device__ __forceinline__ uint32_t dint3_quantize(float x, float s, int z, float lower, float upper)
+{
+    if (x > lower && x <= upper) return 6u;
+    if (x < -lower && x >= -upper) return 7u;
+    float r = rintf(__fdiv_rn(x, s));
+    r = fminf(fmaxf(r, -1048576.0f), 1048576.0f);
+    int q = (int)r + z;
+    q = q < 0 ? 0 : (q > 5 ? 5 : q);
+    return (uint32_t)q;
 }
 
 __device__ __forceinline__ float scaled(const __half h, const float *s_in, int k)
@@ -60,6 +74,7 @@ __device__ __forceinline__ void write_header(uint8_t *blob, const BlobLayout &L,
     h.off_codes = L.off_codes; h.total_bytes = L.total_bytes;
     h.clip = clip;
     h.level_shift = (uint32_t)L.shift;
+    h.bits = (uint32_t)L.bits;
     *reinterpret_cast<BlobHeader *>(blob) = h;
 }
 
@@ -183,6 +198,92 @@ pack_groups_kernel(const __half *__restrict__ W, const float *__restrict__ s_in,
     }
 }
 
+// 3-bit codes (dINT3), per-channel or group-128: one CTA of 128 threads per output row.  A
+// thread takes 32-k quarters of the row; the four threads of a 128-wide chunk combine their
+// ranges by shuffles, the chunks' ranges wait in shared memory (the whole row's for
+// per-channel weights), then every thread re-reads its quarters and writes three words each.
+__global__ void __launch_bounds__(128)
+pack3_kernel(const __half *__restrict__ W, const float *__restrict__ s_in, BlobLayout L, float clip,
+             uint8_t *__restrict__ blob)
+{
+    extern __shared__ float s_range[];               // lo[chunks], hi[chunks]
+    const int n = blockIdx.x, tid = threadIdx.x;
+    float *scales = reinterpret_cast<float *>(blob + L.off_scales);
+    uint8_t *zeros = blob + L.off_zeros;
+    uint8_t *codes = blob + L.off_codes;
+    if (n == 0 && tid == 0) write_header(blob, L, clip);
+    const bool real = n < L.N;
+    const __half *row = W + (size_t)n * L.K;
+    const int chunks = L.k_blocks, quarters = 4 * chunks;
+    float *s_lo = s_range, *s_hi = s_range + chunks;
+    for (int qi = tid; qi < (quarters + 127) / 128 * 128; qi += 128) {
+        float lo = 0.0f, hi = 0.0f;
+        if (real && qi < quarters) {
+            for (int i = 0; i < 32; ++i) {
+                const float w = scaled(row[qi * 32 + i], s_in, qi * 32 + i);
+                if (w < lo) lo = w;
+                if (w > hi) hi = w;
+            }
+        }
+        for (int o = 1; o <= 2; o <<= 1) {
+            const float l2 = __shfl_xor_sync(0xffffffffu, lo, o);
+            const float h2 = __shfl_xor_sync(0xffffffffu, hi, o);
+            if (l2 < lo) lo = l2;
+            if (h2 > hi) hi = h2;
+        }
+        if ((tid & 3) == 0 && qi < quarters) { s_lo[qi >> 2] = lo; s_hi[qi >> 2] = hi; }
+    }
+    __syncthreads();
+    if (L.group == 0) {
+        if (tid == 0) {
+            float lo = 0.0f, hi = 0.0f;
+            for (int c = 0; c < chunks; ++c) {
+                if (s_lo[c] < lo) lo = s_lo[c];
+                if (s_hi[c] > hi) hi = s_hi[c];
+            }
+            float s; int z;
+            step_and_zero(lo, hi, clip, s, z, 5);
+            scales[n] = s;
+            zeros[n] = (uint8_t)z;
+            s_lo[0] = s;
+            s_hi[0] = __int_as_float(z);
+        }
+    } else {
+        for (int c = tid; c < chunks; c += 128) {
+            float s; int z;
+            step_and_zero(s_lo[c], s_hi[c], clip, s, z, 5);
+            scales[(size_t)c * L.n_pad + n] = s;
+            zeros[(size_t)c * L.n_pad + n] = (uint8_t)z;
+            s_lo[c] = s;
+            s_hi[c] = __int_as_float(z);
+        }
+    }
+    __syncthreads();
+    for (int qi = tid; qi < quarters; qi += 128) {
+        const int c = L.group == 0 ? 0 : (qi >> 2);
+        const float s = s_lo[c];
+        const int z = __float_as_int(s_hi[c]);
+        float lower, upper;
+        special_band(s, L.shift, lower, upper);
+        uint32_t w[3] = {0u, 0u, 0u};
+        if (real) {
+            for (int i = 0; i < 32; ++i) {
+                const uint32_t code = dint3_quantize(scaled(row[qi * 32 + i], s_in, qi * 32 + i), s, z, lower, upper);
+                if (i < 24) {
+                    w[i >> 3] |= code << (4 * (i & 7));
+                } else {
+                    const int sh = 4 * (i - 24) + 3;
+                    w[0] |= (code & 1u) << sh;
+                    w[1] |= ((code >> 1) & 1u) << sh;
+                    w[2] |= ((code >> 2) & 1u) << sh;
+                }
+            }
+        }
+        for (int j = 0; j < 3; ++j)
+            *reinterpret_cast<uint32_t *>(codes + code3_word_offset(L, n, qi >> 2, qi & 3, j)) = w[j];
+    }
+}
+
 __global__ void unpack_kernel(const uint8_t *__restrict__ blob, BlobLayout L,
                               uint8_t *__restrict__ out_codes, float *__restrict__ out_scales,
                               uint8_t *__restrict__ out_zeros)
@@ -196,6 +297,14 @@ __global__ void unpack_kernel(const uint8_t *__restrict__ blob, BlobLayout L,
          i += (size_t)gridDim.x * blockDim.x) {
         const int n = (int)(i / half_k);
         const int k = (int)(i % half_k) * 2;
+        if (L.bits == 3) {
+            const int kb = k / kTileK, q = (k % kTileK) / 32, j = k % 32;
+            const uint32_t w0 = *reinterpret_cast<const uint32_t *>(codes + code3_word_offset(L, n, kb, q, 0));
+            const uint32_t w1 = *reinterpret_cast<const uint32_t *>(codes + code3_word_offset(L, n, kb, q, 1));
+            const uint32_t w2 = *reinterpret_cast<const uint32_t *>(codes + code3_word_offset(L, n, kb, q, 2));
+            out_codes[i] = (uint8_t)(code3_of(w0, w1, w2, j) | (code3_of(w0, w1, w2, j + 1) << 4));
+            continue;
+        }
         out_codes[i] = codes[code_byte_offset(L, n, k)];
     }
     const size_t meta = (size_t)L.G * L.N;
@@ -247,7 +356,9 @@ rowsum_kernel(const uint8_t *__restrict__ blob, BlobLayout L, int kb_per_slice,
 cudaError_t launch_pack(const __half *W, const float *s_in, const BlobLayout &L, float clip,
                         uint8_t *blob, cudaStream_t st)
 {
-    if (L.group == 0)
+    if (L.bits == 3)
+        pack3_kernel<<<L.n_pad, 128, 2 * L.k_blocks * sizeof(float), st>>>(W, s_in, L, clip, blob);
+    else if (L.group == 0)
         pack_rows_kernel<<<L.n_pad, kPackThreads, 0, st>>>(W, s_in, L, clip, blob);
     else
         pack_groups_kernel<<<L.n_pad, kPackThreads, 0, st>>>(W, s_in, L, clip, blob);
