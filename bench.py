@@ -842,6 +842,42 @@ def main():
         down.clear()
         torch.cuda.empty_cache()
 
+    if legs_on:
+        # -------------------------------------------------------------- attention value path (W4A8V4)
+        Hh, Dh = 32, 128
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(5005)
+        pv = {}
+        for name, T, S in (("prefill_T2048_S2048", 2048, 2048), ("decode_T1_S4096", 1, 4096)):
+            V = torch.randn((S, Hh, Dh), generator=gen, device=dev, dtype=torch.float16)
+            P = torch.softmax(2.0 * torch.randn((Hh, T, S), generator=gen, device=dev, dtype=torch.float32), -1).half()
+            blobs = [w4a8.pack_value(V)]
+            blobs += [blobs[0].clone() for _ in range(3)]
+            Pq = torch.empty((Hh * T, S), dtype=torch.int8, device=dev)
+            ps = torch.empty((Hh * T,), dtype=torch.float32, device=dev)
+            O = torch.empty((T, Hh, Dh), dtype=torch.bfloat16, device=dev)
+            wsv = w4a8.new_attn_pv_workspace(T, S, Hh, Dh)
+
+            def fn(it, P=P, Pq=Pq, ps=ps, blobs=blobs, O=O, wsv=wsv, T=T, S=S):
+                w4a8.quantize_act(P.view(Hh * T, S), None, out=(Pq, ps))
+                w4a8.attn_pv(Pq.view(Hh, T, S), ps.view(Hh, T), blobs[it % 4], Dh, wsv, out=O)
+            ms_pv = graph_ms(fn, 20)
+            w4a8.check_status(wsv)
+            ops_pv = 2.0 * T * S * Hh * Dh
+            bytes_pv = S * Hh * Dh // 2 + 5 * Hh * Dh + Hh * T * (S + 4) + 2 * T * Hh * Dh
+            pv[name] = {"ms": ms_pv, "tops": ops_pv / (ms_pv * 1e-3) / 1e12,
+                        "gbs": bytes_pv / (ms_pv * 1e-3) / 1e9,
+                        "frac_of_burst_tensor": ops_pv / (ms_pv * 1e-3) / 1e12 / (2.0 * peaks["bf16_burst"]),
+                        "frac_of_measured_copy": bytes_pv / (ms_pv * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+            del V, P, blobs, Pq, ps, O, wsv
+        torch.cuda.empty_cache()
+        legs["attn_pv_value4"] = {
+            "workload": "attention map x values, 32 heads of dimension 128, channel-wise dINT4 values "
+                        "(W4A8V4), token-wise INT8 attention map", **pv,
+            "note": "per step: quantize_act on the FP16 attention map + attn_pv (all heads in one "
+                    "launch of the tensor-core kernel); random map and values drawn on the device; "
+                    "CUDA graph replay of 20 steps"}
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()

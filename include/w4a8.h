@@ -291,6 +291,28 @@ w4a8_status w4a8_linear_asym(const int8_t *Xq, const float *tok_scale, const int
                              int M, int N, int K, void *Y_bf16, int32_t *acc, void *workspace,
                              size_t workspace_bytes, void *stream, const w4a8_opts *opts);
 
+/* ---- attention value path: "W4A8V4" (Section 5; Appendix A.1: channel-wise 4-bit Value) ----
+ * The product of the attention map and the values, O[t][h][d] = sum_s P[h][t][s] V[s][h][d], with
+ * V quantized to dINT4 per channel (h, d) - the dimension along which the partial sums
+ * accumulate is the sequence s, so one step size and zero-point per channel factor out of the sum
+ * - and the attention map quantized token-wise to INT8 like every other activation.  With the
+ * channels (h, d) as output features and the sequence as input features this is Eq. 1 once per
+ * head, and the tensor-core kernel runs all heads in one launch (head h = 128-row tile h).
+ * Head dimension D = 128; S % 128 == 0.
+ *
+ * w4a8_pack_value: V_f16 [S][H][D] binary16 (the value projection's output, token-major) ->
+ *   blob of w4a8_packed_bytes(H * D, S, 0) bytes (Eq. 5 per channel over the S positions).
+ * w4a8_attn_pv: Pq [H][T][S] INT8 and p_scale [H][T] FP32 as written by w4a8_quantize_act on
+ *   the attention map viewed as [H * T][S]; O_bf16 [T][H][D] bfloat16:
+ *   o = (float(sum_s Pq * t2(code)) * p_scale[h][t]) * (0.5 * step[h][d]).
+ *   workspace >= w4a8_attn_pv_workspace_bytes(T, S, H, D), zero-filled once. */
+w4a8_status w4a8_pack_value(const void *V_f16, int S, int H, int D, float clip, void *packed,
+                            size_t packed_bytes, void *stream);
+size_t w4a8_attn_pv_workspace_bytes(int T, int S, int H, int D);
+w4a8_status w4a8_attn_pv(const int8_t *Pq, const float *p_scale, const void *packed, int T, int S,
+                         int H, int D, void *O_bf16, void *workspace, size_t workspace_bytes,
+                         void *stream);
+
 /* Test export: the INT32 accumulators of the contraction, acc [G][M][N], before any
  * rescale (Eq. 6 in units of step/2).  Uses the same kernels as w4a8_linear_ex. */
 w4a8_status w4a8_linear_acc_i32(const int8_t *Xq, const void *packed, int M, int N, int K,

@@ -394,6 +394,30 @@ def linear_bits(Xq, tok_scale, codes, scales, zeros, bias, group: int, bits: int
     return acc, Y, wide
 
 
+def pack_value(V: np.ndarray, clip: float = 1.0):
+    """Channel-wise dINT4 quantization of the attention values (Appendix A.1, "W4A8V4"):
+    V is [S, H, D] float16; a channel is one (h, d), its Min-Max range is taken over the S
+    positions (the dimension the attention map sums over).  Returns (codes [H*D, S/2],
+    scales [1, H*D], zeros [1, H*D]) as pack_weights does for the matrix V^T."""
+    V = _c(V, np.float16)
+    S, H, D = V.shape
+    return pack_weights(np.ascontiguousarray(V.reshape(S, H * D).T), None, 0, clip)
+
+
+def attn_pv(Pq: np.ndarray, p_scale: np.ndarray, codes, scales, zeros, D: int) -> np.ndarray:
+    """O[t, h, d] = (float(sum_s Pq[h, t, s] * t2(code[h*D + d, s])) * p_scale[h, t]) * (0.5 * step[h*D + d]),
+    BF16 bits [T, H, D]: Eq. 1 once per head with the channels (h, d) as output features."""
+    Pq = _c(Pq, np.int8)
+    p_scale = _c(p_scale, np.float32)
+    H, T, S = Pq.shape
+    out = np.empty((T, H, D), dtype=np.uint16)
+    for h in range(H):
+        sl = slice(h * D, (h + 1) * D)
+        out[:, h, :] = linear(Pq[h], p_scale[h], np.ascontiguousarray(codes[sl]),
+                              np.ascontiguousarray(scales[:, sl]), np.ascontiguousarray(zeros[:, sl]), None, 0)
+    return out
+
+
 def bf16_bits_to_float(bits: np.ndarray) -> np.ndarray:
     """Widen BF16 bit patterns (uint16) to float32 values (exact)."""
     return (bits.astype(np.uint32) << 16).view(np.float32)

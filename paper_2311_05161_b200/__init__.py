@@ -12,4 +12,5 @@ from .binding import (  # noqa: F401
     workspace_init, quantize_act_asym, weight_rowsum, linear_asym,
     quantize_linear, quantize_linear_workspace_bytes, new_quantize_linear_workspace, linear_plan,
     norm_quantize_act, NORM_RMS, NORM_LAYER, dint_table,
+    pack_value, attn_pv, new_attn_pv_workspace,
 )

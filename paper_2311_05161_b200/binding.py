@@ -31,6 +31,7 @@ EXPORTS = (
     "w4a8_pack_weights_fmt", "w4a8_dint4_table_fmt",
     "w4a8_quantize_linear", "w4a8_quantize_linear_workspace_bytes", "w4a8_linear_plan", "w4a8_norm_quantize_act",
     "w4a8_packed_bytes_bits", "w4a8_pack_weights_bits", "w4a8_unpack_codes_bits", "w4a8_dint_table_bits",
+    "w4a8_pack_value", "w4a8_attn_pv", "w4a8_attn_pv_workspace_bytes",
 )
 
 
@@ -89,6 +90,12 @@ def _load() -> ctypes.CDLL:
     lib.w4a8_unpack_codes_bits.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp]
     lib.w4a8_dint_table_bits.restype = None
     lib.w4a8_dint_table_bits.argtypes = [ci, ci, ci, vp]
+    lib.w4a8_pack_value.restype = ci
+    lib.w4a8_pack_value.argtypes = [vp, ci, ci, ci, cf, vp, sz, vp]
+    lib.w4a8_attn_pv_workspace_bytes.restype = sz
+    lib.w4a8_attn_pv_workspace_bytes.argtypes = [ci, ci, ci, ci]
+    lib.w4a8_attn_pv.restype = ci
+    lib.w4a8_attn_pv.argtypes = [vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, vp]
     lib.w4a8_pack_weights_fmt.restype = ci
     lib.w4a8_pack_weights_fmt.argtypes = [vp, vp, ci, ci, ci, cf, ci, vp, sz, vp]
     lib.w4a8_quantize_act_asym.restype = ci
@@ -337,6 +344,40 @@ def linear_asym(Xq, tok_scale, tok_zero, packed, rowsum, bias, N: int, workspace
                               ctypes.byref(opts) if opts is not None else None)
     _check(st, "w4a8_linear_asym")
     return (out, acc) if want_acc else out
+
+
+def pack_value(V, clip: float = 1.0, out=None):
+    """Attention values V [S, H, D] float16 (CUDA) -> dINT4 blob, one step per channel (h, d)."""
+    V = _dev(V, torch.float16, "V")
+    S, H, D = V.shape
+    nbytes = packed_bytes(H * D, S, 0)
+    if nbytes == 0:
+        raise W4A8Error(2, "w4a8_packed_bytes")
+    if out is None:
+        out = torch.empty(nbytes, dtype=torch.uint8, device=V.device)
+    _check(lib.w4a8_pack_value(_ptr(V), S, H, D, clip, _ptr(out), out.numel(), _stream()), "w4a8_pack_value")
+    return out
+
+
+def new_attn_pv_workspace(T: int, S: int, H: int, D: int, device="cuda"):
+    nbytes = int(lib.w4a8_attn_pv_workspace_bytes(T, S, H, D))
+    if nbytes == 0:
+        raise W4A8Error(2, "w4a8_attn_pv_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    workspace_init(ws)
+    return ws
+
+
+def attn_pv(Pq, p_scale, packed, D: int, workspace, out=None):
+    """Pq [H, T, S] int8, p_scale [H, T] float32, packed values -> O [T, H, D] bfloat16."""
+    Pq = _dev(Pq, torch.int8, "Pq")
+    p_scale = _dev(p_scale, torch.float32, "p_scale")
+    H, T, S = Pq.shape
+    if out is None:
+        out = torch.empty((T, H, D), dtype=torch.bfloat16, device=Pq.device)
+    _check(lib.w4a8_attn_pv(_ptr(Pq), _ptr(p_scale), _ptr(packed), T, S, H, D, _ptr(out),
+                            _ptr(workspace), workspace.numel(), _stream()), "w4a8_attn_pv")
+    return out
 
 
 def linear_static(Xq, tok_scale, packed, bias, N: int, group: int, out):

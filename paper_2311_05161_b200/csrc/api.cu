@@ -327,6 +327,60 @@ w4a8_status w4a8_quantize_linear(const void *X_f16, const float *inv_s_in, const
                               static_cast<const __half *>(X_f16), inv_s_in);
 }
 
+// ---- attention value path (W4A8V4): P * V with channel-wise dINT4 values ----
+w4a8_status w4a8_pack_value(const void *V_f16, int S, int H, int D, float clip, void *packed,
+                            size_t packed_bytes, void *stream)
+{
+    if (!V_f16 || !packed) return W4A8_ERR_NULL;
+    if (D != kTileN || H < 1 || H > 4096 || !shape_ok(H * D, S, 0) || !(clip > 0.0f && clip <= 1.0f))
+        return W4A8_ERR_SHAPE;
+    if (!depth_ok(S, 1, 127)) return W4A8_ERR_SHAPE;
+    if (!aligned(V_f16, 16) || !aligned(packed, 256)) return W4A8_ERR_ALIGN;
+    const BlobLayout L = make_layout(H * D, S, 0);
+    if (packed_bytes < L.total_bytes) return W4A8_ERR_BUFFER_TOO_SMALL;
+    const w4a8_status arch = check_arch();
+    if (arch != W4A8_OK) return arch;
+    const cudaError_t e = launch_pack_transposed(static_cast<const __half *>(V_f16), L, clip,
+                                                 static_cast<uint8_t *>(packed),
+                                                 static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+}
+
+size_t w4a8_attn_pv_workspace_bytes(int T, int S, int H, int D)
+{
+    if (D != kTileN || H < 1 || T < 1 || !shape_ok(H * D, S, 0)) return 0;
+    LinearPlan plan;
+    w4a8_opts o = {};
+    o.path = W4A8_PATH_TCGEN05;
+    if (!make_plan(T, make_layout(H * D, S, 0), &o, &plan)) return 0;
+    return plan.workspace_bytes;
+}
+
+w4a8_status w4a8_attn_pv(const int8_t *Pq, const float *p_scale, const void *packed, int T, int S,
+                         int H, int D, void *O_bf16, void *workspace, size_t workspace_bytes,
+                         void *stream)
+{
+    if (!Pq || !p_scale || !packed || !O_bf16 || !workspace) return W4A8_ERR_NULL;
+    if (D != kTileN || H < 1 || T < 1 || !shape_ok(H * D, S, 0) || !depth_ok(S, 1, 127))
+        return W4A8_ERR_SHAPE;
+    if (!aligned(Pq, 16) || !aligned(p_scale, 4) || !aligned(O_bf16, 16) || !aligned(packed, 256) ||
+        !aligned(workspace, 256))
+        return W4A8_ERR_ALIGN;
+    const BlobLayout L = make_layout(H * D, S, 0);
+    LinearPlan plan;
+    w4a8_opts o = {};
+    o.path = W4A8_PATH_TCGEN05;
+    if (!make_plan(T, L, &o, &plan)) return W4A8_ERR_SHAPE;
+    if (workspace_bytes < plan.workspace_bytes) return W4A8_ERR_BUFFER_TOO_SMALL;
+    const w4a8_status arch = check_arch();
+    if (arch != W4A8_OK) return arch;
+    plan.batched = 1;            // head h = row tile h reads its own [T][S] block of Pq and p_scale
+    return launch_linear_tcgen05(Pq, p_scale, static_cast<const uint8_t *>(packed), L, nullptr, T,
+                                 static_cast<__nv_bfloat16 *>(O_bf16), nullptr,
+                                 static_cast<uint8_t *>(workspace), plan,
+                                 static_cast<cudaStream_t>(stream));
+}
+
 w4a8_status w4a8_linear_acc_i32(const int8_t *Xq, const void *packed, int M, int N, int K,
                                 int group_size, int32_t *acc, void *workspace,
                                 size_t workspace_bytes, void *stream, const w4a8_opts *opts)

@@ -268,6 +268,7 @@ struct LinearPlan {
     int decode_warps; // warps converting codes to INT8: 4, 8 or 16
     int cluster;      // CTAs per cluster: 1, or 2 (each CTA expands half of every code tile for both)
     int debug_wait_ms, debug_skip_load;   // test hooks of w4a8_opts (0 = off)
+    int batched;      // every 128-row tile has its own block of tokens (attention P*V form)
     int kb_per_split; // k-blocks per slice (last slice may be shorter)
     size_t off_counters, off_partials, workspace_bytes;
 };
@@ -286,6 +287,8 @@ int device_sms();
 // launchers (defined in the .cu files, called by api.cu)
 cudaError_t launch_pack(const __half *W, const float *s_in, const BlobLayout &L, float clip,
                         uint8_t *blob, cudaStream_t st);
+cudaError_t launch_pack_transposed(const __half *Wt, const BlobLayout &L, float clip, uint8_t *blob,
+                                   cudaStream_t st);
 cudaError_t launch_unpack(const uint8_t *blob, const BlobLayout &L, uint8_t *codes,
                           float *scales, uint8_t *zeros, cudaStream_t st);
 cudaError_t launch_quantize_act(const __half *X, const float *inv_s, int M, int K, int8_t *Xq,

@@ -122,6 +122,8 @@ struct Params {
     LevelTables lt;
     float unit;          // level unit as a factor of the step: 2^-shift
     unsigned long long wait_ns, drain_ns;   // limits of the bounded waits
+    int batch_rows;      // 0, or M when every 128-row tile has its own [M][K] block of tokens (and
+                         // token steps), stacked in tile order: the attention P*V form
     int skip_load;       // test hook: every producer leaves out the token load of its k-block
                          // number skip_load - 1 (0 = none), so that a wait runs out
 };
@@ -570,6 +572,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             for (int u = unit0; u < P.total_units && ok; u += unit_step) {
                 const int s = u % P.split_k, rest = u / P.split_k;
                 const int tt = (rest / n_tiles) * CL + (int)rank;
+                const int nt_of_unit = rest % n_tiles;
                 const int kb0 = s * P.kb_per_split;
                 const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
@@ -583,7 +586,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     const uint32_t stage = base + st * C::kStageBytes;
                     const uint32_t tok_bar = bar_dec + 8 * st;
                     mbar_arrive_expect_tx(tok_bar, C::kTokBytes + (CL > 1 ? kABytes / CL : 0));
-                    tma_load_2d(stage + C::kTokOff, &tok_map, kb * kTileK, tt * TOK, tok_bar);
+                    tma_load_2d(stage + C::kTokOff, &tok_map, kb * kTileK, nt_of_unit * P.batch_rows + tt * TOK, tok_bar);
                     if (P.prefetch_codes) {
                         // keep the code stream kPrefetchAhead k-blocks ahead of the decode warps
                         while (pf.valid() && pf.it < it + C::kPrefetchAhead) {
@@ -870,7 +873,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 named_bar_sync(1, kEpiThreads);
                 for (int i = et; i < TOK; i += kEpiThreads) {
                     const bool in = tt * TOK + i < P.M;
-                    s_tok[i] = (in && P.tok_scale) ? __ldg(P.tok_scale + tt * TOK + i) : 0.0f;
+                    s_tok[i] = (in && P.tok_scale) ? __ldg(P.tok_scale + nt * P.batch_rows + tt * TOK + i) : 0.0f;
                     s_tz[i] = (in && P.zp.tok_zero) ? __ldg(P.zp.tok_zero + tt * TOK + i) : 0;
                 }
                 named_bar_sync(1, kEpiThreads);
@@ -1285,6 +1288,7 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     if (dw != 4 && dw != 8 && !((dw == 12 || dw == 16) && !grouped)) return false;
     plan->decode_warps = dw;
     plan->cluster = cluster;
+    plan->batched = 0;
     plan->debug_wait_ms = opts ? opts->debug_wait_ms : 0;
     plan->debug_skip_load = opts ? opts->debug_skip_load : 0;
     plan->tok_tile = tok;
@@ -1308,7 +1312,8 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     if (!enc) return W4A8_ERR_CUDA;
     Maps maps;
     memset(&maps, 0, sizeof(maps));
-    const cuuint64_t dims[2] = {(cuuint64_t)L.K, (cuuint64_t)M};
+    // (P*V form: the token blocks of all row tiles are stacked, one after the other)
+    const cuuint64_t dims[2] = {(cuuint64_t)L.K, (cuuint64_t)M * (plan.batched ? L.n_tiles : 1)};
     const cuuint64_t strides[1] = {(cuuint64_t)L.K};
     const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)plan.tok_tile};
     const cuuint32_t estr[2] = {1, 1};
@@ -1356,6 +1361,7 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     P.wait_ns = plan.debug_wait_ms > 0 ? (unsigned long long)plan.debug_wait_ms * 1000000ull : kWaitLimitNs;
     P.drain_ns = plan.debug_wait_ms > 0 ? P.wait_ns : kDrainLimitNs;
     P.skip_load = plan.debug_skip_load;
+    P.batch_rows = plan.batched ? M : 0;
 
     const bool g = L.group != 0;
     switch (plan.tok_tile) {

@@ -284,6 +284,63 @@ pack3_kernel(const __half *__restrict__ W, const float *__restrict__ s_in, BlobL
     }
 }
 
+// Per-output-channel packing of a matrix that arrives transposed, Wt[K][N] (the attention
+// value tensor V[s][h * D + d]: its channels are the outputs, the sequence is the reduction
+// dimension).  A CTA takes 32 consecutive channels n (lane = channel, so a warp reads 64
+// contiguous bytes of a row of Wt); its 8 warps split the k range.
+__global__ void __launch_bounds__(kPackThreads)
+pack_transposed_kernel(const __half *__restrict__ Wt, BlobLayout L, float clip,
+                       uint8_t *__restrict__ blob)
+{
+    __shared__ float s_lo[8][32], s_hi[8][32];
+    __shared__ float s_step[32];
+    __shared__ int s_zero[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n = blockIdx.x * 32 + lane;
+    float *scales = reinterpret_cast<float *>(blob + L.off_scales);
+    uint8_t *zeros = blob + L.off_zeros;
+    uint8_t *codes = blob + L.off_codes;
+    if (blockIdx.x == 0 && threadIdx.x == 0) write_header(blob, L, clip);
+    const bool real = n < L.N;
+    float lo = 0.0f, hi = 0.0f;
+    if (real) {
+        for (int k = warp; k < L.K; k += 8) {
+            const float w = __half2float(Wt[(size_t)k * L.N + n]);
+            if (w < lo) lo = w;
+            if (w > hi) hi = w;
+        }
+    }
+    s_lo[warp][lane] = lo;
+    s_hi[warp][lane] = hi;
+    __syncthreads();
+    if (warp == 0) {
+        for (int w = 1; w < 8; ++w) {
+            if (s_lo[w][lane] < lo) lo = s_lo[w][lane];
+            if (s_hi[w][lane] > hi) hi = s_hi[w][lane];
+        }
+        float s; int z;
+        step_and_zero(lo, hi, clip, s, z);
+        s_step[lane] = s;
+        s_zero[lane] = z;
+        if (n < L.n_pad) { scales[n] = s; zeros[n] = (uint8_t)z; }
+    }
+    __syncthreads();
+    const float s = s_step[lane];
+    const int z = s_zero[lane];
+    float quarter, threeq;
+    special_band(s, L.shift, quarter, threeq);
+    if (n >= L.n_pad) return;
+    for (int k = 2 * warp; k < L.K; k += 16) {
+        uint32_t byte = 0;
+        if (real) {
+            const float w0 = __half2float(Wt[(size_t)k * L.N + n]);
+            const float w1 = __half2float(Wt[(size_t)(k + 1) * L.N + n]);
+            byte = dint4_quantize(w0, s, z, quarter, threeq) | (dint4_quantize(w1, s, z, quarter, threeq) << 4);
+        }
+        codes[code_byte_offset(L, n, k)] = (uint8_t)byte;
+    }
+}
+
 __global__ void unpack_kernel(const uint8_t *__restrict__ blob, BlobLayout L,
                               uint8_t *__restrict__ out_codes, float *__restrict__ out_scales,
                               uint8_t *__restrict__ out_zeros)
@@ -362,6 +419,13 @@ cudaError_t launch_pack(const __half *W, const float *s_in, const BlobLayout &L,
         pack_rows_kernel<<<L.n_pad, kPackThreads, 0, st>>>(W, s_in, L, clip, blob);
     else
         pack_groups_kernel<<<L.n_pad, kPackThreads, 0, st>>>(W, s_in, L, clip, blob);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pack_transposed(const __half *Wt, const BlobLayout &L, float clip, uint8_t *blob,
+                                   cudaStream_t st)
+{
+    pack_transposed_kernel<<<L.n_pad / 32, kPackThreads, 0, st>>>(Wt, L, clip, blob);
     return cudaGetLastError();
 }
 
