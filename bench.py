@@ -825,6 +825,36 @@ def main():
             "per_linear_ms": dict(zip([d["label"] for d in L3], lin3)),
             "per_linear_tops": {d["label"]: 2.0 * M_PREFILL * d["K"] * d["N"] / (t * 1e-3) / 1e12
                                 for d, t in zip(L3, lin3)}}
+        # the gated feed-forward block as two launches per matmul stage: gate and up rows interleaved
+        # in one blob, silu(gate) * up in the epilogue (binary16), quantizer, down projection
+        gate, up, down_l = L3[0], L3[1], L3[2]
+        Wgu = w4a8.interleave_gate_up(torch.from_numpy(layers3[0]["W"]).to(dev), torch.from_numpy(layers3[1]["W"]).to(dev))
+        F3, K3 = gate["N"], gate["K"]
+        packed_gu = w4a8.pack_weights(Wgu, gate["s"], 128)
+        del Wgu
+        ws_gu = w4a8.new_linear_swiglu_workspace(M_PREFILL, F3, K3, 128)
+        Hbuf = torch.empty((M_PREFILL, F3), dtype=torch.float16, device=dev)
+
+        def pass_mlp(it=None):
+            w4a8.quantize_act(gate["X"], gate["inv_s"], out=(gate["Xq"], gate["tok"]))
+            w4a8.linear_swiglu(gate["Xq"], gate["tok"], packed_gu, None, F3, 128, ws_gu, out=Hbuf)
+            w4a8.quantize_act(Hbuf, down_l["inv_s"], out=(down_l["Xq"], down_l["tok"]))
+            w4a8.linear(down_l["Xq"], down_l["tok"], down_l["packed"], down_l["bias"], down_l["N"], 128,
+                        down_l["ws"], out=down_l["Y"])
+        for _ in range(3):
+            pass_mlp()
+        ms_mlp = timed(pass_mlp, 50) / 50
+        w4a8.check_status(ws_gu)
+        ops_mlp = 2.0 * M_PREFILL * K3 * F3 * 3
+        group_leg["gated_mlp_fused"] = {
+            "metric": "w4a8_dint_linear_tops", "value": ops_mlp / (ms_mlp * 1e-3) / 1e12, "unit": "TOPS",
+            "ms_per_pass": ms_mlp,
+            "unfused_linears_ms": lin3[0] + lin3[1] + lin3[2],
+            "note": "llama-7b feed-forward block at M=2048, group-128: quantize_act, linear_swiglu "
+                    "(4096 -> 2 x 11008 with silu(gate) * up in the epilogue), quantize_act, linear "
+                    "(11008 -> 4096); unfused_linears_ms is the sum of the three separate tensor-core "
+                    "launches of the block above (without the unit and without the quantizers)"}
+        del packed_gu, ws_gu, Hbuf
         for d in L3:
             d.clear()
         del L3, layers3

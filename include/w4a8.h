@@ -291,6 +291,24 @@ w4a8_status w4a8_linear_asym(const int8_t *Xq, const float *tok_scale, const int
                              int M, int N, int K, void *Y_bf16, int32_t *acc, void *workspace,
                              size_t workspace_bytes, void *stream, const w4a8_opts *opts);
 
+/* ---- gate and up projections of a gated feed-forward block with the unit in the epilogue ----
+ * In a LLaMA-style block the two projections that read the same quantized input (gate and up)
+ * feed h = silu(gate) * up, which is the next quantized matmul's input ("all matrix
+ * multiplications in the Decoder layer", Appendix A.1): here both run as ONE quantized linear
+ * layer over a weight matrix of 2 F rows in which row 2 i is row i of the gate projection and row
+ * 2 i + 1 row i of the up projection (interleave, then w4a8_pack_weights), and the epilogue
+ * writes h instead of the two BF16 outputs: per element the FP32 value of w4a8_linear before its
+ * BF16 rounding (g for the even row, u for the odd row, bias included), then
+ *   h = (g / (1 + exp(-g))) * u   in FP32, rounded to binary16.
+ * H_f16 [M][F] is what w4a8_quantize_act takes next.  F % 8 == 0.  bias_gate_up [2 F]
+ * interleaved like the rows, or NULL.  workspace >= w4a8_linear_swiglu_workspace_bytes(...),
+ * zero-filled once.  The exponential is the GPU's fast one: results agree with a binary64
+ * evaluation of the formula to one binary16 step. */
+size_t w4a8_linear_swiglu_workspace_bytes(int M, int F, int K, int group_size);
+w4a8_status w4a8_linear_swiglu(const int8_t *Xq, const float *tok_scale, const void *packed_gate_up,
+                               const float *bias_gate_up, int M, int F, int K, int group_size,
+                               void *H_f16, void *workspace, size_t workspace_bytes, void *stream);
+
 /* ---- attention value path: "W4A8V4" (Section 5; Appendix A.1: channel-wise 4-bit Value) ----
  * The product of the attention map and the values, O[t][h][d] = sum_s P[h][t][s] V[s][h][d], with
  * V quantized to dINT4 per channel (h, d) - the dimension along which the partial sums

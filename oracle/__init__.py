@@ -394,6 +394,26 @@ def linear_bits(Xq, tok_scale, codes, scales, zeros, bias, group: int, bits: int
     return acc, Y, wide
 
 
+def linear_swiglu(Xq, tok_scale, codes, scales, zeros, bias=None, group: int = 0):
+    """Gate / up projections (rows interleaved: 2 i gate, 2 i + 1 up) and h = silu(g) * u.
+    Returns (H binary64 [M, F], the layer's FP32 values [M, 2 F])."""
+    Xq = _c(Xq, np.int8)
+    codes = _c(codes, np.uint8)
+    zeros = _c(zeros, np.uint8)
+    scales = _c(scales, np.float32)
+    tok_scale = _c(tok_scale, np.float32)
+    M, N, K, G = _shape(Xq, codes, zeros, group)
+    assert N % 2 == 0
+    if bias is not None:
+        bias = _c(bias, np.float32)
+    H = np.empty((M, N // 2), dtype=np.float64)
+    T = np.empty((M, N), dtype=np.float32)
+    lib().oracle_linear_swiglu(_p(Xq), _p(tok_scale), _p(codes), _p(scales), _p(zeros),
+                               _p(bias) if bias is not None else None, ctypes.c_int(M),
+                               ctypes.c_int(N // 2), ctypes.c_int(K), ctypes.c_int(group), _p(H), _p(T))
+    return H, T
+
+
 def pack_value(V: np.ndarray, clip: float = 1.0):
     """Channel-wise dINT4 quantization of the attention values (Appendix A.1, "W4A8V4"):
     V is [S, H, D] float16; a channel is one (h, d), its Min-Max range is taken over the S

@@ -280,9 +280,11 @@ void oracle_linear_acc_i32(const int8_t *Xq, const uint8_t *codes,
  *   G groups  : u = 0; for g ascending u = fmaf(float(acc_g), 0.5f * s[g][n], u);
  *               t = u * tok_scale[m]
  *   then t = t + bias[n] when bias is given, and Y = bf16(t), nearest-even. */
-void oracle_linear(const int8_t *Xq, const float *tok_scale, const uint8_t *codes,
-                   const float *scales, const uint8_t *zeros, const float *bias,
-                   int M, int N, int K, int group, uint16_t *Y)
+/* The layer's FP32 value t before the BF16 rounding (Y, may be NULL) and, optionally, that
+ * value itself (T32, may be NULL). */
+void oracle_linear_f32(const int8_t *Xq, const float *tok_scale, const uint8_t *codes,
+                       const float *scales, const uint8_t *zeros, const float *bias,
+                       int M, int N, int K, int group, uint16_t *Y, float *T32)
 {
     const int glen = group ? group : K;
     const int G = K / glen;
@@ -309,9 +311,36 @@ void oracle_linear(const int8_t *Xq, const float *tok_scale, const uint8_t *code
             }
             if (G != 1) t = u * tok_scale[m];
             if (bias) t = t + bias[n];
-            Y[(size_t)m * N + n] = float_to_bf16_bits(t);
+            if (Y) Y[(size_t)m * N + n] = float_to_bf16_bits(t);
+            if (T32) T32[(size_t)m * N + n] = t;
         }
     }
+}
+
+void oracle_linear(const int8_t *Xq, const float *tok_scale, const uint8_t *codes,
+                   const float *scales, const uint8_t *zeros, const float *bias,
+                   int M, int N, int K, int group, uint16_t *Y)
+{
+    oracle_linear_f32(Xq, tok_scale, codes, scales, zeros, bias, M, N, K, group, Y, NULL);
+}
+
+/* Gate and up projections with the gated unit h = silu(g) * u between them and the next
+ * quantized matmul ("all matrix multiplications in the Decoder layer", Appendix A.1; the unit
+ * itself is the LLaMA block's, not the paper's).  Row 2 i of the weight matrix is row i of the
+ * gate projection, row 2 i + 1 row i of the up projection; g and u are the layer's FP32 values
+ * (bias included) before any BF16 rounding; h = (g / (1 + exp(-g))) * u is evaluated in binary64
+ * on those FP32 values (H64, [M][F]) and rounded once to binary16 (H16 bits, may be NULL). */
+void oracle_linear_swiglu(const int8_t *Xq, const float *tok_scale, const uint8_t *codes,
+                          const float *scales, const uint8_t *zeros, const float *bias, int M,
+                          int F, int K, int group, double *H64, float *T32)
+{
+    oracle_linear_f32(Xq, tok_scale, codes, scales, zeros, bias, M, 2 * F, K, group, NULL, T32);
+    for (int m = 0; m < M; ++m)
+        for (int f = 0; f < F; ++f) {
+            const double g = (double)T32[(size_t)m * 2 * F + 2 * f];
+            const double u = (double)T32[(size_t)m * 2 * F + 2 * f + 1];
+            H64[(size_t)m * F + f] = g / (1.0 + exp(-g)) * u;
+        }
 }
 
 /* The same value in binary64, not rounded to BF16: the tolerance reference. */

@@ -32,6 +32,7 @@ EXPORTS = (
     "w4a8_quantize_linear", "w4a8_quantize_linear_workspace_bytes", "w4a8_linear_plan", "w4a8_norm_quantize_act",
     "w4a8_packed_bytes_bits", "w4a8_pack_weights_bits", "w4a8_unpack_codes_bits", "w4a8_dint_table_bits",
     "w4a8_pack_value", "w4a8_attn_pv", "w4a8_attn_pv_workspace_bytes",
+    "w4a8_linear_swiglu", "w4a8_linear_swiglu_workspace_bytes",
 )
 
 
@@ -90,6 +91,10 @@ def _load() -> ctypes.CDLL:
     lib.w4a8_unpack_codes_bits.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp]
     lib.w4a8_dint_table_bits.restype = None
     lib.w4a8_dint_table_bits.argtypes = [ci, ci, ci, vp]
+    lib.w4a8_linear_swiglu_workspace_bytes.restype = sz
+    lib.w4a8_linear_swiglu_workspace_bytes.argtypes = [ci, ci, ci, ci]
+    lib.w4a8_linear_swiglu.restype = ci
+    lib.w4a8_linear_swiglu.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, vp]
     lib.w4a8_pack_value.restype = ci
     lib.w4a8_pack_value.argtypes = [vp, ci, ci, ci, cf, vp, sz, vp]
     lib.w4a8_attn_pv_workspace_bytes.restype = sz
@@ -344,6 +349,36 @@ def linear_asym(Xq, tok_scale, tok_zero, packed, rowsum, bias, N: int, workspace
                               ctypes.byref(opts) if opts is not None else None)
     _check(st, "w4a8_linear_asym")
     return (out, acc) if want_acc else out
+
+
+def interleave_gate_up(Wg, Wu):
+    """[F, K] gate and up weights -> [2 F, K] with row 2 i = gate row i, row 2 i + 1 = up row i."""
+    F, K = Wg.shape
+    return torch.stack((Wg, Wu), dim=1).reshape(2 * F, K).contiguous()
+
+
+def new_linear_swiglu_workspace(M: int, F: int, K: int, group: int = 0, device="cuda"):
+    nbytes = int(lib.w4a8_linear_swiglu_workspace_bytes(M, F, K, group))
+    if nbytes == 0:
+        raise W4A8Error(2, "w4a8_linear_swiglu_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    workspace_init(ws)
+    return ws
+
+
+def linear_swiglu(Xq, tok_scale, packed_gate_up, bias_gate_up, F: int, group: int, workspace, out=None):
+    """Gate and up projections (rows interleaved in one blob) with silu(gate) * up in the epilogue:
+    returns H [M, F] float16."""
+    Xq = _dev(Xq, torch.int8, "Xq")
+    tok_scale = _dev(tok_scale, torch.float32, "tok_scale")
+    bias_gate_up = _dev(bias_gate_up, torch.float32, "bias_gate_up")
+    M, K = Xq.shape
+    if out is None:
+        out = torch.empty((M, F), dtype=torch.float16, device=Xq.device)
+    _check(lib.w4a8_linear_swiglu(_ptr(Xq), _ptr(tok_scale), _ptr(packed_gate_up), _ptr(bias_gate_up), M, F,
+                                  K, group, _ptr(out), _ptr(workspace), workspace.numel(), _stream()),
+           "w4a8_linear_swiglu")
+    return out
 
 
 def pack_value(V, clip: float = 1.0, out=None):

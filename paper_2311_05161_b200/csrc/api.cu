@@ -327,6 +327,46 @@ w4a8_status w4a8_quantize_linear(const void *X_f16, const float *inv_s_in, const
                               static_cast<const __half *>(X_f16), inv_s_in);
 }
 
+// ---- gate / up projections with the gated unit in the epilogue ----
+static bool swiglu_plan(int M, int F, int K, int group, BlobLayout *L, LinearPlan *plan)
+{
+    if (F < 8 || F % 8 != 0 || M < 1 || !shape_ok(2 * F, K, group)) return false;   // (bulk stores: rows of 16-byte multiples)
+    *L = make_layout(2 * F, K, group);
+    w4a8_opts o = {};
+    o.path = W4A8_PATH_TCGEN05;
+    o.split_k = 1;                      // the epilogue pairs rows inside one accumulator tile
+    if (!make_plan(M, *L, &o, plan)) return false;
+    plan->swiglu = 1;
+    return true;
+}
+
+size_t w4a8_linear_swiglu_workspace_bytes(int M, int F, int K, int group_size)
+{
+    BlobLayout L;
+    LinearPlan plan;
+    return swiglu_plan(M, F, K, group_size, &L, &plan) ? plan.workspace_bytes : 0;
+}
+
+w4a8_status w4a8_linear_swiglu(const int8_t *Xq, const float *tok_scale, const void *packed_gate_up,
+                               const float *bias_gate_up, int M, int F, int K, int group_size,
+                               void *H_f16, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!Xq || !tok_scale || !packed_gate_up || !H_f16 || !workspace) return W4A8_ERR_NULL;
+    BlobLayout L;
+    LinearPlan plan;
+    if (!swiglu_plan(M, F, K, group_size, &L, &plan) || !depth_ok(K, 1, 127)) return W4A8_ERR_SHAPE;
+    if (!aligned(Xq, 16) || !aligned(tok_scale, 4) || !aligned(bias_gate_up, 4) || !aligned(H_f16, 16) ||
+        !aligned(packed_gate_up, 256) || !aligned(workspace, 256))
+        return W4A8_ERR_ALIGN;
+    if (workspace_bytes < plan.workspace_bytes) return W4A8_ERR_BUFFER_TOO_SMALL;
+    const w4a8_status arch = check_arch();
+    if (arch != W4A8_OK) return arch;
+    return launch_linear_tcgen05(Xq, tok_scale, static_cast<const uint8_t *>(packed_gate_up), L,
+                                 bias_gate_up, M, static_cast<__nv_bfloat16 *>(H_f16), nullptr,
+                                 static_cast<uint8_t *>(workspace), plan,
+                                 static_cast<cudaStream_t>(stream));
+}
+
 // ---- attention value path (W4A8V4): P * V with channel-wise dINT4 values ----
 w4a8_status w4a8_pack_value(const void *V_f16, int S, int H, int D, float clip, void *packed,
                             size_t packed_bytes, void *stream)

@@ -268,6 +268,7 @@ struct LinearPlan {
     int decode_warps; // warps converting codes to INT8: 4, 8 or 16
     int cluster;      // CTAs per cluster: 1, or 2 (each CTA expands half of every code tile for both)
     int debug_wait_ms, debug_skip_load;   // test hooks of w4a8_opts (0 = off)
+    int swiglu;       // gated-unit epilogue (see w4a8_linear_swiglu)
     int batched;      // every 128-row tile has its own block of tokens (attention P*V form)
     int kb_per_split; // k-blocks per slice (last slice may be shorter)
     size_t off_counters, off_partials, workspace_bytes;

@@ -33,6 +33,7 @@ namespace w4a8 {
 namespace {
 
 constexpr int kFirstDecodeWarp = 2;
+constexpr int kSwigluVariant = 5;
 constexpr int kMaxDevices = 64;
 constexpr int kABytes = kTileN * kTileK;            // decoded INT8 tile, 16 KiB
 constexpr int kDefaultTeamWarps = 4;               // warps per decode team
@@ -122,6 +123,7 @@ struct Params {
     LevelTables lt;
     float unit;          // level unit as a factor of the step: 2^-shift
     unsigned long long wait_ns, drain_ns;   // limits of the bounded waits
+    int swiglu;          // gated-unit epilogue: Y is [M][N / 2] binary16, silu(row 2i) * row 2i + 1
     int batch_rows;      // 0, or M when every 128-row tile has its own [M][K] block of tokens (and
                          // token steps), stacked in tile order: the attention P*V form
     int skip_load;       // test hook: every producer leaves out the token load of its k-block
@@ -483,12 +485,17 @@ __device__ __forceinline__ void decode8(uint32_t w, const uint32_t (&t)[4], uint
 }
 
 // --------------------------------------------------------------------------- the kernel
-template <int TOK, bool GROUPED, int DW, int CL, int BITS>
+// VARIANT: 4 = 4-bit codes, 3 = 3-bit codes, kSwigluVariant = 4-bit codes with the gated-unit
+// epilogue (rows 2i / 2i + 1 of the weight matrix are feature i of the gate / up projection;
+// the output is silu(gate) * up in binary16, half as wide as the weight matrix is tall)
+template <int TOK, bool GROUPED, int DW, int CL, int VARIANT>
 __global__ void __launch_bounds__(Cfg<TOK, GROUPED, DW, CL>::kThreads, 1)
 linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                       const __grid_constant__ CUtensorMap y_map, const Params P)
 {
     using C = Cfg<TOK, GROUPED, DW, CL>;
+    constexpr int BITS = VARIANT == 3 ? 3 : 4;
+    constexpr bool SWIGLU = VARIANT == kSwigluVariant;
     constexpr int kFirstEpiWarp = C::kFirstEpiWarp;
     constexpr int S = C::kStages;
     extern __shared__ uint8_t smem_raw[];
@@ -843,14 +850,28 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             const uint32_t sbuf = stores % C::kStageBufs;
             if (elected) bulk_wait_read<C::kStageBufs - 1>();   // the buffer's last store has been read
             named_bar_sync(group_bar, 128);
-            __nv_bfloat16 *dst = stg + sbuf * (C::kChunk * kTileN) + f;
+            if constexpr (SWIGLU) {
+                // lanes 2i and 2i + 1 hold the gate and the up value of feature i: the even
+                // lane takes its neighbour's value and writes silu(gate) * up, 64 features per
+                // token in the staging buffer
+                __half *dst = reinterpret_cast<__half *>(stg + sbuf * (C::kChunk * kTileN)) + (f >> 1);
 #pragma unroll
-            for (int j = 0; j < C::kChunk; ++j) dst[j * kTileN] = __float2bfloat16_rn(tv[j]);
+                for (int j = 0; j < C::kChunk; ++j) {
+                    const float up = __shfl_xor_sync(0xffffffffu, tv[j], 1);
+                    const float gate = tv[j];
+                    const float h = __fmul_rn(__fdiv_rn(gate, __fadd_rn(1.0f, __expf(-gate))), up);
+                    if ((lane & 1) == 0) dst[j * (kTileN / 2)] = __float2half_rn(h);
+                }
+            } else {
+                __nv_bfloat16 *dst = stg + sbuf * (C::kChunk * kTileN) + f;
+#pragma unroll
+                for (int j = 0; j < C::kChunk; ++j) dst[j * kTileN] = __float2bfloat16_rn(tv[j]);
+            }
             fence_proxy_async();
             named_bar_sync(group_bar, 128);
             if (elected) {
-                tma_store_2d(&y_map, smem_u32(stg + sbuf * (C::kChunk * kTileN)), nt * kTileN,
-                             tok_row);
+                tma_store_2d(&y_map, smem_u32(stg + sbuf * (C::kChunk * kTileN)),
+                             SWIGLU ? nt * (kTileN / 2) : nt * kTileN, tok_row);
                 bulk_commit();
             }
             ++stores;
@@ -1143,7 +1164,7 @@ struct Maps {
 
 // Clusters of CL CTAs of this kernel that the current device can hold at once (one CTA per
 // SM); asked once per kernel instance and device.
-template <int TOK, bool GROUPED, int DW, int CL, int BITS>
+template <int TOK, bool GROUPED, int DW, int CL, int VARIANT>
 int resident_clusters()
 {
     using C = Cfg<TOK, GROUPED, DW, CL>;
@@ -1152,7 +1173,7 @@ int resident_clusters()
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
     int n = cached[dev].load(std::memory_order_acquire);
     if (n > 0) return n;
-    auto kern = linear_tcgen05_kernel<TOK, GROUPED, DW, CL, BITS>;
+    auto kern = linear_tcgen05_kernel<TOK, GROUPED, DW, CL, VARIANT>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) !=
         cudaSuccess)
         return 0;
@@ -1179,12 +1200,12 @@ int resident_clusters()
     return n;
 }
 
-template <int TOK, bool GROUPED, int DW, int CL, int BITS = 4>
+template <int TOK, bool GROUPED, int DW, int CL, int VARIANT = 4>
 w4a8_status launch_cl(const Maps &maps, const Params &P, cudaStream_t st)
 {
     using C = Cfg<TOK, GROUPED, DW, CL>;
-    auto kern = linear_tcgen05_kernel<TOK, GROUPED, DW, CL, BITS>;
-    const int resident = resident_clusters<TOK, GROUPED, DW, CL, BITS>();   // also sizes the kernel's shared memory
+    auto kern = linear_tcgen05_kernel<TOK, GROUPED, DW, CL, VARIANT>;
+    const int resident = resident_clusters<TOK, GROUPED, DW, CL, VARIANT>();   // also sizes the kernel's shared memory
     if (resident < 1) return W4A8_ERR_CUDA;
     const int clusters = P.total_units < resident ? P.total_units : resident;
     const cudaError_t e =
@@ -1209,6 +1230,11 @@ w4a8_status launch_one(const Maps &maps, const Params &P, int dw, int cluster, c
 {
     // 3-bit codes: eight decode warps, no clusters (make_plan picks nothing else)
     if (P.L.bits == 3) return dw == 8 && cluster == 1 ? launch_cl<TOK, GROUPED, 8, 1, 3>(maps, P, st) : W4A8_ERR_SHAPE;
+    // gated-unit epilogue: the default warps, no clusters, no K split (make_plan picks nothing else)
+    if (P.swiglu) {
+        if (cluster != 1 || P.split_k != 1 || dw != (GROUPED ? 8 : 16)) return W4A8_ERR_SHAPE;
+        return launch_cl<TOK, GROUPED, GROUPED ? 8 : 16, 1, kSwigluVariant>(maps, P, st);
+    }
     if (dw == 4) return launch_dw<TOK, GROUPED, 4>(maps, P, cluster, st);
     if (dw == 8) return launch_dw<TOK, GROUPED, 8>(maps, P, cluster, st);
     if (dw == 12 && !GROUPED) return launch_dw<TOK, false, 12>(maps, P, cluster, st);
@@ -1289,6 +1315,7 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     plan->decode_warps = dw;
     plan->cluster = cluster;
     plan->batched = 0;
+    plan->swiglu = 0;
     plan->debug_wait_ms = opts ? opts->debug_wait_ms : 0;
     plan->debug_skip_load = opts ? opts->debug_skip_load : 0;
     plan->tok_tile = tok;
@@ -1323,11 +1350,14 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
         return W4A8_ERR_CUDA;
     if (Y && plan.split_k == 1) {
         // output tiles of 128 features x 16 or 32 tokens; parts beyond N or M are clipped
-        const cuuint64_t ydims[2] = {(cuuint64_t)L.N, (cuuint64_t)M};
-        const cuuint64_t ystrides[1] = {(cuuint64_t)L.N * 2};
+        // (gated-unit epilogue: half as many features per tile and per row, binary16)
+        const int width = plan.swiglu ? L.N / 2 : L.N, tile_w = plan.swiglu ? kTileN / 2 : kTileN;
+        const cuuint64_t ydims[2] = {(cuuint64_t)width, (cuuint64_t)M};
+        const cuuint64_t ystrides[1] = {(cuuint64_t)width * 2};
         for (int rows = 16; rows <= 32; rows += 16) {
-            const cuuint32_t ybox[2] = {(cuuint32_t)kTileN, (cuuint32_t)rows};
-            if (enc(rows == 16 ? &maps.y16 : &maps.y32, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y,
+            const cuuint32_t ybox[2] = {(cuuint32_t)tile_w, (cuuint32_t)rows};
+            if (enc(rows == 16 ? &maps.y16 : &maps.y32,
+                    plan.swiglu ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y,
                     ydims, ystrides, ybox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -1362,6 +1392,7 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     P.drain_ns = plan.debug_wait_ms > 0 ? P.wait_ns : kDrainLimitNs;
     P.skip_load = plan.debug_skip_load;
     P.batch_rows = plan.batched ? M : 0;
+    P.swiglu = plan.swiglu;
 
     const bool g = L.group != 0;
     switch (plan.tok_tile) {
