@@ -296,6 +296,31 @@ def linear_asym(Q, tok_scale, tok_zero, codes, scales, zeros, bias=None, wide: b
     return (Y, W) if wide else Y
 
 
+def linear_asym_group(Q, tok_scale, tok_zero, codes, scales, zeros, bias, group: int):
+    """Asymmetric activations with group-wise weight steps: (acc int64 [G, M, N], Y BF16 bits
+    [M, N], Y binary64 [M, N])."""
+    Q = _c(Q, np.uint8)
+    tok_scale = _c(tok_scale, np.float32)
+    tok_zero = _c(tok_zero, np.int32)
+    codes = _c(codes, np.uint8)
+    zeros = _c(zeros, np.uint8)
+    scales = _c(scales, np.float32)
+    M, K = Q.shape
+    N = codes.shape[0]
+    G = K // group
+    assert codes.shape == (N, K // 2) and zeros.shape == (G, N) and scales.shape == (G, N)
+    if bias is not None:
+        bias = _c(bias, np.float32)
+    acc = np.empty((G, M, N), dtype=np.int64)
+    Y = np.empty((M, N), dtype=np.uint16)
+    wide = np.empty((M, N), dtype=np.float64)
+    lib().oracle_linear_asym_group(_p(Q), _p(tok_scale), _p(tok_zero), _p(codes), _p(scales), _p(zeros),
+                                   _p(bias) if bias is not None else None, ctypes.c_int(M),
+                                   ctypes.c_int(N), ctypes.c_int(K), ctypes.c_int(group), _p(acc),
+                                   _p(Y), _p(wide))
+    return acc, Y, wide
+
+
 # ---- special value s / 2^shift (App. A.5): shift = 1 is Eq. 5 / Eq. 6 --------------------
 
 def dint_quantize_fmt(x: float, s: float, z: int, shift: int, b: int = 4) -> int:

@@ -468,6 +468,45 @@ void oracle_linear_asym(const uint8_t *Q, const float *tok_scale, const int32_t 
     }
 }
 
+/* The same layer with group-wise weight steps (128 consecutive k share a step and a
+ * zero-point): the token's zero-point leaves every group's integer sum before that sum is
+ * scaled, acc_g = sum_{k in g} (Q - zx) * t2, then the FP32 accumulation over the groups of
+ * oracle_linear: u = fmaf(float(acc_g), 0.5 s_g, u), y = u * tok_scale (+ bias).  acc
+ * ([G][M][N], may be NULL), Y (BF16 bits, may be NULL), wide (binary64, may be NULL). */
+void oracle_linear_asym_group(const uint8_t *Q, const float *tok_scale, const int32_t *tok_zero,
+                              const uint8_t *codes, const float *scales, const uint8_t *zeros,
+                              const float *bias, int M, int N, int K, int group, int64_t *acc,
+                              uint16_t *Y, double *wide)
+{
+    const int G = K / group;
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        for (int m = 0; m < M; ++m) {
+            float u = 0.0f;
+            double w = 0.0;
+            for (int g = 0; g < G; ++g) {
+                int8_t t2[16];
+                oracle_dint_table2(zeros[(size_t)g * N + n], 4, t2);
+                int32_t sum = 0;
+                for (int k = g * group; k < (g + 1) * group; ++k) {
+                    const uint8_t byte = codes[(size_t)n * (K / 2) + k / 2];
+                    const int code = (k & 1) ? (byte >> 4) : (byte & 15);
+                    sum += ((int32_t)Q[(size_t)m * K + k] - tok_zero[m]) * (int32_t)t2[code];
+                }
+                if (acc) acc[((size_t)g * M + m) * N + n] = sum;
+                const float h = 0.5f * scales[(size_t)g * N + n];
+                u = fmaf((float)sum, h, u);
+                w += (double)sum * (double)h;
+            }
+            float t = u * tok_scale[m];
+            w *= (double)tok_scale[m];
+            if (bias) { t = t + bias[n]; w += (double)bias[n]; }
+            if (Y) Y[(size_t)m * N + n] = float_to_bf16_bits(t);
+            if (wide) wide[(size_t)m * N + n] = w;
+        }
+    }
+}
+
 /* ------------------------------------------------------------------------- */
 /* other special values: c = s / 2^j (App. A.5 sweeps c/s = 0.5, 0.25, 0.125)  */
 /* ------------------------------------------------------------------------- */

@@ -187,3 +187,37 @@ def test_output_against_float64_and_real_matmul():
     Y0 = oracle.linear_asym(Q, step, np.zeros_like(zx), codes, scales, zeros, bias)
     got0 = oracle.bf16_bits_to_float(Y0).astype(np.float64)
     assert np.linalg.norm(got0 - real) / np.linalg.norm(real) > 3 * rel
+
+
+def test_group_wise_weights_with_asymmetric_activations():
+    """Group-128 steps: per group the integer sum of (Q - zx) * level by numpy, the real-valued
+    meaning "dequantize both operands, multiply", and the one-group case equal to the
+    per-channel function."""
+    rng = np.random.default_rng(21)
+    M, N, K, group = 5, 24, 384, 128
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float16)
+    X = (rng.standard_normal((M, K)) + 1.5).astype(np.float16)
+    bias = (rng.standard_normal(N) * 0.1).astype(np.float32)
+    codes, scales, zeros = oracle.pack_weights(W, None, group)
+    Q, step, zx = oracle.quantize_act_asym(X)
+    acc, Y, wide = oracle.linear_asym_group(Q, step, zx, codes, scales, zeros, bias, group)
+    c = np.empty((N, K), dtype=np.int64)
+    c[:, 0::2], c[:, 1::2] = codes & 15, codes >> 4
+    zf = np.repeat(zeros.T.astype(np.int64), group, axis=1)
+    lv = np.where(c == 14, 1, np.where(c == 15, -1, 2 * (c - zf)))
+    A = Q.astype(np.int64) - zx.astype(np.int64)[:, None]
+    want = np.stack([A[:, g * group:(g + 1) * group] @ lv[:, g * group:(g + 1) * group].T for g in range(K // group)])
+    assert np.array_equal(acc, want)
+    sf = np.repeat(scales.T.astype(np.float64), group, axis=1)
+    deq_w = lv * sf / 2
+    deq_x = A * step.astype(np.float64)[:, None]
+    assert np.allclose(wide, deq_x @ deq_w.T + bias, rtol=1e-9, atol=1e-12)
+    got = oracle.bf16_bits_to_float(Y).astype(np.float64)
+    assert np.all(np.abs(got - wide) <= np.abs(wide) * 2.0 ** -8 + 1e-6)
+    # one group covering all of K is the per-channel layer (same integer, one scaling order apart)
+    c1, s1, z1 = oracle.pack_weights(W[:, :128], None, 128)
+    Q1, st1, zx1 = oracle.quantize_act_asym(X[:, :128])
+    a1, _, w1 = oracle.linear_asym_group(Q1, st1, zx1, c1, s1, z1, bias, 128)
+    assert np.array_equal(a1[0], oracle.linear_asym_acc(Q1, zx1, c1, z1))
+    _, w0 = oracle.linear_asym(Q1, st1, zx1, c1, s1, z1, bias, wide=True)
+    assert np.allclose(w1, w0, rtol=1e-12)
