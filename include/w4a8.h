@@ -331,6 +331,18 @@ w4a8_status w4a8_attn_pv(const int8_t *Pq, const float *p_scale, const void *pac
                          int H, int D, void *O_bf16, void *workspace, size_t workspace_bytes,
                          void *stream);
 
+/* w4a8_linear_asym for any group_size: with group_size 128 the token's zero-point leaves every
+ * group's integer sum before that sum is scaled,
+ *   acc_g[m][n] = sum_{k in g} Xq[m][k] * t2(code[n][k]) - tok_zero[m] * rowsum[g][n],
+ *   y = (sum_g float(acc_g) * (0.5 * step[g][n])) * tok_scale[m] + bias[n],
+ * rowsum [G][N] as written by w4a8_weight_rowsum with the same group_size; acc, if given, is
+ * [G][M][N].  (The paper's W4A8 uses per-channel steps; its group-128 results are weight-only.) */
+w4a8_status w4a8_linear_asym_group(const int8_t *Xq, const float *tok_scale, const int32_t *tok_zero,
+                                   const void *packed, const int32_t *rowsum, const float *bias,
+                                   int M, int N, int K, int group_size, void *Y_bf16, int32_t *acc,
+                                   void *workspace, size_t workspace_bytes, void *stream,
+                                   const w4a8_opts *opts);
+
 /* Test export: the INT32 accumulators of the contraction, acc [G][M][N], before any
  * rescale (Eq. 6 in units of step/2).  Uses the same kernels as w4a8_linear_ex. */
 w4a8_status w4a8_linear_acc_i32(const int8_t *Xq, const void *packed, int M, int N, int K,

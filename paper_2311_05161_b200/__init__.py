@@ -13,5 +13,5 @@ from .binding import (  # noqa: F401
     quantize_linear, quantize_linear_workspace_bytes, new_quantize_linear_workspace, linear_plan,
     norm_quantize_act, NORM_RMS, NORM_LAYER, dint_table,
     pack_value, attn_pv, new_attn_pv_workspace,
-    interleave_gate_up, linear_swiglu, new_linear_swiglu_workspace,
+    interleave_gate_up, linear_swiglu, new_linear_swiglu_workspace, linear_asym_group,
 )

@@ -32,7 +32,7 @@ EXPORTS = (
     "w4a8_quantize_linear", "w4a8_quantize_linear_workspace_bytes", "w4a8_linear_plan", "w4a8_norm_quantize_act",
     "w4a8_packed_bytes_bits", "w4a8_pack_weights_bits", "w4a8_unpack_codes_bits", "w4a8_dint_table_bits",
     "w4a8_pack_value", "w4a8_attn_pv", "w4a8_attn_pv_workspace_bytes",
-    "w4a8_linear_swiglu", "w4a8_linear_swiglu_workspace_bytes",
+    "w4a8_linear_swiglu", "w4a8_linear_swiglu_workspace_bytes", "w4a8_linear_asym_group",
 )
 
 
@@ -109,6 +109,8 @@ def _load() -> ctypes.CDLL:
     lib.w4a8_weight_rowsum.argtypes = [vp, ci, ci, ci, vp, vp]
     lib.w4a8_linear_asym.restype = ci
     lib.w4a8_linear_asym.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, vp, vp, vp, sz, vp, op]
+    lib.w4a8_linear_asym_group.restype = ci
+    lib.w4a8_linear_asym_group.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, vp, sz, vp, op]
     lib.w4a8_linear_acc_i32.restype = ci
     lib.w4a8_linear_acc_i32.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, sz, vp, op]
     lib.w4a8_unpack_codes.restype = ci
@@ -328,6 +330,28 @@ def weight_rowsum(packed, N: int, K: int, group: int = 0):
     _check(lib.w4a8_weight_rowsum(_ptr(packed), N, K, group, _ptr(out), _stream()),
            "w4a8_weight_rowsum")
     return out
+
+
+def linear_asym_group(Xq, tok_scale, tok_zero, packed, rowsum, bias, N: int, group: int, workspace,
+                      opts: Opts | None = None, out=None, want_acc: bool = False):
+    """linear_asym for group-wise weight steps: rowsum is [G, N]; returns Y [M, N] bfloat16, or
+    (Y, acc [G, M, N] int32) with `want_acc`."""
+    Xq = _dev(Xq, torch.int8, "Xq")
+    tok_scale = _dev(tok_scale, torch.float32, "tok_scale")
+    tok_zero = _dev(tok_zero, torch.int32, "tok_zero")
+    rowsum = _dev(rowsum, torch.int32, "rowsum")
+    bias = _dev(bias, torch.float32, "bias")
+    M, K = Xq.shape
+    G = K // group if group else 1
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=Xq.device)
+    acc = torch.empty((G, M, N), dtype=torch.int32, device=Xq.device) if want_acc else None
+    st = lib.w4a8_linear_asym_group(_ptr(Xq), _ptr(tok_scale), _ptr(tok_zero), _ptr(packed), _ptr(rowsum),
+                                    _ptr(bias), M, N, K, group, _ptr(out), _ptr(acc), _ptr(workspace),
+                                    workspace.numel(), _stream(),
+                                    ctypes.byref(opts) if opts is not None else None)
+    _check(st, "w4a8_linear_asym_group")
+    return (out, acc) if want_acc else out
 
 
 def linear_asym(Xq, tok_scale, tok_zero, packed, rowsum, bias, N: int, workspace,

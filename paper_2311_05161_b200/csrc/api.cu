@@ -474,6 +474,21 @@ w4a8_status w4a8_linear_asym(const int8_t *Xq, const float *tok_scale, const int
                          workspace_bytes, stream, opts, zp);
 }
 
+w4a8_status w4a8_linear_asym_group(const int8_t *Xq, const float *tok_scale, const int32_t *tok_zero,
+                                   const void *packed, const int32_t *rowsum, const float *bias,
+                                   int M, int N, int K, int group_size, void *Y_bf16, int32_t *acc,
+                                   void *workspace, size_t workspace_bytes, void *stream,
+                                   const w4a8_opts *opts)
+{
+    if (!tok_zero || !rowsum) return W4A8_ERR_NULL;
+    if (!aligned(tok_zero, 4) || !aligned(rowsum, 4)) return W4A8_ERR_ALIGN;
+    ZeroPoint zp;
+    zp.tok_zero = tok_zero;
+    zp.rowsum = rowsum;
+    return linear_common(Xq, tok_scale, packed, bias, M, N, K, group_size, Y_bf16, acc, workspace,
+                         workspace_bytes, stream, opts, zp);
+}
+
 w4a8_status w4a8_unpack_codes(const void *packed, int N, int K, int group_size, uint8_t *codes,
                               float *scales, uint8_t *zeros, void *stream)
 {

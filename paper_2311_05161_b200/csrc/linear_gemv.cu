@@ -358,8 +358,11 @@ linear_gemv_kernel(const GemvParams P)
                 }
                 if (GROUPED) {
                     const float h = __fmul_rn(P.unit, P.scales[(size_t)kb * P.L.n_pad + n]);
+                    // asymmetric activations: the token's zero-point times this group's level sum
+                    const int rs = (P.zp.tok_zero && n < P.L.N) ? P.zp.rowsum[(size_t)kb * P.L.N + n] : 0;
 #pragma unroll
                     for (int m = 0; m < MT; ++m) {
+                        if (P.zp.tok_zero && m < P.M) acc[m] -= P.zp.tok_zero[m] * rs;
                         usum[m] = fmaf((float)acc[m], h, usum[m]);
                         if (P.acc_out && m < P.M && n < P.L.N)
                             P.acc_out[((size_t)kb * P.M + m) * P.L.N + n] = acc[m];
@@ -563,8 +566,10 @@ linear_gemv_rows_kernel(const GemvParams P)
         }
         if (GROUPED) {
             const float h = __fmul_rn(P.unit, P.scales[(size_t)kbi * P.L.n_pad + n]);
+            const int rs = (P.zp.tok_zero && n < P.L.N) ? P.zp.rowsum[(size_t)kbi * P.L.N + n] : 0;
 #pragma unroll
             for (int m = 0; m < MT; ++m) {
+                if (P.zp.tok_zero && m < P.M) acc[m] -= P.zp.tok_zero[m] * rs;
                 usum[m] = fmaf((float)acc[m], h, usum[m]);
                 if (P.acc_out && m < P.M && n < P.L.N)
                     P.acc_out[((size_t)kbi * P.M + m) * P.L.N + n] = acc[m];

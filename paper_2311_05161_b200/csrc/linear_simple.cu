@@ -49,6 +49,7 @@ linear_simple_kernel(const int8_t *__restrict__ Xq, const float *__restrict__ to
             }
         }
         if (grouped && n < L.N) {
+            if (zp.tok_zero) acc -= zp.tok_zero[m] * zp.rowsum[(size_t)kb * L.N + n];
             if (acc_out) acc_out[((size_t)kb * M + m) * L.N + n] = acc;
             u = fmaf((float)acc, __fmul_rn(level_unit(L.shift), scales[(size_t)kb * L.n_pad + n]), u);
         }

@@ -1014,11 +1014,18 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 // the next group's step is loaded one k-block ahead and only touched when used,
                 // so the warp never stalls on that load
                 float step_next = P.scales[(size_t)kb0 * P.L.n_pad + n];
+                // asymmetric activations: the group's level sum of this row, one k-block ahead too
+                const bool asym = P.zp.tok_zero != nullptr;
+                int rs_next = (asym && n_ok) ? __ldg(P.zp.rowsum + (size_t)kb0 * P.L.N + n) : 0;
                 constexpr int kAcc = 16;          // columns per tensor-memory load while accumulating
                 for (int kb = kb0; kb < kb1; ++kb) {
                     const uint32_t h_bits = __float_as_uint(__fmul_rn(P.unit, step_next));
                     const uint64_t h2 = pack_f32x2(h_bits, h_bits);
-                    if (kb + 1 < kb1) step_next = P.scales[(size_t)(kb + 1) * P.L.n_pad + n];
+                    const int rs = rs_next;
+                    if (kb + 1 < kb1) {
+                        step_next = P.scales[(size_t)(kb + 1) * P.L.n_pad + n];
+                        if (asym && n_ok) rs_next = __ldg(P.zp.rowsum + (size_t)(kb + 1) * P.L.N + n);
+                    }
                     const uint32_t buf = phase % NB;
                     ok = wait_bounded(bar_acc_full + 8 * buf, (phase / NB) & 1u, ctl, P.sb, 41);
                     ok = __all_sync(0xffffffffu, ok);
@@ -1035,6 +1042,13 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                             tc_fence_before();
                             __syncwarp();
                             if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+                        }
+                        if (asym) {
+                            // the token's zero-point times the group's level sum leaves the
+                            // integer partial before it is scaled
+#pragma unroll
+                            for (int j = 0; j < kAcc; ++j)
+                                v[j] = (uint32_t)((int)v[j] - s_tz[col0 + c + j] * rs);
                         }
 #pragma unroll
                         for (int j = 0; j < kAcc; j += 2) {

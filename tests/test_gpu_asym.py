@@ -174,3 +174,44 @@ def test_full_size_opt_6_7b_shapes_sampled(shape_index, M):
     rows = np.unique(np.concatenate([[0, 127, 128, N - 1], rng.choice(N, 60, replace=False)]))
     toks = np.unique(np.concatenate([[0, M - 1], rng.choice(M, min(M, 24), replace=False)]))
     check(lay, Y[np.ix_(toks, rows)], acc[np.ix_(toks, rows)], rows=rows, toks=toks)
+
+
+# ---- group-128 weight steps with asymmetric activations ----
+def run_group(K, N, M, opts, seed):
+    lay = make(K, N, M, seed=seed, dist="laplace")
+    d = {k: to_dev(v) for k, v in lay.items()}
+    packed = w4a8.pack_weights(d["W"], d["s"], 128)
+    rowsum = w4a8.weight_rowsum(packed, N, K, 128).contiguous()
+    Xq, tok, tz = w4a8.quantize_act_asym(d["X"], d["inv_s"])
+    ws = w4a8.new_workspace(M, N, K, 128, opts)
+    codes, scales, zeros = oracle.pack_weights(lay["W"], lay["s"], 128)
+    Q, step, zx = oracle.quantize_act_asym(lay["X"], lay["inv_s"])
+    acc_w, y_w, wide = oracle.linear_asym_group(Q, step, zx, codes, scales, zeros, lay["bias"], 128)
+    from util import bf16_ulp
+    for _ in range(2):
+        Y, acc = w4a8.linear_asym_group(Xq, tok, tz, packed, rowsum, d["bias"], N, 128, ws, opts, want_acc=True)
+        w4a8.check_status(ws)
+        assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_w), "group sums"
+        mag = (np.abs(acc_w) * (0.5 * scales.astype(np.float64))[:, None, :]).sum(0)
+        tol = bf16_ulp(wide) + 2.0 ** -20 * step.astype(np.float64)[:, None] * mag
+        got = oracle.bf16_bits_to_float(bf16_bits(Y)).astype(np.float64)
+        assert np.all(np.abs(got - wide) <= tol)
+
+
+def test_group_weights_simple_path():
+    run_group(768, 768, 16, w4a8.make_opts(w4a8.PATH_SIMPLE), seed=1300)
+
+
+@pytest.mark.parametrize("tok_tile", [16, 64, 128])
+def test_group_weights_tensor_core_path(tok_tile):
+    run_group(1024, 200, 2 * tok_tile + 5, w4a8.make_opts(w4a8.PATH_TCGEN05, tok_tile=tok_tile), seed=1310 + tok_tile)
+
+
+def test_group_weights_split_k_and_automatic_plan():
+    run_group(1024, 384, 16, w4a8.make_opts(w4a8.PATH_TCGEN05, split_k=4), seed=1320)
+    run_group(2048, 640, 300, None, seed=1321)
+
+
+@pytest.mark.parametrize("M,N", [(1, 200), (2, 200), (3, 200), (1, 3080), (4, 3080)])
+def test_group_weights_weight_streaming_kernels(M, N):
+    run_group(1280, N, M, w4a8.make_opts(w4a8.PATH_GEMV), seed=1330 + M + N)
