@@ -80,7 +80,11 @@ typedef struct {
     int bits;        /* code width of the blob: 0 or 4 (dINT4), or 3 (dINT3, packed by
                         w4a8_pack_weights_bits); must match the blob.  3-bit blobs run on the
                         tensor-core kernel (any M) or the simple kernel, with symmetric activations */
-    int reserved;    /* must be zero */
+    int offset_tables; /* 0 = off; 1 = the tensor-core kernel expands codes through level tables
+                        stored with an offset (fewer logic instructions per code) and takes the
+                        offset out again with the tokens' sums, which a small kernel in front
+                        computes into the workspace.  Per-channel 4-bit weights, level_shift
+                        1 or 2.  Same bits as without. */
 } w4a8_opts;
 
 /* Bytes of the packed-weight blob for an [N][K] matrix; 0 if the shape is invalid.

@@ -271,7 +271,9 @@ struct LinearPlan {
     int swiglu;       // gated-unit epilogue (see w4a8_linear_swiglu)
     int batched;      // every 128-row tile has its own block of tokens (attention P*V form)
     int kb_per_split; // k-blocks per slice (last slice may be shorter)
-    size_t off_counters, off_partials, workspace_bytes;
+    int offset;       // 0, or the offset of the decode tables (13 * 2^shift)
+    size_t toksum_slots;
+    size_t off_counters, off_partials, off_toksum, workspace_bytes;
 };
 
 // Asymmetric activations: acc[m][n] -= tok_zero[m] * rowsum[n] before the rescale (both

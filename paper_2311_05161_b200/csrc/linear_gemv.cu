@@ -16,6 +16,7 @@
 // runs the permutes is what bounds them, not HBM), and both can quantize their one to four
 // FP16 tokens themselves (w4a8_quantize_linear), which saves the quantizer's launch.
 #include "common.cuh"
+#include "decode.cuh"
 #include "quant_math.cuh"
 
 namespace w4a8 {
@@ -27,58 +28,6 @@ constexpr int kGemvMaxSteps = 8;    // steps per CTA: a K slice is at most 16 k-
 constexpr int kGemvDepth = 2;       // steps of codes in flight per thread (asynchronous copies)
 constexpr int kGemvRingBytes = kGemvDepth * kGemvKb * 4 * 128 * 16;   // 32 KiB per CTA
 constexpr int kGemvMaxTokens = 4;
-
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
-{
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
-}
-
-__device__ __forceinline__ void decode8(uint32_t w, const uint32_t (&t)[4], uint32_t &o0,
-                                        uint32_t &o1)
-{
-    const uint32_t idx = w & 0x77777777u;
-    const uint32_t e = w << 4;
-    const uint32_t idx_hi = idx >> 16;
-    const uint32_t a0 = prmt(t[0], t[1], idx), b0 = prmt(t[2], t[3], idx);
-    const uint32_t a1 = prmt(t[0], t[1], idx_hi), b1 = prmt(t[2], t[3], idx_hi);
-    const uint32_t m0 = prmt(e, w, 0xD9C8u), m1 = prmt(e, w, 0xFBEAu);
-    o0 = (a0 & ~m0) | (b0 & m0);
-    o1 = (a1 & ~m1) | (b1 & m1);
-}
-
-__device__ __forceinline__ uint4 ld_stream(const uint4 *p)
-{
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-
-// Cheaper expansion for special values step/2 and step/4.  The levels are stored with an offset
-// `off` = 13 * 2^shift, so every table byte lies in [0, 2 off] <= 104 and has its top bit clear.
-// A permute whose selector nibble has bit 3 set returns the selected byte's sign spread over the
-// byte, which is zero for such a table.  So the raw code nibbles pick from the table of codes
-// 0..7 and give 0 for codes 8..15, the nibbles with bit 3 flipped do the opposite on the table
-// of codes 8..15, and the two results go to dp4a as they are (one of them is zero in every
-// byte): no mask, no select.  The sums then carry off * (sum of the tokens' INT8 values over the
-// k-block), which is subtracted per k-block from a small table of those sums.  Integer
-// arithmetic modulo 2^32 throughout, so the result is exact whenever the true sum fits.
-__device__ __forceinline__ void build_offset_tables(int z, const LevelTables &lt, int shift,
-                                                    uint32_t (&t)[4])
-{
-    const uint32_t off = 13u << shift;
-    const uint32_t kc = (128u - off) * 0x01010101u;      // the tables' 0x80 bias minus the offset
-    const uint32_t zz = (uint32_t)z * lt.zmul;
-    t[0] = lt.base[0] - zz - kc;
-    t[1] = lt.base[1] - zz - kc;
-    t[2] = lt.base[2] - zz - kc;
-    // codes 12 and 13, then the two special values +1 and -1
-    t[3] = ((lt.base[3] - (zz & 0xFFFFu) - (kc & 0xFFFFu)) & 0xFFFFu) | ((off + 1u) << 16) |
-           ((off - 1u) << 24);
-}
 
 // One k-block (128 input features) of one output row against MT tokens: w = the row's 64 bytes
 // of codes, xk = the tokens' INT8 values of this k-block (token stride in bytes).

@@ -27,6 +27,7 @@
 #include <atomic>
 
 #include "common.cuh"
+#include "decode.cuh"
 
 namespace w4a8 {
 
@@ -85,7 +86,7 @@ struct Cfg {
     // output staging: two buffers of kChunk tokens x 128 features BF16 per epilogue group
     static constexpr int kStagingBytes = kEpiGroups * kStageBufs * kChunk * kTileN * 2;
     static constexpr int kTailBytes =
-        kStagingBytes + 2048 /* token steps and zero-points */ + 1024 /* barriers */;
+        kStagingBytes + 3072 /* token steps, zero-points, offset sums */ + 1024 /* barriers */;
     static constexpr int kMaxStages = (232448 - 1024 - kTailBytes) / kStageBytes;
     static constexpr int kStages = kMaxStages > 9 ? 9 : kMaxStages;
     // accumulator buffers in tensor memory: two for per-channel weights (epilogue of one unit
@@ -97,7 +98,7 @@ struct Cfg {
                                      : kTmemNeed <= 256 ? 256 : 512;
     static constexpr int kOffStaging = kStages * kStageBytes;
     static constexpr int kOffTok = kOffStaging + kStagingBytes;
-    static constexpr int kOffBarriers = kOffTok + 2048;
+    static constexpr int kOffBarriers = kOffTok + 3072;
     static constexpr int kSmemBytes = kOffBarriers + 1024 + 1024 /* alignment slack */;
     static_assert(kStages >= 3, "pipeline depth");
     static_assert(kTmemNeed <= 512, "tensor memory budget");
@@ -123,6 +124,9 @@ struct Params {
     LevelTables lt;
     float unit;          // level unit as a factor of the step: 2^-shift
     unsigned long long wait_ns, drain_ns;   // limits of the bounded waits
+    int offset;          // 0, or 13 * 2^shift: the decode warps use the offset tables (decode.cuh)
+                         // and the epilogue subtracts tok_offsum[m] = offset * (sum of token m)
+    const int32_t *tok_offsum;
     int swiglu;          // gated-unit epilogue: Y is [M][N / 2] binary16, silu(row 2i) * row 2i + 1
     int batch_rows;      // 0, or M when every 128-row tile has its own [M][K] block of tokens (and
                          // token steps), stacked in tile order: the attention P*V form
@@ -327,12 +331,6 @@ __device__ __forceinline__ uint32_t biased_float_bits(uint32_t acc, uint32_t one
     asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(acc), "r"(one), "r"(kMagicBits));
     return r;
 }
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
-{
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
-}
 __device__ __forceinline__ void named_bar_sync(int id, int threads)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
@@ -459,29 +457,33 @@ __device__ __forceinline__ void prefetch_l2(const void *p, uint32_t bytes)
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 
-// 16-byte global load that does not allocate in L1 (each code byte is used once per CTA).
-__device__ __forceinline__ uint4 ld_stream(const uint4 *p)
+// --------------------------------------------------------------------------- token sums
+// out[m] = offset * sum_k Xq[m][k]: what the offset form of the decode tables adds to every
+// accumulator of token m.  One CTA per token; launched in front of the main kernel.
+__global__ void __launch_bounds__(256)
+token_offsum_kernel(const int8_t *__restrict__ Xq, int K, int offset, int32_t *__restrict__ out)
 {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-
-// --------------------------------------------------------------------------- decode
-// Eight codes (nibble i = code of k0 + i) -> eight INT8 values, bytes in k order.
-__device__ __forceinline__ void decode8(uint32_t w, const uint32_t (&t)[4], uint32_t &o0,
-                                        uint32_t &o1)
-{
-    const uint32_t idx = w & 0x77777777u;
-    const uint32_t e = w << 4;
-    const uint32_t idx_hi = idx >> 16;
-    const uint32_t a0 = prmt(t[0], t[1], idx), b0 = prmt(t[2], t[3], idx);
-    const uint32_t a1 = prmt(t[0], t[1], idx_hi), b1 = prmt(t[2], t[3], idx_hi);
-    const uint32_t m0 = prmt(e, w, 0xD9C8u), m1 = prmt(e, w, 0xFBEAu);   // bit 3 -> byte mask
-    o0 = (a0 & ~m0) | (b0 & m0);
-    o1 = (a1 & ~m1) | (b1 & m1);
+    __shared__ int red[8];
+    allow_dependents();
+    dependent_wait();                      // Xq may be the output of the kernel before
+    const int4 *row = reinterpret_cast<const int4 *>(Xq + (size_t)blockIdx.x * K);
+    int s = 0;
+    for (int i = threadIdx.x; i < K / 16; i += 256) {
+        const int4 v = __ldg(row + i);
+        s = __dp4a(v.x, 0x01010101, s);
+        s = __dp4a(v.y, 0x01010101, s);
+        s = __dp4a(v.z, 0x01010101, s);
+        s = __dp4a(v.w, 0x01010101, s);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int t = 0;
+        for (int w = 0; w < 8; ++w) t += red[w];
+        out[blockIdx.x] = t * offset;
+    }
 }
 
 // --------------------------------------------------------------------------- the kernel
@@ -761,6 +763,9 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         };
         if (cur.valid()) fetch(cur, w, z);
         bool ok = true;
+        const bool use_offset = P.offset != 0;
+        uint32_t one = 1u;                       // opaque to the compiler: see decode8_offset
+        asm volatile("" : "+r"(one));
         while (cur.valid() && ok) {
             KbCursor nxt = cur;
             nxt.advance(T);
@@ -770,9 +775,21 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             const int st = cur.it % S;
             const uint32_t fill = cur.it / S;
             uint32_t t[4];
-            build_level_tables(z, P.lt, t);
+            if (use_offset) build_offset_tables(z, P.lt, P.L.shift, t);
+            else build_level_tables(z, P.lt, t);
             uint4 lv[2 * QT];                    // the thread's INT8 levels, 16 per register quad
             auto expand = [&]() {
+                if (use_offset) {
+#pragma unroll
+                    for (int q = 0; q < QT; ++q) {
+                        const uint4 wq = w[q];
+                        decode8_offset(wq.x, t, one, lv[2 * q].x, lv[2 * q].y);
+                        decode8_offset(wq.y, t, one, lv[2 * q].z, lv[2 * q].w);
+                        decode8_offset(wq.z, t, one, lv[2 * q + 1].x, lv[2 * q + 1].y);
+                        decode8_offset(wq.w, t, one, lv[2 * q + 1].z, lv[2 * q + 1].w);
+                    }
+                    return;
+                }
 #pragma unroll
                 for (int q = 0; q < QT; ++q) {
                     const uint4 wq = w[q];
@@ -836,6 +853,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         float *s_tok = reinterpret_cast<float *>(gen_base + C::kOffTok);
         int *s_tz = reinterpret_cast<int *>(gen_base + C::kOffTok + 1024);   // tokens' zero-points
+        int *s_off = reinterpret_cast<int *>(gen_base + C::kOffTok + 2048);  // offset * token sum
         __nv_bfloat16 *stg =
             reinterpret_cast<__nv_bfloat16 *>(gen_base + C::kOffStaging) +
             col_group * C::kStageBufs * C::kChunk * kTileN;
@@ -889,13 +907,14 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             valid = valid < 0 ? 0 : (valid > C::kColsPerThread ? C::kColsPerThread : valid);
             const float bias_n = (P.bias && n_ok) ? P.bias[n] : 0.0f;
 
-            if (P.Y || P.zp.tok_zero) {
+            if (P.Y || P.zp.tok_zero || P.offset) {
                 // token step sizes (and zero-points) of this tile, shared by all epilogue threads
                 named_bar_sync(1, kEpiThreads);
                 for (int i = et; i < TOK; i += kEpiThreads) {
                     const bool in = tt * TOK + i < P.M;
                     s_tok[i] = (in && P.tok_scale) ? __ldg(P.tok_scale + nt * P.batch_rows + tt * TOK + i) : 0.0f;
                     s_tz[i] = (in && P.zp.tok_zero) ? __ldg(P.zp.tok_zero + tt * TOK + i) : 0;
+                    s_off[i] = (in && P.offset) ? __ldcg(P.tok_offsum + nt * P.batch_rows + tt * TOK + i) : 0;
                 }
                 named_bar_sync(1, kEpiThreads);
             }
@@ -925,10 +944,12 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
                     }
                     if (c >= valid) continue;             // uniform over the column group
-                    if (P.zp.tok_zero && P.split_k == 1) {
+                    if ((P.zp.tok_zero || P.offset) && P.split_k == 1) {
+                        // the token's zero-point times the row's level sum, and the offset of the
+                        // decode tables times the token's own sum, leave the accumulator
 #pragma unroll
                         for (int j = 0; j < C::kChunk; ++j)
-                            v[j] = (uint32_t)((int)v[j] - s_tz[col0 + c + j] * row_sum);
+                            v[j] = (uint32_t)((int)v[j] - s_tz[col0 + c + j] * row_sum - s_off[col0 + c + j]);   // (both staged: zero when unused)
                     }
                     if (P.acc_out && P.split_k == 1 && n_ok) {
 #pragma unroll
@@ -989,7 +1010,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                                 const int j = j0 + t;
                                 if (j >= valid) break;
                                 const int m = tok0 + j;
-                                acc[t] -= s_tz[col0 + j] * row_sum;
+                                if (P.zp.tok_zero) acc[t] -= s_tz[col0 + j] * row_sum;
+                                if (P.offset) acc[t] -= s_off[col0 + j];
                                 if (P.acc_out) P.acc_out[(size_t)m * P.L.N + n] = acc[t];
                                 if (P.Y) {
                                     float x = rescale_channel(acc[t], s_tok[col0 + j], half_step);
@@ -1339,8 +1361,23 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     plan->off_counters = sizeof(StatusBlock);
     plan->off_partials = align_up(plan->off_counters + (size_t)tiles * sizeof(int), 256);
     const size_t m_pad = (size_t)tok_tiles * tok;
-    plan->workspace_bytes =
-        plan->off_partials + (split > 1 ? (size_t)split * m_pad * L.n_pad * 4 : 0);
+    plan->off_toksum = align_up(plan->off_partials + (split > 1 ? (size_t)split * m_pad * L.n_pad * 4 : 0), 256);
+    // Offset form of the decode tables (decode.cuh), on request: per-channel 4-bit weights whose
+    // special value is step/2 or step/4, and a K short enough for the offset sums to stay inside
+    // INT32.  It needs offset * (sum of each token), computed by a small kernel in front into the
+    // workspace (one INT32 per token and row tile in the P*V form, so the slot is sized for the
+    // padded rows).  Measured: seven instead of eleven logic-pipe instructions per eight codes let
+    // the SM clock rise under the power cap (1440 against 1370 MHz on the 9216-wide block), but the
+    // per-k-block time does not follow the logic pipe and the extra launch costs what the clock
+    // gains (2350 against 2380 TOPS sustained; 53.8 against 52.3 us at 16 tokens), so the
+    // automatic plan leaves it off.
+    const int off = 13 << L.shift;
+    const bool want = opts && opts->offset_tables == 1;
+    if (want && !(!grouped && L.bits == 4 && L.shift <= 2 && (long long)L.K * 127 * (2 * off) < (1LL << 31)))
+        return false;
+    plan->offset = want ? off : 0;
+    plan->toksum_slots = (size_t)L.n_tiles * M;
+    plan->workspace_bytes = plan->off_toksum + (plan->offset ? plan->toksum_slots * 4 : 0);
     return true;
 }
 
@@ -1407,6 +1444,14 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     P.skip_load = plan.debug_skip_load;
     P.batch_rows = plan.batched ? M : 0;
     P.swiglu = plan.swiglu;
+    P.offset = plan.offset;
+    P.tok_offsum = reinterpret_cast<const int32_t *>(workspace + plan.off_toksum);
+    if (plan.offset) {
+        const int rows = plan.batched ? M * L.n_tiles : M;
+        if (launch_overlapped(token_offsum_kernel, dim3(rows), dim3(256), 0, st, Xq, L.K, plan.offset,
+                              reinterpret_cast<int32_t *>(workspace + plan.off_toksum)) != cudaSuccess)
+            return W4A8_ERR_CUDA;
+    }
 
     const bool g = L.group != 0;
     switch (plan.tok_tile) {

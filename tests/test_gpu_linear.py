@@ -206,3 +206,43 @@ def test_cluster_option_is_validated():
     assert w4a8.linear_workspace_bytes(300, 256, 256, 0, w4a8.make_opts(tok_tile=128, cluster=3)) == 0
     assert w4a8.linear_plan(2048, 4096, 4096, 0)["cluster"] == 1
     assert w4a8.linear_plan(2048, 4096, 4096, 0, w4a8.make_opts(tok_tile=256, cluster=2))["cluster"] == 2
+
+
+@pytest.mark.parametrize("tok_tile,split", [(16, 1), (16, 4), (128, 1), (256, 1)])
+def test_tcgen05_offset_tables(tok_tile, split):
+    """Level tables stored with an offset (cheaper expansion) and taken out again with the tokens'
+    sums: the same INT32 sums and BF16 bits, every zero-point and both special codes in play."""
+    M = 2 * tok_tile + 5 if tok_tile > 16 else 13
+    prob = Problem(1024, 200, M, 0, seed=800 + tok_tile + split, dist="laplace", outliers=0.01, mult=20.0)
+    opts = w4a8.make_opts(w4a8.PATH_TCGEN05, split_k=split, tok_tile=tok_tile, offset_tables=1)
+    for _ in range(2):
+        Y, acc = run_linear(prob, opts)
+        assert np.array_equal(acc, prob.oracle_acc())
+        check_y(prob, Y, exact=True)
+    assert len(np.unique(prob.zeros)) >= 4                      # several zero-points among the rows
+    assert w4a8.linear_workspace_bytes(16, 256, 256, 128, w4a8.make_opts(offset_tables=1)) == 0
+
+
+def test_tcgen05_offset_tables_every_zero_point():
+    """Rows whose ranges are built to give every zero-point 0..13, values in both special bands."""
+    K, N, M = 512, 168, 40
+    rng = np.random.default_rng(5)
+    W = np.empty((N, K), dtype=np.float16)
+    for n in range(N):
+        z = n % 14
+        vals = rng.uniform(-z, 13 - z, size=K)
+        vals[0], vals[1], vals[2], vals[3] = -z, 13 - z, 0.5, -0.5
+        W[n] = (vals * 0.01).astype(np.float16)
+    prob = Problem.__new__(Problem)
+    X = (rng.standard_normal((M, K)) * 2).astype(np.float16)
+    prob.K, prob.N, prob.M, prob.group, prob.rows = K, N, M, 0, None
+    prob.host = {"W": W, "X": X, "s": None, "inv_s": None, "bias": None}
+    prob.dev = {k: (torch.from_numpy(v).cuda() if v is not None else None) for k, v in prob.host.items()}
+    prob.codes, prob.scales, prob.zeros = oracle.pack_weights(W, None, 0)
+    prob.Xq, prob.tok = oracle.quantize_act(X, None)
+    prob.bias_sel = None
+    assert set(np.unique(prob.zeros)) == set(range(14))
+    for tok_tile in (16, 64):
+        Y, acc = run_linear(prob, w4a8.make_opts(w4a8.PATH_TCGEN05, tok_tile=tok_tile, offset_tables=1))
+        assert np.array_equal(acc, prob.oracle_acc())
+        check_y(prob, Y, exact=True)
