@@ -66,10 +66,17 @@ typedef struct {
                         or 32) */
     int level_shift; /* special value of the blob = step / 2^level_shift: 0 or 1 (the paper's
                         step/2), 2 or 3 (w4a8_pack_weights_fmt); must match the blob */
-    int cluster;     /* 0 = automatic; else CTAs per thread-block cluster of the tensor-core kernel:
-                        1, or 2 (token tiles of 128 and more): the two CTAs work on two token
-                        tiles of the same weight rows and each expands half of every code tile
-                        for both */
+    int cluster;     /* 0 = automatic (one CTA); else the cluster form of the tensor-core kernel:
+                        1 = one CTA per cluster;
+                        2 = sharing pair (token tiles of 128 and more, symmetric activations
+                            when the weights are grouped): two CTAs work on two token tiles of
+                            the same weight rows and each expands half of every code tile for both;
+                        3 = MMA pair (token tile 256, per-channel 4-bit weights, an even number
+                            of 128-row tiles, 8 or 16 decode warps): two CTAs on two row tiles
+                            and one token tile issue every MMA as one 256-row instruction, each
+                            loads half of the tokens.
+                        Same bits in every form; a form that does not fit the call is refused
+                        with W4A8_ERR_SHAPE. */
     int debug_wait_ms;   /* test hook, 0 = off: limit of every bounded wait inside the tensor-core
                             kernel in milliseconds (normally 2 s) */
     int debug_skip_load; /* test hook, 0 = off: the copy thread of every CTA leaves out the token

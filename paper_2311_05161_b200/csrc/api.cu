@@ -37,10 +37,10 @@ bool opts_ok(const w4a8_opts *o)
     if (o->path < W4A8_PATH_AUTO || o->path > W4A8_PATH_GEMV) return false;
     if (o->split_k < 0 || o->tok_tile < 0 || o->decode_warps < 0) return false;
     if (o->level_shift < 0 || o->level_shift > 3) return false;
-    if (o->cluster < 0 || o->cluster > 2) return false;
+    if (o->cluster < 0 || o->cluster > 3) return false;
     if (o->offset_tables < 0 || o->offset_tables > 1 || (o->bits != 0 && !bits_ok(o->bits))) return false;
     if (o->offset_tables && (o->path == W4A8_PATH_GEMV || o->path == W4A8_PATH_SIMPLE)) return false;
-    if (o->bits == 3 && (o->path == W4A8_PATH_GEMV || o->cluster == 2)) return false;
+    if (o->bits == 3 && (o->path == W4A8_PATH_GEMV || o->cluster >= 2)) return false;
 #ifdef W4A8_DEBUG_HOOKS
     if (o->debug_wait_ms < 0 || o->debug_wait_ms > 2000 || o->debug_skip_load < 0) return false;
     if ((o->debug_wait_ms || o->debug_skip_load) && o->path != W4A8_PATH_TCGEN05) return false;

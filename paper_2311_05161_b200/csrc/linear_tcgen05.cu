@@ -35,6 +35,7 @@ namespace {
 
 constexpr int kFirstDecodeWarp = 2;
 constexpr int kSwigluVariant = 5;
+constexpr int kAsymGroupVariant = 6;
 constexpr int kMaxDevices = 64;
 constexpr int kABytes = kTileN * kTileK;            // decoded INT8 tile, 16 KiB
 constexpr int kDefaultTeamWarps = 4;               // warps per decode team
@@ -51,7 +52,9 @@ struct Cfg {
     // epilogue warpgroups: group mode spreads the per-k-block FP32 accumulation over
     // 32 columns per thread (more warps in flight, fewer registers each)
     static constexpr int kEpiGroups = !GROUPED ? 1 : (TOK >= 128 ? 4 : TOK >= 64 ? 2 : 1);
-    static constexpr int kStageBufs = GROUPED ? 1 : 2;      // output staging buffers per group
+    // output staging buffers per group (one where the token ring needs the room)
+    static constexpr int kStageBufs = (GROUPED || (TOK >= 256 && CL != 3)) ? 1 : 2;
+    static constexpr int kAStagesWanted = GROUPED ? 5 : (TOK >= 256 && CL != 3) ? 3 : 4;
     static constexpr int kEpiWarps = 4 * kEpiGroups;
     static constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
     // With at most 512 threads a thread has the registers to expand its codes before the stage
@@ -59,7 +62,15 @@ struct Cfg {
     static constexpr bool kExpandAhead = kThreads <= 512;
     static constexpr int kColsPerThread = TOK / kEpiGroups;
     static constexpr int kChunk = kColsPerThread >= 32 ? 32 : 16;
-    static constexpr int kTokBytes = TOK * kTileK;
+    // CL = 1: one CTA.  CL = 2 (kShare): two CTAs on the same row tile, each on its own token
+    // tile, share the expansion of the codes.  CL = 3 (kPair): two CTAs on two row tiles and the
+    // same token tile run as one MMA pair (cta_group::2): every MMA instruction covers both row
+    // tiles, CTA r holds (and loads) tokens 128 r .. 128 r + 127 of the tile, and the leader's one
+    // issuing thread serves both, so the token bytes per SM and the issue cost per CTA halve.
+    static constexpr bool kShare = CL == 2, kPair = CL == 3;
+    static constexpr int kCtas = CL == 1 ? 1 : 2;
+    static constexpr int kTokRows = kPair ? TOK / 2 : TOK;     // token rows this CTA loads per k-block
+    static constexpr int kTokBytes = kTokRows * kTileK;
     // Codes go from global memory straight into the decode threads' registers (shared-memory
     // bandwidth and capacity are the scarce resources); for weight-streaming shapes the
     // producer thread runs ahead with L2 prefetches of the code tiles.
@@ -73,22 +84,28 @@ struct Cfg {
     // each on its own token tile.  With CL = 2 each expands 64 of the tile's 128 rows into its own
     // stage and sends them to its peer's stage with a bulk copy through distributed shared memory
     // that completes on the peer's barrier, so the table lookups per MMA halve.
-    static constexpr int kRowsPerCta = kTileN / CL;
-    static constexpr int kQuartersPerThread = 4 / CL;            // 32-k quarters of a row per thread
-    static_assert(CL == 1 || CL == 2, "cluster of one or two CTAs");
+    static constexpr int kRowsPerCta = kShare ? kTileN / 2 : kTileN;
+    static constexpr int kQuartersPerThread = kShare ? 2 : 4;   // 32-k quarters of a row per thread
+    static_assert(CL >= 1 && CL <= 3, "one CTA, a sharing pair or an MMA pair");
+    static_assert(!kPair || (TOK == 256 && !GROUPED), "the MMA pair: 256 tokens, per-channel weights");
     static_assert(DW % kTeamWarps == 0 && kTeamWarps == 4, "decode warps form whole teams of four");
-    // One stage holds the decoded INT8 weights of a k-block (operand A, 16 KiB, written by the
-    // decode warps) and the tokens of the same k-block (operand B, written by TMA).  Keeping
-    // operand A in tensor memory instead was measured slower at every token tile.
-    static constexpr int kStageBytes = kABytes + kTokBytes;
-    static constexpr int kTokOff = kABytes;             // tokens inside a stage
+    // Two rings of operand buffers, one set of barriers.  Ring A holds decoded INT8 weights of a
+    // k-block (16 KiB, written by the decode warps), ring B the tokens of a k-block (written by
+    // TMA).  K-block number `it` uses A buffer it % kAStages, B buffer it % kStages and the barrier
+    // pair it % kStages.  The rings differ in depth because they hide different latencies: a
+    // token tile comes from L2 and is on its way for a few thousand cycles when all SMs pull
+    // tiles at once (the bytes in flight bound the rate), decoded weights come from registers.
+    // (Keeping operand A in tensor memory instead was measured slower at every token tile.)
     static constexpr int kPrefetchAhead = 16;          // k-blocks of codes requested into L2
-    // output staging: two buffers of kChunk tokens x 128 features BF16 per epilogue group
+    // output staging: kStageBufs buffers of kChunk tokens x 128 features BF16 per epilogue group
     static constexpr int kStagingBytes = kEpiGroups * kStageBufs * kChunk * kTileN * 2;
     static constexpr int kTailBytes =
         kStagingBytes + 3072 /* token steps, zero-points, offset sums */ + 1024 /* barriers */;
-    static constexpr int kMaxStages = (232448 - 1024 - kTailBytes) / kStageBytes;
-    static constexpr int kStages = kMaxStages > 9 ? 9 : kMaxStages;
+    static constexpr int kRingBytes = 232448 - 1024 - kTailBytes;
+    static constexpr int kAStages = kAStagesWanted;
+    static constexpr int kMaxStages = (kRingBytes - kAStages * kABytes) / kTokBytes;
+    static constexpr int kStages = kMaxStages > 12 ? 12 : kMaxStages;
+    static constexpr int kOffTokRing = kAStages * kABytes;
     // accumulator buffers in tensor memory: two for per-channel weights (epilogue of one unit
     // overlaps the main loop of the next); group mode hands over every k-block, and a hand-over
     // costs several hundred cycles of latency, so it rotates over as many buffers as fit
@@ -96,11 +113,11 @@ struct Cfg {
     static constexpr int kTmemNeed = kAccBufs * TOK;
     static constexpr int kTmemCols = kTmemNeed <= 32 ? 32 : kTmemNeed <= 64 ? 64 : kTmemNeed <= 128 ? 128
                                      : kTmemNeed <= 256 ? 256 : 512;
-    static constexpr int kOffStaging = kStages * kStageBytes;
+    static constexpr int kOffStaging = kOffTokRing + kStages * kTokBytes;
     static constexpr int kOffTok = kOffStaging + kStagingBytes;
     static constexpr int kOffBarriers = kOffTok + 3072;
     static constexpr int kSmemBytes = kOffBarriers + 1024 + 1024 /* alignment slack */;
-    static_assert(kStages >= 3, "pipeline depth");
+    static_assert(kStages >= kAStages && kAStages >= 2, "pipeline depth");
     static_assert(kTmemNeed <= 512, "tensor memory budget");
     static_assert(kSmemBytes <= 232448, "shared memory budget");
     static_assert(!GROUPED || TOK <= 128, "group mode keeps its FP32 sums in registers");
@@ -194,6 +211,36 @@ __device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_in_cluster, uint32
         "r"(src), "r"(bytes), "r"(bar_in_cluster)
         : "memory");
 }
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_in_cluster)
+{
+    // (default semantics, as for a local arrival: asking for a cluster-scope release here was
+    // measured to cost the arriving thread more than half a microsecond per arrival)
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_in_cluster) : "memory");
+}
+// wait with cluster-scope acquire: what a peer CTA released by its arrival is visible afterwards
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
+        : "memory");
+    return ok != 0;
+}
+// Tile load of a CTA of an MMA pair: the bytes land in this CTA, the completion counts on the
+// barrier `bar_in_cluster`, which may belong to the pair's other CTA (no multicast: one copy).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int x, int y,
+                                                 uint32_t bar_in_cluster)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+        "l"(map), "r"(bar_in_cluster), "r"(x), "r"(y)
+        : "memory");
+}
 __device__ __forceinline__ void cluster_sync_all()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -259,6 +306,25 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
         "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The pair forms: one instruction of the leader CTA drives the tensor cores of both CTAs.
+__device__ __forceinline__ void tc_mma_i8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                               uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t mask)
+{
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::
+            "r"(bar),
+        "h"(mask)
         : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
@@ -354,9 +420,9 @@ __device__ __forceinline__ bool named_bar_and(int id, int threads, bool pred)
 // rows and 128-byte swizzle, 8-row groups 1024 bytes apart; the start address advances by 32
 // bytes per 32-deep MMA step inside the swizzle span.
 // Instruction descriptor: signed 8-bit A and B, both K-major, INT32 accumulate, M = 128.
-__host__ __device__ constexpr uint32_t instr_desc_i8(int n)
+__host__ __device__ constexpr uint32_t instr_desc_i8(int n, int m = 128)
 {
-    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // --------------------------------------------------------------------------- bounded wait
@@ -369,14 +435,18 @@ struct Ctl {
 
 // `draining`: the CTA has given up and only waits for what it has in flight (copies, MMAs):
 // such a wait does not end because of the abort flag, and it has the shorter limit.
+template <bool CLUSTER_ACQUIRE = false>
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, Ctl *ctl,
                                              StatusBlock *sb, int where, bool draining = false)
 {
-    if (mbar_try_wait(bar, parity)) return true;
+    auto test = [&]() {
+        return CLUSTER_ACQUIRE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity);
+    };
+    if (test()) return true;
     // the timer is slow to read: it is only consulted after many failed polls
     unsigned long long t0 = 0;
     for (uint32_t i = 1;; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (test()) return true;
         if ((i & 63u) == 0u) {
             if (ctl->abort && !draining) return false;
             if (t0 == 0) {
@@ -487,7 +557,10 @@ token_offsum_kernel(const int8_t *__restrict__ Xq, int K, int offset, int32_t *_
 }
 
 // --------------------------------------------------------------------------- the kernel
-// VARIANT: 4 = 4-bit codes, 3 = 3-bit codes, kSwigluVariant = 4-bit codes with the gated-unit
+// VARIANT: 4 = 4-bit codes, 3 = 3-bit codes, kAsymGroupVariant = 4-bit codes in groups with
+// asymmetric activations (a kernel of its own: the zero-point correction in the loop over the
+// groups, even as an untaken branch, was measured to cost the symmetric path a quarter of its
+// throughput through register pressure), kSwigluVariant = 4-bit codes with the gated-unit
 // epilogue (rows 2i / 2i + 1 of the weight matrix are feature i of the gate / up projection;
 // the output is silu(gate) * up in binary16, half as wide as the weight matrix is tall)
 template <int TOK, bool GROUPED, int DW, int CL, int VARIANT>
@@ -498,6 +571,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     using C = Cfg<TOK, GROUPED, DW, CL>;
     constexpr int BITS = VARIANT == 3 ? 3 : 4;
     constexpr bool SWIGLU = VARIANT == kSwigluVariant;
+    constexpr bool ASYM_GROUP = VARIANT == kAsymGroupVariant;
+    static_assert(!ASYM_GROUP || GROUPED, "the asymmetric group variant is a group-mode kernel");
     constexpr int kFirstEpiWarp = C::kFirstEpiWarp;
     constexpr int S = C::kStages;
     extern __shared__ uint8_t smem_raw[];
@@ -523,22 +598,33 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     else if (warp == 1) role = kMma;
     else if (warp < kFirstEpiWarp) { role = kDecode; role_idx = warp - kFirstDecodeWarp; }
     else { role = kEpilogue; role_idx = warp - kFirstEpiWarp; }
-    // Units (token-tile group, row tile, K slice) are dealt round-robin to the clusters; CTA
-    // `rank` of a cluster takes token tile CL * group + rank of the unit.
+    // Units (token-tile group, row-tile group, K slice) are dealt round-robin to the clusters.
+    // Sharing pair: CTA `rank` takes token tile 2 * group + rank of the unit.  MMA pair: CTA
+    // `rank` takes row tile 2 * group + rank.
+    constexpr bool kShare = C::kShare, kPair = C::kPair;
     const uint32_t rank = CL > 1 ? cluster_ctarank() : 0u;
-    const int unit0 = (int)blockIdx.x / CL, unit_step = (int)gridDim.x / CL;
+    const int unit0 = (int)blockIdx.x / C::kCtas, unit_step = (int)gridDim.x / C::kCtas;
+    // row-tile groups of the unit list, and this CTA's row / token tile inside a unit
+    const int nt_groups = kPair ? P.L.n_tiles / 2 : P.L.n_tiles;
+    auto row_tile = [&](int g) { return kPair ? 2 * g + (int)rank : g; };
+    auto tok_tile_of = [&](int g) { return kShare ? 2 * g + (int)rank : g; };
+    // the barriers the MMA thread waits on live in the leader CTA of an MMA pair
+    const bool leader = !kPair || rank == 0u;
+    auto at_leader = [&](uint32_t bar) { return kPair ? map_to_cta(bar, 0u) : bar; };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             // the warps of a decode team and the producer's arrival; the token copy and, in a
             // cluster, the peer's half of the expanded rows complete on it too
-            mbar_init(bar_dec + 8 * s, C::kTeamWarps + 1);
-            // the MMA threads of all CTAs of the cluster: they all read rows this CTA wrote
-            mbar_init(bar_empty + 8 * s, CL);
+            // (MMA pair: the leader's barrier collects both CTAs' arrivals)
+            // (MMA pair: the leader's barrier collects the decode warps of both CTAs)
+            mbar_init(bar_dec + 8 * s, kPair ? 2 * C::kTeamWarps + 1 : C::kTeamWarps + 1);
+            // sharing pair: the MMA threads of both CTAs, which all read rows this CTA wrote
+            mbar_init(bar_empty + 8 * s, kShare ? 2 : 1);
         }
         for (int b = 0; b < NB; ++b) {
             mbar_init(bar_acc_full + 8 * b, 1);
-            mbar_init(bar_acc_empty + 8 * b, C::kEpiWarps);
+            mbar_init(bar_acc_empty + 8 * b, C::kEpiWarps * (kPair ? 2 : 1));
         }
         mbar_init(bar_drain, 1);
         ctl->abort = 0;
@@ -549,11 +635,20 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         fence_proxy_async();
     }
     if (role == kMma) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                         smem_u32(&ctl->tmem_base)),
-                     "r"((uint32_t)C::kTmemCols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (kPair) {
+            // the MMA warps of both CTAs allocate the same columns together
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                             smem_u32(&ctl->tmem_base)),
+                         "r"((uint32_t)C::kTmemCols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                             smem_u32(&ctl->tmem_base)),
+                         "r"((uint32_t)C::kTmemCols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -577,11 +672,11 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             uint32_t it = 0;
             bool ok = true;
             KbCursor pf;
-            pf.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, n_tiles);
+            pf.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, nt_groups);
             for (int u = unit0; u < P.total_units && ok; u += unit_step) {
                 const int s = u % P.split_k, rest = u / P.split_k;
-                const int tt = (rest / n_tiles) * CL + (int)rank;
-                const int nt_of_unit = rest % n_tiles;
+                const int tt = tok_tile_of(rest / nt_groups);
+                const int nt_of_unit = row_tile(rest % nt_groups);
                 const int kb0 = s * P.kb_per_split;
                 const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
@@ -592,14 +687,26 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         break;
                     }
                     if (P.skip_load != 0 && it == (uint32_t)(P.skip_load - 1)) continue;
-                    const uint32_t stage = base + st * C::kStageBytes;
+                    const uint32_t tok_dst = base + C::kOffTokRing + st * C::kTokBytes;
                     const uint32_t tok_bar = bar_dec + 8 * st;
-                    mbar_arrive_expect_tx(tok_bar, C::kTokBytes + (CL > 1 ? kABytes / CL : 0));
-                    tma_load_2d(stage + C::kTokOff, &tok_map, kb * kTileK, nt_of_unit * P.batch_rows + tt * TOK, tok_bar);
+                    if (kPair) {
+                        // this CTA's 128 of the tile's 256 tokens; completion counts at the leader
+                        // (the leader's copy thread announces both CTAs' bytes with its own
+                        // arrival; the other CTA only issues its copy: a release-arrival on a
+                        // remote barrier was measured to cost that thread about a microsecond)
+                        const uint32_t lead_bar = at_leader(tok_bar);
+                        if (rank == 0u) mbar_arrive_expect_tx(tok_bar, 2 * C::kTokBytes);
+                        tma_load_2d_pair(tok_dst, &tok_map, kb * kTileK,
+                                         tt * TOK + (int)rank * C::kTokRows, lead_bar);
+                    } else {
+                        mbar_arrive_expect_tx(tok_bar, C::kTokBytes + (kShare ? kABytes / 2 : 0));
+                        tma_load_2d(tok_dst, &tok_map, kb * kTileK,
+                                    nt_of_unit * P.batch_rows + tt * TOK, tok_bar);
+                    }
                     if (P.prefetch_codes) {
                         // keep the code stream kPrefetchAhead k-blocks ahead of the decode warps
                         while (pf.valid() && pf.it < it + C::kPrefetchAhead) {
-                            const int pnt = pf.nt;
+                            const int pnt = row_tile(pf.nt);
                             prefetch_l2(P.codes + ((size_t)pnt * k_blocks + pf.kb) * (BITS == 3 ? kTileBytes3 : kTileBytes),
                                         BITS == 3 ? kTileBytes3 : kTileBytes);
                             pf.advance(1);
@@ -607,8 +714,10 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     }
                 }
             }
-            if (!ok) {
-                // copies already issued must land before the CTA gives its memory back
+            if (!ok && leader) {
+                // copies already issued must land before the CTA gives its memory back (in an MMA
+                // pair the leader's barriers count both CTAs' copies, and the other CTA stays
+                // until the leader is through: the cluster barrier at the end)
                 const uint32_t first = it > (uint32_t)S ? it - S : 0u;
                 for (uint32_t j = first; j < it; ++j)
                     wait_bounded(bar_dec + 8 * (j % S), (j / S) & 1u, ctl, P.sb, 11, true);
@@ -617,14 +726,16 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         __syncwarp();
     } else if (role == kMma) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        if (lane == 0 && leader) {
             // This loop is the serial spine of the kernel (one thread, once per k-block): all
             // counters are kept incrementally and the descriptors are an add away.
-            constexpr uint32_t idesc = instr_desc_i8(TOK);
+            constexpr uint32_t idesc = instr_desc_i8(TOK, kPair ? 256 : 128);
+            constexpr uint16_t kBoth = 3;                // both CTAs of the cluster
             constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
             const uint32_t a_lo0 = ((base & 0x3FFFFu) >> 4) | (1u << 16);
-            const uint32_t b_lo0 = (((base + C::kTokOff) & 0x3FFFFu) >> 4) | (1u << 16);
-            uint32_t st = 0, st_par = 0;                 // stage and its fill parity
+            const uint32_t b_lo0 = (((base + C::kOffTokRing) & 0x3FFFFu) >> 4) | (1u << 16);
+            uint32_t st = 0, st_par = 0;                 // token buffer (= barrier slot), fill parity
+            uint32_t sa = 0;                             // weight buffer
             uint32_t buf = 0, buf_par = 0;               // accumulator buffer and its parity
             bool ok = true;
             for (int u = unit0; u < P.total_units && ok; u += unit_step) {
@@ -635,37 +746,43 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     const bool first = GROUPED || i == 0;
                     const bool last = GROUPED || i == nkb - 1;
                     if (first &&
-                        !wait_bounded(bar_acc_empty + 8 * buf, buf_par ^ 1u, ctl, P.sb, 20)) {
+                        !wait_bounded<kPair>(bar_acc_empty + 8 * buf, buf_par ^ 1u, ctl, P.sb, 20)) {
                         ok = false;
                         break;
                     }
                     // decoded weights and tokens of the stage
-                    if (!wait_bounded(bar_dec + 8 * st, st_par, ctl, P.sb, 21)) {
+                    if (!wait_bounded<kPair>(bar_dec + 8 * st, st_par, ctl, P.sb, 21)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
                     const uint32_t d = tmem_base + buf * TOK;
-                    const uint32_t soff = st * (C::kStageBytes >> 4);
-                    const uint64_t a_desc = ((uint64_t)kDescHi << 32) | (a_lo0 + soff);
-                    const uint64_t b_desc = ((uint64_t)kDescHi << 32) | (b_lo0 + soff);
+                    const uint64_t a_desc = ((uint64_t)kDescHi << 32) | (a_lo0 + sa * (kABytes >> 4));
+                    const uint64_t b_desc = ((uint64_t)kDescHi << 32) | (b_lo0 + st * (C::kTokBytes >> 4));
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
                         const uint32_t acc_flag = (!first || ks > 0) ? 1u : 0u;
-                        tc_mma_i8(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
-                                  acc_flag);
+                        if (kPair)
+                            tc_mma_i8_pair(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
+                                           acc_flag);
+                        else
+                            tc_mma_i8(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
+                                      acc_flag);
                     }
-                    if (CL > 1) tc_commit_multicast(bar_empty + 8 * st, (uint16_t)((1u << CL) - 1u));
+                    if (kPair) tc_commit_pair(bar_empty + 8 * st, kBoth);
+                    else if (kShare) tc_commit_multicast(bar_empty + 8 * st, kBoth);
                     else tc_commit(bar_empty + 8 * st);
                     if (last) {
-                        tc_commit(bar_acc_full + 8 * buf);
+                        if (kPair) tc_commit_pair(bar_acc_full + 8 * buf, kBoth);
+                        else tc_commit(bar_acc_full + 8 * buf);
                         if (++buf == (uint32_t)NB) { buf = 0; buf_par ^= 1u; }
                     }
                     if (++st == (uint32_t)S) { st = 0; st_par ^= 1u; }
+                    if (++sa == (uint32_t)C::kAStages) sa = 0;
                 }
             }
             // nothing issued may still be running when tensor memory is freed
-            tc_commit(bar_drain);
+            if (kPair) tc_commit_pair(bar_drain, 1); else tc_commit(bar_drain);
             wait_bounded(bar_drain, 0u, ctl, P.sb, 22, !ok);
         }
         __syncwarp();
@@ -679,16 +796,23 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         // One thread per row of the tile; in a cluster this CTA takes 64 of the rows, a warp 16 of
         // them, and a thread half a row, so that a warp's rows are one contiguous 2 KiB piece of
         // the stage.
-        const int r = CL == 1 ? (dt & 127)
+        const int r = !kShare ? (dt & 127)
                               : (int)rank * C::kRowsPerCta + ((dt >> 5) & 3) * 16 + (lane & 15);
-        const int q0 = CL == 1 ? 0 : (lane >> 4) * QT;       // first 32-k quarter of this thread
+        const int q0 = !kShare ? 0 : (lane >> 4) * QT;       // first 32-k quarter of this thread
         const int team = dt / (32 * C::kTeamWarps);
         constexpr int T = C::kTeams;
         // the same stage and barrier in the peer CTA
         const uint32_t peer = rank ^ 1u;
         KbCursor cur;
-        cur.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, n_tiles);
+        cur.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, nt_groups);
         cur.advance(team);
+        // the weight buffer of k-block `it` is free once the MMAs of k-block it - kAStages, its
+        // last user, have retired (their commit completed a phase of that k-block's barrier slot)
+        auto wait_a_free = [&](uint32_t it) -> bool {
+            if (it < (uint32_t)C::kAStages) return true;
+            const uint32_t j = it - (uint32_t)C::kAStages;
+            return wait_bounded(bar_empty + 8 * (j % S), (j / S) & 1u, ctl, P.sb, 31);
+        };
         if constexpr (BITS == 3) {
             // 3-bit codes: twelve words per row and k-block (three per 32-k quarter, each read
             // as 128 contiguous bytes by a warp); the selector nibbles of eight codes are the
@@ -718,14 +842,13 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 uint32_t wn3[12];
                 int zn3 = 0;
                 if (nxt.valid()) fetch3(nxt, wn3, zn3);
-                const int st = cur.it % S;
-                const uint32_t fill = cur.it / S;
+                const int st = cur.it % S, sa = cur.it % C::kAStages;
                 uint32_t t3[2];
                 build_level_tables3(z3, P.L.shift, t3);
-                ok3 = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
+                ok3 = wait_a_free(cur.it);
                 ok3 = __all_sync(0xffffffffu, ok3);
                 if (!ok3) break;
-                uint8_t *arow = gen_base + st * C::kStageBytes + r * 128;
+                uint8_t *arow = gen_base + sa * kABytes + r * 128;
                 const int sw = r & 7;
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
@@ -753,7 +876,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         uint4 w[QT];
         int z = 0;
         auto fetch = [&](const KbCursor &c, uint4 (&dst)[QT], int &zz) {
-            const int nt = c.nt;
+            const int nt = row_tile(c.nt);
             const int n = nt * kTileN + r;
             zz = GROUPED ? P.zeros[(size_t)c.kb * P.L.n_pad + n] : P.zeros[n];
             const uint4 *src = reinterpret_cast<const uint4 *>(
@@ -763,7 +886,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         };
         if (cur.valid()) fetch(cur, w, z);
         bool ok = true;
-        const bool use_offset = P.offset != 0;
+        const bool use_offset = !GROUPED && P.offset != 0;   // (per-channel weights only)
         uint32_t one = 1u;                       // opaque to the compiler: see decode8_offset
         asm volatile("" : "+r"(one));
         while (cur.valid() && ok) {
@@ -772,8 +895,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             uint4 wn[QT];
             int zn = 0;
             if (nxt.valid()) fetch(nxt, wn, zn);                 // prefetch the team's next k-block
-            const int st = cur.it % S;
-            const uint32_t fill = cur.it / S;
+            const int st = cur.it % S, sa = cur.it % C::kAStages;
             uint32_t t[4];
             if (use_offset) build_offset_tables(z, P.lt, P.L.shift, t);
             else build_level_tables(z, P.lt, t);
@@ -808,13 +930,12 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     asm volatile("" : "+r"(lv[q].x), "+r"(lv[q].y), "+r"(lv[q].z), "+r"(lv[q].w));
             }
             {
-                // the operand buffer is free once the MMAs of its last use have retired
-                ok = wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 31);
+                // (all lanes poll: one polling lane per warp was measured a quarter slower)
+                ok = wait_a_free(cur.it);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (!C::kExpandAhead) expand();
-                uint8_t *stage = gen_base + st * C::kStageBytes;
-                uint8_t *arow = stage + r * 128;
+                uint8_t *arow = gen_base + sa * kABytes + r * 128;
                 const int sw = r & 7;
 #pragma unroll
                 for (int q = 0; q < QT; ++q) {
@@ -824,10 +945,11 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(bar_dec + 8 * st);
-                    if (CL > 1) {
+                    if (kPair && rank != 0u) mbar_arrive_cluster(at_leader(bar_dec + 8 * st));
+                    else mbar_arrive(bar_dec + 8 * st);
+                    if (kShare) {
                         // this warp's 16 rows, now complete in the local stage, go to the peer
-                        const uint32_t piece = base + st * C::kStageBytes + (uint32_t)(r * 128);
+                        const uint32_t piece = base + sa * kABytes + (uint32_t)(r * 128);
                         bulk_copy_to_cta(map_to_cta(piece, peer), piece, 16 * 128,
                                          map_to_cta(bar_dec + 8 * st, peer));
                     }
@@ -897,7 +1019,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
 
         for (int u = unit0; u < P.total_units && ok; u += unit_step) {
             const int s = u % P.split_k, rest = u / P.split_k;
-            const int nt = rest % n_tiles, tt = (rest / n_tiles) * CL + (int)rank;
+            const int nt = row_tile(rest % nt_groups), tt = tok_tile_of(rest / nt_groups);
             const int kb0 = s * P.kb_per_split;
             const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
             const int n = nt * kTileN + f;
@@ -941,7 +1063,10 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                         // the accumulator is in registers: hand the buffer back
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+                        if (lane == 0) {
+                            if (kPair && rank != 0u) mbar_arrive_cluster(at_leader(bar_acc_empty + 8 * buf));
+                            else mbar_arrive(bar_acc_empty + 8 * buf);
+                        }
                     }
                     if (c >= valid) continue;             // uniform over the column group
                     if ((P.zp.tok_zero || P.offset) && P.split_k == 1) {
@@ -1033,58 +1158,61 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 asm volatile("" : "+r"(one));
                 const uint32_t neg_magic = __float_as_uint(-12582912.0f);
                 const uint64_t neg_magic2 = pack_f32x2(neg_magic, neg_magic);
-                // the next group's step is loaded one k-block ahead and only touched when used,
-                // so the warp never stalls on that load
-                float step_next = P.scales[(size_t)kb0 * P.L.n_pad + n];
-                // asymmetric activations: the group's level sum of this row, one k-block ahead too
-                const bool asym = P.zp.tok_zero != nullptr;
-                int rs_next = (asym && n_ok) ? __ldg(P.zp.rowsum + (size_t)kb0 * P.L.N + n) : 0;
                 constexpr int kAcc = 16;          // columns per tensor-memory load while accumulating
-                for (int kb = kb0; kb < kb1; ++kb) {
-                    const uint32_t h_bits = __float_as_uint(__fmul_rn(P.unit, step_next));
-                    const uint64_t h2 = pack_f32x2(h_bits, h_bits);
-                    const int rs = rs_next;
-                    if (kb + 1 < kb1) {
-                        step_next = P.scales[(size_t)(kb + 1) * P.L.n_pad + n];
-                        if (asym && n_ok) rs_next = __ldg(P.zp.rowsum + (size_t)(kb + 1) * P.L.N + n);
-                    }
-                    const uint32_t buf = phase % NB;
-                    ok = wait_bounded(bar_acc_full + 8 * buf, (phase / NB) & 1u, ctl, P.sb, 41);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    tc_fence_after();
-                    ++phase;
-#pragma unroll
-                    for (int c = 0; c < C::kColsPerThread; c += kAcc) {
-                        uint32_t v[32];
-                        const uint32_t taddr = tmem_base + lane_base + buf * TOK + col0 + c;
-                        tc_ld16(taddr, v);
-                        tc_wait_ld();
-                        if (c + kAcc >= C::kColsPerThread) {
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+                {
+                    constexpr bool ASYM = ASYM_GROUP;
+                    // the next group's step is loaded one k-block ahead and only touched when
+                    // used, so the warp never stalls on that load; the group's level sum of this
+                    // row (asymmetric activations) likewise
+                    float step_next = P.scales[(size_t)kb0 * P.L.n_pad + n];
+                    int rs_next = 0;
+                    if (ASYM) rs_next = n_ok ? __ldg(P.zp.rowsum + (size_t)kb0 * P.L.N + n) : 0;
+                    for (int kb = kb0; kb < kb1; ++kb) {
+                        const uint32_t h_bits = __float_as_uint(__fmul_rn(P.unit, step_next));
+                        const uint64_t h2 = pack_f32x2(h_bits, h_bits);
+                        const int rs = rs_next;
+                        if (kb + 1 < kb1) {
+                            step_next = P.scales[(size_t)(kb + 1) * P.L.n_pad + n];
+                            if (ASYM && n_ok) rs_next = __ldg(P.zp.rowsum + (size_t)(kb + 1) * P.L.N + n);
                         }
-                        if (asym) {
-                            // the token's zero-point times the group's level sum leaves the
-                            // integer partial before it is scaled
+                        const uint32_t buf = phase % NB;
+                        ok = wait_bounded(bar_acc_full + 8 * buf, (phase / NB) & 1u, ctl, P.sb, 41);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                        tc_fence_after();
+                        ++phase;
 #pragma unroll
-                            for (int j = 0; j < kAcc; ++j)
-                                v[j] = (uint32_t)((int)v[j] - s_tz[col0 + c + j] * rs);
-                        }
+                        for (int c = 0; c < C::kColsPerThread; c += kAcc) {
+                            uint32_t v[32];
+                            const uint32_t taddr = tmem_base + lane_base + buf * TOK + col0 + c;
+                            tc_ld16(taddr, v);
+                            tc_wait_ld();
+                            if (c + kAcc >= C::kColsPerThread) {
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+                            }
+                            if (ASYM) {
+                                // the token's zero-point times the group's level sum leaves the
+                                // integer partial before it is scaled
 #pragma unroll
-                        for (int j = 0; j < kAcc; j += 2) {
-                            const uint64_t biased =
-                                pack_f32x2(biased_float_bits(v[j], one), biased_float_bits(v[j + 1], one));
-                            usum2[(c + j) >> 1] =
-                                fma_f32x2(add_f32x2(biased, neg_magic2), h2, usum2[(c + j) >> 1]);
-                        }
-                        if (P.acc_out && n_ok) {
+                                for (int j = 0; j < kAcc; ++j)
+                                    v[j] = (uint32_t)((int)v[j] - s_tz[col0 + c + j] * rs);
+                            }
 #pragma unroll
-                            for (int j = 0; j < kAcc; ++j)
-                                if (c + j < valid)
-                                    P.acc_out[((size_t)kb * P.M + tok0 + c + j) * P.L.N + n] =
-                                        (int)v[j];
+                            for (int j = 0; j < kAcc; j += 2) {
+                                const uint64_t biased =
+                                    pack_f32x2(biased_float_bits(v[j], one), biased_float_bits(v[j + 1], one));
+                                usum2[(c + j) >> 1] =
+                                    fma_f32x2(add_f32x2(biased, neg_magic2), h2, usum2[(c + j) >> 1]);
+                            }
+                            if (P.acc_out && n_ok) {
+#pragma unroll
+                                for (int j = 0; j < kAcc; ++j)
+                                    if (c + j < valid)
+                                        P.acc_out[((size_t)kb * P.M + tok0 + c + j) * P.L.N + n] =
+                                            (int)v[j];
+                            }
                         }
                     }
                 }
@@ -1166,9 +1294,14 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     if (CL > 1) cluster_sync_all();
     if (role == kMma) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                     "r"((uint32_t)C::kTmemCols)
-                     : "memory");
+        if (kPair)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                         "r"((uint32_t)C::kTmemCols)
+                         : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                         "r"((uint32_t)C::kTmemCols)
+                         : "memory");
     }
 }
 
@@ -1217,12 +1350,12 @@ int resident_clusters()
         n = device_sms();
     } else {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(CL * device_sms());
+        cfg.gridDim = dim3(C::kCtas * device_sms());
         cfg.blockDim = dim3(C::kThreads);
         cfg.dynamicSmemBytes = C::kSmemBytes;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = CL;
+        attr[0].val.clusterDim.x = C::kCtas;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
@@ -1245,7 +1378,7 @@ w4a8_status launch_cl(const Maps &maps, const Params &P, cudaStream_t st)
     if (resident < 1) return W4A8_ERR_CUDA;
     const int clusters = P.total_units < resident ? P.total_units : resident;
     const cudaError_t e =
-        launch_overlapped_cluster(kern, dim3(clusters * CL), dim3(C::kThreads), (size_t)C::kSmemBytes, st, CL,
+        launch_overlapped_cluster(kern, dim3(clusters * C::kCtas), dim3(C::kThreads), (size_t)C::kSmemBytes, st, C::kCtas,
                           maps.tok, C::kChunk == 32 ? maps.y32 : maps.y16, P);
     return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
 }
@@ -1256,6 +1389,9 @@ w4a8_status launch_dw(const Maps &maps, const Params &P, int cluster, cudaStream
     // two-CTA clusters exist for the wide token tiles: narrow ones serve few tokens
     if constexpr (TOK >= 128) {
         if (cluster == 2) return launch_cl<TOK, GROUPED, DW, 2>(maps, P, st);
+    }
+    if constexpr (TOK == 256 && !GROUPED && (DW == 8 || DW == 16)) {
+        if (cluster == 3) return launch_cl<TOK, false, DW, 3>(maps, P, st);
     }
     if (cluster == 1) return launch_cl<TOK, GROUPED, DW, 1>(maps, P, st);
     return W4A8_ERR_SHAPE;
@@ -1270,6 +1406,15 @@ w4a8_status launch_one(const Maps &maps, const Params &P, int dw, int cluster, c
     if (P.swiglu) {
         if (cluster != 1 || P.split_k != 1 || dw != (GROUPED ? 8 : 16)) return W4A8_ERR_SHAPE;
         return launch_cl<TOK, GROUPED, GROUPED ? 8 : 16, 1, kSwigluVariant>(maps, P, st);
+    }
+    if constexpr (GROUPED) {
+        // asymmetric activations with group steps: a kernel variant of its own, one CTA per cluster
+        if (P.zp.tok_zero) {
+            if (cluster != 1) return W4A8_ERR_SHAPE;
+            if (dw == 4) return launch_cl<TOK, true, 4, 1, kAsymGroupVariant>(maps, P, st);
+            if (dw == 8) return launch_cl<TOK, true, 8, 1, kAsymGroupVariant>(maps, P, st);
+            return W4A8_ERR_SHAPE;
+        }
     }
     if (dw == 4) return launch_dw<TOK, GROUPED, 4>(maps, P, cluster, st);
     if (dw == 8) return launch_dw<TOK, GROUPED, 8>(maps, P, cluster, st);
@@ -1336,10 +1481,14 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     // that gains (2200 against 2380 TOPS sustained), so the automatic plan stays with one CTA.
     int cluster = opts ? opts->cluster : 0;
     if (cluster == 0) cluster = 1;
-    if (cluster != 1 && !(cluster == 2 && tok >= 128)) return false;
-    const int tok_groups = (tok_tiles + cluster - 1) / cluster;
+    // (3: the MMA pair - 256-token tiles, per-channel 4-bit weights, an even number of row tiles)
+    const bool pair = cluster == 3;
+    if (pair && !(tok == 256 && !grouped && L.bits == 4 && L.n_tiles % 2 == 0)) return false;
+    if (cluster != 1 && !pair && !(cluster == 2 && tok >= 128)) return false;
+    const int share = cluster == 2 ? 2 : 1;
+    const int tok_groups = (tok_tiles + share - 1) / share;
     // one counter per (token tile, row tile), empty partner tiles included
-    const long long tiles = (long long)tok_groups * cluster * L.n_tiles;
+    const long long tiles = (long long)tok_groups * share * L.n_tiles;
     if (split < 1 || split > L.k_blocks) return false;
     const int kb_per = (L.k_blocks + split - 1) / split;
     split = (L.k_blocks + kb_per - 1) / kb_per;              // no empty slice
@@ -1393,7 +1542,8 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     // (P*V form: the token blocks of all row tiles are stacked, one after the other)
     const cuuint64_t dims[2] = {(cuuint64_t)L.K, (cuuint64_t)M * (plan.batched ? L.n_tiles : 1)};
     const cuuint64_t strides[1] = {(cuuint64_t)L.K};
-    const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)plan.tok_tile};
+    // (an MMA pair: each CTA loads half of the token tile)
+    const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)(plan.cluster == 3 ? plan.tok_tile / 2 : plan.tok_tile)};
     const cuuint32_t estr[2] = {1, 1};
     if (enc(&maps.tok, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(Xq), dims, strides,
             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -1434,7 +1584,11 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     P.m_pad = plan.tok_tiles * plan.tok_tile;
     P.split_k = plan.split_k;
     P.kb_per_split = plan.kb_per_split;
-    P.total_units = (plan.tok_tiles + plan.cluster - 1) / plan.cluster * L.n_tiles * plan.split_k;
+    // units: (token-tile group, row-tile group, K slice); a sharing pair groups two token tiles,
+    // an MMA pair two row tiles
+    P.total_units = plan.cluster == 2 ? (plan.tok_tiles + 1) / 2 * L.n_tiles * plan.split_k
+                  : plan.cluster == 3 ? plan.tok_tiles * (L.n_tiles / 2) * plan.split_k
+                                      : plan.tok_tiles * L.n_tiles * plan.split_k;
     P.prefetch_codes = plan.tok_tiles == 1 ? 1 : 0;   // every code tile is read exactly once
     P.zp = zp;
     P.lt = make_level_tables(L.shift);

@@ -246,3 +246,21 @@ def test_tcgen05_offset_tables_every_zero_point():
         Y, acc = run_linear(prob, w4a8.make_opts(w4a8.PATH_TCGEN05, tok_tile=tok_tile, offset_tables=1))
         assert np.array_equal(acc, prob.oracle_acc())
         check_y(prob, Y, exact=True)
+
+
+def test_tcgen05_mma_pair():
+    """Two CTAs as one MMA pair (cta_group::2): two row tiles per instruction, each CTA loads half
+    of the 256-token tile; the leader's barriers collect both CTAs' arrivals.  Ragged token tile,
+    several units per cluster, a K split; same bits as the one-CTA form."""
+    prob = Problem(1536, 128 * 44, 2 * 256 + 37, 0, seed=721)
+    packed = w4a8.pack_weights(prob.dev["W"], prob.dev["s"], 0)
+    want = prob.oracle_acc()
+    for split, dw in ((1, 16), (1, 8), (3, 16)):
+        opts = w4a8.make_opts(w4a8.PATH_TCGEN05, split_k=split, tok_tile=256, decode_warps=dw, cluster=3)
+        for _ in range(2):
+            Y, acc = run_linear(prob, opts, packed)
+            assert np.array_equal(acc, want)
+            check_y(prob, Y, exact=True)
+    assert w4a8.linear_workspace_bytes(300, 384, 256, 0, w4a8.make_opts(tok_tile=256, cluster=3)) == 0   # odd row tiles
+    assert w4a8.linear_workspace_bytes(300, 512, 256, 0, w4a8.make_opts(tok_tile=128, cluster=3)) == 0
+    assert w4a8.linear_workspace_bytes(300, 512, 256, 128, w4a8.make_opts(tok_tile=256, cluster=3)) == 0
