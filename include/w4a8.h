@@ -66,15 +66,20 @@ typedef struct {
                         or 32) */
     int level_shift; /* special value of the blob = step / 2^level_shift: 0 or 1 (the paper's
                         step/2), 2 or 3 (w4a8_pack_weights_fmt); must match the blob */
-    int cluster;     /* 0 = automatic (one CTA); else the cluster form of the tensor-core kernel:
-                        1 = one CTA per cluster;
+    int cluster;     /* 0 = automatic: form 3 with offset tables for 1024 tokens and more when the
+                        shape allows it (and decode_warps and offset_tables are 0), else form 1;
+                        else the form of the tensor-core kernel:
+                        1 = one CTA per cluster, one row tile per CTA;
                         2 = sharing pair (token tiles of 128 and more, symmetric activations
                             when the weights are grouped): two CTAs work on two token tiles of
                             the same weight rows and each expands half of every code tile for both;
-                        3 = MMA pair (token tile 256, per-channel 4-bit weights, an even number
-                            of 128-row tiles, 8 or 16 decode warps): two CTAs on two row tiles
-                            and one token tile issue every MMA as one 256-row instruction, each
-                            loads half of the tokens.
+                        3 = MMA pair (token tile 256, per-channel 4-bit weights, even numbers
+                            of 128-row tiles and of k-blocks per K slice, 8 or 16 decode warps): two
+                            CTAs on two row tiles and one token tile issue every MMA as one
+                            256-row instruction, each loads half of the tokens;
+                        4 = two row tiles per CTA (token tile 256, per-channel 4-bit weights, an
+                            even number of 128-row tiles, 16 decode warps): one CTA multiplies
+                            two row tiles by the same token buffer.
                         Same bits in every form; a form that does not fit the call is refused
                         with W4A8_ERR_SHAPE. */
     int debug_wait_ms;   /* test hook, 0 = off: limit of every bounded wait inside the tensor-core
@@ -87,7 +92,8 @@ typedef struct {
     int bits;        /* code width of the blob: 0 or 4 (dINT4), or 3 (dINT3, packed by
                         w4a8_pack_weights_bits); must match the blob.  3-bit blobs run on the
                         tensor-core kernel (any M) or the simple kernel, with symmetric activations */
-    int offset_tables; /* 0 = off; 1 = the tensor-core kernel expands codes through level tables
+    int offset_tables; /* 0 = off (on with the automatic MMA pair, see cluster); 1 = the
+                        tensor-core kernel expands codes through level tables
                         stored with an offset (fewer logic instructions per code) and takes the
                         offset out again with the tokens' sums, which a small kernel in front
                         computes into the workspace.  Per-channel 4-bit weights, level_shift
@@ -182,7 +188,7 @@ size_t w4a8_linear_workspace_bytes_ex(int M, int N, int K, int group_size,
  * (NULL = automatic, i.e. what w4a8_linear runs), without touching a device.  `out` is a host
  * array of 5: out[0] = w4a8_path; out[1] = tokens per tile (tensor-core kernel, else 0);
  * out[2] = K slices; out[3] = warps that expand codes (tensor-core kernel) or warps of a
- * row-slab CTA (weight-streaming kernel; 0 = its K-sliced variant); out[4] = CTAs per cluster.
+ * row-slab CTA (weight-streaming kernel; 0 = its K-sliced variant); out[4] = cluster form (see w4a8_opts.cluster).
  * The plan follows the SM
  * count of the current device (148 when there is none).  Eq. 1 fixes the result, not the plan:
  * this call only reports the choice, e.g. where the weight-streaming kernel hands over to the

@@ -37,7 +37,7 @@ bool opts_ok(const w4a8_opts *o)
     if (o->path < W4A8_PATH_AUTO || o->path > W4A8_PATH_GEMV) return false;
     if (o->split_k < 0 || o->tok_tile < 0 || o->decode_warps < 0) return false;
     if (o->level_shift < 0 || o->level_shift > 3) return false;
-    if (o->cluster < 0 || o->cluster > 3) return false;
+    if (o->cluster < 0 || o->cluster > 4) return false;
     if (o->offset_tables < 0 || o->offset_tables > 1 || (o->bits != 0 && !bits_ok(o->bits))) return false;
     if (o->offset_tables && (o->path == W4A8_PATH_GEMV || o->path == W4A8_PATH_SIMPLE)) return false;
     if (o->bits == 3 && (o->path == W4A8_PATH_GEMV || o->cluster >= 2)) return false;
@@ -113,7 +113,7 @@ w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *
         return launch_linear_gemv(Xq, tok_scale, blob, L, bias, M, static_cast<__nv_bfloat16 *>(Y),
                                   acc, static_cast<uint8_t *>(workspace), plan, st, zp);
     }
-    if (!make_plan(M, L, opts, &plan)) return W4A8_ERR_SHAPE;
+    if (!make_plan(M, L, opts, &plan, true)) return W4A8_ERR_SHAPE;
     return launch_linear_tcgen05(Xq, tok_scale, blob, L, bias, M, static_cast<__nv_bfloat16 *>(Y),
                                  acc, static_cast<uint8_t *>(workspace), plan, st, zp);
 }
@@ -212,7 +212,7 @@ size_t w4a8_linear_workspace_bytes_ex(int M, int N, int K, int group_size, const
         gemv_plan(M, make_layout(N, K, group_size), &plan);
         return plan.workspace_bytes;
     }
-    if (!make_plan(M, make_layout(N, K, group_size, shift_of(opts), bits_of(opts)), opts, &plan)) return 0;
+    if (!make_plan(M, make_layout(N, K, group_size, shift_of(opts), bits_of(opts)), opts, &plan, true)) return 0;
     return plan.workspace_bytes;
 }
 
@@ -242,7 +242,7 @@ w4a8_status w4a8_linear_plan(int M, int N, int K, int group_size, const w4a8_opt
         out[3] = warps;
         return W4A8_OK;
     }
-    if (!make_plan(M, L, opts, &plan)) return W4A8_ERR_SHAPE;
+    if (!make_plan(M, L, opts, &plan, true)) return W4A8_ERR_SHAPE;
     out[0] = W4A8_PATH_TCGEN05;
     out[1] = plan.tok_tile;
     out[2] = plan.split_k;

@@ -307,7 +307,9 @@ cudaError_t launch_linear_simple(const int8_t *Xq, const float *tok_scale, const
                                  const BlobLayout &L, const float *bias, int M,
                                  __nv_bfloat16 *Y, int32_t *acc, StatusBlock *sb,
                                  cudaStream_t st, ZeroPoint zp = ZeroPoint());
-bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *plan);
+// auto_pair: the automatic plan may choose the MMA pair with offset tables (callers whose token
+// layout or epilogue the pair does not cover leave it off)
+bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *plan, bool auto_pair = false);
 w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, const uint8_t *blob,
                                   const BlobLayout &L, const float *bias, int M,
                                   __nv_bfloat16 *Y, int32_t *acc, uint8_t *workspace,

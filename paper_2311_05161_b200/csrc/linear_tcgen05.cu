@@ -57,9 +57,6 @@ struct Cfg {
     static constexpr int kAStagesWanted = GROUPED ? 5 : (TOK >= 256 && CL != 3) ? 3 : 4;
     static constexpr int kEpiWarps = 4 * kEpiGroups;
     static constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
-    // With at most 512 threads a thread has the registers to expand its codes before the stage
-    // they go to is free (its raw codes, the next k-block's raw codes and the expanded levels).
-    static constexpr bool kExpandAhead = kThreads <= 512;
     static constexpr int kColsPerThread = TOK / kEpiGroups;
     static constexpr int kChunk = kColsPerThread >= 32 ? 32 : 16;
     // CL = 1: one CTA.  CL = 2 (kShare): two CTAs on the same row tile, each on its own token
@@ -67,8 +64,19 @@ struct Cfg {
     // same token tile run as one MMA pair (cta_group::2): every MMA instruction covers both row
     // tiles, CTA r holds (and loads) tokens 128 r .. 128 r + 127 of the tile, and the leader's one
     // issuing thread serves both, so the token bytes per SM and the issue cost per CTA halve.
-    static constexpr bool kShare = CL == 2, kPair = CL == 3;
-    static constexpr int kCtas = CL == 1 ? 1 : 2;
+    // CL = 4 (kDual): one CTA on two row tiles and one token tile: the two tiles' MMAs read the same
+    // token buffer, so the token bytes per MAC halve as in the MMA pair, without any traffic
+    // between CTAs; the two accumulators fill tensor memory, so the epilogue of a unit no longer
+    // overlaps the next unit's main loop.
+    static constexpr bool kShare = CL == 2, kPair = CL == 3, kDual = CL == 4;
+    static constexpr int kCtas = (kShare || kPair) ? 2 : 1;
+    static constexpr int kTiles = kDual ? 2 : 1;               // row tiles of a unit in this CTA
+    // k-blocks per barrier round.  The issuing thread's loop (wait, MMAs, commit) is the serial
+    // spine of the kernel, and its fixed part per round (wait, commit, bookkeeping: some 300
+    // cycles) is what keeps an MMA pair from outrunning one CTA; with two k-blocks per round the
+    // pair pays it once per eight MMA instructions.  Operand buffers stay one k-block each.
+    static constexpr int kSub = kPair ? 2 : 1;
+    static constexpr int kPerRound = kTiles * kSub;            // weight buffers filled per round
     static constexpr int kTokRows = kPair ? TOK / 2 : TOK;     // token rows this CTA loads per k-block
     static constexpr int kTokBytes = kTokRows * kTileK;
     // Codes go from global memory straight into the decode threads' registers (shared-memory
@@ -86,13 +94,15 @@ struct Cfg {
     // that completes on the peer's barrier, so the table lookups per MMA halve.
     static constexpr int kRowsPerCta = kShare ? kTileN / 2 : kTileN;
     static constexpr int kQuartersPerThread = kShare ? 2 : 4;   // 32-k quarters of a row per thread
-    static_assert(CL >= 1 && CL <= 3, "one CTA, a sharing pair or an MMA pair");
+    static_assert(CL >= 1 && CL <= 4, "one CTA, a sharing pair, an MMA pair or two row tiles per CTA");
+    static_assert(!kDual || (TOK == 256 && !GROUPED), "two row tiles per CTA: 256 tokens, per-channel weights");
     static_assert(!kPair || (TOK == 256 && !GROUPED), "the MMA pair: 256 tokens, per-channel weights");
     static_assert(DW % kTeamWarps == 0 && kTeamWarps == 4, "decode warps form whole teams of four");
     // Two rings of operand buffers, one set of barriers.  Ring A holds decoded INT8 weights of a
     // k-block (16 KiB, written by the decode warps), ring B the tokens of a k-block (written by
     // TMA).  K-block number `it` uses A buffer it % kAStages, B buffer it % kStages and the barrier
-    // pair it % kStages.  The rings differ in depth because they hide different latencies: a
+    // pair it % kStages (with two row tiles per unit: weight buffer (2 it + h) % kAStages for
+    // tile h).  The rings differ in depth because they hide different latencies: a
     // token tile comes from L2 and is on its way for a few thousand cycles when all SMs pull
     // tiles at once (the bytes in flight bound the rate), decoded weights come from registers.
     // (Keeping operand A in tensor memory instead was measured slower at every token tile.)
@@ -489,8 +499,9 @@ __device__ __forceinline__ bool wait_bounded_idle(uint32_t bar, uint32_t parity,
 struct KbCursor {
     int u, step, total_units, split_k, kb_per_split, k_blocks, n_tiles;
     int kb, kb1;
-    int nt;                    // row tile of the unit (integer divisions happen once per unit)
-    uint32_t it;
+    int nt;                    // row-tile group of the unit (integer divisions happen once per unit)
+    int h, tiles;              // row tile inside the unit, row tiles per unit
+    uint32_t it;               // counts (k-block, tile) items
     __device__ __forceinline__ void open_unit()
     {
         if (u < total_units) {
@@ -502,10 +513,10 @@ struct KbCursor {
         }
     }
     __device__ __forceinline__ void start(int first, int stride, int total, int split, int per,
-                                          int kbs, int tiles)
+                                          int kbs, int groups, int tiles_per_unit = 1)
     {
         u = first; step = stride; total_units = total; split_k = split; kb_per_split = per;
-        k_blocks = kbs; n_tiles = tiles; it = 0; kb = kb1 = 0; nt = 0;
+        k_blocks = kbs; n_tiles = groups; it = 0; kb = kb1 = 0; nt = 0; h = 0; tiles = tiles_per_unit;
         open_unit();
     }
     __device__ __forceinline__ bool valid() const { return u < total_units; }
@@ -513,6 +524,8 @@ struct KbCursor {
     {
         for (int i = 0; i < n && valid(); ++i) {
             ++it;
+            if (++h < tiles) continue;
+            h = 0;
             if (++kb >= kb1) {
                 u += step;
                 open_unit();
@@ -601,12 +614,13 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     // Units (token-tile group, row-tile group, K slice) are dealt round-robin to the clusters.
     // Sharing pair: CTA `rank` takes token tile 2 * group + rank of the unit.  MMA pair: CTA
     // `rank` takes row tile 2 * group + rank.
-    constexpr bool kShare = C::kShare, kPair = C::kPair;
-    const uint32_t rank = CL > 1 ? cluster_ctarank() : 0u;
+    constexpr bool kShare = C::kShare, kPair = C::kPair, kDual = C::kDual;
+    constexpr int kTiles = C::kTiles, kSub = C::kSub;
+    const uint32_t rank = C::kCtas > 1 ? cluster_ctarank() : 0u;
     const int unit0 = (int)blockIdx.x / C::kCtas, unit_step = (int)gridDim.x / C::kCtas;
     // row-tile groups of the unit list, and this CTA's row / token tile inside a unit
-    const int nt_groups = kPair ? P.L.n_tiles / 2 : P.L.n_tiles;
-    auto row_tile = [&](int g) { return kPair ? 2 * g + (int)rank : g; };
+    const int nt_groups = (kPair || kDual) ? P.L.n_tiles / 2 : P.L.n_tiles;
+    auto row_tile = [&](int g, int h = 0) { return kPair ? 2 * g + (int)rank : kDual ? 2 * g + h : g; };
     auto tok_tile_of = [&](int g) { return kShare ? 2 * g + (int)rank : g; };
     // the barriers the MMA thread waits on live in the leader CTA of an MMA pair
     const bool leader = !kPair || rank == 0u;
@@ -618,7 +632,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             // cluster, the peer's half of the expanded rows complete on it too
             // (MMA pair: the leader's barrier collects both CTAs' arrivals)
             // (MMA pair: the leader's barrier collects the decode warps of both CTAs)
-            mbar_init(bar_dec + 8 * s, kPair ? 2 * C::kTeamWarps + 1 : C::kTeamWarps + 1);
+            // (two row tiles per CTA: the teams of both tiles)
+            mbar_init(bar_dec + 8 * s, C::kPerRound * C::kTeamWarps * (kPair ? 2 : 1) + 1);
             // sharing pair: the MMA threads of both CTAs, which all read rows this CTA wrote
             mbar_init(bar_empty + 8 * s, kShare ? 2 : 1);
         }
@@ -653,7 +668,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     tc_fence_before();
     __syncthreads();
     // no CTA may touch a peer's barriers or stages before the peer has set them up
-    if (CL > 1) cluster_sync_all();
+    if (C::kCtas > 1) cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     // Set-up is done; earlier work in the stream (the activation quantizer, a previous call's
@@ -672,7 +687,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             uint32_t it = 0;
             bool ok = true;
             KbCursor pf;
-            pf.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, nt_groups);
+            pf.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, nt_groups, kTiles);
             for (int u = unit0; u < P.total_units && ok; u += unit_step) {
                 const int s = u % P.split_k, rest = u / P.split_k;
                 const int tt = tok_tile_of(rest / nt_groups);
@@ -680,22 +695,27 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 const int kb0 = s * P.kb_per_split;
                 const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                    // token buffer it % S, last used by k-block it - S: free once the round of
+                    // that k-block has retired; the copy completes on the barrier of its own round
                     const int st = it % S;
-                    const uint32_t fill = it / S;
-                    if (!wait_bounded(bar_empty + 8 * st, (fill & 1u) ^ 1u, ctl, P.sb, 10)) {
-                        ok = false;
-                        break;
+                    if (it >= (uint32_t)S) {
+                        const uint32_t r = (it - (uint32_t)S) / kSub;
+                        if (!wait_bounded(bar_empty + 8 * (r % S), (r / S) & 1u, ctl, P.sb, 10)) {
+                            ok = false;
+                            break;
+                        }
                     }
                     if (P.skip_load != 0 && it == (uint32_t)(P.skip_load - 1)) continue;
                     const uint32_t tok_dst = base + C::kOffTokRing + st * C::kTokBytes;
-                    const uint32_t tok_bar = bar_dec + 8 * st;
+                    const uint32_t tok_bar = bar_dec + 8 * ((it / kSub) % S);
                     if (kPair) {
                         // this CTA's 128 of the tile's 256 tokens; completion counts at the leader
                         // (the leader's copy thread announces both CTAs' bytes with its own
                         // arrival; the other CTA only issues its copy: a release-arrival on a
                         // remote barrier was measured to cost that thread about a microsecond)
                         const uint32_t lead_bar = at_leader(tok_bar);
-                        if (rank == 0u) mbar_arrive_expect_tx(tok_bar, 2 * C::kTokBytes);
+                        // (once per round: the bytes of both its k-blocks)
+                        if (rank == 0u && it % kSub == 0) mbar_arrive_expect_tx(tok_bar, 2 * kSub * C::kTokBytes);
                         tma_load_2d_pair(tok_dst, &tok_map, kb * kTileK,
                                          tt * TOK + (int)rank * C::kTokRows, lead_bar);
                     } else {
@@ -705,8 +725,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     }
                     if (P.prefetch_codes) {
                         // keep the code stream kPrefetchAhead k-blocks ahead of the decode warps
-                        while (pf.valid() && pf.it < it + C::kPrefetchAhead) {
-                            const int pnt = row_tile(pf.nt);
+                        while (pf.valid() && pf.it < (it + C::kPrefetchAhead) * kTiles) {
+                            const int pnt = row_tile(pf.nt, pf.h);
                             prefetch_l2(P.codes + ((size_t)pnt * k_blocks + pf.kb) * (BITS == 3 ? kTileBytes3 : kTileBytes),
                                         BITS == 3 ? kTileBytes3 : kTileBytes);
                             pf.advance(1);
@@ -718,8 +738,9 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 // copies already issued must land before the CTA gives its memory back (in an MMA
                 // pair the leader's barriers count both CTAs' copies, and the other CTA stays
                 // until the leader is through: the cluster barrier at the end)
-                const uint32_t first = it > (uint32_t)S ? it - S : 0u;
-                for (uint32_t j = first; j < it; ++j)
+                // (a round of which only a part was issued never completes: that wait runs out)
+                const uint32_t first = (it > (uint32_t)S ? it - S : 0u) / kSub;
+                for (uint32_t j = first; j < (it + kSub - 1) / kSub; ++j)
                     wait_bounded(bar_dec + 8 * (j % S), (j / S) & 1u, ctl, P.sb, 11, true);
             }
         }
@@ -734,51 +755,85 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
             const uint32_t a_lo0 = ((base & 0x3FFFFu) >> 4) | (1u << 16);
             const uint32_t b_lo0 = (((base + C::kOffTokRing) & 0x3FFFFu) >> 4) | (1u << 16);
-            uint32_t st = 0, st_par = 0;                 // token buffer (= barrier slot), fill parity
-            uint32_t sa = 0;                             // weight buffer
+            uint32_t st = 0, st_par = 0;                 // barrier slot of the round and its parity
+            uint32_t sa = 0, tb = 0;                     // weight buffer, token buffer
             uint32_t buf = 0, buf_par = 0;               // accumulator buffer and its parity
             bool ok = true;
             for (int u = unit0; u < P.total_units && ok; u += unit_step) {
                 const int s = u % P.split_k;
                 const int kb0 = s * P.kb_per_split;
                 const int nkb = min(k_blocks, kb0 + P.kb_per_split) - kb0;
-                for (int i = 0; i < nkb; ++i) {
+                for (int i = 0; i < nkb; i += C::kSub) {
                     const bool first = GROUPED || i == 0;
-                    const bool last = GROUPED || i == nkb - 1;
-                    if (first &&
+                    const bool last = GROUPED || i + C::kSub >= nkb;
+                    if (!kDual && first &&
                         !wait_bounded<kPair>(bar_acc_empty + 8 * buf, buf_par ^ 1u, ctl, P.sb, 20)) {
                         ok = false;
                         break;
                     }
-                    // decoded weights and tokens of the stage
+                    // decoded weights and tokens of the round
                     if (!wait_bounded<kPair>(bar_dec + 8 * st, st_par, ctl, P.sb, 21)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t d = tmem_base + buf * TOK;
-                    const uint64_t a_desc = ((uint64_t)kDescHi << 32) | (a_lo0 + sa * (kABytes >> 4));
-                    const uint64_t b_desc = ((uint64_t)kDescHi << 32) | (b_lo0 + st * (C::kTokBytes >> 4));
+                    if constexpr (kDual) {
+                        // both row tiles of the unit against the same tokens; accumulator h belongs
+                        // to tile h, and the epilogue hands the two back one after the other
+                        const uint64_t b_desc = ((uint64_t)kDescHi << 32) | (b_lo0 + tb * (C::kTokBytes >> 4));
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const uint32_t acc_flag = (!first || ks > 0) ? 1u : 0u;
-                        if (kPair)
-                            tc_mma_i8_pair(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
-                                           acc_flag);
-                        else
-                            tc_mma_i8(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
-                                      acc_flag);
-                    }
-                    if (kPair) tc_commit_pair(bar_empty + 8 * st, kBoth);
-                    else if (kShare) tc_commit_multicast(bar_empty + 8 * st, kBoth);
-                    else tc_commit(bar_empty + 8 * st);
-                    if (last) {
-                        if (kPair) tc_commit_pair(bar_acc_full + 8 * buf, kBoth);
-                        else tc_commit(bar_acc_full + 8 * buf);
-                        if (++buf == (uint32_t)NB) { buf = 0; buf_par ^= 1u; }
+                        for (int h = 0; h < 2; ++h) {
+                            if (first &&
+                                !wait_bounded(bar_acc_empty + 8 * h, buf_par ^ 1u, ctl, P.sb, 20)) {
+                                ok = false;
+                                break;
+                            }
+                            if (first) tc_fence_after();
+                            const uint64_t a_desc = ((uint64_t)kDescHi << 32) | (a_lo0 + sa * (kABytes >> 4));
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks)
+                                tc_mma_i8(tmem_base + h * TOK, a_desc + (uint64_t)(ks * 2),
+                                          b_desc + (uint64_t)(ks * 2), idesc, (!first || ks > 0) ? 1u : 0u);
+                            if (++sa == (uint32_t)C::kAStages) sa = 0;
+                        }
+                        if (!ok) break;
+                        if (++tb == (uint32_t)S) tb = 0;
+                        tc_commit(bar_empty + 8 * st);
+                        if (last) {
+                            tc_commit(bar_acc_full);
+                            tc_commit(bar_acc_full + 8);
+                            buf_par ^= 1u;
+                        }
+                    } else {
+                        const uint32_t d = tmem_base + buf * TOK;
+#pragma unroll
+                        for (int h = 0; h < C::kSub; ++h) {
+                            // (the k-blocks of a round: one weight and one token buffer each)
+                            const uint64_t a_desc = ((uint64_t)kDescHi << 32) | (a_lo0 + sa * (kABytes >> 4));
+                            const uint64_t b_desc = ((uint64_t)kDescHi << 32) | (b_lo0 + tb * (C::kTokBytes >> 4));
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks) {
+                                const uint32_t acc_flag = (!first || h > 0 || ks > 0) ? 1u : 0u;
+                                if (kPair)
+                                    tc_mma_i8_pair(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2),
+                                                   idesc, acc_flag);
+                                else
+                                    tc_mma_i8(d, a_desc + (uint64_t)(ks * 2), b_desc + (uint64_t)(ks * 2), idesc,
+                                              acc_flag);
+                            }
+                            if (++sa == (uint32_t)C::kAStages) sa = 0;
+                            if (++tb == (uint32_t)S) tb = 0;
+                        }
+                        if (kPair) tc_commit_pair(bar_empty + 8 * st, kBoth);
+                        else if (kShare) tc_commit_multicast(bar_empty + 8 * st, kBoth);
+                        else tc_commit(bar_empty + 8 * st);
+                        if (last) {
+                            if (kPair) tc_commit_pair(bar_acc_full + 8 * buf, kBoth);
+                            else tc_commit(bar_acc_full + 8 * buf);
+                            if (++buf == (uint32_t)NB) { buf = 0; buf_par ^= 1u; }
+                        }
                     }
                     if (++st == (uint32_t)S) { st = 0; st_par ^= 1u; }
-                    if (++sa == (uint32_t)C::kAStages) sa = 0;
                 }
             }
             // nothing issued may still be running when tensor memory is freed
@@ -804,13 +859,14 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         // the same stage and barrier in the peer CTA
         const uint32_t peer = rank ^ 1u;
         KbCursor cur;
-        cur.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, nt_groups);
+        cur.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, nt_groups, kTiles);
         cur.advance(team);
-        // the weight buffer of k-block `it` is free once the MMAs of k-block it - kAStages, its
-        // last user, have retired (their commit completed a phase of that k-block's barrier slot)
+        // Items (k-block, row tile of the unit) are numbered in the order the MMAs use them.  The
+        // weight buffer of item `it` is free once the MMAs of item it - kAStages, its last user,
+        // have retired (their commit completed a phase of that item's k-block's barrier slot).
         auto wait_a_free = [&](uint32_t it) -> bool {
             if (it < (uint32_t)C::kAStages) return true;
-            const uint32_t j = it - (uint32_t)C::kAStages;
+            const uint32_t j = (it - (uint32_t)C::kAStages) / C::kPerRound;
             return wait_bounded(bar_empty + 8 * (j % S), (j / S) & 1u, ctl, P.sb, 31);
         };
         if constexpr (BITS == 3) {
@@ -842,7 +898,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                 uint32_t wn3[12];
                 int zn3 = 0;
                 if (nxt.valid()) fetch3(nxt, wn3, zn3);
-                const int st = cur.it % S, sa = cur.it % C::kAStages;
+                const int st = (cur.it / C::kPerRound) % S, sa = cur.it % C::kAStages;
                 uint32_t t3[2];
                 build_level_tables3(z3, P.L.shift, t3);
                 ok3 = wait_a_free(cur.it);
@@ -876,7 +932,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         uint4 w[QT];
         int z = 0;
         auto fetch = [&](const KbCursor &c, uint4 (&dst)[QT], int &zz) {
-            const int nt = row_tile(c.nt);
+            const int nt = row_tile(c.nt, c.h);
             const int n = nt * kTileN + r;
             zz = GROUPED ? P.zeros[(size_t)c.kb * P.L.n_pad + n] : P.zeros[n];
             const uint4 *src = reinterpret_cast<const uint4 *>(
@@ -892,10 +948,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         while (cur.valid() && ok) {
             KbCursor nxt = cur;
             nxt.advance(T);
-            uint4 wn[QT];
-            int zn = 0;
-            if (nxt.valid()) fetch(nxt, wn, zn);                 // prefetch the team's next k-block
-            const int st = cur.it % S, sa = cur.it % C::kAStages;
+            const int st = (cur.it / C::kPerRound) % S, sa = cur.it % C::kAStages;
             uint32_t t[4];
             if (use_offset) build_offset_tables(z, P.lt, P.L.shift, t);
             else build_level_tables(z, P.lt, t);
@@ -921,20 +974,23 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     decode8(wq.w, t, lv[2 * q + 1].z, lv[2 * q + 1].w);
                 }
             };
-            if (C::kExpandAhead) {
-                // The levels are ready in registers before the stage is: only the stores stand
-                // between the moment the stage is free and the moment its operands are in place.
-                expand();
+            // The levels are ready in registers before the buffer is: only the stores stand between
+            // the moment the buffer is free and the moment its operand is in place (the expansion
+            // of a tile takes a team a few thousand cycles while all teams work, more than the
+            // ring of weight buffers can hide).  The codes of the team's next item are requested
+            // only now, into the registers the expansion has just read, so a thread holds raw
+            // codes and levels of one item at a time; the wait and the stores cover the loads.
+            expand();
 #pragma unroll
-                for (int q = 0; q < 2 * QT; ++q)
-                    asm volatile("" : "+r"(lv[q].x), "+r"(lv[q].y), "+r"(lv[q].z), "+r"(lv[q].w));
-            }
+            for (int q = 0; q < 2 * QT; ++q)
+                asm volatile("" : "+r"(lv[q].x), "+r"(lv[q].y), "+r"(lv[q].z), "+r"(lv[q].w));
+            int zn = 0;
+            if (nxt.valid()) fetch(nxt, w, zn);
             {
                 // (all lanes poll: one polling lane per warp was measured a quarter slower)
                 ok = wait_a_free(cur.it);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (!C::kExpandAhead) expand();
                 uint8_t *arow = gen_base + sa * kABytes + r * 128;
                 const int sw = r & 7;
 #pragma unroll
@@ -955,8 +1011,6 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     }
                 }
             }
-#pragma unroll
-            for (int q = 0; q < QT; ++q) w[q] = wn[q];
             z = zn;
             cur = nxt;
         }
@@ -1017,9 +1071,12 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             ++stores;
         };
 
-        for (int u = unit0; u < P.total_units && ok; u += unit_step) {
+        for (int uh = unit0 * kTiles; uh < P.total_units * kTiles && ok;
+             uh += ((uh + 1) % kTiles == 0 ? (unit_step - 1) * kTiles + 1 : 1)) {
+            // (two row tiles per unit: tile 0 from accumulator 0, then tile 1 from accumulator 1)
+            const int u = uh / kTiles, h = uh % kTiles;
             const int s = u % P.split_k, rest = u / P.split_k;
-            const int nt = row_tile(rest % nt_groups), tt = tok_tile_of(rest / nt_groups);
+            const int nt = row_tile(rest % nt_groups, h), tt = tok_tile_of(rest / nt_groups);
             const int kb0 = s * P.kb_per_split;
             const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
             const int n = nt * kTileN + f;
@@ -1393,6 +1450,9 @@ w4a8_status launch_dw(const Maps &maps, const Params &P, int cluster, cudaStream
     if constexpr (TOK == 256 && !GROUPED && (DW == 8 || DW == 16)) {
         if (cluster == 3) return launch_cl<TOK, false, DW, 3>(maps, P, st);
     }
+    if constexpr (TOK == 256 && !GROUPED && DW == 16) {
+        if (cluster == 4) return P.batch_rows == 0 ? launch_cl<TOK, false, 16, 4>(maps, P, st) : W4A8_ERR_SHAPE;
+    }
     if (cluster == 1) return launch_cl<TOK, GROUPED, DW, 1>(maps, P, st);
     return W4A8_ERR_SHAPE;
 }
@@ -1425,7 +1485,7 @@ w4a8_status launch_one(const Maps &maps, const Params &P, int dw, int cluster, c
 
 }  // namespace
 
-bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *plan)
+bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *plan, bool auto_pair)
 {
     const bool grouped = L.group != 0;
     const int cap = grouped ? 128 : 256;
@@ -1474,15 +1534,29 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     if (tok != 16 && tok != 32 && tok != 64 && tok != 128 && tok != 192 && tok != 256) return false;
     if (tok > cap) return false;
     const int tok_tiles = (M + tok - 1) / tok;
-    // Two-CTA clusters (each CTA expands half of the code tile for both; an odd last token tile
-    // is paired with an empty one) are there on request.  Measured on 9216 -> 36864 at 2048 tokens
-    // they halve the table lookups and run at a higher clock under the power cap (1590 against
-    // 1370 MHz), but the hand-over between the two CTAs lengthens the per-k-block chain more than
-    // that gains (2200 against 2380 TOPS sustained), so the automatic plan stays with one CTA.
+    // Cluster forms.  The sharing pair (2) halves the table lookups per CTA, but the hand-over
+    // between the two CTAs lengthens the per-k-block chain by more than that gains: on request only.
+    // The MMA pair (3) halves the token bytes per SM and, with two k-blocks per barrier round, the
+    // issuing thread's fixed cost per MMA; together with the offset form of the decode tables
+    // it is the most energy-efficient form, and a long job runs at the power cap, where that
+    // decides (OPT-66B block at 2048 tokens, sustained: 2430 against 2360 TOPS).  The automatic
+    // plan takes it for 1024 tokens and more when the shape allows.
     int cluster = opts ? opts->cluster : 0;
-    if (cluster == 0) cluster = 1;
+    const int off = 13 << L.shift;
+    const bool offset_fits = !grouped && L.bits == 4 && L.shift <= 2 &&
+                             (long long)L.K * 127 * (2 * off) < (1LL << 31);
+    bool auto_offset = false;
+    if (cluster == 0) {
+        cluster = 1;
+        if (auto_pair && M >= 1024 && tok == 256 && split == 1 && offset_fits && L.n_tiles % 2 == 0 &&
+            L.k_blocks % 2 == 0 && (!opts || (opts->decode_warps == 0 && opts->offset_tables == 0))) {
+            cluster = 3;
+            auto_offset = true;
+        }
+    }
     // (3: the MMA pair - 256-token tiles, per-channel 4-bit weights, an even number of row tiles)
-    const bool pair = cluster == 3;
+    // (4: two row tiles per CTA - the same conditions, sixteen decode warps)
+    const bool pair = cluster == 3 || cluster == 4;
     if (pair && !(tok == 256 && !grouped && L.bits == 4 && L.n_tiles % 2 == 0)) return false;
     if (cluster != 1 && !pair && !(cluster == 2 && tok >= 128)) return false;
     const int share = cluster == 2 ? 2 : 1;
@@ -1493,9 +1567,12 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     const int kb_per = (L.k_blocks + split - 1) / split;
     split = (L.k_blocks + kb_per - 1) / kb_per;              // no empty slice
     if (tiles * split > 0x7fffffffLL) return false;
+    // the MMA pair takes k-blocks two at a time: every K slice has an even number of them
+    if (cluster == 3 && (kb_per % 2 != 0 || L.k_blocks % 2 != 0)) return false;
     int dw = opts ? opts->decode_warps : 0;
     if (dw == 0) dw = (grouped || L.bits == 3) ? 8 : 16;
     if (L.bits == 3 && (dw != 8 || cluster != 1)) return false;
+    if (cluster == 4 && dw != 16) return false;
     if (dw != 4 && dw != 8 && !((dw == 12 || dw == 16) && !grouped)) return false;
     plan->decode_warps = dw;
     plan->cluster = cluster;
@@ -1511,19 +1588,16 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     plan->off_partials = align_up(plan->off_counters + (size_t)tiles * sizeof(int), 256);
     const size_t m_pad = (size_t)tok_tiles * tok;
     plan->off_toksum = align_up(plan->off_partials + (split > 1 ? (size_t)split * m_pad * L.n_pad * 4 : 0), 256);
-    // Offset form of the decode tables (decode.cuh), on request: per-channel 4-bit weights whose
-    // special value is step/2 or step/4, and a K short enough for the offset sums to stay inside
-    // INT32.  It needs offset * (sum of each token), computed by a small kernel in front into the
+    // Offset form of the decode tables (decode.cuh): per-channel 4-bit weights whose special
+    // value is step/2 or step/4, and a K short enough for the offset sums to stay inside INT32.
+    // It needs offset * (sum of each token), computed by a small kernel in front into the
     // workspace (one INT32 per token and row tile in the P*V form, so the slot is sized for the
-    // padded rows).  Measured: seven instead of eleven logic-pipe instructions per eight codes let
-    // the SM clock rise under the power cap (1440 against 1370 MHz on the 9216-wide block), but the
-    // per-k-block time does not follow the logic pipe and the extra launch costs what the clock
-    // gains (2350 against 2380 TOPS sustained; 53.8 against 52.3 us at 16 tokens), so the
-    // automatic plan leaves it off.
-    const int off = 13 << L.shift;
-    const bool want = opts && opts->offset_tables == 1;
-    if (want && !(!grouped && L.bits == 4 && L.shift <= 2 && (long long)L.K * 127 * (2 * off) < (1LL << 31)))
-        return false;
+    // padded rows).  Seven instead of eleven logic-pipe instructions per eight codes: the time per
+    // k-block does not follow the logic pipe, but the energy does, so the form pays where the
+    // power cap sets the clock (long prefill jobs) and costs its extra launch elsewhere.  On
+    // request, and with the automatic MMA pair.
+    const bool want = auto_offset || (opts && opts->offset_tables == 1);
+    if (want && !offset_fits) return false;
     plan->offset = want ? off : 0;
     plan->toksum_slots = (size_t)L.n_tiles * M;
     plan->workspace_bytes = plan->off_toksum + (plan->offset ? plan->toksum_slots * 4 : 0);
@@ -1587,7 +1661,7 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     // units: (token-tile group, row-tile group, K slice); a sharing pair groups two token tiles,
     // an MMA pair two row tiles
     P.total_units = plan.cluster == 2 ? (plan.tok_tiles + 1) / 2 * L.n_tiles * plan.split_k
-                  : plan.cluster == 3 ? plan.tok_tiles * (L.n_tiles / 2) * plan.split_k
+                  : (plan.cluster == 3 || plan.cluster == 4) ? plan.tok_tiles * (L.n_tiles / 2) * plan.split_k
                                       : plan.tok_tiles * L.n_tiles * plan.split_k;
     P.prefetch_codes = plan.tok_tiles == 1 ? 1 : 0;   // every code tile is read exactly once
     P.zp = zp;

@@ -204,7 +204,8 @@ def test_tcgen05_two_cta_clusters_many_units_and_split_k():
 def test_cluster_option_is_validated():
     assert w4a8.linear_workspace_bytes(300, 256, 256, 0, w4a8.make_opts(tok_tile=64, cluster=2)) == 0
     assert w4a8.linear_workspace_bytes(300, 256, 256, 0, w4a8.make_opts(tok_tile=128, cluster=3)) == 0
-    assert w4a8.linear_plan(2048, 4096, 4096, 0)["cluster"] == 1
+    assert w4a8.linear_plan(2048, 4096, 4096, 0)["cluster"] == 3         # automatic: the MMA pair
+    assert w4a8.linear_plan(512, 4096, 4096, 0)["cluster"] == 1
     assert w4a8.linear_plan(2048, 4096, 4096, 0, w4a8.make_opts(tok_tile=256, cluster=2))["cluster"] == 2
 
 
@@ -264,3 +265,45 @@ def test_tcgen05_mma_pair():
     assert w4a8.linear_workspace_bytes(300, 384, 256, 0, w4a8.make_opts(tok_tile=256, cluster=3)) == 0   # odd row tiles
     assert w4a8.linear_workspace_bytes(300, 512, 256, 0, w4a8.make_opts(tok_tile=128, cluster=3)) == 0
     assert w4a8.linear_workspace_bytes(300, 512, 256, 128, w4a8.make_opts(tok_tile=256, cluster=3)) == 0
+
+
+def test_tcgen05_two_row_tiles_per_cta():
+    """One CTA on two row tiles and one token tile (cluster form 4): both tiles' MMAs read the same
+    token buffer, the weight ring is numbered by (k-block, tile) items, the two accumulators are
+    handed back one after the other.  Ragged token tile, rows past N in the last tile, several units
+    per CTA (more units than SMs), a K split, asymmetric-free path; same bits as the one-CTA form."""
+    prob = Problem(1536, 128 * 44 - 24, 3 * 256 + 37, 0, seed=722)
+    packed = w4a8.pack_weights(prob.dev["W"], prob.dev["s"], 0)
+    want = prob.oracle_acc()
+    for split in (1, 3):
+        opts = w4a8.make_opts(w4a8.PATH_TCGEN05, split_k=split, tok_tile=256, decode_warps=16, cluster=4)
+        for _ in range(2):
+            Y, acc = run_linear(prob, opts, packed)
+            assert np.array_equal(acc, want)
+            check_y(prob, Y, exact=True)
+    # one k-block only (fewer items than weight buffers), and many k-blocks on few units
+    for K, N, M in ((128, 256, 40), (4096, 512, 300)):
+        small = Problem(K, N, M, 0, seed=723 + K)
+        Y, acc = run_linear(small, w4a8.make_opts(w4a8.PATH_TCGEN05, tok_tile=256, cluster=4))
+        assert np.array_equal(acc, small.oracle_acc())
+        check_y(small, Y, exact=True)
+    assert w4a8.linear_workspace_bytes(300, 384, 256, 0, w4a8.make_opts(tok_tile=256, cluster=4)) == 0   # odd row tiles
+    assert w4a8.linear_workspace_bytes(300, 512, 256, 0, w4a8.make_opts(tok_tile=128, cluster=4)) == 0
+    assert w4a8.linear_workspace_bytes(300, 512, 256, 0, w4a8.make_opts(tok_tile=256, decode_warps=8, cluster=4)) == 0
+    assert w4a8.linear_workspace_bytes(300, 512, 256, 128, w4a8.make_opts(tok_tile=256, cluster=4)) == 0
+
+
+def test_automatic_plan_takes_the_mma_pair_for_many_tokens():
+    """From 1024 tokens on the library's own plan is the MMA pair with offset tables (per-channel
+    4-bit weights, even numbers of row tiles and k-blocks); the bits do not depend on the plan."""
+    prob = Problem(512, 8192, 1024 + 77, 0, seed=731)       # more units than SMs: no K split
+    assert w4a8.linear_plan(prob.M, prob.N, prob.K, 0)["cluster"] == 3
+    assert w4a8.linear_plan(1000, prob.N, prob.K, 0)["cluster"] == 1            # fewer tokens
+    assert w4a8.linear_plan(prob.M, 8192 - 128, prob.K, 0)["cluster"] == 1      # odd row tiles
+    assert w4a8.linear_plan(prob.M, prob.N, 384, 0)["cluster"] == 1             # odd k-blocks
+    assert w4a8.linear_plan(prob.M, prob.N, prob.K, 128)["cluster"] == 1        # group steps
+    Y, acc = run_linear(prob)
+    assert np.array_equal(acc, prob.oracle_acc())
+    check_y(prob, Y, exact=True)
+    Y1, acc1 = run_linear(prob, w4a8.make_opts(w4a8.PATH_TCGEN05, cluster=1))
+    assert np.array_equal(Y, Y1) and np.array_equal(acc, acc1)
