@@ -396,12 +396,12 @@ def main():
     ap.add_argument("--no-legs", action="store_true",
                     help="only the headline workload (resident and host-buffer timings)")
     ap.add_argument("--plan", default=None,
-                    help="tok_tile,split_k,decode_warps,cluster[,offset_tables] for the tensor-core kernel of the headline "
+                    help="tok_tile,split_k,decode_warps,cluster[,offset_tables[,tok_run]] for the tensor-core kernel of the headline "
                          "instead of the library's own choice (sweeps)")
     ap.add_argument("--no-graph", action="store_true",
                     help="--case only: time with per-launch events, no CUDA graph replay")
     ap.add_argument("--case", default=None,
-                    help="K,N,M,group[,tok_tile[,split_k[,decode_warps[,cluster]]]]: time one linear shape instead of "
+                    help="K,N,M,group[,tok_tile[,split_k[,decode_warps[,cluster[,offset_tables[,tok_run]]]]]]: time one linear shape instead of "
                          "(tok_tile -1: the weight-streaming kernel, decode_warps = warps per CTA) "
                          "the block (profiling and sweeps); prints its own JSON line")
     args = ap.parse_args()
@@ -454,9 +454,9 @@ def main():
 
     plan_opts = None
     if args.plan:
-        pv = [int(v) for v in args.plan.split(",")] + [0]
-        pt, ps, pd, pc, po = pv[:5]
-        plan_opts = w4a8.make_opts(w4a8.PATH_TCGEN05, ps, pt, pd, cluster=pc, offset_tables=po)
+        pv = [int(v) for v in args.plan.split(",")] + [0, 0]
+        pt, ps, pd, pc, po, pr = pv[:6]
+        plan_opts = w4a8.make_opts(w4a8.PATH_TCGEN05, ps, pt, pd, cluster=pc, offset_tables=po, tok_run=pr)
 
     def device_block(layers, M, rot=1, host_buffers=False, asym=False, opts=None):
         """Device tensors of a list of layers: packed weights (rot rotating copies), inputs,

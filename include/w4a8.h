@@ -98,6 +98,12 @@ typedef struct {
                         offset out again with the tokens' sums, which a small kernel in front
                         computes into the workspace.  Per-channel 4-bit weights, level_shift
                         1 or 2.  Same bits as without. */
+    int tok_run;     /* 0 = automatic; else the token tiles per run in the order in which the
+                        tensor-core kernel's CTAs take their work: inside a run the token tile
+                        changes fastest, then the 128-row tile (1: every token tile walks through
+                        all row tiles; many: CTAs that work side by side read the same codes).
+                        The automatic choice streams whichever operand does not fit in L2 once.
+                        Same bits either way. */
 } w4a8_opts;
 
 /* Bytes of the packed-weight blob for an [N][K] matrix; 0 if the shape is invalid.

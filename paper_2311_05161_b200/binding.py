@@ -46,7 +46,8 @@ class Opts(ctypes.Structure):
     _fields_ = [("path", ctypes.c_int), ("split_k", ctypes.c_int), ("tok_tile", ctypes.c_int),
                 ("decode_warps", ctypes.c_int), ("level_shift", ctypes.c_int),
                 ("cluster", ctypes.c_int), ("debug_wait_ms", ctypes.c_int), ("debug_skip_load", ctypes.c_int),
-                ("bits", ctypes.c_int), ("offset_tables", ctypes.c_int)]
+                ("bits", ctypes.c_int), ("offset_tables", ctypes.c_int),
+                ("tok_run", ctypes.c_int)]
 
 
 def _load() -> ctypes.CDLL:
@@ -151,7 +152,7 @@ def _dev(t, dtype, what):
 def make_opts(path: int = PATH_AUTO, split_k: int = 0, tok_tile: int = 0,
               decode_warps: int = 0, level_shift: int = 0, cluster: int = 0,
               debug_wait_ms: int = 0, debug_skip_load: int = 0, bits: int = 0,
-              offset_tables: int = 0) -> Opts:
+              offset_tables: int = 0, tok_run: int = 0) -> Opts:
     o = Opts()
     o.path, o.split_k, o.tok_tile, o.decode_warps = path, split_k, tok_tile, decode_warps
     o.level_shift = level_shift
@@ -159,6 +160,7 @@ def make_opts(path: int = PATH_AUTO, split_k: int = 0, tok_tile: int = 0,
     o.debug_wait_ms, o.debug_skip_load = debug_wait_ms, debug_skip_load
     o.bits = bits
     o.offset_tables = offset_tables
+    o.tok_run = tok_run
     return o
 
 

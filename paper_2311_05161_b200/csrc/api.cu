@@ -15,6 +15,16 @@ int device_sms()
     return 148;
 }
 
+long long device_l2_bytes()
+{
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&v, cudaDevAttrL2CacheSize, dev) == cudaSuccess && v > 0)
+        return v;
+    cudaGetLastError();
+    return 126ll << 20;
+}
+
 }  // namespace w4a8
 
 namespace {
@@ -38,6 +48,7 @@ bool opts_ok(const w4a8_opts *o)
     if (o->split_k < 0 || o->tok_tile < 0 || o->decode_warps < 0) return false;
     if (o->level_shift < 0 || o->level_shift > 3) return false;
     if (o->cluster < 0 || o->cluster > 4) return false;
+    if (o->tok_run < 0 || (o->tok_run && (o->path == W4A8_PATH_GEMV || o->path == W4A8_PATH_SIMPLE))) return false;
     if (o->offset_tables < 0 || o->offset_tables > 1 || (o->bits != 0 && !bits_ok(o->bits))) return false;
     if (o->offset_tables && (o->path == W4A8_PATH_GEMV || o->path == W4A8_PATH_SIMPLE)) return false;
     if (o->bits == 3 && (o->path == W4A8_PATH_GEMV || o->cluster >= 2)) return false;
@@ -69,7 +80,7 @@ bool use_gemv(int M, const w4a8_opts *o)
     const int path = o ? o->path : W4A8_PATH_AUTO;
     if (path == W4A8_PATH_GEMV) return true;
     if (bits_of(o) == 3) return false;       // the weight-streaming kernels read 4-bit tiles
-    if (path != W4A8_PATH_AUTO || (o && (o->split_k || o->tok_tile || o->decode_warps || o->cluster || o->offset_tables)))
+    if (path != W4A8_PATH_AUTO || (o && (o->split_k || o->tok_tile || o->decode_warps || o->cluster || o->offset_tables || o->tok_run)))
         return false;
     return M <= 2;
 }

@@ -269,6 +269,7 @@ struct LinearPlan {
     int cluster;      // CTAs per cluster: 1, or 2 (each CTA expands half of every code tile for both)
     int debug_wait_ms, debug_skip_load;   // test hooks of w4a8_opts (0 = off)
     int swiglu;       // gated-unit epilogue (see w4a8_linear_swiglu)
+    int tok_run;      // token tiles per run of the unit order on request, 0 = automatic
     int batched;      // every 128-row tile has its own block of tokens (attention P*V form)
     int kb_per_split; // k-blocks per slice (last slice may be shorter)
     int offset;       // 0, or the offset of the decode tables (13 * 2^shift)
@@ -286,6 +287,8 @@ struct ZeroPoint {
 // SM count of the current device (asked on every call: a process may drive several devices;
 // 148, a B200, when no device answers, so that the size queries work without one)
 int device_sms();
+// L2 size of the current device in bytes
+long long device_l2_bytes();
 
 // launchers (defined in the .cu files, called by api.cu)
 cudaError_t launch_pack(const __half *W, const float *s_in, const BlobLayout &L, float clip,

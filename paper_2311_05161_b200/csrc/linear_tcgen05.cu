@@ -147,6 +147,7 @@ struct Params {
     void *partials;
     BlobLayout L;
     int M, tok_tiles, m_pad, split_k, kb_per_split, total_units, prefetch_codes;
+    int tok_groups, tok_run;   // token-tile groups of the unit list, and how many form a run (unit_tiles)
     ZeroPoint zp;
     LevelTables lt;
     float unit;          // level unit as a factor of the step: 2^-shift
@@ -494,10 +495,28 @@ __device__ __forceinline__ bool wait_bounded_idle(uint32_t bar, uint32_t parity,
     }
 }
 
+// Order of the units.  Unit number `rest` (K slices taken out) belongs to a run of `tok_run`
+// consecutive token tiles; inside a run the token tile changes fastest, then the row tile, and the
+// runs follow one another.  CTAs work on consecutive units at the same time, so with a run of one
+// token tile they share the tokens and walk through the whole weight matrix once per token tile
+// (right when the packed weights stay in L2), and with longer runs tok_run CTAs read the same code
+// tile at about the same time (one DRAM read, the others hit L2) while the run's tokens stay in L2:
+// the host picks the run so that whichever operand does not fit in L2 is streamed once.
+__device__ __forceinline__ void unit_tiles(int rest, int row_groups, int tok_groups, int tok_run,
+                                           int &row_group, int &tok_group)
+{
+    const int per_run = tok_run * row_groups;
+    const int run = rest / per_run, r = rest - run * per_run;
+    const int first = run * tok_run;
+    const int width = min(tok_run, tok_groups - first);
+    row_group = r / width;
+    tok_group = first + (r - row_group * width);
+}
+
 // Position of a CTA in its list of k-blocks: units (token tile, row tile, K slice) are dealt
 // round-robin to the CTAs, each unit is a run of k-blocks, `it` counts k-blocks from zero.
 struct KbCursor {
-    int u, step, total_units, split_k, kb_per_split, k_blocks, n_tiles;
+    int u, step, total_units, split_k, kb_per_split, k_blocks, n_tiles, tok_groups, tok_run;
     int kb, kb1;
     int nt;                    // row-tile group of the unit (integer divisions happen once per unit)
     int h, tiles;              // row tile inside the unit, row tiles per unit
@@ -507,16 +526,17 @@ struct KbCursor {
         if (u < total_units) {
             const int rest = u / split_k;
             const int s = u - rest * split_k;
-            nt = rest % n_tiles;
+            int tg;
+            unit_tiles(rest, n_tiles, tok_groups, tok_run, nt, tg);
             kb = s * kb_per_split;
             kb1 = min(k_blocks, kb + kb_per_split);
         }
     }
     __device__ __forceinline__ void start(int first, int stride, int total, int split, int per,
-                                          int kbs, int groups, int tiles_per_unit = 1)
+                                          int kbs, int groups, int tgroups, int trun, int tiles_per_unit = 1)
     {
         u = first; step = stride; total_units = total; split_k = split; kb_per_split = per;
-        k_blocks = kbs; n_tiles = groups; it = 0; kb = kb1 = 0; nt = 0; h = 0; tiles = tiles_per_unit;
+        k_blocks = kbs; n_tiles = groups; tok_groups = tgroups; tok_run = trun; it = 0; kb = kb1 = 0; nt = 0; h = 0; tiles = tiles_per_unit;
         open_unit();
     }
     __device__ __forceinline__ bool valid() const { return u < total_units; }
@@ -687,11 +707,14 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             uint32_t it = 0;
             bool ok = true;
             KbCursor pf;
-            pf.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, nt_groups, kTiles);
+            pf.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, nt_groups,
+                     P.tok_groups, P.tok_run, kTiles);
             for (int u = unit0; u < P.total_units && ok; u += unit_step) {
                 const int s = u % P.split_k, rest = u / P.split_k;
-                const int tt = tok_tile_of(rest / nt_groups);
-                const int nt_of_unit = row_tile(rest % nt_groups);
+                int row_group, tok_group;
+                unit_tiles(rest, nt_groups, P.tok_groups, P.tok_run, row_group, tok_group);
+                const int tt = tok_tile_of(tok_group);
+                const int nt_of_unit = row_tile(row_group);
                 const int kb0 = s * P.kb_per_split;
                 const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
@@ -859,7 +882,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         // the same stage and barrier in the peer CTA
         const uint32_t peer = rank ^ 1u;
         KbCursor cur;
-        cur.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, nt_groups, kTiles);
+        cur.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, nt_groups,
+                  P.tok_groups, P.tok_run, kTiles);
         cur.advance(team);
         // Items (k-block, row tile of the unit) are numbered in the order the MMAs use them.  The
         // weight buffer of item `it` is free once the MMAs of item it - kAStages, its last user,
@@ -1076,7 +1100,9 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             // (two row tiles per unit: tile 0 from accumulator 0, then tile 1 from accumulator 1)
             const int u = uh / kTiles, h = uh % kTiles;
             const int s = u % P.split_k, rest = u / P.split_k;
-            const int nt = row_tile(rest % nt_groups, h), tt = tok_tile_of(rest / nt_groups);
+            int row_group, tok_group;
+            unit_tiles(rest, nt_groups, P.tok_groups, P.tok_run, row_group, tok_group);
+            const int nt = row_tile(row_group, h), tt = tok_tile_of(tok_group);
             const int kb0 = s * P.kb_per_split;
             const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
             const int n = nt * kTileN + f;
@@ -1577,6 +1603,7 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     plan->decode_warps = dw;
     plan->cluster = cluster;
     plan->batched = 0;
+    plan->tok_run = opts ? opts->tok_run : 0;
     plan->swiglu = 0;
     plan->debug_wait_ms = opts ? opts->debug_wait_ms : 0;
     plan->debug_skip_load = opts ? opts->debug_skip_load : 0;
@@ -1663,6 +1690,20 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     P.total_units = plan.cluster == 2 ? (plan.tok_tiles + 1) / 2 * L.n_tiles * plan.split_k
                   : (plan.cluster == 3 || plan.cluster == 4) ? plan.tok_tiles * (L.n_tiles / 2) * plan.split_k
                                       : plan.tok_tiles * L.n_tiles * plan.split_k;
+    // Order of the units (unit_tiles): packed weights that stay in L2 are walked once per token
+    // tile; larger ones are read by a run of token tiles at the same time, the run as long as its
+    // tokens fit in a third of L2 (the codes of the row tiles in flight and the outputs take the rest).
+    {
+        const int share = plan.cluster == 2 ? 2 : 1;
+        P.tok_groups = (plan.tok_tiles + share - 1) / share;
+        const long long l2 = device_l2_bytes();
+        const long long code_bytes = (long long)L.n_tiles * L.k_blocks * L.tile_bytes;
+        const long long run_bytes = (long long)plan.tok_tile * share * L.K;      // tokens of one group
+        long long run = code_bytes <= l2 / 3 ? 1 : (l2 / 3) / run_bytes;
+        if (plan.tok_run > 0) run = plan.tok_run;
+        if (plan.batched) run = 1;                      // every row tile has its own tokens
+        P.tok_run = (int)(run < 1 ? 1 : run > P.tok_groups ? P.tok_groups : run);
+    }
     P.prefetch_codes = plan.tok_tiles == 1 ? 1 : 0;   // every code tile is read exactly once
     P.zp = zp;
     P.lt = make_level_tables(L.shift);
