@@ -40,9 +40,10 @@ HEADLINE_NAME = ("opt-66b block linears (qkv 9216->27648, out 9216->9216, fc1 92
 M_PREFILL = 2048
 MIN_REGION_S = 1.2                  # length of the headline's timed region
 SUSTAINED_FROM_S = 1.0              # regions at least this long are compared with the sustained peak
-# DRAM bytes per launch of the dominant kernel from an ncu capture; None while the kernel has
-# changed since the counters were taken.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum, mean
+# over the four linears of the headline block, from the ncu launch list of this program); None
+# while the kernel has changed since the counters were taken.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 404.5e6
 CPU_SAMPLE_TOKENS = 48
 CPU_SAMPLE_ROWS = 4096
 NOMINAL_INT8_TOPS = 4500.0
