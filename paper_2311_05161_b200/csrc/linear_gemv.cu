@@ -15,6 +15,8 @@
 // codes with the offset tables described at build_offset_tables (the 16-lane logic pipe that
 // runs the permutes is what bounds them, not HBM), and both can quantize their one to four
 // FP16 tokens themselves (w4a8_quantize_linear), which saves the quantizer's launch.
+#include <atomic>
+
 #include "common.cuh"
 #include "decode.cuh"
 #include "quant_math.cuh"
@@ -28,6 +30,7 @@ constexpr int kGemvMaxSteps = 8;    // steps per CTA: a K slice is at most 16 k-
 constexpr int kGemvDepth = 2;       // steps of codes in flight per thread (asynchronous copies)
 constexpr int kGemvRingBytes = kGemvDepth * kGemvKb * 4 * 128 * 16;   // 32 KiB per CTA
 constexpr int kGemvMaxTokens = 4;
+constexpr int kMaxGemvDevices = 64;
 
 // One k-block (128 input features) of one output row against MT tokens: w = the row's 64 bytes
 // of codes, xk = the tokens' INT8 values of this k-block (token stride in bytes).
@@ -560,12 +563,25 @@ linear_gemv_rows_kernel(const GemvParams P)
     }
 }
 
+// Raise a kernel's dynamic shared-memory limit to `bytes` unless an earlier call on this device
+// already set it at least that high (one slot per kernel instance and device).
+template <typename Kernel>
+void ensure_dynamic_smem(Kernel kern, int bytes, std::atomic<int> (&set_bytes)[kMaxGemvDevices])
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxGemvDevices) dev = -1;
+    if (dev >= 0 && set_bytes[dev].load(std::memory_order_acquire) >= bytes) return;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess &&
+        dev >= 0)
+        set_bytes[dev].store(bytes, std::memory_order_release);
+}
+
 template <int MT, bool GROUPED, int W>
 void launch_rows(const GemvParams &P, cudaStream_t st)
 {
     const int smem = MT * P.L.K + W * MT * 32 * 4 + MT * P.L.k_blocks * 4;
-    cudaFuncSetAttribute(linear_gemv_rows_kernel<MT, GROUPED, W>,
-                         cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    static std::atomic<int> set_bytes[kMaxGemvDevices] = {};
+    ensure_dynamic_smem(linear_gemv_rows_kernel<MT, GROUPED, W>, smem, set_bytes);
     launch_overlapped(linear_gemv_rows_kernel<MT, GROUPED, W>, dim3(P.L.n_tiles * 4), dim3(32 * W),
                       (size_t)smem, st, P);
 }
@@ -615,8 +631,8 @@ template <int MT, bool GROUPED>
 void launch_gemv(dim3 grid, const GemvParams &P, cudaStream_t st)
 {
     constexpr int smem = kGemvRingBytes + MT * kGemvMaxSteps * kGemvKb * kTileK;
-    cudaFuncSetAttribute(linear_gemv_kernel<MT, GROUPED>,
-                         cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    static std::atomic<int> set_bytes[kMaxGemvDevices] = {};
+    ensure_dynamic_smem(linear_gemv_kernel<MT, GROUPED>, smem, set_bytes);
     launch_overlapped(linear_gemv_kernel<MT, GROUPED>, grid, dim3(128), smem, st, P);
 }
 

@@ -505,6 +505,14 @@ __device__ __forceinline__ bool wait_bounded_idle(uint32_t bar, uint32_t parity,
 __device__ __forceinline__ void unit_tiles(int rest, int row_groups, int tok_groups, int tok_run,
                                            int &row_group, int &tok_group)
 {
+    // (The one-tile run keeps its short form: with only the general form below in the code, group
+    // mode, whose runs are always one tile, measured 15 % slower; as a call that is not inlined
+    // the general form cost both modes.)
+    if (tok_run == 1) {                 // the row group changes fastest
+        tok_group = rest / row_groups;
+        row_group = rest - tok_group * row_groups;
+        return;
+    }
     const int per_run = tok_run * row_groups;
     const int run = rest / per_run, r = rest - run * per_run;
     const int first = run * tok_run;
@@ -513,42 +521,42 @@ __device__ __forceinline__ void unit_tiles(int rest, int row_groups, int tok_gro
     tok_group = first + (r - row_group * width);
 }
 
-// Position of a CTA in its list of k-blocks: units (token tile, row tile, K slice) are dealt
-// round-robin to the CTAs, each unit is a run of k-blocks, `it` counts k-blocks from zero.
+// What does not change while a cursor walks: kept apart from the cursor, so that a copy of the
+// cursor (the decode warps hold the current and the next position) copies six registers, not fifteen.
+struct CursorEnv {
+    int step, total_units, split_k, kb_per_split, k_blocks, row_groups, tok_groups, tok_run, tiles;
+};
 struct KbCursor {
-    int u, step, total_units, split_k, kb_per_split, k_blocks, n_tiles, tok_groups, tok_run;
-    int kb, kb1;
+    int u, kb, kb1;
     int nt;                    // row-tile group of the unit (integer divisions happen once per unit)
-    int h, tiles;              // row tile inside the unit, row tiles per unit
+    int h;                     // row tile inside the unit
     uint32_t it;               // counts (k-block, tile) items
-    __device__ __forceinline__ void open_unit()
+    __device__ __forceinline__ void open_unit(const CursorEnv &e)
     {
-        if (u < total_units) {
-            const int rest = u / split_k;
-            const int s = u - rest * split_k;
+        if (u < e.total_units) {
+            const int rest = u / e.split_k;
+            const int s = u - rest * e.split_k;
             int tg;
-            unit_tiles(rest, n_tiles, tok_groups, tok_run, nt, tg);
-            kb = s * kb_per_split;
-            kb1 = min(k_blocks, kb + kb_per_split);
+            unit_tiles(rest, e.row_groups, e.tok_groups, e.tok_run, nt, tg);
+            kb = s * e.kb_per_split;
+            kb1 = min(e.k_blocks, kb + e.kb_per_split);
         }
     }
-    __device__ __forceinline__ void start(int first, int stride, int total, int split, int per,
-                                          int kbs, int groups, int tgroups, int trun, int tiles_per_unit = 1)
+    __device__ __forceinline__ void start(int first, const CursorEnv &e)
     {
-        u = first; step = stride; total_units = total; split_k = split; kb_per_split = per;
-        k_blocks = kbs; n_tiles = groups; tok_groups = tgroups; tok_run = trun; it = 0; kb = kb1 = 0; nt = 0; h = 0; tiles = tiles_per_unit;
-        open_unit();
+        u = first; it = 0; kb = kb1 = 0; nt = 0; h = 0;
+        open_unit(e);
     }
-    __device__ __forceinline__ bool valid() const { return u < total_units; }
-    __device__ __forceinline__ void advance(int n)
+    __device__ __forceinline__ bool valid(const CursorEnv &e) const { return u < e.total_units; }
+    __device__ __forceinline__ void advance(int n, const CursorEnv &e)
     {
-        for (int i = 0; i < n && valid(); ++i) {
+        for (int i = 0; i < n && valid(e); ++i) {
             ++it;
-            if (++h < tiles) continue;
+            if (++h < e.tiles) continue;
             h = 0;
             if (++kb >= kb1) {
-                u += step;
-                open_unit();
+                u += e.step;
+                open_unit(e);
             }
         }
     }
@@ -697,6 +705,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     const bool blob_ok = header_matches(P.blob, P.L);
 
     const int n_tiles = P.L.n_tiles, k_blocks = P.L.k_blocks;
+    const CursorEnv env = {unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, nt_groups,
+                           P.tok_groups, P.tok_run, kTiles};
 
     if (!blob_ok) {
         // not the blob the caller described: nothing is read or written, only the status
@@ -707,8 +717,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             uint32_t it = 0;
             bool ok = true;
             KbCursor pf;
-            pf.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, nt_groups,
-                     P.tok_groups, P.tok_run, kTiles);
+            pf.start(unit0, env);
             for (int u = unit0; u < P.total_units && ok; u += unit_step) {
                 const int s = u % P.split_k, rest = u / P.split_k;
                 int row_group, tok_group;
@@ -748,11 +757,11 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     }
                     if (P.prefetch_codes) {
                         // keep the code stream kPrefetchAhead k-blocks ahead of the decode warps
-                        while (pf.valid() && pf.it < (it + C::kPrefetchAhead) * kTiles) {
+                        while (pf.valid(env) && pf.it < (it + C::kPrefetchAhead) * kTiles) {
                             const int pnt = row_tile(pf.nt, pf.h);
                             prefetch_l2(P.codes + ((size_t)pnt * k_blocks + pf.kb) * (BITS == 3 ? kTileBytes3 : kTileBytes),
                                         BITS == 3 ? kTileBytes3 : kTileBytes);
-                            pf.advance(1);
+                            pf.advance(1, env);
                         }
                     }
                 }
@@ -882,9 +891,8 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         // the same stage and barrier in the peer CTA
         const uint32_t peer = rank ^ 1u;
         KbCursor cur;
-        cur.start(unit0, unit_step, P.total_units, P.split_k, P.kb_per_split, k_blocks, nt_groups,
-                  P.tok_groups, P.tok_run, kTiles);
-        cur.advance(team);
+        cur.start(unit0, env);
+        cur.advance(team, env);
         // Items (k-block, row tile of the unit) are numbered in the order the MMAs use them.  The
         // weight buffer of item `it` is free once the MMAs of item it - kAStages, its last user,
         // have retired (their commit completed a phase of that item's k-block's barrier slot).
@@ -914,14 +922,14 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                     dst[i] = v;
                 }
             };
-            if (cur.valid()) fetch3(cur, w3, z3);
+            if (cur.valid(env)) fetch3(cur, w3, z3);
             bool ok3 = true;
-            while (cur.valid() && ok3) {
+            while (cur.valid(env) && ok3) {
                 KbCursor nxt = cur;
-                nxt.advance(C::kTeams);
+                nxt.advance(C::kTeams, env);
                 uint32_t wn3[12];
                 int zn3 = 0;
-                if (nxt.valid()) fetch3(nxt, wn3, zn3);
+                if (nxt.valid(env)) fetch3(nxt, wn3, zn3);
                 const int st = (cur.it / C::kPerRound) % S, sa = cur.it % C::kAStages;
                 uint32_t t3[2];
                 build_level_tables3(z3, P.L.shift, t3);
@@ -964,14 +972,14 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
 #pragma unroll
             for (int q = 0; q < QT; ++q) dst[q] = ld_stream(src + (q0 + q) * (kQuarterBytes / 16));
         };
-        if (cur.valid()) fetch(cur, w, z);
+        if (cur.valid(env)) fetch(cur, w, z);
         bool ok = true;
         const bool use_offset = !GROUPED && P.offset != 0;   // (per-channel weights only)
         uint32_t one = 1u;                       // opaque to the compiler: see decode8_offset
         asm volatile("" : "+r"(one));
-        while (cur.valid() && ok) {
+        while (cur.valid(env) && ok) {
             KbCursor nxt = cur;
-            nxt.advance(T);
+            nxt.advance(T, env);
             const int st = (cur.it / C::kPerRound) % S, sa = cur.it % C::kAStages;
             uint32_t t[4];
             if (use_offset) build_offset_tables(z, P.lt, P.L.shift, t);
@@ -1004,17 +1012,27 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             // ring of weight buffers can hide).  The codes of the team's next item are requested
             // only now, into the registers the expansion has just read, so a thread holds raw
             // codes and levels of one item at a time; the wait and the stores cover the loads.
-            expand();
-#pragma unroll
-            for (int q = 0; q < 2 * QT; ++q)
-                asm volatile("" : "+r"(lv[q].x), "+r"(lv[q].y), "+r"(lv[q].z), "+r"(lv[q].w));
+            // Group mode keeps the older order (next codes requested first, expansion after the
+            // wait): its MMAs are short and its promotion warps own the issue slots, and there the
+            // early expansion measured 15 % slower.
+            constexpr bool kFetchFirst = GROUPED;
+            uint4 wn[kFetchFirst ? QT : 1];
             int zn = 0;
-            if (nxt.valid()) fetch(nxt, w, zn);
+            if constexpr (kFetchFirst) {
+                if (nxt.valid(env)) fetch(nxt, wn, zn);
+            } else {
+                expand();
+#pragma unroll
+                for (int q = 0; q < 2 * QT; ++q)
+                    asm volatile("" : "+r"(lv[q].x), "+r"(lv[q].y), "+r"(lv[q].z), "+r"(lv[q].w));
+                if (nxt.valid(env)) fetch(nxt, w, zn);
+            }
             {
                 // (all lanes poll: one polling lane per warp was measured a quarter slower)
                 ok = wait_a_free(cur.it);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+                if constexpr (kFetchFirst) expand();
                 uint8_t *arow = gen_base + sa * kABytes + r * 128;
                 const int sw = r & 7;
 #pragma unroll
@@ -1034,6 +1052,10 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                                          map_to_cta(bar_dec + 8 * st, peer));
                     }
                 }
+            }
+            if constexpr (kFetchFirst) {
+#pragma unroll
+                for (int q = 0; q < QT; ++q) w[q] = wn[q];
             }
             z = zn;
             cur = nxt;
@@ -1566,7 +1588,10 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     // issuing thread's fixed cost per MMA; together with the offset form of the decode tables
     // it is the most energy-efficient form, and a long job runs at the power cap, where that
     // decides (OPT-66B block at 2048 tokens, sustained: 2430 against 2360 TOPS).  The automatic
-    // plan takes it for 1024 tokens and more when the shape allows.
+    // plan takes it for 1024 tokens and more on layers of at least 8192 x 8192: the token sums of
+    // the offset tables cost a launch whose time goes with M x K while the layer's goes with
+    // M x N x K, and with few k-blocks per unit the pair's longer rounds do not pay (4096 -> 4096
+    // at 2048 tokens: 39.6 against 31.5 us, 16384 -> 4096: 112 against 103 us).
     int cluster = opts ? opts->cluster : 0;
     const int off = 13 << L.shift;
     const bool offset_fits = !grouped && L.bits == 4 && L.shift <= 2 &&
@@ -1574,7 +1599,8 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     bool auto_offset = false;
     if (cluster == 0) {
         cluster = 1;
-        if (auto_pair && M >= 1024 && tok == 256 && split == 1 && offset_fits && L.n_tiles % 2 == 0 &&
+        if (auto_pair && M >= 1024 && L.N >= 8192 && L.K >= 8192 && tok == 256 && split == 1 &&
+            offset_fits && L.n_tiles % 2 == 0 &&
             L.k_blocks % 2 == 0 && (!opts || (opts->decode_warps == 0 && opts->offset_tables == 0))) {
             cluster = 3;
             auto_offset = true;

@@ -204,8 +204,9 @@ def test_tcgen05_two_cta_clusters_many_units_and_split_k():
 def test_cluster_option_is_validated():
     assert w4a8.linear_workspace_bytes(300, 256, 256, 0, w4a8.make_opts(tok_tile=64, cluster=2)) == 0
     assert w4a8.linear_workspace_bytes(300, 256, 256, 0, w4a8.make_opts(tok_tile=128, cluster=3)) == 0
-    assert w4a8.linear_plan(2048, 4096, 4096, 0)["cluster"] == 3         # automatic: the MMA pair
-    assert w4a8.linear_plan(512, 4096, 4096, 0)["cluster"] == 1
+    assert w4a8.linear_plan(2048, 8192, 8192, 0)["cluster"] == 3         # automatic: the MMA pair
+    assert w4a8.linear_plan(2048, 4096, 4096, 0)["cluster"] == 1         # small layers: one CTA
+    assert w4a8.linear_plan(512, 8192, 8192, 0)["cluster"] == 1
     assert w4a8.linear_plan(2048, 4096, 4096, 0, w4a8.make_opts(tok_tile=256, cluster=2))["cluster"] == 2
 
 
@@ -294,19 +295,32 @@ def test_tcgen05_two_row_tiles_per_cta():
 
 
 def test_automatic_plan_takes_the_mma_pair_for_many_tokens():
-    """From 1024 tokens on the library's own plan is the MMA pair with offset tables (per-channel
-    4-bit weights, even numbers of row tiles and k-blocks); the bits do not depend on the plan."""
-    prob = Problem(512, 8192, 1024 + 77, 0, seed=731)       # more units than SMs: no K split
-    assert w4a8.linear_plan(prob.M, prob.N, prob.K, 0)["cluster"] == 3
-    assert w4a8.linear_plan(1000, prob.N, prob.K, 0)["cluster"] == 1            # fewer tokens
-    assert w4a8.linear_plan(prob.M, 8192 - 128, prob.K, 0)["cluster"] == 1      # odd row tiles
-    assert w4a8.linear_plan(prob.M, prob.N, 384, 0)["cluster"] == 1             # odd k-blocks
-    assert w4a8.linear_plan(prob.M, prob.N, prob.K, 128)["cluster"] == 1        # group steps
-    Y, acc = run_linear(prob)
-    assert np.array_equal(acc, prob.oracle_acc())
-    check_y(prob, Y, exact=True)
-    Y1, acc1 = run_linear(prob, w4a8.make_opts(w4a8.PATH_TCGEN05, cluster=1))
-    assert np.array_equal(Y, Y1) and np.array_equal(acc, acc1)
+    """From 1024 tokens on, on layers of at least 8192 x 8192, the library's own plan is the MMA
+    pair with offset tables (per-channel 4-bit weights, even numbers of row tiles and k-blocks); the
+    bits do not depend on the plan.  The oracle recomputes a sample of rows (every output element
+    depends only on its own weight row and token)."""
+    K, N, M = 8192, 8192, 1024 + 77
+    assert w4a8.linear_plan(M, N, K, 0)["cluster"] == 3
+    assert w4a8.linear_plan(1000, N, K, 0)["cluster"] == 1            # fewer tokens
+    assert w4a8.linear_plan(M, N - 128, K, 0)["cluster"] == 1         # odd row tiles
+    assert w4a8.linear_plan(M, N, K + 128, 0)["cluster"] == 1         # odd k-blocks
+    assert w4a8.linear_plan(M, N, K, 128)["cluster"] == 1             # group steps
+    assert w4a8.linear_plan(M, 4096, K, 0)["cluster"] == 1            # a narrow layer
+    rows = np.array([0, 1, 127, 128, 129, 255, 256, 4095, 4096, N - 129, N - 128, N - 1])
+    prob = Problem(K, N, M, 0, seed=731, rows=rows)
+    d = prob.dev
+    packed = w4a8.pack_weights(d["W"], d["s"], 0)
+    Xq, tok = w4a8.quantize_act(d["X"], d["inv_s"])
+    outs = []
+    for opts in (None, w4a8.make_opts(w4a8.PATH_TCGEN05, cluster=1)):
+        ws = w4a8.new_workspace(M, N, K, 0, opts)
+        Y = w4a8.linear(Xq, tok, packed, d["bias"], N, 0, ws, opts)
+        acc = w4a8.linear_acc_i32(Xq, packed, N, 0, ws, opts)
+        w4a8.check_status(ws)
+        outs.append((bf16_bits(Y), acc.cpu().numpy().reshape(M, N)))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    assert np.array_equal(outs[0][1][:, rows], prob.oracle_acc().reshape(M, len(rows)))
+    assert np.array_equal(outs[0][0][:, rows], prob.oracle_y_bits())
 
 
 def test_unit_order_runs_of_token_tiles():
