@@ -287,22 +287,21 @@ def run_case(args):
     import paper_2311_05161_b200 as w4a8
     from paper_2311_05161_b200 import synth
 
-    vals = [int(v) for v in args.case.split(",")]
-    K, N, M, group = vals[:4]
-    tok_tile = vals[4] if len(vals) > 4 else 0
-    split_k = vals[5] if len(vals) > 5 else 0
-    dw = vals[6] if len(vals) > 6 else 0
-    cluster = vals[7] if len(vals) > 7 else 0
+    vals = [int(v) for v in args.case.split(",")] + [0] * 7
+    K, N, M, group, tok_tile, split_k, dw, cluster, offset_tables, tok_run, bits = vals[:11]
+    plan_given = bool(tok_tile or split_k or dw or cluster or offset_tables or tok_run)
     if tok_tile < 0:            # the weight-streaming kernel on request; dw = warps of a row-slab CTA
         opts = w4a8.make_opts(w4a8.PATH_GEMV, 0, 0, dw)
+    elif plan_given or bits:
+        opts = w4a8.make_opts(w4a8.PATH_TCGEN05 if plan_given else w4a8.PATH_AUTO, split_k, tok_tile, dw,
+                              cluster=cluster, offset_tables=offset_tables, tok_run=tok_run, bits=bits)
     else:
-        opts = (w4a8.make_opts(w4a8.PATH_TCGEN05, split_k, tok_tile, dw, cluster=cluster)
-                if (tok_tile or split_k or dw or cluster) else None)
+        opts = None
     torch.cuda.set_device(0)
     peaks = read_peaks()
     lay = synth.make_layer(K, N, M, seed=7, dist="normal", outliers=0.001, mult=60.0)
     d = {k: torch.from_numpy(lay[k]).cuda() for k in ("W", "X", "s", "inv_s", "bias")}
-    packed = w4a8.pack_weights(d["W"], d["s"], group)
+    packed = w4a8.pack_weights(d["W"], d["s"], group, bits=bits) if bits else w4a8.pack_weights(d["W"], d["s"], group)
     del d["W"]
     per_copy = packed.numel() + M * K * 3 + M * N * 2
     copies = max(1, min(8, -(-(256 << 20) // per_copy)))
@@ -402,7 +401,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true",
                     help="--case only: time with per-launch events, no CUDA graph replay")
     ap.add_argument("--case", default=None,
-                    help="K,N,M,group[,tok_tile[,split_k[,decode_warps[,cluster[,offset_tables[,tok_run]]]]]]: time one linear shape instead of "
+                    help="K,N,M,group[,tok_tile[,split_k[,decode_warps[,cluster[,offset_tables[,tok_run[,bits]]]]]]]: time one linear shape instead of "
                          "(tok_tile -1: the weight-streaming kernel, decode_warps = warps per CTA) "
                          "the block (profiling and sweeps); prints its own JSON line")
     args = ap.parse_args()

@@ -104,6 +104,8 @@ typedef struct {
                         changes fastest, then the 128-row tile (1: every token tile walks through
                         all row tiles; many: CTAs that work side by side read the same codes).
                         The automatic choice streams whichever operand does not fit in L2 once.
+                        Runs longer than one exist for per-channel 4-bit weights with token tiles
+                        of 128 and more; elsewhere the field is accepted and has no effect.
                         Same bits either way. */
 } w4a8_opts;
 

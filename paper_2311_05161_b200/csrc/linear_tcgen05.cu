@@ -502,13 +502,16 @@ __device__ __forceinline__ bool wait_bounded_idle(uint32_t bar, uint32_t parity,
 // (right when the packed weights stay in L2), and with longer runs tok_run CTAs read the same code
 // tile at about the same time (one DRAM read, the others hit L2) while the run's tokens stay in L2:
 // the host picks the run so that whichever operand does not fit in L2 is streamed once.
+// RUNS = false: the kernel instance has only the one-tile form (the host then never asks for longer
+// runs).  The general form costs the instances that never need it - group mode and 3-bit codes
+// measured 15-20 % slower with it compiled in, as a call that is not inlined it cost all of them -
+// so only the wide per-channel 4-bit instances, the ones that meet code matrices larger than L2
+// with many token tiles, carry it.
+template <bool RUNS>
 __device__ __forceinline__ void unit_tiles(int rest, int row_groups, int tok_groups, int tok_run,
                                            int &row_group, int &tok_group)
 {
-    // (The one-tile run keeps its short form: with only the general form below in the code, group
-    // mode, whose runs are always one tile, measured 15 % slower; as a call that is not inlined
-    // the general form cost both modes.)
-    if (tok_run == 1) {                 // the row group changes fastest
+    if (!RUNS || tok_run == 1) {        // the row group changes fastest
         tok_group = rest / row_groups;
         row_group = rest - tok_group * row_groups;
         return;
@@ -526,6 +529,7 @@ __device__ __forceinline__ void unit_tiles(int rest, int row_groups, int tok_gro
 struct CursorEnv {
     int step, total_units, split_k, kb_per_split, k_blocks, row_groups, tok_groups, tok_run, tiles;
 };
+template <bool RUNS>
 struct KbCursor {
     int u, kb, kb1;
     int nt;                    // row-tile group of the unit (integer divisions happen once per unit)
@@ -537,7 +541,7 @@ struct KbCursor {
             const int rest = u / e.split_k;
             const int s = u - rest * e.split_k;
             int tg;
-            unit_tiles(rest, e.row_groups, e.tok_groups, e.tok_run, nt, tg);
+            unit_tiles<RUNS>(rest, e.row_groups, e.tok_groups, e.tok_run, nt, tg);
             kb = s * e.kb_per_split;
             kb1 = min(e.k_blocks, kb + e.kb_per_split);
         }
@@ -613,6 +617,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
     constexpr int BITS = VARIANT == 3 ? 3 : 4;
     constexpr bool SWIGLU = VARIANT == kSwigluVariant;
     constexpr bool ASYM_GROUP = VARIANT == kAsymGroupVariant;
+    constexpr bool kRuns = !GROUPED && TOK >= 128 && VARIANT == 4;   // see unit_tiles
     static_assert(!ASYM_GROUP || GROUPED, "the asymmetric group variant is a group-mode kernel");
     constexpr int kFirstEpiWarp = C::kFirstEpiWarp;
     constexpr int S = C::kStages;
@@ -716,12 +721,12 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            KbCursor pf;
+            KbCursor<kRuns> pf;
             pf.start(unit0, env);
             for (int u = unit0; u < P.total_units && ok; u += unit_step) {
                 const int s = u % P.split_k, rest = u / P.split_k;
                 int row_group, tok_group;
-                unit_tiles(rest, nt_groups, P.tok_groups, P.tok_run, row_group, tok_group);
+                unit_tiles<kRuns>(rest, nt_groups, P.tok_groups, P.tok_run, row_group, tok_group);
                 const int tt = tok_tile_of(tok_group);
                 const int nt_of_unit = row_tile(row_group);
                 const int kb0 = s * P.kb_per_split;
@@ -890,7 +895,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         constexpr int T = C::kTeams;
         // the same stage and barrier in the peer CTA
         const uint32_t peer = rank ^ 1u;
-        KbCursor cur;
+        KbCursor<kRuns> cur;
         cur.start(unit0, env);
         cur.advance(team, env);
         // Items (k-block, row tile of the unit) are numbered in the order the MMAs use them.  The
@@ -910,7 +915,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             static_assert(CL == 1, "3-bit codes: one CTA per cluster");
             uint32_t w3[12];
             int z3 = 0;
-            auto fetch3 = [&](const KbCursor &c, uint32_t (&dst)[12], int &zz) {
+            auto fetch3 = [&](const KbCursor<kRuns> &c, uint32_t (&dst)[12], int &zz) {
                 const int n = c.nt * kTileN + r;
                 zz = GROUPED ? P.zeros[(size_t)c.kb * P.L.n_pad + n] : P.zeros[n];
                 const uint32_t *src = reinterpret_cast<const uint32_t *>(
@@ -925,7 +930,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             if (cur.valid(env)) fetch3(cur, w3, z3);
             bool ok3 = true;
             while (cur.valid(env) && ok3) {
-                KbCursor nxt = cur;
+                KbCursor<kRuns> nxt = cur;
                 nxt.advance(C::kTeams, env);
                 uint32_t wn3[12];
                 int zn3 = 0;
@@ -963,7 +968,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         } else {
         uint4 w[QT];
         int z = 0;
-        auto fetch = [&](const KbCursor &c, uint4 (&dst)[QT], int &zz) {
+        auto fetch = [&](const KbCursor<kRuns> &c, uint4 (&dst)[QT], int &zz) {
             const int nt = row_tile(c.nt, c.h);
             const int n = nt * kTileN + r;
             zz = GROUPED ? P.zeros[(size_t)c.kb * P.L.n_pad + n] : P.zeros[n];
@@ -978,7 +983,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
         uint32_t one = 1u;                       // opaque to the compiler: see decode8_offset
         asm volatile("" : "+r"(one));
         while (cur.valid(env) && ok) {
-            KbCursor nxt = cur;
+            KbCursor<kRuns> nxt = cur;
             nxt.advance(T, env);
             const int st = (cur.it / C::kPerRound) % S, sa = cur.it % C::kAStages;
             uint32_t t[4];
@@ -1123,7 +1128,7 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             const int u = uh / kTiles, h = uh % kTiles;
             const int s = u % P.split_k, rest = u / P.split_k;
             int row_group, tok_group;
-            unit_tiles(rest, nt_groups, P.tok_groups, P.tok_run, row_group, tok_group);
+            unit_tiles<kRuns>(rest, nt_groups, P.tok_groups, P.tok_run, row_group, tok_group);
             const int nt = row_tile(row_group, h), tt = tok_tile_of(tok_group);
             const int kb0 = s * P.kb_per_split;
             const int kb1 = min(k_blocks, kb0 + P.kb_per_split);
@@ -1728,6 +1733,8 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
         long long run = code_bytes <= l2 / 3 ? 1 : (l2 / 3) / run_bytes;
         if (plan.tok_run > 0) run = plan.tok_run;
         if (plan.batched) run = 1;                      // every row tile has its own tokens
+        // only the wide per-channel 4-bit instances of the kernel know longer runs
+        if (L.group != 0 || plan.tok_tile < 128 || L.bits != 4 || plan.swiglu) run = 1;
         P.tok_run = (int)(run < 1 ? 1 : run > P.tok_groups ? P.tok_groups : run);
     }
     P.prefetch_codes = plan.tok_tiles == 1 ? 1 : 0;   // every code tile is read exactly once

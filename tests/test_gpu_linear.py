@@ -327,12 +327,12 @@ def test_unit_order_runs_of_token_tiles():
     """The order in which CTAs take (token tile, row tile) units - runs of tok_run token tiles,
     token tile fastest inside a run - changes no bit: every run length, a ragged last run, with a
     K split, in the cluster forms."""
-    prob = Problem(512, 128 * 6, 5 * 64 + 9, 0, seed=741)
+    prob = Problem(512, 128 * 6, 5 * 128 + 9, 0, seed=741)
     packed = w4a8.pack_weights(prob.dev["W"], prob.dev["s"], 0)
     want = prob.oracle_acc()
     for run in (1, 2, 3, 6, 50):
         for split in (1, 2):
-            Y, acc = run_linear(prob, w4a8.make_opts(w4a8.PATH_TCGEN05, split_k=split, tok_tile=64, tok_run=run), packed)
+            Y, acc = run_linear(prob, w4a8.make_opts(w4a8.PATH_TCGEN05, split_k=split, tok_tile=128, tok_run=run), packed)
             assert np.array_equal(acc, want)
             check_y(prob, Y, exact=True)
     big = Problem(256, 128 * 6, 5 * 256 + 9, 0, seed=742)
@@ -343,6 +343,7 @@ def test_unit_order_runs_of_token_tiles():
             Y, acc = run_linear(big, w4a8.make_opts(w4a8.PATH_TCGEN05, tok_tile=tok_tile, cluster=cluster, tok_run=run), packed)
             assert np.array_equal(acc, want)
             check_y(big, Y, exact=True)
+    # (group steps, narrow tiles, 3-bit codes: the request is accepted and the order stays one tile per run)
     grp = Problem(512, 128 * 3, 3 * 64 + 5, 128, seed=743)
     Y, acc = run_linear(grp, w4a8.make_opts(w4a8.PATH_TCGEN05, tok_tile=64, tok_run=2))
     assert np.array_equal(acc, grp.oracle_acc())
