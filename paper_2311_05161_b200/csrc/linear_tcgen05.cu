@@ -583,12 +583,22 @@ token_offsum_kernel(const int8_t *__restrict__ Xq, int K, int offset, int32_t *_
     dependent_wait();                      // Xq may be the output of the kernel before
     const int4 *row = reinterpret_cast<const int4 *>(Xq + (size_t)blockIdx.x * K);
     int s = 0;
-    for (int i = threadIdx.x; i < K / 16; i += 256) {
-        const int4 v = __ldg(row + i);
-        s = __dp4a(v.x, 0x01010101, s);
-        s = __dp4a(v.y, 0x01010101, s);
-        s = __dp4a(v.z, 0x01010101, s);
-        s = __dp4a(v.w, 0x01010101, s);
+    const int n16 = K / 16;
+    // four independent 16-byte loads per thread and round: the kernel is a pure read of Xq
+    for (int i0 = threadIdx.x; i0 < n16; i0 += 4 * 256) {
+        int4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = i0 + j * 256;
+            v[j] = i < n16 ? __ldg(row + i) : make_int4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            s = __dp4a(v[j].x, 0x01010101, s);
+            s = __dp4a(v[j].y, 0x01010101, s);
+            s = __dp4a(v[j].z, 0x01010101, s);
+            s = __dp4a(v[j].w, 0x01010101, s);
+        }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
