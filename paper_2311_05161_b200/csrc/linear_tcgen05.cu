@@ -1451,6 +1451,48 @@ struct Maps {
     CUtensorMap tok, y16, y32;      // activations; output with 16- and 32-token boxes
 };
 
+// Tensor maps of a two-dimensional row-major tensor, kept per host thread: a serving loop calls
+// with the same pointers and shapes over and over, and a map depends on nothing else (addresses
+// are unique across the devices of a process).  Eight entries, replaced in turn.
+struct MapKey {
+    const void *base;
+    unsigned long long dim0, dim1, stride;
+    unsigned box0, box1;
+    int dtype, swizzle, promotion;
+    bool operator==(const MapKey &o) const
+    {
+        return base == o.base && dim0 == o.dim0 && dim1 == o.dim1 && stride == o.stride && box0 == o.box0 &&
+               box1 == o.box1 && dtype == o.dtype && swizzle == o.swizzle && promotion == o.promotion;
+    }
+};
+bool encode_2d(EncodeTiledFn enc, CUtensorMap *out, CUtensorMapDataType dtype, const void *base,
+               cuuint64_t dim0, cuuint64_t dim1, cuuint64_t stride_bytes, cuuint32_t box0, cuuint32_t box1,
+               CUtensorMapSwizzle swizzle, CUtensorMapL2promotion promotion)
+{
+    constexpr int kEntries = 8;
+    thread_local MapKey keys[kEntries] = {};
+    thread_local CUtensorMap maps[kEntries];
+    thread_local int next = 0;
+    const MapKey key = {base, dim0, dim1, stride_bytes, box0, box1, (int)dtype, (int)swizzle, (int)promotion};
+    for (int i = 0; i < kEntries; ++i) {
+        if (keys[i].base != nullptr && keys[i] == key) {
+            *out = maps[i];
+            return true;
+        }
+    }
+    const cuuint64_t dims[2] = {dim0, dim1};
+    const cuuint64_t strides[1] = {stride_bytes};
+    const cuuint32_t box[2] = {box0, box1};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(out, dtype, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            swizzle, promotion, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    keys[next] = key;
+    maps[next] = *out;
+    next = (next + 1) % kEntries;
+    return true;
+}
+
 // Clusters of CL CTAs of this kernel that the current device can hold at once (one CTA per
 // SM); asked once per kernel instance and device.
 template <int TOK, bool GROUPED, int DW, int CL, int VARIANT>
@@ -1681,29 +1723,22 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     if (!enc) return W4A8_ERR_CUDA;
     Maps maps;
     memset(&maps, 0, sizeof(maps));
-    // (P*V form: the token blocks of all row tiles are stacked, one after the other)
-    const cuuint64_t dims[2] = {(cuuint64_t)L.K, (cuuint64_t)M * (plan.batched ? L.n_tiles : 1)};
-    const cuuint64_t strides[1] = {(cuuint64_t)L.K};
-    // (an MMA pair: each CTA loads half of the token tile)
-    const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)(plan.cluster == 3 ? plan.tok_tile / 2 : plan.tok_tile)};
-    const cuuint32_t estr[2] = {1, 1};
-    if (enc(&maps.tok, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(Xq), dims, strides,
-            box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    // (P*V form: the token blocks of all row tiles are stacked, one after the other; an MMA
+    // pair: each CTA loads half of the token tile)
+    if (!encode_2d(enc, &maps.tok, CU_TENSOR_MAP_DATA_TYPE_UINT8, Xq, (cuuint64_t)L.K,
+                   (cuuint64_t)M * (plan.batched ? L.n_tiles : 1), (cuuint64_t)L.K, (cuuint32_t)kTileK,
+                   (cuuint32_t)(plan.cluster == 3 ? plan.tok_tile / 2 : plan.tok_tile),
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B))
         return W4A8_ERR_CUDA;
     if (Y && plan.split_k == 1) {
         // output tiles of 128 features x 16 or 32 tokens; parts beyond N or M are clipped
         // (gated-unit epilogue: half as many features per tile and per row, binary16)
         const int width = plan.swiglu ? L.N / 2 : L.N, tile_w = plan.swiglu ? kTileN / 2 : kTileN;
-        const cuuint64_t ydims[2] = {(cuuint64_t)width, (cuuint64_t)M};
-        const cuuint64_t ystrides[1] = {(cuuint64_t)width * 2};
         for (int rows = 16; rows <= 32; rows += 16) {
-            const cuuint32_t ybox[2] = {(cuuint32_t)tile_w, (cuuint32_t)rows};
-            if (enc(rows == 16 ? &maps.y16 : &maps.y32,
-                    plan.swiglu ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y,
-                    ydims, ystrides, ybox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            if (!encode_2d(enc, rows == 16 ? &maps.y16 : &maps.y32,
+                           plan.swiglu ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, Y,
+                           (cuuint64_t)width, (cuuint64_t)M, (cuuint64_t)width * 2, (cuuint32_t)tile_w,
+                           (cuuint32_t)rows, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE))
                 return W4A8_ERR_CUDA;
         }
     }

@@ -28,7 +28,7 @@ def sample(total, count, seed, edges):
     return np.array(sorted(picked))
 
 
-def check_shape(config, shape_index, tokens):
+def check_shape(config, shape_index, tokens, acc_for_M=None):
     wl = synth.WORKLOADS[config]
     K, N, label = wl.shapes[shape_index]
     seed = wl.seed(shape_index)
@@ -61,6 +61,15 @@ def check_shape(config, shape_index, tokens):
                               oscales.view(np.uint32)), (label, M, "steps")
         assert np.array_equal(Xq[toks_t].cpu().numpy(), oXq), (label, M, "Xq")
         assert np.array_equal(tok[toks_t].cpu().numpy().view(np.uint32), otok.view(np.uint32))
+        if acc_for_M == M:
+            # the INT32 accumulators of the same launch configuration, on the same sample
+            acc = w4a8.linear_acc_i32(Xq, packed, N, group, ws)
+            w4a8.check_status(ws)
+            G = acc.shape[0]
+            got_acc = acc[:, toks_t][:, :, rows_t].cpu().numpy()
+            want_acc = oracle.linear_acc(oXq, ocodes, ozeros, group).reshape(G, len(toks), len(rows))
+            assert np.array_equal(got_acc, want_acc), (label, M, "INT32 accumulators")
+            del acc
         got = bf16_bits(Y[toks_t][:, rows_t].contiguous())
         want = oracle.linear(oXq, otok, ocodes, oscales, ozeros, bias[rows], group)
         plan_splits = w4a8.linear_workspace_bytes(M, N, K, group) > 4096 + 4 * 4096
@@ -93,7 +102,8 @@ def test_config3_llama_7b_block_group128(shape_index):
 
 @pytest.mark.parametrize("shape_index", [0, 1, 2, 3, 4, 5, 6, 7])
 def test_config4_large_linears(shape_index):
-    check_shape(4, shape_index, (2048, 16))
+    # (the first shape, 9216 -> 36864, also compares the INT32 accumulators at 2048 tokens)
+    check_shape(4, shape_index, (2048, 16), acc_for_M=2048 if shape_index == 0 else None)
 
 
 def test_config5_token_sweep_group128():
