@@ -275,11 +275,16 @@ w4a8_status w4a8_quantize_linear(const void *X_f16, const float *inv_s_in, const
  *   All calls on one device share the array: the call clears the part that must start at
  *   zero, on `stream`, before its kernel.  Two calls that can overlap on the GPU (different
  *   streams without an ordering between them) race on it and give undefined results.
- *   Failures inside the kernel are not reported through this call: there is no workspace
- *   to poll. */
+ *   Failures inside the kernel are not reported through this call: poll them with
+ *   w4a8_static_poll_status before the next call. */
 w4a8_status w4a8_linear_static(const int8_t *Xq, const float *tok_scale, const void *packed,
                                const float *bias, int M, int N, int K, int group_size,
                                void *Y_bf16, void *stream);
+
+/* Synchronizes `stream` and returns what the kernel of the last w4a8_linear_static call on the
+ * current device reported (W4A8_OK, W4A8_ERR_TIMEOUT, W4A8_ERR_BAD_BLOB).  The next
+ * w4a8_linear_static call clears that status, so poll before it.  Allocates nothing. */
+w4a8_status w4a8_static_poll_status(void *stream);
 
 /* ---- asymmetric token-wise activations (the paper's own activation quantizer) ----
  * Appendix A.1 quantizes activations token-wise with an asymmetric Min-Max quantizer; the

@@ -7,7 +7,7 @@ been built: there is no CPU or other fallback path.
 from . import synth  # noqa: F401
 from .binding import (  # noqa: F401
     EXPORTS, LIB_PATH, PATH_AUTO, PATH_GEMV, PATH_SIMPLE, PATH_TCGEN05, Opts, W4A8Error, check_status,
-    dint4_table, lib, linear, linear_acc_i32, linear_static, linear_workspace_bytes, make_opts, new_workspace,
+    dint4_table, lib, linear, linear_acc_i32, linear_static, static_poll_status, linear_workspace_bytes, make_opts, new_workspace,
     pack_weights, packed_bytes, poll_status, quantize_act, unpack_codes, version,
     workspace_init, quantize_act_asym, weight_rowsum, linear_asym,
     quantize_linear, quantize_linear_workspace_bytes, new_quantize_linear_workspace, linear_plan,

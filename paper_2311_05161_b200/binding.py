@@ -25,7 +25,8 @@ PATH_AUTO, PATH_SIMPLE, PATH_TCGEN05, PATH_GEMV = 0, 1, 2, 3
 EXPORTS = (
     "w4a8_packed_bytes", "w4a8_pack_weights", "w4a8_quantize_act",
     "w4a8_linear_workspace_bytes", "w4a8_linear_workspace_bytes_ex", "w4a8_workspace_init",
-    "w4a8_linear", "w4a8_linear_ex", "w4a8_linear_static", "w4a8_linear_acc_i32", "w4a8_unpack_codes",
+    "w4a8_linear", "w4a8_linear_ex", "w4a8_linear_static", "w4a8_static_poll_status", "w4a8_linear_acc_i32",
+    "w4a8_unpack_codes",
     "w4a8_poll_status", "w4a8_dint4_table", "w4a8_version",
     "w4a8_quantize_act_asym", "w4a8_weight_rowsum", "w4a8_linear_asym",
     "w4a8_pack_weights_fmt", "w4a8_dint4_table_fmt",
@@ -80,6 +81,8 @@ def _load() -> ctypes.CDLL:
     lib.w4a8_linear_ex.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp, sz, vp, op]
     lib.w4a8_linear_static.restype = ci
     lib.w4a8_linear_static.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, vp, vp]
+    lib.w4a8_static_poll_status.restype = ci
+    lib.w4a8_static_poll_status.argtypes = [vp]
     lib.w4a8_quantize_linear_workspace_bytes.restype = sz
     lib.w4a8_quantize_linear_workspace_bytes.argtypes = [ci, ci, ci, ci]
     lib.w4a8_quantize_linear.restype = ci
@@ -455,6 +458,11 @@ def linear_static(Xq, tok_scale, packed, bias, N: int, group: int, out):
     _check(lib.w4a8_linear_static(_ptr(Xq), _ptr(tok_scale), _ptr(packed), _ptr(bias), M, N, K,
                                   group, _ptr(out), _stream()), "w4a8_linear_static")
     return out
+
+
+def static_poll_status() -> int:
+    """Status the kernel of the last linear_static call on this device reported (0 = none)."""
+    return int(lib.w4a8_static_poll_status(_stream()))
 
 
 def linear_acc_i32(Xq, packed, N: int, group: int, workspace, opts: Opts | None = None, out=None):

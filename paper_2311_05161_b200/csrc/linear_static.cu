@@ -68,3 +68,18 @@ extern "C" w4a8_status w4a8_linear_static(const int8_t *Xq, const float *tok_sca
     return launch_linear_tcgen05(Xq, tok_scale, static_cast<const uint8_t *>(packed), L, bias, M,
                                  static_cast<__nv_bfloat16 *>(Y_bf16), nullptr, scratch, plan, st);
 }
+
+// What the kernel of the last w4a8_linear_static call on this device reported: the status block
+// at the head of the array, read after `stream` has drained (the next call clears it).  Copies
+// twelve bytes to the host; allocates nothing.
+extern "C" w4a8_status w4a8_static_poll_status(void *stream)
+{
+    unsigned char *scratch = nullptr;
+    const w4a8_status s = scratch_for_current_device(&scratch);
+    if (s != W4A8_OK) return s;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return W4A8_ERR_CUDA;
+    int host[3] = {0, 0, 0};
+    if (cudaMemcpy(host, scratch, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess) return W4A8_ERR_CUDA;
+    if (host[0] == 0) return W4A8_OK;
+    return host[0] == W4A8_ERR_BAD_BLOB ? W4A8_ERR_BAD_BLOB : W4A8_ERR_TIMEOUT;
+}

@@ -48,6 +48,7 @@ def test_static_scratch_entry_point_matches_linear_twice(group):
         if call == 1:       # (the first call on a device may load the kernel's code)
             assert torch.cuda.mem_get_info()[0] == free_before, "the call took device memory"
         assert torch.cuda.memory_allocated() == held_before
+        assert w4a8.static_poll_status() == 0
         got = bf16_bits(out)
         assert np.array_equal(got, want_bits), f"call {call}: differs from w4a8_linear"
         check_y(prob, got, exact=(group == 0))
@@ -69,6 +70,24 @@ def test_static_scratch_entry_point_with_two_tokens():
         torch.cuda.synchronize()
         assert np.array_equal(bf16_bits(out), want_bits), f"call {call}"
         check_y(prob, bf16_bits(out), exact=True)
+
+
+def test_static_scratch_reports_a_blob_that_does_not_match():
+    # a blob packed per channel, described to the call as group-128: the kernel touches nothing
+    # but the status block, and the status is readable until the next call clears it
+    prob = Problem(1024, 384, 16, 0, seed=322)
+    d = prob.dev
+    packed = w4a8.pack_weights(d["W"], d["s"], 0)
+    Xq, tok = w4a8.quantize_act(d["X"], d["inv_s"])
+    room = torch.zeros(w4a8.packed_bytes(384, 1024, 128), dtype=torch.uint8, device="cuda")
+    room[:packed.numel()] = packed
+    out = torch.zeros((16, 384), dtype=torch.bfloat16, device="cuda")
+    w4a8.linear_static(Xq, tok, room, d["bias"], 384, 128, out)
+    assert w4a8.static_poll_status() == 8            # W4A8_ERR_BAD_BLOB
+    assert torch.count_nonzero(out).item() == 0
+    w4a8.linear_static(Xq, tok, packed, d["bias"], 384, 0, out)
+    assert w4a8.static_poll_status() == 0
+    check_y(prob, bf16_bits(out), exact=True)
 
 
 def test_static_scratch_rejects_plans_beyond_its_size():
