@@ -176,6 +176,24 @@ def test_full_size_opt_6_7b_shapes_sampled(shape_index, M):
     check(lay, Y[np.ix_(toks, rows)], acc[np.ix_(toks, rows)], rows=rows, toks=toks)
 
 
+def test_large_layer_in_the_mma_pair_with_offset_tables_sampled():
+    """A layer large enough for the automatic MMA pair with offset tables (8192 x 8192, more than
+    1024 tokens): the zero-point term and the offset term leave the accumulator together."""
+    K, N, M = 8192, 8192, 1024 + 53
+    assert w4a8.linear_plan(M, N, K, 0)["cluster"] == 3
+    seed = 4711
+    rng = np.random.Generator(np.random.PCG64([seed, 99]))
+    W = synth.make_weights(N, K, seed)
+    X = synth.make_activations(M, K, seed, "normal", 8, 60.0)
+    X = (X.astype(np.float32) + (rng.standard_normal((M, 1)) * 0.5).astype(np.float32)).astype(np.float16)
+    s, inv = synth.make_channel_scales(X, W)
+    lay = {"W": W, "X": X, "s": s, "inv_s": inv, "bias": synth.make_bias(N, seed)}
+    Y, acc = run(lay, K, N, M, None)
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, N - 1], rng.choice(N, 40, replace=False)]))
+    toks = np.unique(np.concatenate([[0, 255, 256, M - 1], rng.choice(M, 24, replace=False)]))
+    check(lay, Y[np.ix_(toks, rows)], acc[np.ix_(toks, rows)], rows=rows, toks=toks)
+
+
 # ---- group-128 weight steps with asymmetric activations ----
 def run_group(K, N, M, opts, seed):
     lay = make(K, N, M, seed=seed, dist="laplace")
