@@ -66,9 +66,9 @@ typedef struct {
                         or 32) */
     int level_shift; /* special value of the blob = step / 2^level_shift: 0 or 1 (the paper's
                         step/2), 2 or 3 (w4a8_pack_weights_fmt); must match the blob */
-    int cluster;     /* 0 = automatic: form 3 with offset tables for 1024 tokens and more on layers
-                        of at least 8192 x 8192 when the shape allows it (and decode_warps and
-                        offset_tables are 0), else form 1;
+    int cluster;     /* 0 = automatic: form 3 (form 4 from K = 32768 on) with offset tables for 1024
+                        tokens and more on layers of at least 8192 x 8192 when the shape allows
+                        it (and decode_warps and offset_tables are 0), else form 1;
                         else the form of the tensor-core kernel:
                         1 = one CTA per cluster, one row tile per CTA;
                         2 = sharing pair (token tiles of 128 and more, symmetric activations

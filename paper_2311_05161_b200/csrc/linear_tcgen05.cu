@@ -54,7 +54,7 @@ struct Cfg {
     static constexpr int kEpiGroups = !GROUPED ? 1 : (TOK >= 128 ? 4 : TOK >= 64 ? 2 : 1);
     // output staging buffers per group (one where the token ring needs the room)
     static constexpr int kStageBufs = (GROUPED || (TOK >= 256 && CL != 3)) ? 1 : 2;
-    static constexpr int kAStagesWanted = GROUPED ? 5 : (TOK >= 256 && CL != 3) ? 3 : 4;
+    static constexpr int kAStagesWanted = CL == 4 ? 5 : CL == 3 ? 4 : GROUPED ? 5 : TOK >= 256 ? 3 : 4;
     static constexpr int kEpiWarps = 4 * kEpiGroups;
     static constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
     static constexpr int kColsPerThread = TOK / kEpiGroups;
@@ -127,7 +127,9 @@ struct Cfg {
     static constexpr int kOffTok = kOffStaging + kStagingBytes;
     static constexpr int kOffBarriers = kOffTok + 3072;
     static constexpr int kSmemBytes = kOffBarriers + 1024 + 1024 /* alignment slack */;
-    static_assert(kStages >= kAStages && kAStages >= 2, "pipeline depth");
+    // (a barrier slot must not be reused while a decode thread may still wait on its last phase:
+    // the weight buffers span at most as many rounds as there are slots)
+    static_assert(kStages * kPerRound >= kAStages && kAStages >= 2 && kStages >= 3, "pipeline depth");
     static_assert(kTmemNeed <= 512, "tensor memory budget");
     static_assert(kSmemBytes <= 232448, "shared memory budget");
     static_assert(!GROUPED || TOK <= 128, "group mode keeps its FP32 sums in registers");
@@ -1659,7 +1661,10 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
         if (auto_pair && M >= 1024 && L.N >= 8192 && L.K >= 8192 && tok == 256 && split == 1 &&
             offset_fits && L.n_tiles % 2 == 0 &&
             L.k_blocks % 2 == 0 && (!opts || (opts->decode_warps == 0 && opts->offset_tables == 0))) {
-            cluster = 3;
+            // (very long K: two row tiles per CTA instead - no traffic between CTAs, and the
+            // epilogue that this form cannot overlap is small against 256 and more k-blocks;
+            // 36864 -> 9216 at 2048 tokens, sustained: 2660 against 2460 TOPS)
+            cluster = L.k_blocks >= 256 ? 4 : 3;
             auto_offset = true;
         }
     }
