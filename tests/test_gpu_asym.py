@@ -176,6 +176,18 @@ def test_full_size_opt_6_7b_shapes_sampled(shape_index, M):
     check(lay, Y[np.ix_(toks, rows)], acc[np.ix_(toks, rows)], rows=rows, toks=toks)
 
 
+@pytest.mark.parametrize("cluster", [2, 3, 4])
+@pytest.mark.parametrize("offset_tables", [0, 1])
+def test_cluster_forms_with_zero_points(cluster, offset_tables):
+    """The zero-point term (and the offset term of the offset tables) in every cluster form of the
+    tensor-core kernel: ragged token tile, rows past N in the last tile."""
+    K, N, M = 512, 128 * 6 - 24, 2 * 256 + 37
+    lay = make(K, N, M, seed=80 + cluster)
+    Y, acc = run(lay, K, N, M, w4a8.make_opts(w4a8.PATH_TCGEN05, tok_tile=256, cluster=cluster,
+                                              offset_tables=offset_tables))
+    check(lay, Y, acc)
+
+
 def test_large_layer_in_the_mma_pair_with_offset_tables_sampled():
     """A layer large enough for the automatic MMA pair with offset tables (8192 x 8192, more than
     1024 tokens): the zero-point term and the offset term leave the accumulator together."""
