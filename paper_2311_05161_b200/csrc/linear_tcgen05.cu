@@ -1029,27 +1029,18 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
             // ring of weight buffers can hide).  The codes of the team's next item are requested
             // only now, into the registers the expansion has just read, so a thread holds raw
             // codes and levels of one item at a time; the wait and the stores cover the loads.
-            // Group mode keeps the older order (next codes requested first, expansion after the
-            // wait): its MMAs are short and its promotion warps own the issue slots, and there the
-            // early expansion measured 15 % slower.
-            constexpr bool kFetchFirst = GROUPED;
-            uint4 wn[kFetchFirst ? QT : 1];
+            // (Group mode measured the same with either order.)
             int zn = 0;
-            if constexpr (kFetchFirst) {
-                if (nxt.valid(env)) fetch(nxt, wn, zn);
-            } else {
-                expand();
+            expand();
 #pragma unroll
-                for (int q = 0; q < 2 * QT; ++q)
-                    asm volatile("" : "+r"(lv[q].x), "+r"(lv[q].y), "+r"(lv[q].z), "+r"(lv[q].w));
-                if (nxt.valid(env)) fetch(nxt, w, zn);
-            }
+            for (int q = 0; q < 2 * QT; ++q)
+                asm volatile("" : "+r"(lv[q].x), "+r"(lv[q].y), "+r"(lv[q].z), "+r"(lv[q].w));
+            if (nxt.valid(env)) fetch(nxt, w, zn);
             {
                 // (all lanes poll: one polling lane per warp was measured a quarter slower)
                 ok = wait_a_free(cur.it);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if constexpr (kFetchFirst) expand();
                 uint8_t *arow = gen_base + sa * kABytes + r * 128;
                 const int sw = r & 7;
 #pragma unroll
@@ -1069,10 +1060,6 @@ linear_tcgen05_kernel(const __grid_constant__ CUtensorMap tok_map,
                                          map_to_cta(bar_dec + 8 * st, peer));
                     }
                 }
-            }
-            if constexpr (kFetchFirst) {
-#pragma unroll
-                for (int q = 0; q < QT; ++q) w[q] = wn[q];
             }
             z = zn;
             cur = nxt;
