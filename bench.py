@@ -740,8 +740,8 @@ def main():
             "decode": {"metric": "w4a8_dint_linear_hbm_gbs", "M": 1, "value": bytes3 / (ms_d3_dec * 1e-3) / 1e9,
                        "unit": "GB/s", "ms_per_step": ms_d3_dec, "bytes_per_step": bytes3,
                        "frac_of_measured_copy": bytes3 / (ms_d3_dec * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                       "note": "tensor-core kernel with a 16-token tile (the weight-streaming kernels "
-                               "read 4-bit tiles only), 3 rotating blob copies, CUDA graph replay"}}
+                       "note": "quantize_act + linear per shape (weight-streaming kernel, row slabs, 3-bit "
+                               "tiles), 3 rotating blob copies, CUDA graph replay"}}
 
         # decode, M = 1: eight launches of a few microseconds per step, timed from a CUDA graph
         for d in L2:

@@ -92,7 +92,9 @@ typedef struct {
                             and only w4a8_linear_ex with W4A8_PATH_TCGEN05 takes them */
     int bits;        /* code width of the blob: 0 or 4 (dINT4), or 3 (dINT3, packed by
                         w4a8_pack_weights_bits); must match the blob.  3-bit blobs run on the
-                        tensor-core kernel (any M) or the simple kernel, with symmetric activations */
+                        tensor-core kernel (any M), the row-slab form of the weight-streaming
+                        kernel (one or two tokens, layers of 3072 rows and more) or the simple
+                        kernel, with symmetric activations */
     int offset_tables; /* 0 = off (on with the automatic MMA pair, see cluster); 1 = the
                         tensor-core kernel expands codes through level tables
                         stored with an offset (fewer logic instructions per code) and takes the

@@ -51,7 +51,7 @@ bool opts_ok(const w4a8_opts *o)
     if (o->tok_run < 0 || (o->tok_run && (o->path == W4A8_PATH_GEMV || o->path == W4A8_PATH_SIMPLE))) return false;
     if (o->offset_tables < 0 || o->offset_tables > 1 || (o->bits != 0 && !bits_ok(o->bits))) return false;
     if (o->offset_tables && (o->path == W4A8_PATH_GEMV || o->path == W4A8_PATH_SIMPLE)) return false;
-    if (o->bits == 3 && (o->path == W4A8_PATH_GEMV || o->cluster >= 2)) return false;
+    if (o->bits == 3 && o->cluster >= 2) return false;
 #ifdef W4A8_DEBUG_HOOKS
     if (o->debug_wait_ms < 0 || o->debug_wait_ms > 2000 || o->debug_skip_load < 0) return false;
     if ((o->debug_wait_ms || o->debug_skip_load) && o->path != W4A8_PATH_TCGEN05) return false;
@@ -75,13 +75,15 @@ bool depth_ok(int K, int shift, int amax)
 // default it takes one and two tokens: measured, it is as fast or faster there on every shape
 // (two tokens: 5.0 against 9.3 us on 4096 -> 4096, 13.2 against 17.7 us on 16384 -> 4096, equal on
 // 9216 -> 36864), and the tensor-core kernel with its 16-token tile wins from four tokens on.
-bool use_gemv(int M, const w4a8_opts *o)
+bool use_gemv(int M, const BlobLayout &L, const w4a8_opts *o)
 {
     const int path = o ? o->path : W4A8_PATH_AUTO;
     if (path == W4A8_PATH_GEMV) return true;
-    if (bits_of(o) == 3) return false;       // the weight-streaming kernels read 4-bit tiles
     if (path != W4A8_PATH_AUTO || (o && (o->split_k || o->tok_tile || o->decode_warps || o->cluster || o->offset_tables || o->tok_run)))
         return false;
+    // 3-bit tiles are read by the row-slab kernel only: layers too narrow for it stay on the
+    // tensor-core kernel
+    if (L.bits == 3) return M <= 2 && gemv_row_slab_warps(M, L, 0) > 0;
     return M <= 2;
 }
 
@@ -115,7 +117,7 @@ w4a8_status linear_common(const int8_t *Xq, const float *tok_scale, const void *
         return e == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
     }
     LinearPlan plan;
-    if (use_gemv(M, opts)) {
+    if (use_gemv(M, L, opts)) {
         gemv_plan(M, L, &plan);
         // on request, the warps of a CTA of the row-slab variant (else chosen by the length of K)
         const int dw = opts ? opts->decode_warps : 0;
@@ -218,12 +220,14 @@ size_t w4a8_linear_workspace_bytes_ex(int M, int N, int K, int group_size, const
     if (!shape_ok(N, K, group_size) || M < 1 || !opts_ok(opts)) return 0;
     if (opts && opts->path == W4A8_PATH_SIMPLE) return sizeof(StatusBlock);
     LinearPlan plan;
-    if (use_gemv(M, opts)) {
+    const BlobLayout L = make_layout(N, K, group_size, shift_of(opts), bits_of(opts));
+    if (use_gemv(M, L, opts)) {
         if (M > gemv_max_tokens()) return 0;
-        gemv_plan(M, make_layout(N, K, group_size), &plan);
+        if (L.bits == 3 && gemv_row_slab_warps(M, L, opts ? opts->decode_warps : 0) == 0) return 0;
+        gemv_plan(M, L, &plan);
         return plan.workspace_bytes;
     }
-    if (!make_plan(M, make_layout(N, K, group_size, shift_of(opts), bits_of(opts)), opts, &plan, true)) return 0;
+    if (!make_plan(M, L, opts, &plan, true)) return 0;
     return plan.workspace_bytes;
 }
 
@@ -244,7 +248,7 @@ w4a8_status w4a8_linear_plan(int M, int N, int K, int group_size, const w4a8_opt
         return W4A8_OK;
     }
     LinearPlan plan;
-    if (use_gemv(M, opts)) {
+    if (use_gemv(M, L, opts)) {
         if (M > gemv_max_tokens()) return W4A8_ERR_SHAPE;
         gemv_plan(M, L, &plan);
         const int warps = gemv_row_slab_warps(M, L, opts ? opts->decode_warps : 0);

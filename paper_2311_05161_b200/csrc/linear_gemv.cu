@@ -385,7 +385,10 @@ linear_gemv_kernel(const GemvParams P)
 constexpr int kRowsPerCta = 32;
 constexpr int kRowSlabMaxTokenBytes = 96 * 1024;
 
-template <int MT, bool GROUPED, int W>
+// BITS = 3: the 3-bit tile layout (twelve 32-bit words per row and k-block, word w of all 128 rows
+// contiguous, so a warp's 32 lanes read 128 contiguous bytes per word) and the 8-entry level
+// table; no offset tables there (one permute per four codes already).
+template <int MT, bool GROUPED, int W, int BITS = 4>
 __global__ void __launch_bounds__(32 * W)
 linear_gemv_rows_kernel(const GemvParams P)
 {
@@ -400,12 +403,24 @@ linear_gemv_rows_kernel(const GemvParams P)
     const int r = slab * kRowsPerCta + lane;                  // row inside the 128-row tile
     const int n = nt * kTileN + r;
     const int k_blocks = P.L.k_blocks;
-    const uint8_t *src = P.codes + (size_t)nt * k_blocks * kTileBytes + r * 16;
+    const uint8_t *src = BITS == 3 ? P.codes + (size_t)nt * k_blocks * kTileBytes3 + r * 4
+                                   : P.codes + (size_t)nt * k_blocks * kTileBytes + r * 16;
     auto fetch = [&](int kb, uint4 (&dst)[4]) {
+        if constexpr (BITS == 3) {
+            uint32_t *d = reinterpret_cast<uint32_t *>(dst);        // twelve of the sixteen words
+            const uint32_t *p = reinterpret_cast<const uint32_t *>(src + (size_t)kb * kTileBytes3);
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-            dst[q] = ld_stream(reinterpret_cast<const uint4 *>(src + (size_t)kb * kTileBytes +
-                                                               q * kQuarterBytes));
+            for (int i = 0; i < 12; ++i) {
+                uint32_t v;
+                asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p + i * 128));
+                d[i] = v;
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                dst[q] = ld_stream(reinterpret_cast<const uint4 *>(src + (size_t)kb * kTileBytes +
+                                                                   q * kQuarterBytes));
+        }
     };
     // Before the wait only prefetch hints are allowed: ask L2 for this warp's first two
     // k-blocks (its 32 rows x 16 bytes x 4 quarters each = sixteen 128-byte lines per k-block, one
@@ -413,7 +428,7 @@ linear_gemv_rows_kernel(const GemvParams P)
     // (Hints further ahead inside the main loop were measured slower on the large shapes.)
     auto prefetch_pair = [&](int kb0) {      // k-blocks kb0 and kb0 + W of this warp
         const int kbp = kb0 + (lane >> 4) * W;
-        if (kbp < k_blocks) {
+        if (BITS == 4 && kbp < k_blocks) {
             const uint8_t *line = P.codes + ((size_t)nt * k_blocks + kbp) * kTileBytes +
                                   ((lane >> 2) & 3) * kQuarterBytes + slab * (kRowsPerCta * 16) + (lane & 3) * 128;
             asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
@@ -465,7 +480,7 @@ linear_gemv_rows_kernel(const GemvParams P)
     }
     // offset-table expansion (see build_offset_tables) for special values step/2 and step/4;
     // a warp sums the token values of its own k-blocks (written and read by the same warp)
-    const bool offset_tables = P.L.shift <= 2;
+    const bool offset_tables = BITS == 4 && P.L.shift <= 2;
     const int off = 13 << P.L.shift;
     if (offset_tables) {
         for (int kbi = warp; kbi < k_blocks; kbi += W)
@@ -481,19 +496,46 @@ linear_gemv_rows_kernel(const GemvParams P)
 #pragma unroll
     for (int m = 0; m < MT; ++m) { acc[m] = 0; usum[m] = 0.0f; }
     uint32_t t[4];
-    if (!GROUPED) {
-        if (offset_tables) build_offset_tables(P.zeros[n], P.lt, P.L.shift, t);
-        else build_level_tables(P.zeros[n], P.lt, t);
-    }
-    auto consume = [&](int kbi, const uint4 (&w)[4]) {
-        if (GROUPED) {
-            const int z = P.zeros[(size_t)kbi * P.L.n_pad + n];
+    auto tables = [&](int z) {
+        if constexpr (BITS == 3) {
+            uint32_t t3[2];
+            build_level_tables3(z, P.L.shift, t3);
+            t[0] = t3[0]; t[1] = t3[1];
+        } else {
             if (offset_tables) build_offset_tables(z, P.lt, P.L.shift, t);
             else build_level_tables(z, P.lt, t);
+        }
+    };
+    if (!GROUPED) tables(P.zeros[n]);
+    auto consume = [&](int kbi, const uint4 (&w)[4]) {
+        if (GROUPED) {
+            tables(P.zeros[(size_t)kbi * P.L.n_pad + n]);
 #pragma unroll
             for (int m = 0; m < MT; ++m) acc[m] = 0;
         }
-        if (offset_tables) {
+        if constexpr (BITS == 3) {
+            // per 32-k quarter: three words whose nibbles (top bit cleared) select eight levels
+            // each, and a fourth selector put together from the top bits
+            const uint32_t *w3 = reinterpret_cast<const uint32_t *>(w);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint32_t a = w3[3 * q], b = w3[3 * q + 1], c = w3[3 * q + 2];
+                const uint32_t sel[4] = {a & 0x77777777u, b & 0x77777777u, c & 0x77777777u,
+                                         ((a >> 3) & 0x11111111u) | ((b >> 2) & 0x22222222u) |
+                                             ((c >> 1) & 0x44444444u)};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t d0 = prmt(t[0], t[1], sel[j]), d1 = prmt(t[0], t[1], sel[j] >> 16);
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) {
+                        const uint2 x = *reinterpret_cast<const uint2 *>(
+                            s_x + (size_t)m * P.L.K + kbi * kTileK + q * 32 + j * 8);
+                        acc[m] = __dp4a((int)d0, (int)x.x, acc[m]);
+                        acc[m] = __dp4a((int)d1, (int)x.y, acc[m]);
+                    }
+                }
+            }
+        } else if (offset_tables) {
             block_dot_offset<MT>(w, t, s_x + kbi * kTileK, (size_t)P.L.K, acc);
 #pragma unroll
             for (int m = 0; m < MT; ++m)
@@ -576,13 +618,13 @@ void ensure_dynamic_smem(Kernel kern, int bytes, std::atomic<int> (&set_bytes)[k
         set_bytes[dev].store(bytes, std::memory_order_release);
 }
 
-template <int MT, bool GROUPED, int W>
+template <int MT, bool GROUPED, int W, int BITS = 4>
 void launch_rows(const GemvParams &P, cudaStream_t st)
 {
     const int smem = MT * P.L.K + W * MT * 32 * 4 + MT * P.L.k_blocks * 4;
     static std::atomic<int> set_bytes[kMaxGemvDevices] = {};
-    ensure_dynamic_smem(linear_gemv_rows_kernel<MT, GROUPED, W>, smem, set_bytes);
-    launch_overlapped(linear_gemv_rows_kernel<MT, GROUPED, W>, dim3(P.L.n_tiles * 4), dim3(32 * W),
+    ensure_dynamic_smem(linear_gemv_rows_kernel<MT, GROUPED, W, BITS>, smem, set_bytes);
+    launch_overlapped(linear_gemv_rows_kernel<MT, GROUPED, W, BITS>, dim3(P.L.n_tiles * 4), dim3(32 * W),
                       (size_t)smem, st, P);
 }
 
@@ -646,6 +688,10 @@ int gemv_row_slab_warps(int M, const BlobLayout &L, int requested_warps)
     const int mt = M == 1 ? 1 : (M == 2 ? 2 : 4);
     int w = requested_warps ? requested_warps : row_slab_warps(mt, L);
     if (w == 32 && mt > 2) w = 16;
+    if (L.bits == 3) {                 // 3-bit codes: one or two tokens, 8 or 16 warps
+        if (M > 2) return 0;
+        w = w >= 16 ? 16 : 8;
+    }
     return w;
 }
 
@@ -715,6 +761,20 @@ w4a8_status launch_linear_gemv(const int8_t *Xq, const float *tok_scale, const u
     if (P.slices > 65535) return W4A8_ERR_SHAPE;
     const dim3 grid(L.n_tiles, P.slices);
     const bool g = L.group != 0;
+    if (L.bits == 3) {
+        // 3-bit codes: the row-slab kernel only, one or two tokens, 8 or 16 warps per CTA
+        if (M > 2 || X != nullptr || !row_slabs_fit(M, L, plan.decode_warps != 0)) return W4A8_ERR_SHAPE;
+        int w = plan.decode_warps ? plan.decode_warps : row_slab_warps(M, L);
+        w = w >= 16 ? 16 : 8;
+        if (M == 1) {
+            if (g) { if (w == 16) launch_rows<1, true, 16, 3>(P, st); else launch_rows<1, true, 8, 3>(P, st); }
+            else { if (w == 16) launch_rows<1, false, 16, 3>(P, st); else launch_rows<1, false, 8, 3>(P, st); }
+        } else {
+            if (g) { if (w == 16) launch_rows<2, true, 16, 3>(P, st); else launch_rows<2, true, 8, 3>(P, st); }
+            else { if (w == 16) launch_rows<2, false, 16, 3>(P, st); else launch_rows<2, false, 8, 3>(P, st); }
+        }
+        return cudaGetLastError() == cudaSuccess ? W4A8_OK : W4A8_ERR_CUDA;
+    }
     if (row_slabs_fit(M, L, plan.decode_warps != 0)) {
         const int w = plan.decode_warps;
         if (M == 1) { if (g) launch_rows_w<1, true>(P, st, w); else launch_rows_w<1, false>(P, st, w); }

@@ -78,11 +78,27 @@ def test_split_k_automatic_plan_and_single_token(group):
     run(768, 128 * 40, 130, group, 1, dict(path=w4a8.PATH_TCGEN05, tok_tile=16), seed=80 + group)  # many tiles per CTA
 
 
+@pytest.mark.parametrize("group", [0, 128])
+@pytest.mark.parametrize("M", [1, 2])
+def test_weight_streaming_kernel_reads_three_bit_tiles(M, group):
+    """One and two tokens on layers wide enough for row slabs: the weight-streaming kernel with
+    the 3-bit tile layout and the 8-entry table (automatic plan and 8 / 16 warps on request)."""
+    K, N = 1280, 3072 + 128
+    assert w4a8.linear_plan(M, N, K, group, w4a8.make_opts(bits=3))["kernel"] == "weight-streaming"
+    run(K, N, M, group, 1, {}, seed=90 + M + group)
+    run(K, N, M, group, 2, dict(path=w4a8.PATH_GEMV, decode_warps=16), seed=95 + M + group)
+    run(K, N - 24, M, group, 1, dict(path=w4a8.PATH_GEMV, decode_warps=8), seed=99 + M + group)   # rows past N
+
+
 def test_unsupported_combinations_are_refused():
+    # narrow layers have no row slabs, and the K-sliced weight-streaming kernel reads 4-bit tiles
     assert w4a8.linear_workspace_bytes(2, 256, 256, 0, w4a8.make_opts(w4a8.PATH_GEMV, bits=3)) == 0
+    assert w4a8.linear_workspace_bytes(4, 4096, 1024, 0, w4a8.make_opts(w4a8.PATH_GEMV, bits=3)) == 0
     assert w4a8.linear_workspace_bytes(300, 256, 256, 0, w4a8.make_opts(tok_tile=128, cluster=2, bits=3)) == 0
     assert w4a8.linear_workspace_bytes(300, 256, 256, 0, w4a8.make_opts(bits=5)) == 0
-    assert w4a8.linear_plan(1, 4096, 4096, 0, w4a8.make_opts(bits=3))["kernel"] == "tcgen05"
+    assert w4a8.linear_plan(1, 1024, 4096, 0, w4a8.make_opts(bits=3))["kernel"] == "tcgen05"
+    assert w4a8.linear_plan(1, 4096, 4096, 0, w4a8.make_opts(bits=3))["kernel"] == "weight-streaming"
+    assert w4a8.linear_plan(4, 4096, 4096, 0, w4a8.make_opts(bits=3))["kernel"] == "tcgen05"
 
 
 @pytest.mark.parametrize("shape_index", [0, 3])
