@@ -66,9 +66,9 @@ typedef struct {
                         or 32) */
     int level_shift; /* special value of the blob = step / 2^level_shift: 0 or 1 (the paper's
                         step/2), 2 or 3 (w4a8_pack_weights_fmt); must match the blob */
-    int cluster;     /* 0 = automatic: form 3 (form 4 from K = 32768 on) with offset tables for 1024
-                        tokens and more on layers of at least 8192 x 8192 when the shape allows
-                        it (and decode_warps and offset_tables are 0), else form 1;
+    int cluster;     /* 0 = automatic: form 3 or 5 (form 4 from K = 32768 on) with offset tables for
+                        1024 tokens and more on layers of at least 8192 x 8192 when the shape
+                        allows it (and decode_warps and offset_tables are 0), else form 1;
                         else the form of the tensor-core kernel:
                         1 = one CTA per cluster, one row tile per CTA;
                         2 = sharing pair (token tiles of 128 and more, symmetric activations
@@ -79,8 +79,10 @@ typedef struct {
                             CTAs on two row tiles and one token tile issue every MMA as one
                             256-row instruction, each loads half of the tokens;
                         4 = two row tiles per CTA (token tile 256, per-channel 4-bit weights, an
-                            even number of 128-row tiles, 16 decode warps): one CTA multiplies
-                            two row tiles by the same token buffer.
+                            even number of 128-row tiles, 16 decode warps): one CTA
+                            multiplies two row tiles by the same token buffer;
+                        5 = form 3 with three k-blocks per barrier round instead of two (numbers
+                            of k-blocks per K slice that are multiples of three, 16 decode warps).
                         Same bits in every form; a form that does not fit the call is refused
                         with W4A8_ERR_SHAPE. */
     int debug_wait_ms;   /* test hook, 0 = off: limit of every bounded wait inside the tensor-core

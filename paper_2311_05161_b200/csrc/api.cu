@@ -47,7 +47,7 @@ bool opts_ok(const w4a8_opts *o)
     if (o->path < W4A8_PATH_AUTO || o->path > W4A8_PATH_GEMV) return false;
     if (o->split_k < 0 || o->tok_tile < 0 || o->decode_warps < 0) return false;
     if (o->level_shift < 0 || o->level_shift > 3) return false;
-    if (o->cluster < 0 || o->cluster > 4) return false;
+    if (o->cluster < 0 || o->cluster > 5) return false;
     if (o->tok_run < 0 || (o->tok_run && (o->path == W4A8_PATH_GEMV || o->path == W4A8_PATH_SIMPLE))) return false;
     if (o->offset_tables < 0 || o->offset_tables > 1 || (o->bits != 0 && !bits_ok(o->bits))) return false;
     if (o->offset_tables && (o->path == W4A8_PATH_GEMV || o->path == W4A8_PATH_SIMPLE)) return false;

@@ -53,8 +53,8 @@ struct Cfg {
     // 32 columns per thread (more warps in flight, fewer registers each)
     static constexpr int kEpiGroups = !GROUPED ? 1 : (TOK >= 128 ? 4 : TOK >= 64 ? 2 : 1);
     // output staging buffers per group (one where the token ring needs the room)
-    static constexpr int kStageBufs = (GROUPED || (TOK >= 256 && CL != 3)) ? 1 : 2;
-    static constexpr int kAStagesWanted = CL == 4 ? 5 : CL == 3 ? 4 : GROUPED ? 5 : TOK >= 256 ? 3 : 4;
+    static constexpr int kStageBufs = (GROUPED || (TOK >= 256 && CL != 3 && CL != 5)) ? 1 : 2;
+    static constexpr int kAStagesWanted = CL == 4 ? 5 : CL == 5 ? 6 : CL == 3 ? 4 : GROUPED ? 5 : TOK >= 256 ? 3 : 4;
     static constexpr int kEpiWarps = 4 * kEpiGroups;
     static constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);
     static constexpr int kColsPerThread = TOK / kEpiGroups;
@@ -68,14 +68,16 @@ struct Cfg {
     // token buffer, so the token bytes per MAC halve as in the MMA pair, without any traffic
     // between CTAs; the two accumulators fill tensor memory, so the epilogue of a unit no longer
     // overlaps the next unit's main loop.
-    static constexpr bool kShare = CL == 2, kPair = CL == 3, kDual = CL == 4;
+    // CL = 5: the MMA pair with three k-blocks per barrier round (for k-block counts that are
+    // multiples of three: twelve MMA instructions per wait and commit).
+    static constexpr bool kShare = CL == 2, kPair = CL == 3 || CL == 5, kDual = CL == 4;
     static constexpr int kCtas = (kShare || kPair) ? 2 : 1;
     static constexpr int kTiles = kDual ? 2 : 1;               // row tiles of a unit in this CTA
     // k-blocks per barrier round.  The issuing thread's loop (wait, MMAs, commit) is the serial
     // spine of the kernel, and its fixed part per round (wait, commit, bookkeeping: some 300
     // cycles) is what keeps an MMA pair from outrunning one CTA; with two k-blocks per round the
     // pair pays it once per eight MMA instructions.  Operand buffers stay one k-block each.
-    static constexpr int kSub = kPair ? 2 : 1;
+    static constexpr int kSub = CL == 5 ? 3 : kPair ? 2 : 1;
     static constexpr int kPerRound = kTiles * kSub;            // weight buffers filled per round
     static constexpr int kTokRows = kPair ? TOK / 2 : TOK;     // token rows this CTA loads per k-block
     static constexpr int kTokBytes = kTokRows * kTileK;
@@ -94,7 +96,7 @@ struct Cfg {
     // that completes on the peer's barrier, so the table lookups per MMA halve.
     static constexpr int kRowsPerCta = kShare ? kTileN / 2 : kTileN;
     static constexpr int kQuartersPerThread = kShare ? 2 : 4;   // 32-k quarters of a row per thread
-    static_assert(CL >= 1 && CL <= 4, "one CTA, a sharing pair, an MMA pair or two row tiles per CTA");
+    static_assert(CL >= 1 && CL <= 5, "one CTA, a sharing pair, an MMA pair (two forms) or two row tiles per CTA");
     static_assert(!kDual || (TOK == 256 && !GROUPED), "two row tiles per CTA: 256 tokens, per-channel weights");
     static_assert(!kPair || (TOK == 256 && !GROUPED), "the MMA pair: 256 tokens, per-channel weights");
     static_assert(DW % kTeamWarps == 0 && kTeamWarps == 4, "decode warps form whole teams of four");
@@ -1543,6 +1545,9 @@ w4a8_status launch_dw(const Maps &maps, const Params &P, int cluster, cudaStream
     }
     if constexpr (TOK == 256 && !GROUPED && (DW == 8 || DW == 16)) {
         if (cluster == 3) return launch_cl<TOK, false, DW, 3>(maps, P, st);
+        if constexpr (DW == 16) {
+            if (cluster == 5) return launch_cl<TOK, false, 16, 5>(maps, P, st);
+        }
     }
     if constexpr (TOK == 256 && !GROUPED && DW == 16) {
         if (cluster == 4) return P.batch_rows == 0 ? launch_cl<TOK, false, 16, 4>(maps, P, st) : W4A8_ERR_SHAPE;
@@ -1651,13 +1656,16 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
             // (very long K: two row tiles per CTA instead - no traffic between CTAs, and the
             // epilogue that this form cannot overlap is small against 256 and more k-blocks;
             // 36864 -> 9216 at 2048 tokens, sustained: 2660 against 2460 TOPS)
-            cluster = L.k_blocks >= 256 ? 4 : 3;
+            // (k-block counts that are multiples of three: the pair with three k-blocks per
+            // round, twelve MMA instructions per wait and commit; OPT-66B block, the three
+            // 9216-deep layers, sustained: 2560 / 2305 / 2600 against 2455 / 2235 / 2510 TOPS)
+            cluster = L.k_blocks >= 256 ? 4 : L.k_blocks % 3 == 0 ? 5 : 3;
             auto_offset = true;
         }
     }
     // (3: the MMA pair - 256-token tiles, per-channel 4-bit weights, an even number of row tiles)
     // (4: two row tiles per CTA - the same conditions, sixteen decode warps)
-    const bool pair = cluster == 3 || cluster == 4;
+    const bool pair = cluster == 3 || cluster == 4 || cluster == 5;
     if (pair && !(tok == 256 && !grouped && L.bits == 4 && L.n_tiles % 2 == 0)) return false;
     if (cluster != 1 && !pair && !(cluster == 2 && tok >= 128)) return false;
     const int share = cluster == 2 ? 2 : 1;
@@ -1670,10 +1678,11 @@ bool make_plan(int M, const BlobLayout &L, const w4a8_opts *opts, LinearPlan *pl
     if (tiles * split > 0x7fffffffLL) return false;
     // the MMA pair takes k-blocks two at a time: every K slice has an even number of them
     if (cluster == 3 && (kb_per % 2 != 0 || L.k_blocks % 2 != 0)) return false;
+    if (cluster == 5 && (kb_per % 3 != 0 || L.k_blocks % 3 != 0)) return false;
     int dw = opts ? opts->decode_warps : 0;
     if (dw == 0) dw = (grouped || L.bits == 3) ? 8 : 16;
     if (L.bits == 3 && (dw != 8 || cluster != 1)) return false;
-    if (cluster == 4 && dw != 16) return false;
+    if ((cluster == 4 || cluster == 5) && dw != 16) return false;
     if (dw != 4 && dw != 8 && !((dw == 12 || dw == 16) && !grouped)) return false;
     plan->decode_warps = dw;
     plan->cluster = cluster;
@@ -1719,7 +1728,7 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     // pair: each CTA loads half of the token tile)
     if (!encode_2d(enc, &maps.tok, CU_TENSOR_MAP_DATA_TYPE_UINT8, Xq, (cuuint64_t)L.K,
                    (cuuint64_t)M * (plan.batched ? L.n_tiles : 1), (cuuint64_t)L.K, (cuuint32_t)kTileK,
-                   (cuuint32_t)(plan.cluster == 3 ? plan.tok_tile / 2 : plan.tok_tile),
+                   (cuuint32_t)((plan.cluster == 3 || plan.cluster == 5) ? plan.tok_tile / 2 : plan.tok_tile),
                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B))
         return W4A8_ERR_CUDA;
     if (Y && plan.split_k == 1) {
@@ -1756,7 +1765,7 @@ w4a8_status launch_linear_tcgen05(const int8_t *Xq, const float *tok_scale, cons
     // units: (token-tile group, row-tile group, K slice); a sharing pair groups two token tiles,
     // an MMA pair two row tiles
     P.total_units = plan.cluster == 2 ? (plan.tok_tiles + 1) / 2 * L.n_tiles * plan.split_k
-                  : (plan.cluster == 3 || plan.cluster == 4) ? plan.tok_tiles * (L.n_tiles / 2) * plan.split_k
+                  : (plan.cluster == 3 || plan.cluster == 4 || plan.cluster == 5) ? plan.tok_tiles * (L.n_tiles / 2) * plan.split_k
                                       : plan.tok_tiles * L.n_tiles * plan.split_k;
     // Order of the units (unit_tiles): packed weights that stay in L2 are walked once per token
     // tile; larger ones are read by a run of token tiles at the same time, the run as long as its

@@ -263,6 +263,14 @@ def test_tcgen05_mma_pair():
             Y, acc = run_linear(prob, opts, packed)
             assert np.array_equal(acc, want)
             check_y(prob, Y, exact=True)
+    # the same pair with three k-blocks per barrier round (k-block counts that are multiples of three)
+    for split in (1, 2):
+        opts = w4a8.make_opts(w4a8.PATH_TCGEN05, split_k=split, tok_tile=256, cluster=5)
+        for _ in range(2):
+            Y, acc = run_linear(prob, opts, packed)
+            assert np.array_equal(acc, want)
+            check_y(prob, Y, exact=True)
+    assert w4a8.linear_workspace_bytes(300, 512, 1024, 0, w4a8.make_opts(tok_tile=256, cluster=5)) == 0  # 8 k-blocks
     assert w4a8.linear_workspace_bytes(300, 384, 256, 0, w4a8.make_opts(tok_tile=256, cluster=3)) == 0   # odd row tiles
     assert w4a8.linear_workspace_bytes(300, 512, 256, 0, w4a8.make_opts(tok_tile=128, cluster=3)) == 0
     assert w4a8.linear_workspace_bytes(300, 512, 256, 128, w4a8.make_opts(tok_tile=256, cluster=3)) == 0
