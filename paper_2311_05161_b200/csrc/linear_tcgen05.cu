@@ -558,6 +558,18 @@ struct KbCursor {
     __device__ __forceinline__ bool valid(const CursorEnv &e) const { return u < e.total_units; }
     __device__ __forceinline__ void advance(int n, const CursorEnv &e)
     {
+        // the usual case in one step: the n items ahead lie inside the current unit
+        // (the decode warps call this once per item, in the serial part of their cycle)
+        if (valid(e)) {
+            const int ahead = h + n;
+            const int kb_new = kb + ahead / e.tiles;
+            if (kb_new < kb1) {
+                kb = kb_new;
+                h = ahead % e.tiles;
+                it += (uint32_t)n;
+                return;
+            }
+        }
         for (int i = 0; i < n && valid(e); ++i) {
             ++it;
             if (++h < e.tiles) continue;
