@@ -43,7 +43,7 @@ SUSTAINED_FROM_S = 1.0              # regions at least this long are compared wi
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum, mean
 # over the four linears of the headline block, from the ncu launch list of this program); None
 # while the kernel has changed since the counters were taken.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 303.8e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 292.0e6
 CPU_SAMPLE_TOKENS = 48
 CPU_SAMPLE_ROWS = 4096
 NOMINAL_INT8_TOPS = 4500.0
